@@ -1,0 +1,183 @@
+/*
+ * d2o.h -- C ABI of the B200 (sm_100a) implementation of the D2O KV-cache compression
+ * hot path (Dynamic Discriminative Operations, arXiv 2406.13035).
+ *
+ * The calls follow the paper's own statement of the problem:
+ *   (1) after prompt encoding, from every layer's prompt queries and keys, the attention
+ *       density F_v^l (Eq. 4) and the per-layer cache size S_l (Eq. 5, Appendix A.2);
+ *   (2) per layer, token eviction (Eq. 6-8) and dynamic token merging (Eq. 9-12) of the
+ *       prompt cache into a cache of S_l tokens;
+ *   (3) per generated token, attention over the compressed cache (Eq. 2-3), score
+ *       accumulation (Eq. 6), eviction of one token, and its merge-or-discard under the
+ *       EMA threshold (Eq. 9-12).
+ *
+ * Conventions
+ *   - Every pointer is marked HOST or DEVICE.  Device tensors are contiguous, row-major,
+ *     16-byte aligned, in the element type `dtype` of the config unless a C type is given.
+ *   - The library never allocates or frees device memory.  The caller owns `state` (lives
+ *     as long as the context) and `scratch` (only used while a call's work is in flight)
+ *     and sizes them with d2o_workspace_size().  Inputs are borrowed until the
+ *     stream-ordered work of the call has finished and are never written.
+ *   - All device work is enqueued on the given stream (a cudaStream_t passed as void*).
+ *     Calls return without synchronising, except d2o_layer_budgets and the *_host
+ *     variants, which say so.
+ *   - Every call returns a d2o_status.  Invalid arguments are rejected before anything is
+ *     launched.  Device-side anomalies (a wait that ran out, an empty candidate set) set
+ *     an error word inside `state`, reported by d2o_get_stats(); nothing aborts or traps.
+ *   - A context is not thread-safe; distinct contexts are independent.
+ */
+#ifndef D2O_H_
+#define D2O_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  D2O_OK = 0,
+  D2O_ERR_INVALID_ARG = 1,
+  D2O_ERR_UNSUPPORTED = 2,
+  D2O_ERR_WORKSPACE = 3,   /* state or scratch too small / misaligned */
+  D2O_ERR_STATE = 4,       /* call out of order (e.g. compress before budgets) */
+  D2O_ERR_CUDA = 5,        /* a CUDA runtime call failed; see d2o_last_cuda_error() */
+  D2O_ERR_TIMEOUT = 6
+} d2o_status;
+
+typedef enum { D2O_F32 = 0, D2O_F16 = 1, D2O_BF16 = 2 } d2o_dtype;
+
+/* Hyper-parameters and shapes.  Paper symbols in brackets. */
+typedef struct {
+  int32_t n_layers;        /* [L]                                                          */
+  int32_t batch;           /* independent sequences; budgets, tau and caches are per sequence */
+  int32_t n_q_heads;       /* query heads per layer                                         */
+  int32_t n_kv_heads;      /* KV heads per layer; n_q_heads % n_kv_heads == 0               */
+  int32_t d_head;          /* 64 or 128; softmax scale is 1/sqrt(d_head)                    */
+  int32_t dtype;           /* d2o_dtype of Q/K/V, the cache and the outputs                 */
+  int32_t prompt_len;      /* [L_prompt] = [S] of Eq. 5                                     */
+  int32_t max_new_tokens;  /* upper bound on decode steps                                   */
+  float   rho;             /* [rho] global cache ratio; sum_l S_l = round(rho*L*L_prompt)   */
+  int32_t n_sink;          /* [T] attention-sink tokens always kept                         */
+  int32_t window;          /* [M] recent window; <= 0: derive per layer from nm_ratio       */
+  float   nm_ratio;        /* [N:M], 3.0 in the paper (Section 5.1)                         */
+  float   beta;            /* [beta] weight of the current Max(U_t) in Eq. 10               */
+  float   tau_override;    /* NaN: Eq. 10; +inf: pure eviction; -inf: merge everything      */
+  float   density_temp;    /* gamma in exp(-F/gamma); 1.0 is Eq. 5 as printed               */
+  int32_t min_budget;      /* lower clamp of S_l (>= n_sink + 1)                            */
+  int32_t max_budget;      /* upper clamp of S_l; <= 0 means L_prompt                       */
+  int32_t head_reduce;     /* 0: w_l = sum_h exp(-F_lh/gamma) (Appendix A.5); 1: exp(-mean_h F_lh/gamma) */
+} d2o_config;
+
+typedef struct d2o_ctx d2o_ctx;
+
+/* Device pointers into `state` for inspection / checkpointing.  Per-layer fields refer to the
+ * layer passed to d2o_get_view().  Slices are ordered (b, kv_head); slice (b, h) of the layer
+ * owns rows [row_off + (b*Hkv + h)... see fields.  All DEVICE. */
+typedef struct {
+  const float*   colsum;     /* [B, Hq, P]   column sums of the prompt attention (Eq. 4)      */
+  const double*  density;    /* [B, L, Hq]   F_v per sequence, layer, query head (all layers) */
+  const int32_t* budgets;    /* [B, L]       S_l (all layers)                                  */
+  const int32_t* windows;    /* [B, L]       M_l (all layers)                                  */
+  const int64_t* row_off;    /* [B, L]       first cache row of (b, layer); slice (b,h) starts at row_off + h*S_l */
+  void*          k_cache;    /* base of the K pool, rows of d_head elements (all layers)      */
+  void*          v_cache;    /* base of the V pool                                             */
+  int32_t*       pos;        /* [rows]       original position of each cache row (pool-wide)  */
+  float*         score;      /* [rows]       accumulated attention score (Eq. 6)              */
+  float*         rnorm;      /* [rows]       1/|k| of the stored key (0 for a zero key)       */
+  int32_t*       len;        /* [L, B, Hkv]  tokens currently held (all layers)               */
+  float*         tau;        /* [L, B, Hkv]  EMA threshold (Eq. 10) (all layers)              */
+  const int32_t* evict_idx;  /* [B, Hkv, P]  scratch: evicted prompt positions of the last compressed layer */
+  const float*   evict_mx;   /* [B, Hkv, P]  scratch: Max(U[i,:])                              */
+  const int32_t* evict_nn;   /* [B, Hkv, P]  scratch: Argmax slot (relative to the slice)      */
+  int64_t        pool_rows;  /* total cache rows in the pool                                   */
+} d2o_view;
+
+typedef struct {
+  uint64_t decode_steps;     /* slices x steps processed                                       */
+  uint64_t evictions;        /* tokens evicted during decode                                   */
+  uint64_t merges;           /* ... of which merged (Max(U) >= tau_t)                          */
+  uint64_t discards;         /* ... of which discarded                                         */
+  uint64_t prefill_evicted;  /* tokens evicted at prompt stage                                 */
+  uint64_t prefill_merged;   /* ... of which merged                                            */
+  uint32_t error_word;       /* 0 = none; else first device-side anomaly (d2o_status)         */
+  uint32_t error_detail;
+} d2o_stats;
+
+const char* d2o_status_string(d2o_status s);
+/* Text of the last CUDA runtime error seen by this thread's calls (HOST string). */
+const char* d2o_last_cuda_error(void);
+
+/* Sizes in bytes of the caller-owned DEVICE buffers for this config. */
+d2o_status d2o_workspace_size(const d2o_config* cfg, size_t* state_bytes, size_t* scratch_bytes);
+
+/* Creates a context over caller-owned DEVICE buffers (256-byte aligned).  Zeroes the
+ * bookkeeping part of `state` on `stream`.  The host object is freed by d2o_destroy(). */
+d2o_status d2o_create(const d2o_config* cfg, void* state, size_t state_bytes,
+                      void* scratch, size_t scratch_bytes, void* stream, d2o_ctx** out);
+void d2o_destroy(d2o_ctx* ctx);
+
+/* (1) Eq. 4 for one layer.  Q DEVICE [B, Hq, P, d], K DEVICE [B, Hkv, P, d].
+ * Computes s = column sums of the causal prompt attention Softmax(Q K^T / sqrt(d)) per query
+ * head and F_v = Var(s).  `lse` (DEVICE float [B, Hq, P], natural-log row normalisers of that
+ * attention) may be NULL, in which case it is computed here. */
+d2o_status d2o_layer_stats(d2o_ctx* ctx, int32_t layer, const void* Q, const void* K,
+                           const float* lse, void* stream);
+
+/* (1') Eq. 5 / Appendix A.2 once every layer has been fed: S_l for all layers and sequences.
+ * Writes budgets_host (HOST int32 [B, L], may be NULL).  Synchronises `stream`: the host
+ * needs S_l to lay out the cache.  */
+d2o_status d2o_layer_budgets(d2o_ctx* ctx, int32_t* budgets_host, void* stream);
+
+/* Eq. 5 as a pure function: density DEVICE double [B, L, H] -> budgets DEVICE int32 [B, L]
+ * (and, if not NULL, windows DEVICE int32 [B, L], row offsets DEVICE int64 [B, L]).
+ * No context; asynchronous. */
+d2o_status d2o_budgets_from_density(const double* density, int32_t batch, int32_t n_layers,
+                                    int32_t n_heads, int32_t n_kv_heads, int32_t prompt_len,
+                                    float rho, int32_t min_budget, int32_t max_budget,
+                                    float density_temp, int32_t head_reduce, int32_t n_sink,
+                                    int32_t window, float nm_ratio, int32_t* budgets,
+                                    int32_t* windows, int64_t* row_off, int32_t* status_word,
+                                    void* stream);
+
+/* (2) Eq. 6-12 for one layer's prompt cache.  K, V DEVICE [B, Hkv, P, d].
+ * Keeps T sinks, the Top-N accumulated scores and the last M tokens, matches every evicted
+ * key to its most similar kept key, sets tau_0, merges the tokens at or above it, and
+ * leaves the compressed cache of the layer in `state`. */
+d2o_status d2o_prefill_compress(d2o_ctx* ctx, int32_t layer, const void* K, const void* V,
+                                void* stream);
+
+/* (3) One generated token for layers [l0, l1).  DEVICE tensors:
+ * q [l1-l0, B, Hq, d], k and v [l1-l0, B, Hkv, d], out [l1-l0, B, Hq, d].
+ * Every call advances the token position of those layers by one; all layers must be
+ * stepped equally often. */
+d2o_status d2o_decode_step(d2o_ctx* ctx, int32_t l0, int32_t l1, const void* q, const void* k,
+                           const void* v, void* out, void* stream);
+
+/* Same with HOST buffers (pinned memory recommended): copies q, k, v to the device, runs the
+ * step, copies `out` back and synchronises `stream`. */
+d2o_status d2o_decode_step_host(d2o_ctx* ctx, int32_t l0, int32_t l1, const void* q_host,
+                                const void* k_host, const void* v_host, void* out_host,
+                                void* stream);
+
+/* Uncompressed decode attention (Eq. 2-3), the comparison kernel: appends k, v at row `len`
+ * of k_cache/v_cache DEVICE [n_slices, capacity, d] (n_slices = B*Hkv) and attends over
+ * len+1 rows.  q, out DEVICE [n_slices, group, d]; k, v DEVICE [n_slices, d].
+ * No context, no state; asynchronous. */
+d2o_status d2o_full_decode_step(int32_t dtype, int32_t d_head, int32_t n_slices, int32_t group,
+                                int32_t capacity, int32_t len, void* k_cache, void* v_cache,
+                                const void* q, const void* k, const void* v, void* out,
+                                void* stream);
+
+d2o_status d2o_get_view(d2o_ctx* ctx, int32_t layer, d2o_view* out);
+/* Copies the counters to HOST memory; synchronises `stream`. */
+d2o_status d2o_get_stats(d2o_ctx* ctx, d2o_stats* out_host, void* stream);
+
+/* Launch-shape knobs for measurements (0 = automatic): CTAs per cluster of the decode kernel. */
+d2o_status d2o_set_tuning(d2o_ctx* ctx, int32_t decode_cluster, int32_t reserved);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* D2O_H_ */

@@ -111,22 +111,24 @@ def layer_weights(F: np.ndarray, gamma: float = 1.0, head_reduce: int = 0) -> np
 
 
 def layer_budgets(F: np.ndarray, P: int, rho: float, min_budget: int = 1,
-                  gamma: float = 1.0, head_reduce: int = 0) -> np.ndarray:
+                  gamma: float = 1.0, head_reduce: int = 0, max_budget: int = 0) -> np.ndarray:
     """Integer cache size S_l of every layer (Eq. 5; constraint sum_l S_l = S*L*rho).
 
     Unclamped, S_l = alpha_l * P with alpha_l = L*rho*w_l / sum_l w_l.
     Reading (the paper is silent on all three):
-      * a layer cannot hold fewer than ``min_budget`` or more than ``P`` tokens, so
-        S_l = clip(lam * w_l, min_budget, P) with the single scale ``lam`` chosen so that
-        the total is still S_tot (equal to the unclamped formula when no clamp binds);
+      * a layer cannot hold fewer than ``min_budget`` or more than ``max_budget`` tokens
+        (``P`` unless given: the prompt has no more), so
+        S_l = clip(lam * w_l, min_budget, max_budget) with the single scale ``lam`` chosen so
+        that the total is still S_tot (equal to the unclamped formula when no clamp binds);
       * S_tot = floor(rho*L*P + 1/2);
       * integer sizes by floor + largest remainder (ties: lower layer first)."""
     w = layer_weights(F, gamma, head_reduce)
     L = w.size
     S_tot = int(math.floor(rho * L * P + 0.5))
-    lo, hi = float(min_budget), float(P)
+    cap = max_budget if max_budget > 0 else P
+    lo, hi = float(min_budget), float(cap)
     if not (L * lo <= S_tot <= L * hi):
-        raise ValueError("global budget outside [L*min_budget, L*P]")
+        raise ValueError("global budget outside [L*min_budget, L*max_budget]")
     w = np.maximum(w, 1e-300)        # exp underflow: keep ratios finite
 
     def total(lam: float) -> float:
@@ -160,7 +162,7 @@ def layer_budgets(F: np.ndarray, P: int, rho: float, min_budget: int = 1,
     for l in order:
         if left == 0:
             break
-        if S[l] < P:
+        if S[l] < cap:
             S[l] += 1
             left -= 1
     assert left == 0
@@ -252,6 +254,12 @@ def weighted_merge(Kc: np.ndarray, Vc: np.ndarray, Ke: np.ndarray, Ve: np.ndarra
     return Kn / den[:, None], Vn / den[:, None], den
 
 
+def _merge_with_mask(Kc, Vc, Ke, Ve, mx, nn, mask):
+    """weighted_merge with an explicit mask m_i instead of the threshold test (harness replay)."""
+    passing = np.where(mask, mx, -np.inf)
+    return weighted_merge(Kc, Vc, Ke, Ve, passing, nn, -1e300)
+
+
 @dataclass
 class SliceState:
     """Compressed cache of one (sequence, layer, KV head), kept in ascending position."""
@@ -268,7 +276,10 @@ class SliceState:
 
 
 def prefill_compress_slice(K: np.ndarray, V: np.ndarray, score: np.ndarray, S: int, T: int, M: int,
-                           dtype: str, tau_override: float = float("nan")) -> SliceState:
+                           dtype: str, tau_override: float = float("nan"),
+                           force_retained: Optional[np.ndarray] = None,
+                           force_nn: Optional[np.ndarray] = None,
+                           force_merged: Optional[np.ndarray] = None) -> SliceState:
     """Prompt-stage compression of one slice: eviction (Eq. 7-8), nearest-neighbour
     matching (Eq. 9), tau_0 (Eq. 10) and weighted merging (Eq. 11-12).
 
@@ -276,24 +287,40 @@ def prefill_compress_slice(K: np.ndarray, V: np.ndarray, score: np.ndarray, S: i
     over the query heads that share this KV head (reading for grouped-query attention).
     Reading: similarities use the un-merged keys and all merges happen at once;
     every conserved slot (sinks and window included) can receive merges;
-    a conserved token keeps its own accumulated score."""
+    a conserved token keeps its own accumulated score.
+    ``force_*`` let a harness replay another implementation's choice at a near-tie: the kept
+    positions, the neighbour column of some evicted rows (-1 = keep own), the merge mask."""
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
     retained, evicted = select_retained(score, S, T, M)
+    if force_retained is not None:
+        retained = np.array(sorted(int(j) for j in force_retained), dtype=np.int64)
+        keep = set(retained.tolist())
+        evicted = np.array([j for j in range(K.shape[0]) if j not in keep], dtype=np.int64)
     Kc, Vc = K[retained], V[retained]
     Ke, Ve = K[evicted], V[evicted]
     U = cosine_matrix(Ke, Kc)
     mx, nn = nearest_neighbour(U)
+    if force_nn is not None:
+        for i, j in enumerate(force_nn):
+            if j >= 0:
+                nn[i] = j
+                mx[i] = U[i, j]
     tau0 = initial_threshold(mx)
     thr = tau0 if math.isnan(tau_override) else tau_override
-    Km, Vm, den = weighted_merge(Kc, Vc, Ke, Ve, mx, nn, thr)
+    if force_merged is not None:
+        # a merge mask is replayed by moving the threshold out of the way row by row
+        Km, Vm, den = _merge_with_mask(Kc, Vc, Ke, Ve, mx, nn, np.asarray(force_merged, bool))
+    else:
+        Km, Vm, den = weighted_merge(Kc, Vc, Ke, Ve, mx, nn, thr)
     touched = den > E
     Kn = np.where(touched[:, None], round_storage(Km, dtype), Kc)
     Vn = np.where(touched[:, None], round_storage(Vm, dtype), Vc)
     st = SliceState(pos=retained.copy(), K=Kn, V=Vn, score=np.asarray(score, np.float64)[retained].copy(),
                     tau=tau0, S=S, T=T, M=M, dtype=dtype)
-    st.log = dict(retained=retained, evicted=evicted, mx=mx, nn=nn, den=den,
-                  merged=(mx >= thr) if mx.size else np.zeros(0, bool))
+    st.log = dict(retained=retained, evicted=evicted, mx=mx, nn=nn, den=den, U=U, thr=thr,
+                  merged=(np.asarray(force_merged, bool) if force_merged is not None
+                          else ((mx >= thr) if mx.size else np.zeros(0, bool))))
     return st
 
 
@@ -407,13 +434,14 @@ class OracleStack:
     def __init__(self, *, n_layers: int, batch: int, n_q_heads: int, n_kv_heads: int, d_head: int,
                  dtype: str, prompt_len: int, rho: float, n_sink: int, window: int, nm_ratio: float,
                  beta: float, density_temp: float = 1.0, min_budget: int = 1, head_reduce: int = 0,
-                 tau_override: float = float("nan")):
+                 tau_override: float = float("nan"), max_budget: int = 0):
         self.L, self.B, self.Hq, self.Hkv, self.d = n_layers, batch, n_q_heads, n_kv_heads, d_head
         self.G = n_q_heads // n_kv_heads
         self.dtype, self.P, self.rho = dtype, prompt_len, rho
         self.T, self.window, self.nm_ratio, self.beta = n_sink, window, nm_ratio, beta
         self.gamma, self.min_budget, self.head_reduce = density_temp, min_budget, head_reduce
         self.tau_override = tau_override
+        self.max_budget = max_budget
         self.colsum = np.zeros((self.L, self.B, self.Hq, self.P))
         self.F = np.zeros((self.B, self.L, self.Hq))
         self.budgets: Optional[np.ndarray] = None          # [B, L]
@@ -431,7 +459,7 @@ class OracleStack:
     def layer_budgets(self, F: Optional[np.ndarray] = None) -> np.ndarray:
         F = self.F if F is None else np.asarray(F, np.float64)
         self.budgets = np.stack([layer_budgets(F[b], self.P, self.rho, self.min_budget, self.gamma,
-                                               self.head_reduce) for b in range(self.B)])
+                                               self.head_reduce, self.max_budget) for b in range(self.B)])
         return self.budgets
 
     def slice_params(self, b: int, layer: int) -> Tuple[int, int, int]:
@@ -440,16 +468,20 @@ class OracleStack:
         M = window_size(S, T, self.window, self.nm_ratio)
         return S, T, M
 
+    def group_score(self, layer: int, b: int, h: int) -> np.ndarray:
+        """AttnScore of one KV head at the prompt stage: the sum over its G query heads."""
+        return self.colsum[layer, b, h * self.G:(h + 1) * self.G].sum(axis=0)
+
     def prefill_compress(self, layer: int, K: np.ndarray, V: np.ndarray,
-                         slices: Optional[List[Tuple[int, int]]] = None, colsum: Optional[np.ndarray] = None):
-        """``slices`` restricts to (b, kv head) pairs; ``colsum`` [B,Hq,P] replaces the stored sums."""
-        cs = self.colsum[layer] if colsum is None else np.asarray(colsum, np.float64)
+                         slices: Optional[List[Tuple[int, int]]] = None, force: Optional[dict] = None):
+        """``slices`` restricts to (b, kv head) pairs; ``force[(layer,b,h)]`` may hold the
+        keyword overrides of prefill_compress_slice."""
         todo = slices if slices is not None else [(b, h) for b in range(self.B) for h in range(self.Hkv)]
         for b, h in todo:
             S, T, M = self.slice_params(b, layer)
-            score = cs[b, h * self.G:(h + 1) * self.G].sum(axis=0)
-            self.slices[(layer, b, h)] = prefill_compress_slice(K[b, h], V[b, h], score, S, T, M,
-                                                                self.dtype, self.tau_override)
+            kw = (force or {}).get((layer, b, h), {})
+            self.slices[(layer, b, h)] = prefill_compress_slice(K[b, h], V[b, h], self.group_score(layer, b, h),
+                                                                S, T, M, self.dtype, self.tau_override, **kw)
 
     def decode_step(self, layer: int, q: np.ndarray, k: np.ndarray, v: np.ndarray, t: int,
                     slices: Optional[List[Tuple[int, int]]] = None, force: Optional[dict] = None):

@@ -1,0 +1,181 @@
+// Shared device/host helpers of the D2O library: element-type traits, 16-byte vector access,
+// warp reductions, the context object and the launcher prototypes.  Nothing in here is shared
+// with the CPU oracle.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/d2o.h"
+
+namespace d2o {
+
+constexpr float kEuler = 2.718281828459045f;   // weight of a conserved token: exp(self-similarity 1), Eq. 12
+constexpr float kLog2e = 1.4426950408889634f;
+
+// ----------------------------------------------------------------------------- element traits
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int kPerVec = 4;            // elements per 16-byte vector
+  __device__ static __forceinline__ void unpack(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
+  __device__ static __forceinline__ uint4 pack(const float* f) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+  }
+  __device__ static __forceinline__ float to_float(float x) { return x; }
+  __device__ static __forceinline__ float from_float(float x) { return x; }
+};
+template <> struct Elem<__half> {
+  static constexpr int kPerVec = 8;
+  __device__ static __forceinline__ void unpack(const uint4& v, float* f) {
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { float2 t = __half22float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+  }
+  __device__ static __forceinline__ uint4 pack(const float* f) {
+    uint4 v; __half2* h = reinterpret_cast<__half2*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2half2_rn(f[2 * i], f[2 * i + 1]);
+    return v;
+  }
+  __device__ static __forceinline__ float to_float(__half x) { return __half2float(x); }
+  __device__ static __forceinline__ __half from_float(float x) { return __float2half_rn(x); }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int kPerVec = 8;
+  __device__ static __forceinline__ void unpack(const uint4& v, float* f) {
+    // bf16 -> f32 is a 16-bit shift
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+  __device__ static __forceinline__ uint4 pack(const float* f) {
+    uint4 v; __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    return v;
+  }
+  __device__ static __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+  __device__ static __forceinline__ __nv_bfloat16 from_float(float x) { return __float2bfloat16_rn(x); }
+};
+
+__device__ __forceinline__ uint4 ld_global_v4(const void* p) {
+  return *reinterpret_cast<const uint4*>(p);
+}
+// streaming load: data that is read once per launch should not displace reusable lines in L1
+// (plain coherent load: the cache rows are also written later in the same launch)
+__device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// ----------------------------------------------------------------------------- reductions
+template <typename T> __device__ __forceinline__ T warp_sum(T v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { unsigned long long t = __shfl_xor_sync(0xffffffffu, v, o); v = t < v ? t : v; }
+  return v;
+}
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { unsigned long long t = __shfl_xor_sync(0xffffffffu, v, o); v = t > v ? t : v; }
+  return v;
+}
+// A row of d_head elements is handled by LPR consecutive lanes (one 16-byte segment each).  Groups of
+// one warp may diverge (ragged tails), so their shuffles name only the lanes of the group.
+template <int LPR> __device__ __forceinline__ unsigned group_mask() {
+  if (LPR >= 32) return 0xffffffffu;
+  return ((1u << (LPR & 31)) - 1u) << (((threadIdx.x & 31) / LPR) * LPR);
+}
+template <int LPR> __device__ __forceinline__ float group_sum(float v, unsigned mask) {
+#pragma unroll
+  for (int o = LPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(mask, v, o);
+  return v;
+}
+// monotone map float -> uint32 (a < b  <=>  ord(a) < ord(b)), -0 and +0 distinct but adjacent
+__device__ __forceinline__ uint32_t float_ord(float f) {
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ord_float(uint32_t o) {
+  uint32_t u = (o & 0x80000000u) ? (o & 0x7fffffffu) : ~o;
+  return __uint_as_float(u);
+}
+
+// device-side anomaly report: first writer wins
+__device__ __forceinline__ void report_error(uint32_t* status_word, uint32_t code, uint32_t detail) {
+  if (atomicCAS(status_word, 0u, code) == 0u) status_word[1] = detail;
+}
+
+// ----------------------------------------------------------------------------- counters
+enum Counter { kCntDecodeSteps = 0, kCntEvictions, kCntMerges, kCntDiscards, kCntPrefillEvicted,
+               kCntPrefillMerged, kNumCounters = 8 };
+
+// ----------------------------------------------------------------------------- context
+struct Layout {            // byte offsets into `state`
+  size_t status, counters, density, budgets, windows, row_off, len, tau, colsum, pos, score, rnorm, kpool, vpool, end;
+};
+struct ScratchLayout {     // byte offsets into `scratch`
+  size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, stage_q, stage_k, stage_v, stage_out, end;
+};
+
+}  // namespace d2o
+
+struct d2o_ctx {
+  d2o_config cfg;
+  int group;
+  int elem_size;
+  int max_budget;
+  int64_t total_budget;        // S_tot per sequence = round(rho * L * P)
+  int64_t pool_rows;           // B * Hkv * S_tot
+  d2o::Layout lay;
+  d2o::ScratchLayout slay;
+  char* state;
+  char* scratch;
+  size_t state_bytes, scratch_bytes;
+  // host mirrors, valid after d2o_layer_budgets
+  bool have_budgets;
+  int32_t* h_budgets;          // [B, L]
+  int32_t* h_windows;          // [B, L]
+  int64_t* h_row_off;          // [B, L]
+  uint8_t* layer_fed;          // [L] stats seen
+  uint8_t* layer_compressed;   // [L]
+  int32_t* layer_steps;        // [L] decode steps taken
+  int decode_cluster;          // tuning: 0 = auto
+};
+
+namespace d2o {
+
+// launchers (one per .cu file); all return cudaError_t of the launch
+cudaError_t launch_layer_stats(const d2o_ctx* c, int layer, const void* Q, const void* K, const float* lse,
+                               cudaStream_t st);
+cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, int P, float rho, int min_budget,
+                           int max_budget, float gamma, int head_reduce, int n_sink, int window, float nm_ratio,
+                           int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
+                           cudaStream_t st);
+cudaError_t launch_prefill_compress(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st);
+cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const void* k, const void* v, void* out,
+                          cudaStream_t st, d2o_status* why);
+cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int capacity, int len, void* kc, void* vc,
+                               const void* q, const void* k, const void* v, void* out, cudaStream_t st,
+                               d2o_status* why);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace d2o

@@ -1,0 +1,342 @@
+// Host side of the C ABI: argument validation, workspace layout, context bookkeeping.
+// All device work is delegated to the launchers of the other translation units.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "d2o_common.cuh"
+
+using namespace d2o;
+
+static thread_local char g_cuda_err[256] = "";
+
+static d2o_status cuda_fail(cudaError_t e, const char* where) {
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", where, cudaGetErrorString(e));
+  return D2O_ERR_CUDA;
+}
+#define CUDA_TRY(expr)                                   \
+  do {                                                   \
+    cudaError_t e_ = (expr);                             \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #expr);  \
+  } while (0)
+
+extern "C" const char* d2o_status_string(d2o_status s) {
+  switch (s) {
+    case D2O_OK: return "ok";
+    case D2O_ERR_INVALID_ARG: return "invalid argument";
+    case D2O_ERR_UNSUPPORTED: return "unsupported configuration";
+    case D2O_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case D2O_ERR_STATE: return "call out of order";
+    case D2O_ERR_CUDA: return "CUDA runtime error";
+    case D2O_ERR_TIMEOUT: return "device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+extern "C" const char* d2o_last_cuda_error(void) { return g_cuda_err; }
+
+static int elem_size_of(int dtype) { return dtype == D2O_F32 ? 4 : 2; }
+
+static d2o_status validate(const d2o_config* c, int64_t* total_budget, int* max_budget) {
+  if (!c) return D2O_ERR_INVALID_ARG;
+  if (c->n_layers < 1 || c->n_layers > 1024 || c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1)
+    return D2O_ERR_INVALID_ARG;
+  if (c->n_q_heads % c->n_kv_heads != 0) return D2O_ERR_INVALID_ARG;
+  int g = c->n_q_heads / c->n_kv_heads;
+  if (g != 1 && g != 2 && g != 4 && g != 8) return D2O_ERR_UNSUPPORTED;
+  if (c->d_head != 64 && c->d_head != 128) return D2O_ERR_UNSUPPORTED;
+  if (c->dtype != D2O_F32 && c->dtype != D2O_F16 && c->dtype != D2O_BF16) return D2O_ERR_UNSUPPORTED;
+  if (c->prompt_len < 1 || c->prompt_len > (1 << 20) || c->max_new_tokens < 0) return D2O_ERR_INVALID_ARG;
+  if (!(c->rho > 0.0f) || !isfinite(c->rho)) return D2O_ERR_INVALID_ARG;
+  if (c->n_sink < 0 || c->nm_ratio < 0.0f || !isfinite(c->nm_ratio)) return D2O_ERR_INVALID_ARG;
+  if (!(c->beta >= 0.0f && c->beta <= 1.0f)) return D2O_ERR_INVALID_ARG;
+  if (!(c->density_temp > 0.0f) || !isfinite(c->density_temp)) return D2O_ERR_INVALID_ARG;
+  if (c->head_reduce != 0 && c->head_reduce != 1) return D2O_ERR_UNSUPPORTED;
+  int maxb = c->max_budget > 0 ? c->max_budget : c->prompt_len;
+  if (maxb > c->prompt_len + c->max_new_tokens) return D2O_ERR_INVALID_ARG;
+  if (c->min_budget < 1 || c->min_budget < c->n_sink + 1 || c->min_budget > maxb) return D2O_ERR_INVALID_ARG;
+  double tot = floor((double)c->rho * (double)c->n_layers * (double)c->prompt_len + 0.5);
+  if (tot < (double)c->n_layers * c->min_budget || tot > (double)c->n_layers * maxb) return D2O_ERR_INVALID_ARG;
+  if (maxb + 1 > 8 * 8192) return D2O_ERR_UNSUPPORTED;   // decode kernel: one cluster (<= 8 CTAs) per slice
+  *total_budget = (int64_t)tot;
+  *max_budget = maxb;
+  return D2O_OK;
+}
+
+static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, Layout* l, ScratchLayout* s) {
+  const size_t B = c->batch, L = c->n_layers, Hq = c->n_q_heads, Hkv = c->n_kv_heads, P = c->prompt_len;
+  const size_t d = c->d_head, e = elem_size_of(c->dtype);
+  const size_t rows = B * Hkv * (size_t)total_budget;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  l->status = take(16);
+  l->counters = take(kNumCounters * 8);
+  l->density = take(B * L * Hq * 8);
+  l->budgets = take(B * L * 4);
+  l->windows = take(B * L * 4);
+  l->row_off = take(B * L * 8);
+  l->len = take(L * B * Hkv * 4);
+  l->tau = take(L * B * Hkv * 4);
+  l->colsum = take(L * B * Hq * P * 4);
+  l->pos = take(rows * 4);
+  l->score = take(rows * 4);
+  l->rnorm = take(rows * 4);
+  l->kpool = take(rows * d * e);
+  l->vpool = take(rows * d * e);
+  l->end = o;
+  o = 0;
+  s->lse = take(B * Hq * P * 4);
+  s->evict_idx = take(B * Hkv * P * 4);
+  s->evict_mx = take(B * Hkv * P * 4);
+  s->evict_nn = take(B * Hkv * P * 4);
+  s->seg_start = take(B * Hkv * ((size_t)max_budget + 2) * 4);
+  s->seg_items = take(B * Hkv * P * 4);
+  s->stage_q = take(L * B * Hq * d * e);
+  s->stage_k = take(L * B * Hkv * d * e);
+  s->stage_v = take(L * B * Hkv * d * e);
+  s->stage_out = take(L * B * Hq * d * e);
+  s->end = o;
+}
+
+extern "C" d2o_status d2o_workspace_size(const d2o_config* cfg, size_t* state_bytes, size_t* scratch_bytes) {
+  int64_t tot; int maxb;
+  d2o_status st = validate(cfg, &tot, &maxb);
+  if (st != D2O_OK) return st;
+  if (!state_bytes || !scratch_bytes) return D2O_ERR_INVALID_ARG;
+  Layout l; ScratchLayout s;
+  layouts(cfg, tot, maxb, &l, &s);
+  *state_bytes = l.end;
+  *scratch_bytes = s.end;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t state_bytes, void* scratch,
+                                 size_t scratch_bytes, void* stream, d2o_ctx** out) {
+  int64_t tot; int maxb;
+  d2o_status st = validate(cfg, &tot, &maxb);
+  if (st != D2O_OK) return st;
+  if (!state || !scratch || !out) return D2O_ERR_INVALID_ARG;
+  if (((uintptr_t)state & 255) || ((uintptr_t)scratch & 255)) return D2O_ERR_WORKSPACE;
+  Layout l; ScratchLayout s;
+  layouts(cfg, tot, maxb, &l, &s);
+  if (state_bytes < l.end || scratch_bytes < s.end) return D2O_ERR_WORKSPACE;
+  d2o_ctx* c = (d2o_ctx*)calloc(1, sizeof(d2o_ctx));
+  if (!c) return D2O_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->group = cfg->n_q_heads / cfg->n_kv_heads;
+  c->elem_size = elem_size_of(cfg->dtype);
+  c->max_budget = maxb;
+  c->total_budget = tot;
+  c->pool_rows = (int64_t)cfg->batch * cfg->n_kv_heads * tot;
+  c->lay = l; c->slay = s;
+  c->state = (char*)state; c->scratch = (char*)scratch;
+  c->state_bytes = state_bytes; c->scratch_bytes = scratch_bytes;
+  const size_t BL = (size_t)cfg->batch * cfg->n_layers;
+  c->h_budgets = (int32_t*)calloc(BL, 4);
+  c->h_windows = (int32_t*)calloc(BL, 4);
+  c->h_row_off = (int64_t*)calloc(BL, 8);
+  c->layer_fed = (uint8_t*)calloc(cfg->n_layers, 1);
+  c->layer_compressed = (uint8_t*)calloc(cfg->n_layers, 1);
+  c->layer_steps = (int32_t*)calloc(cfg->n_layers, 4);
+  // bookkeeping (status, counters, density, budgets ... tau) starts at zero
+  cudaError_t e = cudaMemsetAsync(c->state, 0, l.colsum, (cudaStream_t)stream);
+  if (e != cudaSuccess) { d2o_destroy(c); return cuda_fail(e, "cudaMemsetAsync(state)"); }
+  *out = c;
+  return D2O_OK;
+}
+
+extern "C" void d2o_destroy(d2o_ctx* c) {
+  if (!c) return;
+  free(c->h_budgets); free(c->h_windows); free(c->h_row_off);
+  free(c->layer_fed); free(c->layer_compressed); free(c->layer_steps);
+  free(c);
+}
+
+static bool aligned16(const void* p) { return p && (((uintptr_t)p & 15) == 0); }
+
+extern "C" d2o_status d2o_layer_stats(d2o_ctx* c, int32_t layer, const void* Q, const void* K, const float* lse,
+                                      void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return D2O_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || (lse && !aligned16(lse))) return D2O_ERR_INVALID_ARG;
+  CUDA_TRY(launch_layer_stats(c, layer, Q, K, lse, (cudaStream_t)stream));
+  c->layer_fed[layer] = 1;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_budgets_from_density(const double* density, int32_t batch, int32_t n_layers,
+                                               int32_t n_heads, int32_t n_kv_heads, int32_t prompt_len, float rho,
+                                               int32_t min_budget, int32_t max_budget, float density_temp,
+                                               int32_t head_reduce, int32_t n_sink, int32_t window, float nm_ratio,
+                                               int32_t* budgets, int32_t* windows, int64_t* row_off,
+                                               int32_t* status_word, void* stream) {
+  if (!density || !budgets || batch < 1 || n_layers < 1 || n_layers > 1024 || n_heads < 1 || n_kv_heads < 1 ||
+      prompt_len < 1)
+    return D2O_ERR_INVALID_ARG;
+  if (!(rho > 0.0f) || !(density_temp > 0.0f) || (head_reduce != 0 && head_reduce != 1)) return D2O_ERR_INVALID_ARG;
+  if (max_budget <= 0) max_budget = prompt_len;
+  if (min_budget < 1 || min_budget > max_budget) return D2O_ERR_INVALID_ARG;
+  double tot = floor((double)rho * n_layers * prompt_len + 0.5);
+  if (tot < (double)n_layers * min_budget || tot > (double)n_layers * max_budget) return D2O_ERR_INVALID_ARG;
+  CUDA_TRY(launch_budgets(density, batch, n_layers, n_heads, n_kv_heads, prompt_len, rho, min_budget, max_budget,
+                          density_temp, head_reduce, n_sink, window, nm_ratio, budgets, windows, row_off,
+                          (uint32_t*)status_word, (cudaStream_t)stream));
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_layer_budgets(d2o_ctx* c, int32_t* budgets_host, void* stream) {
+  if (!c) return D2O_ERR_INVALID_ARG;
+  for (int l = 0; l < c->cfg.n_layers; ++l)
+    if (!c->layer_fed[l]) return D2O_ERR_STATE;
+  const d2o_config& g = c->cfg;
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t* d_b = (int32_t*)(c->state + c->lay.budgets);
+  int32_t* d_w = (int32_t*)(c->state + c->lay.windows);
+  int64_t* d_o = (int64_t*)(c->state + c->lay.row_off);
+  CUDA_TRY(launch_budgets((const double*)(c->state + c->lay.density), g.batch, g.n_layers, g.n_q_heads,
+                          g.n_kv_heads, g.prompt_len, g.rho, g.min_budget, c->max_budget, g.density_temp,
+                          g.head_reduce, g.n_sink, g.window, g.nm_ratio, d_b, d_w, d_o,
+                          (uint32_t*)(c->state + c->lay.status), st));
+  const size_t BL = (size_t)g.batch * g.n_layers;
+  CUDA_TRY(cudaMemcpyAsync(c->h_budgets, d_b, BL * 4, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaMemcpyAsync(c->h_windows, d_w, BL * 4, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaMemcpyAsync(c->h_row_off, d_o, BL * 8, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  // the device computed offsets for the pool; make sure they fit what the caller gave us
+  for (size_t i = 0; i < BL; ++i) {
+    int64_t end = c->h_row_off[i] + (int64_t)g.n_kv_heads * c->h_budgets[i];
+    if (c->h_budgets[i] < 1 || c->h_budgets[i] > c->max_budget || c->h_row_off[i] < 0 || end > c->pool_rows)
+      return D2O_ERR_STATE;
+  }
+  c->have_budgets = true;
+  if (budgets_host) memcpy(budgets_host, c->h_budgets, BL * 4);
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_prefill_compress(d2o_ctx* c, int32_t layer, const void* K, const void* V, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return D2O_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V)) return D2O_ERR_INVALID_ARG;
+  if (!c->have_budgets) return D2O_ERR_STATE;
+  CUDA_TRY(launch_prefill_compress(c, layer, K, V, (cudaStream_t)stream));
+  c->layer_compressed[layer] = 1;
+  c->layer_steps[layer] = 0;
+  return D2O_OK;
+}
+
+static d2o_status check_decode_range(d2o_ctx* c, int l0, int l1) {
+  if (!c || l0 < 0 || l1 > c->cfg.n_layers || l0 >= l1) return D2O_ERR_INVALID_ARG;
+  for (int l = l0; l < l1; ++l) {
+    if (!c->layer_compressed[l]) return D2O_ERR_STATE;
+    if (c->layer_steps[l] != c->layer_steps[l0]) return D2O_ERR_STATE;
+  }
+  if (c->layer_steps[l0] >= c->cfg.max_new_tokens) return D2O_ERR_STATE;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_decode_step(d2o_ctx* c, int32_t l0, int32_t l1, const void* q, const void* k,
+                                      const void* v, void* out, void* stream) {
+  d2o_status st = check_decode_range(c, l0, l1);
+  if (st != D2O_OK) return st;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return D2O_ERR_INVALID_ARG;
+  d2o_status why = D2O_OK;
+  cudaError_t e = launch_decode(c, l0, l1, q, k, v, out, (cudaStream_t)stream, &why);
+  if (why != D2O_OK) return why;
+  if (e != cudaSuccess) return cuda_fail(e, "launch_decode");
+  for (int l = l0; l < l1; ++l) c->layer_steps[l] += 1;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_decode_step_host(d2o_ctx* c, int32_t l0, int32_t l1, const void* q_host,
+                                           const void* k_host, const void* v_host, void* out_host, void* stream) {
+  d2o_status st = check_decode_range(c, l0, l1);
+  if (st != D2O_OK) return st;
+  if (!q_host || !k_host || !v_host || !out_host) return D2O_ERR_INVALID_ARG;
+  const d2o_config& g = c->cfg;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t nl = (size_t)(l1 - l0);
+  const size_t qb = nl * g.batch * g.n_q_heads * g.d_head * c->elem_size;
+  const size_t kb = nl * g.batch * g.n_kv_heads * g.d_head * c->elem_size;
+  char* dq = c->scratch + c->slay.stage_q;
+  char* dk = c->scratch + c->slay.stage_k;
+  char* dv = c->scratch + c->slay.stage_v;
+  char* dout = c->scratch + c->slay.stage_out;
+  CUDA_TRY(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, s));
+  d2o_status why = D2O_OK;
+  cudaError_t e = launch_decode(c, l0, l1, dq, dk, dv, dout, s, &why);
+  if (why != D2O_OK) return why;
+  if (e != cudaSuccess) return cuda_fail(e, "launch_decode");
+  CUDA_TRY(cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  for (int l = l0; l < l1; ++l) c->layer_steps[l] += 1;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_full_decode_step(int32_t dtype, int32_t d_head, int32_t n_slices, int32_t group,
+                                           int32_t capacity, int32_t len, void* k_cache, void* v_cache,
+                                           const void* q, const void* k, const void* v, void* out, void* stream) {
+  if (dtype != D2O_F32 && dtype != D2O_F16 && dtype != D2O_BF16) return D2O_ERR_UNSUPPORTED;
+  if (d_head != 64 && d_head != 128) return D2O_ERR_UNSUPPORTED;
+  if (group != 1 && group != 2 && group != 4 && group != 8) return D2O_ERR_UNSUPPORTED;
+  if (n_slices < 1 || capacity < 1 || len < 0 || len >= capacity) return D2O_ERR_INVALID_ARG;
+  if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+    return D2O_ERR_INVALID_ARG;
+  d2o_status why = D2O_OK;
+  cudaError_t e = launch_full_decode(dtype, d_head, n_slices, group, capacity, len, k_cache, v_cache, q, k, v, out,
+                                     (cudaStream_t)stream, &why);
+  if (why != D2O_OK) return why;
+  if (e != cudaSuccess) return cuda_fail(e, "launch_full_decode");
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_get_view(d2o_ctx* c, int32_t layer, d2o_view* v) {
+  if (!c || !v || layer < 0 || layer >= c->cfg.n_layers) return D2O_ERR_INVALID_ARG;
+  const d2o_config& g = c->cfg;
+  const size_t per_layer = (size_t)g.batch * g.n_q_heads * g.prompt_len;
+  v->colsum = (const float*)(c->state + c->lay.colsum) + per_layer * layer;
+  v->density = (const double*)(c->state + c->lay.density);
+  v->budgets = (const int32_t*)(c->state + c->lay.budgets);
+  v->windows = (const int32_t*)(c->state + c->lay.windows);
+  v->row_off = (const int64_t*)(c->state + c->lay.row_off);
+  v->k_cache = c->state + c->lay.kpool;
+  v->v_cache = c->state + c->lay.vpool;
+  v->pos = (int32_t*)(c->state + c->lay.pos);
+  v->score = (float*)(c->state + c->lay.score);
+  v->rnorm = (float*)(c->state + c->lay.rnorm);
+  v->len = (int32_t*)(c->state + c->lay.len);
+  v->tau = (float*)(c->state + c->lay.tau);
+  v->evict_idx = (const int32_t*)(c->scratch + c->slay.evict_idx);
+  v->evict_mx = (const float*)(c->scratch + c->slay.evict_mx);
+  v->evict_nn = (const int32_t*)(c->scratch + c->slay.evict_nn);
+  v->pool_rows = c->pool_rows;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_get_stats(d2o_ctx* c, d2o_stats* out, void* stream) {
+  if (!c || !out) return D2O_ERR_INVALID_ARG;
+  uint64_t cnt[kNumCounters];
+  uint32_t word[4];
+  cudaStream_t s = (cudaStream_t)stream;
+  CUDA_TRY(cudaMemcpyAsync(cnt, c->state + c->lay.counters, sizeof(cnt), cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaMemcpyAsync(word, c->state + c->lay.status, sizeof(word), cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  out->decode_steps = cnt[kCntDecodeSteps];
+  out->evictions = cnt[kCntEvictions];
+  out->merges = cnt[kCntMerges];
+  out->discards = cnt[kCntDiscards];
+  out->prefill_evicted = cnt[kCntPrefillEvicted];
+  out->prefill_merged = cnt[kCntPrefillMerged];
+  out->error_word = word[0];
+  out->error_detail = word[1];
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_cluster, int32_t reserved) {
+  (void)reserved;
+  if (!c) return D2O_ERR_INVALID_ARG;
+  if (decode_cluster != 0 && decode_cluster != 1 && decode_cluster != 2 && decode_cluster != 4 && decode_cluster != 8)
+    return D2O_ERR_INVALID_ARG;
+  c->decode_cluster = decode_cluster;
+  return D2O_OK;
+}

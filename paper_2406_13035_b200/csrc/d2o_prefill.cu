@@ -1,0 +1,525 @@
+// Token-level operation at the prompt stage (Section 4.2): eviction (Eq. 7-8), nearest-neighbour
+// matching (Eq. 9), the initial threshold (Eq. 10, t = 0) and weighted merging (Eq. 11-12).
+//
+// Kernels in this file, per layer, one slice = one (sequence, KV head):
+//   select_kernel      group-summed scores, block radix select of the Top-N under the order
+//                      (score desc, position asc), ordered compaction into retained / evicted
+//                      position lists, gather of K_c, V_c, scores and inverse key norms
+//   similarity_kernel  cosine of every evicted key with every retained key, row max / arg-max
+//                      (generic FFMA version; 16-bit inputs take the tcgen05 kernel when built in)
+//   segment_kernel     tau_0 = mean of the row maxima; threshold test; evicted tokens grouped by
+//                      their nearest neighbour in ascending position (deterministic lists)
+//   merge_kernel       per retained row: (e*k_c + sum exp(u)*k_e) / (e + sum exp(u)), same for V
+#include <math.h>
+
+#include "d2o_common.cuh"
+
+namespace d2o {
+
+// ------------------------------------------------------------------------------------ select
+constexpr int kSelThreads = 1024;
+
+struct SelectArgs {
+  const float* colsum;     // [B, Hq, P] of this layer
+  const int32_t* budgets;  // [B, L]
+  const int32_t* windows;  // [B, L]
+  const int64_t* row_off;  // [B, L]
+  int32_t* pos; float* score; float* rnorm;   // pool-wide
+  int32_t* len; float* tau;                   // [L, B, Hkv]
+  int32_t* evict_idx;      // [B, Hkv, P]
+  float* keys_spill;       // [B, Hkv, P] group scores when P does not fit in shared memory (may alias evict_mx)
+  unsigned long long* counters;
+  uint32_t* status;
+  int L, layer, B, Hq, Hkv, G, P, T;
+  int keys_in_smem;
+};
+
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* total) {
+  // exclusive prefix of v over the block (blockDim multiple of 32, <= 1024)
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+  __syncthreads();
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int w = lane < (int)(blockDim.x >> 5) ? warp_tot[lane] : 0;
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xffffffffu, winc, o); if (lane >= o) winc += t; }
+    warp_tot[lane] = winc - w;
+    if (lane == 31) *total = winc;
+  }
+  __syncthreads();
+  return inc - v + warp_tot[warp];
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T* __restrict__ kpool,
+              T* __restrict__ vpool) {
+  extern __shared__ __align__(16) unsigned char sel_smem[];
+  __shared__ int hist[256];
+  __shared__ int warp_tot[32];
+  __shared__ int s_total;
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_need;
+  const int slice = blockIdx.x;                 // b * Hkv + h
+  const int b = slice / a.Hkv, h = slice % a.Hkv;
+  const int P = a.P;
+  const int S = a.budgets[b * a.L + a.layer];
+  const int Tn = a.T < S ? a.T : S;
+  const int M = a.windows[b * a.L + a.layer];
+  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * S;
+  const int sidx = (a.layer * a.B + b) * a.Hkv + h;
+  float* keys = a.keys_in_smem ? reinterpret_cast<float*>(sel_smem) : a.keys_spill + (size_t)slice * P;
+  // group score: sum over the G query heads of this KV head, fixed order (Eq. 6 case 1)
+  const float* cs = a.colsum + ((size_t)b * a.Hq + (size_t)h * a.G) * P;
+  for (int j = threadIdx.x; j < P; j += blockDim.x) {
+    float t = cs[j];
+    for (int g = 1; g < a.G; ++g) t += cs[(size_t)g * P + j];
+    keys[j] = t;
+  }
+  __syncthreads();
+  const bool keep_all = S >= P;
+  const int lo = Tn, hi = keep_all ? Tn : P - M;   // candidate range [lo, hi)
+  const int N = S - Tn - M;
+  uint32_t kth = 0; int need_eq = 0;
+  if (!keep_all && N > 0) {
+    // radix select of the N-th largest key among candidates; scores are >= 0 so the IEEE bit
+    // pattern is monotone, float_ord keeps it monotone for any sign
+    uint32_t prefix = 0, mask = 0; int need = N;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+      __syncthreads();
+      for (int j = lo + threadIdx.x; j < hi; j += blockDim.x) {
+        const uint32_t o = float_ord(keys[j]);
+        if ((o & mask) == prefix) atomicAdd(&hist[(o >> shift) & 255], 1);
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        int acc = 0, bin = 255;
+        for (; bin > 0; --bin) { if (acc + hist[bin] >= need) break; acc += hist[bin]; }
+        s_prefix = prefix | ((uint32_t)bin << shift);
+        s_need = need - acc;
+      }
+      __syncthreads();
+      prefix = s_prefix; need = s_need; mask |= 255u << shift;
+      __syncthreads();
+    }
+    kth = prefix; need_eq = need;                 // keep all keys > kth and the first need_eq keys == kth
+  }
+  // ordered compaction over positions, 1024 at a time
+  int n_ret = 0, n_ev = 0, n_eq = 0;
+  for (int base = 0; base < P; base += blockDim.x) {
+    const int j = base + threadIdx.x;
+    int is_eq = 0, keep = 0;
+    uint32_t o = 0;
+    if (j < P) {
+      if (keep_all || j < Tn || j >= P - M) keep = 1;
+      else if (N > 0) { o = float_ord(keys[j]); if (o > kth) keep = 1; else if (o == kth) is_eq = 1; }
+    }
+    const int eq_rank = block_exclusive_scan(is_eq, warp_tot, &s_total);
+    const int eq_tot = s_total;
+    if (is_eq && n_eq + eq_rank < need_eq) keep = 1;
+    const int kr = block_exclusive_scan(keep, warp_tot, &s_total);
+    const int keep_tot = s_total;
+    if (j < P) {
+      if (keep) {
+        const int slot = n_ret + kr;
+        a.pos[row0 + slot] = j;
+        a.score[row0 + slot] = keys[j];
+      } else {
+        a.evict_idx[(size_t)slice * P + n_ev + (threadIdx.x - kr)] = j;
+      }
+    }
+    const int valid = min((int)blockDim.x, P - base);
+    n_ret += keep_tot; n_ev += valid - keep_tot; n_eq += eq_tot;
+    __syncthreads();
+  }
+  const int n_keep = keep_all ? P : S;
+  if (threadIdx.x == 0) {
+    a.len[sidx] = n_keep;
+    a.tau[sidx] = 0.f;
+    if (n_ret != n_keep) report_error(a.status, D2O_ERR_STATE, 0x5E000000u | (uint32_t)slice);
+    atomicAdd(&a.counters[kCntPrefillEvicted], (unsigned long long)(P - n_keep));
+  }
+  __threadfence_block();
+  __syncthreads();
+  // gather K_c, V_c and 1/|k|: one row per LPR-lane group
+  constexpr int EPV = Elem<T>::kPerVec;
+  constexpr int LPR = D / EPV;                   // lanes per row
+  const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
+  const T* Ks = K + (size_t)slice * P * D;
+  const T* Vs = V + (size_t)slice * P * D;
+  for (int r = grp; r < n_keep; r += blockDim.x / LPR) {
+    const int j = a.pos[row0 + r];
+    const uint4 kv = ld_global_v4(Ks + (size_t)j * D + lig * EPV);
+    const uint4 vv = ld_global_v4(Vs + (size_t)j * D + lig * EPV);
+    *reinterpret_cast<uint4*>(kpool + (row0 + r) * D + lig * EPV) = kv;
+    *reinterpret_cast<uint4*>(vpool + (row0 + r) * D + lig * EPV) = vv;
+    float f[EPV]; Elem<T>::unpack(kv, f);
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < EPV; ++i) ss = fmaf(f[i], f[i], ss);
+    ss = group_sum<LPR>(ss, group_mask<LPR>());
+    if (lig == 0) a.rnorm[row0 + r] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+  }
+}
+
+// ------------------------------------------------------------------------------------ similarity (generic)
+constexpr int kSimTile = 64;
+constexpr int kSimThreads = 256;
+
+struct SimArgs {
+  const int32_t* budgets; const int64_t* row_off;
+  const int32_t* evict_idx; float* evict_mx; int32_t* evict_nn;
+  const float* rnorm; const int32_t* pos;
+  int L, layer, Hkv, P;
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kSimThreads)
+similarity_kernel(SimArgs a, const T* __restrict__ K, const T* __restrict__ kpool) {
+  extern __shared__ __align__(16) float sim_smem[];
+  float* et = sim_smem;                     // [D][64] evicted tile, transposed
+  float* ct = et + D * kSimTile;            // [D][64] retained tile, transposed
+  float* ern = ct + D * kSimTile;           // [64] inverse norms of the evicted rows
+  float* crn = ern + kSimTile;              // [64] inverse norms of the retained rows
+  const int slice = blockIdx.y;
+  const int b = slice / a.Hkv, h = slice % a.Hkv;
+  const int S = a.budgets[b * a.L + a.layer];
+  const int Le = a.P - S;
+  const int i0 = blockIdx.x * kSimTile;
+  if (Le <= 0 || i0 >= Le) return;
+  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * S;
+  const T* Ks = K + (size_t)slice * a.P * D;
+  const int32_t* ev = a.evict_idx + (size_t)slice * a.P;
+  constexpr int EPV = Elem<T>::kPerVec;
+  constexpr int VPR = D / EPV;
+  const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
+  {  // evicted tile: gather rows by index, transposed, plus inverse norms
+    const int r = threadIdx.x % kSimTile;
+    const bool ok = i0 + r < Le;
+    const int j = ok ? ev[i0 + r] : 0;
+    float ss = 0.f;
+    for (int vi = threadIdx.x / kSimTile; vi < VPR; vi += kSimThreads / kSimTile) {
+      float f[EPV];
+      if (ok) { uint4 v = ld_global_v4(Ks + (size_t)j * D + vi * EPV); Elem<T>::unpack(v, f); }
+      else {
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) f[i] = 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < EPV; ++i) { et[(vi * EPV + i) * kSimTile + r] = f[i]; ss = fmaf(f[i], f[i], ss); }
+    }
+    // 4 threads (tid/64 = 0..3) share a row: each partial norm goes to its own cell of ct[]
+    // (not yet in use) and is combined in a fixed order
+    ct[(threadIdx.x / kSimTile) * kSimTile + r] = ss;
+    __syncthreads();
+    if (threadIdx.x < kSimTile) {
+      const float t = (ct[r] + ct[kSimTile + r]) + (ct[2 * kSimTile + r] + ct[3 * kSimTile + r]);
+      ern[r] = t > 0.f ? 1.0f / sqrtf(t) : 0.f;
+    }
+    __syncthreads();
+  }
+  float best[4]; int bidx[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) { best[r] = -INFINITY; bidx[r] = 0x7fffffff; }
+  for (int c0 = 0; c0 < S; c0 += kSimTile) {
+    __syncthreads();
+    {
+      const int r = threadIdx.x % kSimTile;
+      const bool ok = c0 + r < S;
+      for (int vi = threadIdx.x / kSimTile; vi < VPR; vi += kSimThreads / kSimTile) {
+        float f[EPV];
+        if (ok) { uint4 v = ld_global_v4(kpool + (row0 + c0 + r) * D + vi * EPV); Elem<T>::unpack(v, f); }
+        else {
+#pragma unroll
+          for (int i = 0; i < EPV; ++i) f[i] = 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) ct[(vi * EPV + i) * kSimTile + r] = f[i];
+      }
+      if (threadIdx.x < kSimTile) crn[r] = ok ? a.rnorm[row0 + c0 + r] : 0.f;
+    }
+    __syncthreads();
+    float s[4][4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) s[r][c] = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < D; ++k) {
+      const float4 av = *reinterpret_cast<const float4*>(et + k * kSimTile + ty * 4);
+      const float4 bv = *reinterpret_cast<const float4*>(ct + k * kSimTile + tx * 4);
+      const float aa[4] = {av.x, av.y, av.z, av.w};
+      const float bb[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) s[r][c] = fmaf(aa[r], bb[c], s[r][c]);
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const float er = ern[ty * 4 + r];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int col = c0 + tx * 4 + c;
+        if (col < S) {
+          const float u = s[r][c] * er * crn[tx * 4 + c];
+          if (u > best[r]) { best[r] = u; bidx[r] = col; }       // ascending col: first maximum wins
+        }
+      }
+    }
+  }
+  // combine the 16 threads (tx) of a row: max u, ties -> lowest slot
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    unsigned long long key = ((unsigned long long)float_ord(best[r]) << 32) | (uint32_t)(0x7fffffff - bidx[r]);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) {
+      const unsigned long long t = __shfl_xor_sync(0xffffffffu, key, o);
+      key = t > key ? t : key;
+    }
+    const int i = i0 + ty * 4 + r;
+    if (tx == 0 && i < Le) {
+      a.evict_mx[(size_t)slice * a.P + i] = ord_float((uint32_t)(key >> 32));
+      a.evict_nn[(size_t)slice * a.P + i] = 0x7fffffff - (int)(uint32_t)(key & 0xffffffffu);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------ tau_0 + segments
+struct SegArgs {
+  const int32_t* budgets;
+  const float* evict_mx; const int32_t* evict_nn;
+  int32_t* seg_start; int32_t* seg_items; float* tau;
+  unsigned long long* counters;
+  int L, layer, B, Hkv, P, seg_stride;
+  float tau_override;
+};
+
+__global__ void __launch_bounds__(1024)
+segment_kernel(SegArgs a) {
+  extern __shared__ __align__(16) int seg_smem[];       // [S + 1] counts / cursors
+  __shared__ double part[32];
+  __shared__ float s_thr;
+  __shared__ int warp_tot[32];
+  __shared__ int s_total;
+  const int slice = blockIdx.x;
+  const int b = slice / a.Hkv, h = slice % a.Hkv;
+  const int S = a.budgets[b * a.L + a.layer];
+  const int Le = a.P - S;
+  const int sidx = (a.layer * a.B + b) * a.Hkv + h;
+  const float* mx = a.evict_mx + (size_t)slice * a.P;
+  const int32_t* nn = a.evict_nn + (size_t)slice * a.P;
+  int32_t* start = a.seg_start + (size_t)slice * a.seg_stride;
+  int32_t* items = a.seg_items + (size_t)slice * a.P;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (Le <= 0) {
+    for (int j = threadIdx.x; j <= S && j < a.seg_stride; j += blockDim.x) start[j] = 0;
+    if (threadIdx.x == 0) a.tau[sidx] = 0.f;
+    return;
+  }
+  // tau_0 = (1/Le) sum_i mx_i   (Eq. 10, t = 0); fixed reduction tree, double accumulation
+  double t = 0.0;
+  for (int i = threadIdx.x; i < Le; i += blockDim.x) t += (double)mx[i];
+  t = warp_sum(t);
+  if (lane == 0) part[warp] = t;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += part[w];
+    const float tau0 = (float)(s / (double)Le);
+    a.tau[sidx] = tau0;
+    s_thr = isnan(a.tau_override) ? tau0 : a.tau_override;
+  }
+  for (int j = threadIdx.x; j <= S; j += blockDim.x) seg_smem[j] = 0;
+  __syncthreads();
+  const float thr = s_thr;
+  // how many evicted tokens pass the threshold for each retained slot (integer counts: order-free)
+  for (int i = threadIdx.x; i < Le; i += blockDim.x)
+    if (mx[i] >= thr) atomicAdd(&seg_smem[nn[i]], 1);
+  __syncthreads();
+  // exclusive scan of the counts -> segment starts
+  int run = 0;
+  for (int base = 0; base <= S; base += blockDim.x) {
+    const int j = base + threadIdx.x;
+    const int c = j < S ? seg_smem[j] : 0;
+    const int ex = block_exclusive_scan(c, warp_tot, &s_total);
+    if (j <= S) { start[j] = run + ex; }
+    __syncthreads();
+    if (j < S) seg_smem[j] = run + ex;                   // becomes the fill cursor
+    run += s_total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) atomicAdd(&a.counters[kCntPrefillMerged], (unsigned long long)run);
+  // ordered fill by one warp: evicted tokens are visited in ascending index, lanes that share a
+  // target are ranked with match_any, so every list is in ascending position
+  if (warp == 0) {
+    for (int base = 0; base < Le; base += 32) {
+      const int i = base + lane;
+      const bool on = i < Le && mx[i] >= thr;
+      const int j = on ? nn[i] : -1 - lane;               // distinct dummies for idle lanes
+      const unsigned peers = __match_any_sync(0xffffffffu, j);
+      if (on) {
+        const int rank = __popc(peers & ((1u << lane) - 1u));
+        const int cur = seg_smem[j];
+        items[cur + rank] = i;
+        __syncwarp(peers);
+        if (rank == 0) seg_smem[j] = cur + __popc(peers);
+      }
+      __syncwarp();
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------ merge
+struct MergeArgs {
+  const int32_t* budgets; const int64_t* row_off;
+  const int32_t* evict_idx; const float* evict_mx;
+  const int32_t* seg_start; const int32_t* seg_items;
+  float* rnorm;
+  int L, layer, Hkv, P, seg_stride;
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* __restrict__ kpool,
+             T* __restrict__ vpool) {
+  constexpr int EPV = Elem<T>::kPerVec;
+  constexpr int LPR = D / EPV;
+  const int slice = blockIdx.y;
+  const int b = slice / a.Hkv, h = slice % a.Hkv;
+  const int S = a.budgets[b * a.L + a.layer];
+  if (a.P - S <= 0) return;
+  const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
+  const int j = blockIdx.x * (blockDim.x / LPR) + grp;
+  if (j >= S) return;
+  const int32_t* start = a.seg_start + (size_t)slice * a.seg_stride;
+  const int s0 = start[j], s1 = start[j + 1];
+  if (s1 == s0) return;                              // nothing merged: the row stays bit-identical
+  const int64_t row = a.row_off[b * a.L + a.layer] + (int64_t)h * S + j;
+  const int32_t* items = a.seg_items + (size_t)slice * a.P;
+  const int32_t* ev = a.evict_idx + (size_t)slice * a.P;
+  const float* mx = a.evict_mx + (size_t)slice * a.P;
+  const T* Ks = K + (size_t)slice * a.P * D;
+  const T* Vs = V + (size_t)slice * a.P * D;
+  float ka[EPV], va[EPV], f[EPV];
+  Elem<T>::unpack(ld_global_v4(kpool + row * D + lig * EPV), f);
+#pragma unroll
+  for (int i = 0; i < EPV; ++i) ka[i] = kEuler * f[i];
+  Elem<T>::unpack(ld_global_v4(vpool + row * D + lig * EPV), f);
+#pragma unroll
+  for (int i = 0; i < EPV; ++i) va[i] = kEuler * f[i];
+  float den = kEuler;
+  for (int s = s0; s < s1; ++s) {
+    const int i = items[s];
+    const float w = expf(mx[i]);
+    const int pj = ev[i];
+    den += w;
+    Elem<T>::unpack(ld_global_v4(Ks + (size_t)pj * D + lig * EPV), f);
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) ka[e] = fmaf(w, f[e], ka[e]);
+    Elem<T>::unpack(ld_global_v4(Vs + (size_t)pj * D + lig * EPV), f);
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) va[e] = fmaf(w, f[e], va[e]);
+  }
+  const float inv = 1.0f / den;
+#pragma unroll
+  for (int e = 0; e < EPV; ++e) { ka[e] = ka[e] * inv; va[e] = va[e] * inv; }
+  const uint4 kv = Elem<T>::pack(ka);
+  *reinterpret_cast<uint4*>(kpool + row * D + lig * EPV) = kv;
+  *reinterpret_cast<uint4*>(vpool + row * D + lig * EPV) = Elem<T>::pack(va);
+  Elem<T>::unpack(kv, f);                            // the norm of what is actually stored
+  float ss = 0.f;
+#pragma unroll
+  for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
+  ss = group_sum<LPR>(ss, group_mask<LPR>());
+  if (lig == 0) a.rnorm[row] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+}
+
+// ------------------------------------------------------------------------------------ launcher
+template <typename T, int D>
+static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st) {
+  const d2o_config& g = c->cfg;
+  const int B = g.batch, Hkv = g.n_kv_heads, P = g.prompt_len, L = g.n_layers;
+  const int n_slices = B * Hkv;
+  char* S = c->state; char* X = c->scratch;
+  T* kpool = (T*)(S + c->lay.kpool);
+  T* vpool = (T*)(S + c->lay.vpool);
+  int maxS = 0;
+  for (int b = 0; b < B; ++b) maxS = max(maxS, c->h_budgets[b * L + layer]);
+  const int seg_stride = c->max_budget + 2;
+
+  SelectArgs sa;
+  sa.colsum = (const float*)(S + c->lay.colsum) + (size_t)layer * B * g.n_q_heads * P;
+  sa.budgets = (const int32_t*)(S + c->lay.budgets);
+  sa.windows = (const int32_t*)(S + c->lay.windows);
+  sa.row_off = (const int64_t*)(S + c->lay.row_off);
+  sa.pos = (int32_t*)(S + c->lay.pos); sa.score = (float*)(S + c->lay.score); sa.rnorm = (float*)(S + c->lay.rnorm);
+  sa.len = (int32_t*)(S + c->lay.len); sa.tau = (float*)(S + c->lay.tau);
+  sa.evict_idx = (int32_t*)(X + c->slay.evict_idx);
+  sa.keys_spill = (float*)(X + c->slay.evict_mx);
+  sa.counters = (unsigned long long*)(S + c->lay.counters);
+  sa.status = (uint32_t*)(S + c->lay.status);
+  sa.L = L; sa.layer = layer; sa.B = B; sa.Hq = g.n_q_heads; sa.Hkv = Hkv; sa.G = c->group; sa.P = P; sa.T = g.n_sink;
+  const size_t key_bytes = (size_t)P * sizeof(float);
+  sa.keys_in_smem = key_bytes <= 200 * 1024;
+  const size_t sel_sm = sa.keys_in_smem ? key_bytes : 0;
+  cudaError_t e = cudaFuncSetAttribute(select_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)(sel_sm > 48 * 1024 ? sel_sm : 48 * 1024));
+  if (e != cudaSuccess) return e;
+  select_kernel<T, D><<<n_slices, kSelThreads, sel_sm, st>>>(sa, (const T*)K, (const T*)V, kpool, vpool);
+
+  int minS = P;
+  for (int b = 0; b < B; ++b) minS = min(minS, c->h_budgets[b * L + layer]);
+  const int maxLe = P - minS;
+  if (maxLe <= 0) return cudaGetLastError();
+
+  SimArgs ma;
+  ma.budgets = sa.budgets; ma.row_off = sa.row_off;
+  ma.evict_idx = sa.evict_idx; ma.evict_mx = (float*)(X + c->slay.evict_mx); ma.evict_nn = (int32_t*)(X + c->slay.evict_nn);
+  ma.rnorm = sa.rnorm; ma.pos = sa.pos; ma.L = L; ma.layer = layer; ma.Hkv = Hkv; ma.P = P;
+  const size_t sim_sm = ((size_t)2 * D * kSimTile + 2 * kSimTile) * sizeof(float);
+  e = cudaFuncSetAttribute(similarity_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sim_sm);
+  if (e != cudaSuccess) return e;
+  dim3 sgrid((maxLe + kSimTile - 1) / kSimTile, n_slices);
+  similarity_kernel<T, D><<<sgrid, kSimThreads, sim_sm, st>>>(ma, (const T*)K, kpool);
+
+  SegArgs ga;
+  ga.budgets = sa.budgets; ga.evict_mx = ma.evict_mx; ga.evict_nn = ma.evict_nn;
+  ga.seg_start = (int32_t*)(X + c->slay.seg_start); ga.seg_items = (int32_t*)(X + c->slay.seg_items);
+  ga.tau = sa.tau; ga.counters = sa.counters;
+  ga.L = L; ga.layer = layer; ga.B = B; ga.Hkv = Hkv; ga.P = P; ga.seg_stride = seg_stride;
+  ga.tau_override = g.tau_override;
+  const size_t seg_sm = (size_t)(maxS + 1) * sizeof(int);
+  e = cudaFuncSetAttribute(segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)(seg_sm > 48 * 1024 ? seg_sm : 48 * 1024));
+  if (e != cudaSuccess) return e;
+  segment_kernel<<<n_slices, 1024, seg_sm, st>>>(ga);
+
+  MergeArgs mg;
+  mg.budgets = sa.budgets; mg.row_off = sa.row_off; mg.evict_idx = sa.evict_idx; mg.evict_mx = ma.evict_mx;
+  mg.seg_start = ga.seg_start; mg.seg_items = ga.seg_items; mg.rnorm = sa.rnorm;
+  mg.L = L; mg.layer = layer; mg.Hkv = Hkv; mg.P = P; mg.seg_stride = seg_stride;
+  constexpr int LPR = D / Elem<T>::kPerVec;
+  const int rows_per_cta = 256 / LPR;
+  dim3 mgrid((maxS + rows_per_cta - 1) / rows_per_cta, n_slices);
+  merge_kernel<T, D><<<mgrid, 256, 0, st>>>(mg, (const T*)K, (const T*)V, kpool, vpool);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_compress(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st) {
+  const int d = c->cfg.d_head;
+  switch (c->cfg.dtype) {
+    case D2O_F32: return d == 64 ? run_prefill<float, 64>(c, layer, K, V, st) : run_prefill<float, 128>(c, layer, K, V, st);
+    case D2O_F16: return d == 64 ? run_prefill<__half, 64>(c, layer, K, V, st) : run_prefill<__half, 128>(c, layer, K, V, st);
+    default: return d == 64 ? run_prefill<__nv_bfloat16, 64>(c, layer, K, V, st)
+                            : run_prefill<__nv_bfloat16, 128>(c, layer, K, V, st);
+  }
+}
+
+}  // namespace d2o

@@ -1,0 +1,374 @@
+// Layer-level operation (Section 4.1): column sums of the causal prompt attention (Eq. 4 / Eq. 6
+// case 1), the density F_v = Var(s) per query head, and the inverse-variance-softmax budgets
+// (Eq. 5, Appendix A.2).
+//
+// Kernels in this file
+//   lse_kernel      row normalisers log sum_j exp(q_i.k_j/sqrt(d)) of the causal attention
+//   colsum_kernel   s_j = sum_{i>=j} exp(q_i.k_j/sqrt(d) - lse_i); one CTA owns a block of
+//                   columns and walks down the rows, so the column reduction needs neither
+//                   atomics nor scratch and is bit-reproducible
+//   density_kernel  warp-shuffle mean / variance of s per query head (double accumulation)
+//   budget_kernel   Eq. 5 with clamping and exact-sum integerisation, one thread per sequence
+// The two attention sweeps here are the generic FFMA implementation (any dtype, fp32 math);
+// 16-bit inputs take the tensor-core path in d2o_colsum_tc.cu when it is built in.
+#include <math.h>
+
+#include "d2o_common.cuh"
+
+namespace d2o {
+
+constexpr int kTile = 64;        // rows and columns per CTA tile
+constexpr int kStatThreads = 256;
+
+// Loads a [64 x D] tile (rows row0.., zero beyond n_rows) transposed into smem as t[k][r], times `mul`.
+template <typename T, int D>
+__device__ __forceinline__ void load_tile_transposed(float* t, const T* base, int row0, int n_rows, float mul) {
+  constexpr int EPV = Elem<T>::kPerVec;
+  constexpr int VPR = D / EPV;                       // vectors per row
+  const int r = threadIdx.x % kTile;
+  for (int vi = threadIdx.x / kTile; vi < VPR; vi += kStatThreads / kTile) {
+    float f[EPV];
+    if (row0 + r < n_rows) {
+      uint4 v = ld_global_v4(base + (size_t)(row0 + r) * D + vi * EPV);
+      Elem<T>::unpack(v, f);
+    } else {
+#pragma unroll
+      for (int i = 0; i < EPV; ++i) f[i] = 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < EPV; ++i) t[(vi * EPV + i) * kTile + r] = f[i] * mul;
+  }
+}
+
+// 4x4 register tile of S = Q K^T for this thread: rows ty*4.., cols tx*4..
+template <int D>
+__device__ __forceinline__ void tile_dot(const float* qt, const float* kt, int ty, int tx, float s[4][4]) {
+#pragma unroll
+  for (int r = 0; r < 4; ++r)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) s[r][c] = 0.f;
+#pragma unroll 8
+  for (int k = 0; k < D; ++k) {
+    const float4 a = *reinterpret_cast<const float4*>(qt + k * kTile + ty * 4);
+    const float4 b = *reinterpret_cast<const float4*>(kt + k * kTile + tx * 4);
+    const float av[4] = {a.x, a.y, a.z, a.w};
+    const float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) s[r][c] = fmaf(av[r], bv[c], s[r][c]);
+  }
+}
+
+// lse2[b,hq,i] = log2 sum_{j<=i} 2^{(q_i.k_j) * scale * log2e}, stored as natural log.
+template <typename T, int D>
+__global__ void __launch_bounds__(kStatThreads)
+lse_kernel(const T* __restrict__ Q, const T* __restrict__ K, float* __restrict__ lse, int P, int Hq, int group) {
+  extern __shared__ __align__(16) float smem[];
+  float* qt = smem;
+  float* kt = smem + D * kTile;
+  const int it = gridDim.x - 1 - blockIdx.x;          // heaviest row tiles first
+  const int bh = blockIdx.y;
+  const int b = bh / Hq, hq = bh % Hq;
+  const int Hkv = Hq / group;
+  const T* q = Q + ((size_t)b * Hq + hq) * (size_t)P * D;
+  const T* k = K + ((size_t)b * Hkv + hq / group) * (size_t)P * D;
+  const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
+  const float mul = (D == 64 ? 0.125f : 0.08838834764831845f) * kLog2e;
+  load_tile_transposed<T, D>(qt, q, it * kTile, P, mul);
+  float m[4], l[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) { m[r] = -INFINITY; l[r] = 0.f; }
+  for (int jt = 0; jt <= it; ++jt) {
+    __syncthreads();
+    load_tile_transposed<T, D>(kt, k, jt * kTile, P, 1.0f);
+    __syncthreads();
+    float s[4][4];
+    tile_dot<D>(qt, kt, ty, tx, s);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int row = it * kTile + ty * 4 + r;
+      float mx = m[r];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int col = jt * kTile + tx * 4 + c;
+        if (col > row) s[r][c] = -INFINITY;
+        mx = fmaxf(mx, s[r][c]);
+      }
+      if (mx > -INFINITY) {
+        float add = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) add += exp2f(s[r][c] - mx);
+        l[r] = l[r] * exp2f(m[r] - mx) + add;
+        m[r] = mx;
+      }
+    }
+  }
+  // combine the 16 threads (tx) that share a row: contiguous lanes
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) {
+      const float mo = __shfl_xor_sync(0xffffffffu, m[r], o);
+      const float lo = __shfl_xor_sync(0xffffffffu, l[r], o);
+      const float mn = fmaxf(m[r], mo);
+      const float a = (m[r] > -INFINITY) ? l[r] * exp2f(m[r] - mn) : 0.f;
+      const float bb = (mo > -INFINITY) ? lo * exp2f(mo - mn) : 0.f;
+      l[r] = a + bb;
+      m[r] = mn;
+    }
+    const int row = it * kTile + ty * 4 + r;
+    if (tx == 0 && row < P) lse[((size_t)b * Hq + hq) * P + row] = (m[r] + log2f(l[r])) * 0.6931471805599453f;
+  }
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kStatThreads)
+colsum_kernel(const T* __restrict__ Q, const T* __restrict__ K, const float* __restrict__ lse,
+              float* __restrict__ colsum, int P, int Hq, int group) {
+  extern __shared__ __align__(16) float smem[];
+  float* qt = smem;
+  float* kt = smem + D * kTile;
+  float* lse2 = kt + D * kTile;                        // [64]
+  double* red = reinterpret_cast<double*>(lse2 + kTile);  // [16][64]
+  const int jt = blockIdx.x;                          // column tile 0 has the most rows: first
+  const int nT = gridDim.x;
+  const int bh = blockIdx.y;
+  const int b = bh / Hq, hq = bh % Hq;
+  const int Hkv = Hq / group;
+  const T* q = Q + ((size_t)b * Hq + hq) * (size_t)P * D;
+  const T* k = K + ((size_t)b * Hkv + hq / group) * (size_t)P * D;
+  const float* ls = lse + ((size_t)b * Hq + hq) * P;
+  const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
+  const float mul = (D == 64 ? 0.125f : 0.08838834764831845f) * kLog2e;
+  load_tile_transposed<T, D>(kt, k, jt * kTile, P, 1.0f);
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  for (int it = jt; it < nT; ++it) {
+    __syncthreads();
+    load_tile_transposed<T, D>(qt, q, it * kTile, P, mul);
+    if (threadIdx.x < kTile) {
+      const int row = it * kTile + threadIdx.x;
+      lse2[threadIdx.x] = row < P ? ls[row] * kLog2e : INFINITY;    // +inf -> probability 0 for padding rows
+    }
+    __syncthreads();
+    float s[4][4];
+    tile_dot<D>(qt, kt, ty, tx, s);
+    float p[4][4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int row = it * kTile + ty * 4 + r;
+      const float lr = lse2[ty * 4 + r];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int col = jt * kTile + tx * 4 + c;
+        p[r][c] = (col <= row) ? exp2f(s[r][c] - lr) : 0.f;
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) acc[c] += (double)((p[0][c] + p[1][c]) + (p[2][c] + p[3][c]));
+  }
+  __syncthreads();
+#pragma unroll
+  for (int c = 0; c < 4; ++c) red[ty * kTile + tx * 4 + c] = acc[c];
+  __syncthreads();
+  if (threadIdx.x < kTile) {
+    double t = 0.0;
+#pragma unroll
+    for (int y = 0; y < 16; ++y) t += red[y * kTile + threadIdx.x];
+    const int col = jt * kTile + threadIdx.x;
+    if (col < P) colsum[((size_t)b * Hq + hq) * P + col] = (float)t;
+  }
+}
+
+// F[b, layer, hq] = (1/P) sum_j (s_j - mean)^2, mean = (1/P) sum_j s_j   (Eq. 4; population variance)
+__global__ void __launch_bounds__(256)
+density_kernel(const float* __restrict__ colsum, double* __restrict__ density, int P, int Hq, int L, int layer) {
+  __shared__ double part[8];
+  __shared__ double mean_s;
+  const int bh = blockIdx.x;
+  const int b = bh / Hq, hq = bh % Hq;
+  const float* s = colsum + (size_t)bh * P;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  double t = 0.0;
+  for (int j = threadIdx.x; j < P; j += blockDim.x) t += (double)s[j];
+  t = warp_sum(t);
+  if (lane == 0) part[warp] = t;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double a = 0.0;
+    for (int w = 0; w < 8; ++w) a += part[w];
+    mean_s = a / (double)P;
+  }
+  __syncthreads();
+  const double mean = mean_s;
+  t = 0.0;
+  for (int j = threadIdx.x; j < P; j += blockDim.x) { const double dlt = (double)s[j] - mean; t += dlt * dlt; }
+  t = warp_sum(t);
+  __syncthreads();
+  if (lane == 0) part[warp] = t;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double a = 0.0;
+    for (int w = 0; w < 8; ++w) a += part[w];
+    density[((size_t)b * L + layer) * Hq + hq] = a / (double)P;
+  }
+}
+
+// Eq. 5 with S_l = clip(lambda * w_l, S_min, S_max), sum_l S_l = S_tot, then floor + largest remainder.
+// One thread per sequence; per-thread work arrays (w, kinks, x) live in dynamic shared memory.
+__device__ inline double clipd(double v, double lo, double hi) { return v < lo ? lo : (v > hi ? hi : v); }
+
+__global__ void budget_kernel(const double* __restrict__ density, int B, int L, int H, int Hkv, int P, double rho,
+                              int min_budget, int max_budget, double gamma, int head_reduce, int n_sink, int window,
+                              double nm_ratio, int32_t* __restrict__ budgets, int32_t* __restrict__ windows,
+                              int64_t* __restrict__ row_off, uint32_t* status_word) {
+  extern __shared__ __align__(16) double dsm[];
+  double* w = dsm + (size_t)threadIdx.x * 4 * L;
+  double* kinks = w + L;        // [2L]
+  double* x = kinks + 2 * L;    // [L]
+  const double lo = (double)min_budget, hi = (double)max_budget;
+  const long long S_tot = (long long)floor(rho * (double)L * (double)P + 0.5);
+  for (int b = threadIdx.x; b < B; b += blockDim.x) {
+    const double* F = density + (size_t)b * L * H;
+    if (head_reduce == 0) {
+      double fmin = F[0];
+      for (int i = 1; i < L * H; ++i) fmin = fmin < F[i] ? fmin : F[i];
+      for (int l = 0; l < L; ++l) {
+        double a = 0.0;
+        for (int h = 0; h < H; ++h) a = __dadd_rn(a, exp(-__ddiv_rn(__dadd_rn(F[l * H + h], -fmin), gamma)));
+        w[l] = a;
+      }
+    } else {
+      double fmin = INFINITY;
+      for (int l = 0; l < L; ++l) {
+        double a = 0.0;
+        for (int h = 0; h < H; ++h) a = __dadd_rn(a, F[l * H + h]);
+        x[l] = __ddiv_rn(a, (double)H);
+        fmin = fmin < x[l] ? fmin : x[l];
+      }
+      for (int l = 0; l < L; ++l) w[l] = exp(-__ddiv_rn(__dadd_rn(x[l], -fmin), gamma));
+    }
+    for (int l = 0; l < L; ++l) w[l] = w[l] > 1e-300 ? w[l] : 1e-300;
+    // kinks of the piecewise-linear total(lambda), ascending (insertion sort)
+    int nk = 0;
+    for (int l = 0; l < L; ++l) {
+      const double cand[2] = {__ddiv_rn(lo, w[l]), __ddiv_rn(hi, w[l])};
+      for (int c = 0; c < 2; ++c) {
+        int i = nk++;
+        while (i > 0 && kinks[i - 1] > cand[c]) { kinks[i] = kinks[i - 1]; --i; }
+        kinks[i] = cand[c];
+      }
+    }
+    auto total = [&](double lam) {
+      double t = 0.0;
+      for (int l = 0; l < L; ++l) t = __dadd_rn(t, clipd(__dmul_rn(lam, w[l]), lo, hi));
+      return t;
+    };
+    int k = 0;
+    while (k < nk && total(kinks[k]) < (double)S_tot) ++k;
+    double lam;
+    if (k == 0) lam = kinks[0];
+    else if (k == nk) lam = kinks[nk - 1];
+    else {
+      const double a = kinks[k - 1], bb = kinks[k];
+      const double mid = __dmul_rn(0.5, __dadd_rn(a, bb));
+      double fixed = 0.0, wf = 0.0;
+      for (int l = 0; l < L; ++l) {
+        const double v = __dmul_rn(mid, w[l]);
+        if (v > lo && v < hi) wf = __dadd_rn(wf, w[l]);
+        else fixed = __dadd_rn(fixed, clipd(v, lo, hi));
+      }
+      lam = wf > 0.0 ? __ddiv_rn(__dadd_rn((double)S_tot, -fixed), wf) : bb;
+      lam = lam < a ? a : (lam > bb ? bb : lam);
+    }
+    long long sum = 0;
+    for (int l = 0; l < L; ++l) {
+      x[l] = clipd(__dmul_rn(lam, w[l]), lo, hi);
+      const double fl = floor(x[l]);
+      budgets[b * L + l] = (int32_t)fl;
+      x[l] = x[l] - fl;                                   // remainder
+      sum += (long long)fl;
+    }
+    long long left = S_tot - sum;
+    if (left < 0 || left > L) { report_error(status_word, D2O_ERR_STATE, 0xB0000000u | (uint32_t)b); left = 0; }
+    while (left > 0) {                                     // largest remainder first, ties -> lower layer
+      int best = -1;
+      for (int l = 0; l < L; ++l)
+        if (x[l] >= 0.0 && budgets[b * L + l] < max_budget && (best < 0 || x[l] > x[best])) best = l;
+      if (best < 0) { report_error(status_word, D2O_ERR_STATE, 0xB1000000u | (uint32_t)b); break; }
+      budgets[b * L + best] += 1;
+      x[best] = -1.0;                                      // taken
+      --left;
+    }
+    if (windows) {
+      for (int l = 0; l < L; ++l) {
+        const int S = budgets[b * L + l];
+        const int T = n_sink < S ? n_sink : S;
+        int M = window > 0 ? window : (int)floor((double)(S - T) / (1.0 + nm_ratio) + 0.5);
+        M = M < 0 ? 0 : (M > S - T ? S - T : M);
+        windows[b * L + l] = M;
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && row_off) {                       // cache rows laid out layer-major, then sequence
+    long long o = 0;
+    for (int l = 0; l < L; ++l)
+      for (int b = 0; b < B; ++b) { row_off[b * L + l] = o; o += (long long)Hkv * budgets[b * L + l]; }
+  }
+}
+
+template <typename T, int D>
+static cudaError_t run_stats(const d2o_ctx* c, int layer, const void* Q, const void* K, const float* lse_in,
+                             cudaStream_t st) {
+  const d2o_config& g = c->cfg;
+  const int P = g.prompt_len, Hq = g.n_q_heads, B = g.batch;
+  const int nT = (P + kTile - 1) / kTile;
+  float* colsum = (float*)(c->state + c->lay.colsum) + (size_t)layer * B * Hq * P;
+  double* density = (double*)(c->state + c->lay.density);
+  const float* lse = lse_in;
+  dim3 grid(nT, B * Hq);
+  if (!lse) {
+    float* lse_buf = (float*)(c->scratch + c->slay.lse);
+    const size_t sm = (size_t)2 * D * kTile * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(lse_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    if (e != cudaSuccess) return e;
+    lse_kernel<T, D><<<grid, kStatThreads, sm, st>>>((const T*)Q, (const T*)K, lse_buf, P, Hq, c->group);
+    lse = lse_buf;
+  }
+  const size_t sm2 = (size_t)2 * D * kTile * sizeof(float) + kTile * sizeof(float) + 16 * kTile * sizeof(double);
+  cudaError_t e = cudaFuncSetAttribute(colsum_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
+  if (e != cudaSuccess) return e;
+  colsum_kernel<T, D><<<grid, kStatThreads, sm2, st>>>((const T*)Q, (const T*)K, lse, colsum, P, Hq, c->group);
+  density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, g.n_layers, layer);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_layer_stats(const d2o_ctx* c, int layer, const void* Q, const void* K, const float* lse,
+                               cudaStream_t st) {
+  const int d = c->cfg.d_head;
+  switch (c->cfg.dtype) {
+    case D2O_F32: return d == 64 ? run_stats<float, 64>(c, layer, Q, K, lse, st) : run_stats<float, 128>(c, layer, Q, K, lse, st);
+    case D2O_F16: return d == 64 ? run_stats<__half, 64>(c, layer, Q, K, lse, st) : run_stats<__half, 128>(c, layer, Q, K, lse, st);
+    default: return d == 64 ? run_stats<__nv_bfloat16, 64>(c, layer, Q, K, lse, st)
+                            : run_stats<__nv_bfloat16, 128>(c, layer, Q, K, lse, st);
+  }
+}
+
+cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, int P, float rho, int min_budget,
+                           int max_budget, float gamma, int head_reduce, int n_sink, int window, float nm_ratio,
+                           int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
+                           cudaStream_t st) {
+  const size_t per_thread = (size_t)4 * L * sizeof(double);
+  int threads = B < 32 ? B : 32;
+  while (threads > 1 && per_thread * threads > 160 * 1024) threads /= 2;
+  const size_t sm = per_thread * threads;
+  cudaError_t e = cudaFuncSetAttribute(budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+  if (e != cudaSuccess) return e;
+  budget_kernel<<<1, threads, sm, st>>>(density, B, L, H, Hkv, P, (double)rho, min_budget, max_budget, (double)gamma,
+                                        head_reduce, n_sink, window, (double)nm_ratio, budgets, windows, row_off,
+                                        status_word);
+  return cudaGetLastError();
+}
+
+}  // namespace d2o

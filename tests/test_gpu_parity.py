@@ -1,0 +1,201 @@
+"""GPU parity: the CUDA path through the C ABI against the float64 oracle, same seeded inputs."""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import d2o_oracle as O
+from paper_2406_13035_b200 import binding as B
+from paper_2406_13035_b200 import workloads as W
+
+from parity import assert_report, close, np64, run_parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib(cuda_device):
+    from paper_2406_13035_b200 import build
+    build.build_library()
+    B.load_library()
+
+
+def small(name="cfg0", **kw):
+    return dataclasses.replace(W.CONFIGS[name], **kw)
+
+
+def test_cfg0_whole_pipeline():
+    wl = W.CONFIGS["cfg0"]
+    rep = run_parity(wl)
+    assert rep.checked_slices == 8 and rep.steps == 16
+    assert rep.merges + rep.discards == 8 * 16
+    assert_report(rep, wl.dtype)
+    print("cfg0", rep.max_err, rep.ties, rep.merges, rep.discards)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4"])
+def test_scaled_twins(name):
+    wl = W.twin(name)
+    rep = run_parity(wl)
+    assert_report(rep, wl.dtype)
+    assert rep.merges > 0 and rep.discards > 0
+    print(name, rep.max_err, rep.ties, rep.merges, rep.discards)
+
+
+@pytest.mark.parametrize("cluster", [1, 2, 8])
+def test_cluster_sizes_agree(cluster):
+    wl = small(prompt_len=512, decode_steps=8)
+    rep = run_parity(wl, decode_cluster=cluster)
+    assert_report(rep, wl.dtype)
+
+
+def test_layer_by_layer_calls_match():
+    wl = W.twin("cfg1")
+    rep = run_parity(wl, layers_per_call=1, steps=6)
+    assert_report(rep, wl.dtype)
+
+
+@pytest.mark.parametrize("tau", [float("inf"), float("-inf")])
+def test_threshold_overrides(tau):
+    wl = small(prompt_len=384, decode_steps=6)
+    rep = run_parity(wl, ctx_over=dict(tau_override=tau))
+    assert_report(rep, wl.dtype)
+    if tau > 0:
+        assert rep.merges == 0            # pure eviction
+    else:
+        assert rep.discards == 0          # every victim merged
+
+
+@pytest.mark.parametrize("T,window,d,dtype,hq,hkv", [(0, 8, 64, "f16", 4, 4), (4, 0, 128, "f32", 4, 2),
+                                                     (2, 16, 64, "bf16", 8, 1), (1, 0, 128, "bf16", 8, 4)])
+def test_shape_and_hyperparameter_sweep(T, window, d, dtype, hq, hkv):
+    wl = dataclasses.replace(W.CONFIGS["cfg0"], name="sweep", n_q_heads=hq, n_kv_heads=hkv, d_head=d, dtype=dtype,
+                             prompt_len=333, decode_steps=9, n_sink=T, window=window, rho=0.3, n_layers=2,
+                             batch=2, density_temp=50.0, min_budget=max(8, T + 1))
+    rep = run_parity(wl)
+    assert_report(rep, wl.dtype)
+
+
+def test_budget_never_reached_equals_full_attention():
+    """With S_l >= prompt + steps nothing is evicted and the output is plain softmax attention."""
+    wl = small(prompt_len=200, decode_steps=7, rho=1.035)
+    rep = run_parity(wl, ctx_over=dict(max_budget=207))
+    assert rep.merges == 0 and rep.discards == 0
+    assert_report(rep, wl.dtype)
+
+
+def test_budgets_pure_function_matches_oracle(cuda_device):
+    r = np.random.default_rng(5)
+    for trial in range(40):
+        Bn, L, H = int(r.integers(1, 4)), int(r.integers(1, 40)), int(r.integers(1, 9))
+        P = int(r.integers(64, 9000))
+        rho = B.f32(float(r.uniform(0.05, 1.0)))
+        gamma = B.f32(float(r.choice([1.0, 10.0, 1000.0])))
+        smin = int(r.integers(1, 12))
+        F = r.gamma(1.0, size=(Bn, L, H)) * float(r.choice([0.01, 1.0, 30.0, 3000.0]))
+        if L * smin > math.floor(rho * L * P + 0.5):
+            continue
+        hr = int(trial % 2)
+        nm = B.f32(3.0)
+        bud, win, off, status = B.d2o_budgets_from_density(torch.tensor(F, device=cuda_device), n_kv_heads=2,
+                                                           prompt_len=P, rho=rho, min_budget=smin,
+                                                           density_temp=gamma, head_reduce=hr, n_sink=1, window=0,
+                                                           nm_ratio=nm)
+        bud = bud.cpu().numpy()
+        assert int(status[0]) == 0
+        for b in range(Bn):
+            ref = O.layer_budgets(F[b], P, rho, smin, gamma, hr)
+            np.testing.assert_array_equal(bud[b], ref)
+            for l in range(L):
+                assert int(win[b, l]) == O.window_size(int(ref[l]), min(1, int(ref[l])), 0, nm)
+        o = off.cpu().numpy()
+        flat = [(l, b) for l in range(L) for b in range(Bn)]
+        run = 0
+        for l, b in flat:
+            assert o[b, l] == run
+            run += 2 * bud[b, l]
+
+
+@pytest.mark.parametrize("dtype,d,G,n_slices,cap,length", [("f16", 128, 1, 6, 700, 513), ("bf16", 128, 4, 3, 4100, 4099),
+                                                           ("f32", 64, 2, 5, 64, 0), ("f16", 64, 8, 2, 300, 77)])
+def test_full_decode_kernel(cuda_device, dtype, d, G, n_slices, cap, length):
+    td = W.TORCH_DTYPES[dtype]
+    g = torch.Generator(device=cuda_device).manual_seed(11)
+    kc = torch.randn(n_slices, cap, d, generator=g, device=cuda_device).to(td)
+    vc = torch.randn(n_slices, cap, d, generator=g, device=cuda_device).to(td)
+    q = (2 * torch.randn(n_slices, G, d, generator=g, device=cuda_device)).to(td)
+    k = torch.randn(n_slices, d, generator=g, device=cuda_device).to(td)
+    v = torch.randn(n_slices, d, generator=g, device=cuda_device).to(td)
+    out = torch.empty_like(q)
+    kc0, vc0 = kc.clone(), vc.clone()
+    B.d2o_full_decode_step(kc, vc, length, q, k, v, out)
+    torch.cuda.synchronize()
+    assert torch.equal(kc[:, length], k) and torch.equal(vc[:, length], v)          # appended
+    assert torch.equal(kc[:, :length], kc0[:, :length]) and torch.equal(kc[:, length + 1:], kc0[:, length + 1:])
+    for s in range(n_slices):
+        Kf = np.vstack([np64(kc0[s, :length]), np64(k[s])[None]])
+        Vf = np.vstack([np64(vc0[s, :length]), np64(v[s])[None]])
+        ref = O.full_attention_step(np64(q[s]), Kf, Vf)
+        assert close(np64(out[s]), ref, dtype) <= 1.0
+
+
+def test_out_of_order_calls_are_rejected(cuda_device):
+    from parity import make_ctx
+    wl = small(prompt_len=128, decode_steps=2)
+    ctx = make_ctx(wl)
+    s = W.LayerStream(wl, 0, "cuda:0")
+    Q, K, V = s.prompt()
+    with pytest.raises(B.D2OError) as e:
+        ctx.d2o_layer_budgets()
+    assert e.value.status == 4
+    with pytest.raises(B.D2OError) as e:
+        ctx.d2o_prefill_compress(0, K, V)
+    assert e.value.status == 4
+    ctx.d2o_layer_stats(0, Q, K)
+    ctx.d2o_layer_budgets()
+    q, k, v = s.decode()
+    out = torch.empty_like(q)
+    with pytest.raises(B.D2OError) as e:
+        ctx.d2o_decode_step(0, 1, q, k, v, out)
+    assert e.value.status == 4
+    ctx.d2o_prefill_compress(0, K, V)
+    ctx.d2o_decode_step(0, 1, q, k, v, out)
+    ctx.d2o_decode_step(0, 1, q, k, v, out)
+    with pytest.raises(B.D2OError) as e:                      # max_new_tokens = 2
+        ctx.d2o_decode_step(0, 1, q, k, v, out)
+    assert e.value.status == 4
+    assert ctx.d2o_get_stats().error_word == 0
+
+
+def test_host_buffer_entry_matches_device_entry(cuda_device):
+    from parity import make_ctx
+    wl = W.twin("cfg2")
+    outs = []
+    for host in (False, True):
+        ctx = make_ctx(wl)
+        streams = [W.LayerStream(wl, l, "cuda:0") for l in range(wl.n_layers)]
+        kv = []
+        for l, s in enumerate(streams):
+            Q, K, V = s.prompt()
+            ctx.d2o_layer_stats(l, Q, K)
+            kv.append((K, V))
+        ctx.d2o_layer_budgets()
+        for l, (K, V) in enumerate(kv):
+            ctx.d2o_prefill_compress(l, K, V)
+        res = []
+        for step in range(4):
+            q, k, v = (torch.stack(x) for x in zip(*[s.decode() for s in streams]))
+            if host:
+                qh, kh, vh = q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory()
+                oh = torch.empty_like(qh).pin_memory()
+                ctx.d2o_decode_step_host(0, wl.n_layers, qh, kh, vh, oh)
+                res.append(oh.clone())
+            else:
+                o = torch.empty_like(q)
+                ctx.d2o_decode_step(0, wl.n_layers, q, k, v, o)
+                res.append(o.cpu())
+        outs.append(torch.stack(res))
+        ctx.close()
+    assert torch.equal(outs[0], outs[1])
