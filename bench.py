@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the D2O hot path on B200.
+
+One bench *step* is one pass of the whole path over one synthetic batch:
+  per layer: column sums + density (d2o_layer_stats) -> budgets (d2o_layer_budgets)
+  -> per layer: eviction + similarity + merge (d2o_prefill_compress)
+  -> the decode loop (d2o_decode_step, all layers per call, `decode_steps` tokens).
+The headline value is compressed decode steps/s (tokens/s = steps/s x sequences); the
+prompt-stage times are reported beside it.  Inputs are generated once, seeded, and are
+resident in HBM before the timed region; the `e2e` leg repeats the decode loop through the
+host-buffer entry point with pinned host q/k/v/out every step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg1] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2406_13035_b200 import workloads as W  # noqa: E402
+
+METRIC = "compressed decode steps/s (x sequences = tokens/s); prefill-compress ms; fraction of HBM roofline"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="cfg1")
+    ap.add_argument("--decode-steps", type=int, default=0, help="override the config's decode steps")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cluster", type=int, default=0, help="CTAs per cluster of the decode kernel (0 = auto)")
+    ap.add_argument("--nonresident", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers-per-call", type=int, default=0)
+    return ap.parse_args()
+
+
+# --------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------- workload
+def prepare_inputs(wl: W.Workload, device, decode_steps: int):
+    """All prompt tensors and all decode-step tensors, resident on the device."""
+    prompts, dq, dk, dv = [], [], [], []
+    streams = [W.LayerStream(wl, l, device) for l in range(wl.n_layers)]
+    for s in streams:
+        prompts.append(s.prompt())
+    for _ in range(decode_steps):
+        qs, ks, vs = zip(*[s.decode() for s in streams])
+        dq.append(torch.stack(qs)); dk.append(torch.stack(ks)); dv.append(torch.stack(vs))
+    return prompts, torch.stack(dq), torch.stack(dk), torch.stack(dv)
+
+
+def algorithmic_decode_bytes(wl: W.Workload, budgets, step_lens):
+    """Bytes one decode launch must move: K_c and V_c rows once, per-row score/pos/norm read (12 B) and
+    score write (4 B), q/k/v in and out once."""
+    e = 4 if wl.dtype == "f32" else 2
+    rows = float(step_lens) * wl.n_kv_heads
+    per_row = 2 * wl.d_head * e + 16
+    io = wl.n_layers * wl.batch * (2 * wl.n_q_heads + 2 * wl.n_kv_heads) * wl.d_head * e
+    return rows * per_row + io
+
+
+def run_ours(args, wl, rank, world, device):
+    from paper_2406_13035_b200 import binding as B
+    from paper_2406_13035_b200 import build
+    if rank == 0:
+        build.build_library()
+    if world > 1:
+        torch.distributed.barrier()
+    B.load_library()
+    nd = args.decode_steps or wl.decode_steps
+    cfg = B.make_config(n_layers=wl.n_layers, batch=wl.batch, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
+                        d_head=wl.d_head, dtype=wl.dtype, prompt_len=wl.prompt_len, max_new_tokens=nd, rho=wl.rho,
+                        n_sink=wl.n_sink, window=wl.window, nm_ratio=wl.nm_ratio, beta=wl.beta,
+                        density_temp=wl.density_temp, min_budget=wl.min_budget)
+    ctx = B.D2OContext(cfg, device)
+    if args.cluster or args.nonresident:
+        ctx.d2o_set_tuning(args.cluster, args.nonresident)
+    # every rank works on its own sequences: same shapes, rank-dependent seed (weak scaling, no exchange)
+    import dataclasses
+    wl_r = dataclasses.replace(wl, seed=wl.seed + 7919 * rank)
+    prompts, dq, dk, dv = prepare_inputs(wl_r, device, nd)
+    dout = torch.empty_like(dq[0])
+    L = wl.n_layers
+    lpc = args.layers_per_call or L
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+    launches = {"n": 0}
+
+    def one_pass(timed: bool):
+        e = [ev() for _ in range(5)]
+        e[0].record()
+        for l in range(L):
+            ctx.d2o_layer_stats(l, prompts[l][0], prompts[l][1])
+        e[1].record()
+        budgets = ctx.d2o_layer_budgets()
+        e[2].record()
+        for l in range(L):
+            ctx.d2o_prefill_compress(l, prompts[l][1], prompts[l][2])
+        e[3].record()
+        for s in range(nd):
+            for l0 in range(0, L, lpc):
+                l1 = min(L, l0 + lpc)
+                ctx.d2o_decode_step(l0, l1, dq[s, l0:l1], dk[s, l0:l1], dv[s, l0:l1], dout[l0:l1])
+        e[4].record()
+        if timed:
+            launches["n"] += L * 3 + 1 + L * 4 + nd * ((L + lpc - 1) // lpc)
+        return e, budgets
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+
+    for _ in range(args.warmup):
+        one_pass(False)
+    sync_all()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    t_wall = time.perf_counter()
+    passes = []
+    sync_all()
+    for _ in range(args.steps):
+        passes.append(one_pass(True))
+    sync_all()
+    t_wall = time.perf_counter() - t_wall
+    clocks = sampler.stop()
+    seg = [[p[0][i].elapsed_time(p[0][i + 1]) for i in range(4)] for p in passes]          # ms
+    stats_ms = statistics.mean(s[0] for s in seg)
+    budget_ms = statistics.mean(s[1] for s in seg)
+    compress_ms = statistics.mean(s[2] for s in seg)
+    decode_ms = statistics.mean(s[3] for s in seg)
+    pass_ms = stats_ms + budget_ms + compress_ms + decode_ms
+    budgets = passes[-1][1]
+    # max over ranks
+    if world > 1:
+        t = torch.tensor([stats_ms, budget_ms, compress_ms, decode_ms, pass_ms], device=device, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        stats_ms, budget_ms, compress_ms, decode_ms, pass_ms = t.tolist()
+    steps_per_s = nd / (decode_ms * 1e-3)
+    # roofline of the dominant kernel (decode): algorithmic bytes per launch / average launch duration
+    P = wl.prompt_len
+    tot_rows = 0.0
+    for s in range(nd):
+        tot_rows += float(torch.clamp(budgets.double(), max=P + s).sum())          # rows held before step s
+    mean_rows = tot_rows / nd
+    bytes_per_launch = algorithmic_decode_bytes(wl, budgets, mean_rows) / ((L + lpc - 1) // lpc)
+    launch_ms = decode_ms / (nd * ((L + lpc - 1) // lpc))
+    peaks = {}
+    pk_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk_path):
+        peaks = json.load(open(pk_path))
+    peak = float(peaks.get("hbm_gbs", 6650.0))
+    achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": round(achieved, 1), "peak": peak,
+                "unit": "GB/s", "frac": round(achieved / peak, 4),
+                "peak_source": "measured" if "hbm_gbs" in peaks else "fallback",
+                "algorithmic_bytes_per_launch": int(bytes_per_launch), "avg_launch_us": round(launch_ms * 1e3, 2),
+                "traffic": None}
+    # end to end: the decode loop through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        for l in range(L):
+            ctx.d2o_prefill_compress(l, prompts[l][1], prompts[l][2])
+        n_e2e = min(nd, 64)
+        hq = dq[:n_e2e].cpu().pin_memory(); hk = dk[:n_e2e].cpu().pin_memory(); hv = dv[:n_e2e].cpu().pin_memory()
+        ho = torch.empty_like(hq[0]).pin_memory()
+        sync_all()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for s in range(n_e2e):
+            ctx.d2o_decode_step_host(0, L, hq[s], hk[s], hv[s], ho)
+        e1.record()
+        sync_all()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=device, dtype=torch.float64)
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            ms = float(t.item())
+        e2e = {"value": round(world * wl.batch * n_e2e / (ms * 1e-3), 2), "unit": "token-steps/s",
+               "h2d_bytes_per_step": int(hq[0].numel() * hq.element_size() + 2 * hk[0].numel() * hk.element_size()),
+               "d2h_bytes_per_step": int(ho.numel() * ho.element_size()), "steps": n_e2e}
+    st = ctx.d2o_get_stats()
+    if st.error_word != 0:
+        raise RuntimeError(f"device error word {st.error_word} ({st.error_detail:#x})")
+    res = {
+        "metric": METRIC, "value": round(world * wl.batch * steps_per_s, 2), "unit": "token-steps/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(pass_ms, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": f"{wl.name}: L={wl.n_layers} Hq={wl.n_q_heads} Hkv={wl.n_kv_heads} d={wl.d_head} "
+                               f"B={wl.batch} P={wl.prompt_len} rho={wl.rho} decode_steps={nd}",
+                   "l2": "decode working set (K_c+V_c of all layers) exceeds the 126 MB L2; prompt tensors exceed it too",
+                   "layers_per_decode_call": lpc, "decode_cluster": args.cluster or "auto",
+                   "sequences_per_gpu": wl.batch, "parallelism": "replicas (independent sequences per GPU)"},
+        "decode_steps_per_s_per_gpu": round(steps_per_s, 2), "decode_us_per_step": round(decode_ms * 1e3 / nd, 2),
+        "stats_ms": round(stats_ms, 3), "budgets_ms": round(budget_ms, 3), "prefill_compress_ms": round(compress_ms, 3),
+        "decode_ms": round(decode_ms, 3), "wall_s": round(t_wall, 3),
+        "budgets_min_max": [int(budgets.min()), int(budgets.max())],
+        "merges_discards": [int(st.merges), int(st.discards)],
+        "roofline": roofline, "e2e": e2e, "gpu_launches": launches["n"], "clocks": clocks,
+    }
+    ctx.close()
+    return res
+
+
+# --------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(wl: W.Workload, n_slices: int, n_steps: int, threads: int = 1):
+    """Times the oracle on `n_slices` slices of layer 0 of the workload: column sums of their query heads,
+    compression, `n_steps` decode steps.  Returns (seconds for the prompt stage, seconds per decode step of one
+    slice)."""
+    import numpy as np
+    from oracle import d2o_oracle as O
+    from threadpoolctl import threadpool_limits
+    s = W.LayerStream(wl, 0, "cpu")
+    Q, K, V = s.prompt()
+    G = wl.group
+    picks = [(0, h) for h in range(min(n_slices, wl.n_kv_heads))]
+    dec = [s.decode() for _ in range(n_steps)]
+    with threadpool_limits(limits=threads):
+        orc = O.OracleStack(n_layers=1, batch=wl.batch, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
+                            d_head=wl.d_head, dtype=wl.dtype, prompt_len=wl.prompt_len, rho=wl.rho, n_sink=wl.n_sink,
+                            window=wl.window, nm_ratio=wl.nm_ratio, beta=wl.beta, min_budget=wl.min_budget)
+        t0 = time.perf_counter()
+        heads = [(b, h * G + g) for b, h in picks for g in range(G)]
+        Q64 = {(b, hq): Q[b, hq].double().numpy() for b, hq in heads}
+        K64 = {(b, h): K[b, h].double().numpy() for b, h in picks}
+        V64 = {(b, h): V[b, h].double().numpy() for b, h in picks}
+
+        class Idx:
+            def __init__(self, d): self.d = d
+            def __getitem__(self, i): return self.d[i]
+        orc.layer_stats(0, Idx(Q64), Idx({(b, hq): K64[(b, hq // G)] for b, hq in heads}) if False else _KQ(K64, G),
+                        heads)
+        orc.budgets = np.full((wl.batch, 1), int(round(wl.rho * wl.prompt_len)), dtype=np.int64)
+        orc.prefill_compress(0, Idx(K64), Idx(V64), picks)
+        t1 = time.perf_counter()
+        for i, (q, k, v) in enumerate(dec):
+            orc.decode_step(0, q.double().numpy(), k.double().numpy(), v.double().numpy(), wl.prompt_len + i, picks)
+        t2 = time.perf_counter()
+    return (t1 - t0) / len(picks), (t2 - t1) / (len(picks) * max(1, n_steps)), len(picks)
+
+
+class _KQ:
+    """K indexed by (b, kv head) for OracleStack.layer_stats."""
+
+    def __init__(self, d, G):
+        self.d, self.G = d, G
+
+    def __getitem__(self, i):
+        return self.d[i]
+
+
+def cpu_baseline(wl: W.Workload, n_slices=2, n_steps=32):
+    prompt_s, step_s, n = oracle_sample(wl, n_slices, n_steps)
+    total_slices = wl.n_layers * wl.batch * wl.n_kv_heads
+    return {"value": round(wl.batch / (step_s * total_slices), 4), "unit": "token-steps/s", "cores": 1,
+            "kind": "oracle",
+            "sample": f"{n} slices of layer 0 (column sums, compression, {n_steps} decode steps), one thread; "
+                      f"{step_s * 1e3:.3f} ms per slice-step and {prompt_s:.2f} s prompt stage per slice, "
+                      f"extrapolated linearly to all {total_slices} slices"}
+
+
+def run_reference(args, wl):
+    vals = []
+    nd = 16
+    for _ in range(args.warmup):
+        oracle_sample(wl, 1, 2)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        vals.append(oracle_sample(wl, 1, nd))
+    wall = time.perf_counter() - t0
+    step_s = statistics.mean(v[1] for v in vals)
+    prompt_s = statistics.mean(v[0] for v in vals)
+    total_slices = wl.n_layers * wl.batch * wl.n_kv_heads
+    value = round(wl.batch / (step_s * total_slices), 4)
+    sample = (f"per bench step: 1 slice of layer 0 (column sums, compression, {nd} decode steps), one thread; "
+              f"extrapolated linearly to all {total_slices} slices")
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": "token-steps/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(wall / max(1, args.steps) * 1e3, 2),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{wl.name} (bounded sample)"},
+            "prompt_stage_s_per_slice": round(prompt_s, 3),
+            "cpu_baseline": {"value": value, "unit": "token-steps/s", "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "token-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def main():
+    args = parse()
+    wl = W.CONFIGS[args.config] if args.config in W.CONFIGS else W.twin(args.config.replace("_twin", ""))
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args, wl)), flush=True)
+        return
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=torch.device(device))
+    res = run_ours(args, wl, rank, world, device)
+    if rank == 0:
+        if not args.no_cpu_baseline and world == 1:
+            res["cpu_baseline"] = cpu_baseline(wl)
+        print(json.dumps(res), flush=True)
+    if world > 1:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -174,7 +174,8 @@ d2o_status d2o_get_view(d2o_ctx* ctx, int32_t layer, d2o_view* out);
 /* Copies the counters to HOST memory; synchronises `stream`. */
 d2o_status d2o_get_stats(d2o_ctx* ctx, d2o_stats* out_host, void* stream);
 
-/* Launch-shape knobs for measurements (0 = automatic): CTAs per cluster of the decode kernel. */
+/* Launch-shape knobs for measurements (0 = automatic): CTAs per cluster of the decode kernel;
+ * reserved = 1 makes the decode kernel re-read keys from L2 instead of keeping them in shared memory. */
 d2o_status d2o_set_tuning(d2o_ctx* ctx, int32_t decode_cluster, int32_t reserved);
 
 #ifdef __cplusplus

@@ -190,8 +190,8 @@ class D2OContext:
         _check(self.lib.d2o_decode_step_host(self.handle, l0, l1, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream()),
                "d2o_decode_step_host")
 
-    def d2o_set_tuning(self, decode_cluster: int = 0):
-        _check(self.lib.d2o_set_tuning(self.handle, decode_cluster, 0), "d2o_set_tuning")
+    def d2o_set_tuning(self, decode_cluster: int = 0, nonresident: int = 0):
+        _check(self.lib.d2o_set_tuning(self.handle, decode_cluster, nonresident), "d2o_set_tuning")
 
     def d2o_get_stats(self) -> D2OStats:
         s = D2OStats()

@@ -158,6 +158,7 @@ struct d2o_ctx {
   uint8_t* layer_compressed;   // [L]
   int32_t* layer_steps;        // [L] decode steps taken
   int decode_cluster;          // tuning: 0 = auto
+  int decode_nonresident;      // tuning: 1 = do not keep K rows in shared memory (re-read from L2)
 };
 
 namespace d2o {

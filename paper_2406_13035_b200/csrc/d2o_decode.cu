@@ -4,18 +4,18 @@
 // The slice's cache rows are split evenly over the CTAs of the cluster.  Each CTA
 //   1. streams its K rows once from HBM (128-bit loads), keeps them in shared memory, and
 //      computes the G logit vectors; the new token's key is row `len`;
-//   2. streams its V rows once and accumulates un-normalised outputs;
-//   3. exchanges (max, sum, partial output) with its peers through distributed shared memory;
-//      rank 0 writes the attention output, every CTA adds the probabilities of its rows,
-//      summed over the G query heads, to the accumulated scores (Eq. 6 case 2);
-//   4. if the cache exceeds S_l: cluster-wide arg-min of the score over the rows outside the
-//      T sinks and the M most recent positions picks the victim (Eq. 7-8);
-//   5. cosine similarity of the victim's key with every other key, from the copy already in
-//      shared memory (Eq. 9); cluster-wide arg-max;
-//   6. tau_t = beta*max(U) + (1-beta)*tau_{t-1} (Eq. 10); at or above it the victim is merged
-//      into its nearest neighbour with weights e^u/(e^u+e), e/(e^u+e) (Eq. 11-12), else dropped;
-//   7. the new token takes the victim's row.
-// HBM traffic per step is therefore one pass over K_c and V_c plus a few rows.
+//   2. publishes its softmax (max, sum), then streams its V rows once and accumulates
+//      un-normalised outputs while the cluster barrier completes in the background;
+//   3. turns its probabilities into accumulated scores (Eq. 6 case 2) and publishes its lowest
+//      score outside the T sinks and the M most recent positions (Eq. 7-8: the victim candidate);
+//      rank 0 combines the partial outputs;
+//   4. reads the victim's key from its owner's shared memory (distributed shared memory) and takes
+//      the cosine similarity with its own resident rows (Eq. 9); publishes its best neighbour;
+//   5. tau_t = beta*max(U) + (1-beta)*tau_{t-1} (Eq. 10); at or above it the owner of the nearest
+//      neighbour merges the victim into it with weights e^u/(e^u+e), e/(e^u+e) (Eq. 11-12);
+//   6. the new token takes the victim's row.
+// HBM traffic per step is one pass over K_c and V_c plus a few rows.  Cluster barriers are split
+// into arrive / wait so that their latency overlaps the work that does not depend on the peers.
 // The same kernel with COMPRESS=false is the uncompressed decode attention (steps 1-3 and an
 // append), used as the comparison kernel.
 #include <cooperative_groups.h>
@@ -44,28 +44,49 @@ struct DecodeArgs {
   int full_capacity, full_len;
 };
 
-template <int G, int D, typename T>
+template <int G, int D>
 struct alignas(16) Exchange {        // the part of shared memory that peer CTAs read
   float m[G];
   float l[G];
   float acc[G][D];
-  unsigned long long cand_min;       // victim candidate of this CTA
-  unsigned long long cand_max;       // nearest-neighbour candidate of this CTA
-  uint4 vic_k[D * sizeof(T) / 16];   // published by the victim's owner
-  uint4 vic_v[D * sizeof(T) / 16];
-  float vic_rn;
-  int vic_gi;
+  unsigned long long cand_min;       // victim candidate of this CTA: (score bits, 0x7fffffff - pos)
+  unsigned long long cand_max;       // neighbour candidate: (ordered similarity bits, 0x7fffffff - pos)
+  int cand_min_li, cand_max_li;      // their local row indices
+  int pad[2];
 };
 
+__device__ __forceinline__ void cluster_arrive() { __syncwarp(); asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { __syncwarp(); asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+// Block-wide extremum of a 64-bit key with the local row index of the winner (keys are unique per row).
+template <bool MIN>
+__device__ __forceinline__ void block_arg_extreme(unsigned long long key, int li, unsigned long long* s_key,
+                                                   int* s_li, unsigned long long* out_key, int* out_li) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned long long w = MIN ? warp_min_u64(key) : warp_max_u64(key);
+  const unsigned vote = __ballot_sync(0xffffffffu, key == w);
+  const int src = __ffs(vote) - 1;
+  const int wli = __shfl_sync(0xffffffffu, li, src);
+  if (lane == 0) { s_key[warp] = w; s_li[warp] = wli; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long b = s_key[0]; int bl = s_li[0];
+    for (int i = 1; i < kDecWarps; ++i) {
+      const bool better = MIN ? (s_key[i] < b) : (s_key[i] > b);
+      if (better) { b = s_key[i]; bl = s_li[i]; }
+    }
+    *out_key = b; *out_li = bl;
+  }
+}
+
 template <typename T, int D, int G, bool COMPRESS>
-__global__ void __launch_bounds__(kDecThreads)
+__global__ void __launch_bounds__(kDecThreads, (G <= 2 ? 3 : 2))
 decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_in, const T* __restrict__ v_in,
               T* __restrict__ out, T* __restrict__ kpool, T* __restrict__ vpool) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;                  // lanes that share one row (16-byte segment each)
   constexpr int NGRP = kDecThreads / LPR;       // rows in flight per CTA iteration
-  constexpr int GPW = 32 / LPR;                 // row groups per warp
-  using Xch = Exchange<G, D, T>;
+  using Xch = Exchange<G, D>;
 
   cg::cluster_group cluster = cg::this_cluster();
   const int C = (int)cluster.num_blocks();
@@ -100,7 +121,7 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   const float tau_old = COMPRESS ? a.tau[sidx] : 0.f;
   const int Tn = a.T < S ? a.T : S;
 
-  // ---- shared memory carve-up
+  // ---- shared memory carve-up (identical in every CTA of the cluster, so peers can address it)
   extern __shared__ __align__(16) unsigned char dsm[];
   Xch* xch = reinterpret_cast<Xch*>(dsm);
   float* red = reinterpret_cast<float*>(dsm + sizeof(Xch));        // [warps][G][D]
@@ -111,9 +132,9 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   uint4* newkv = reinterpret_cast<uint4*>(ps + a.chunk_cap);        // [2][LPR] staging of the new token's row
   uint4* ks = newkv + 2 * LPR;                                      // [res_rows][LPR]
   __shared__ float s_red[kDecWarps][G];
-  __shared__ unsigned long long s_red64[kDecWarps];
-  __shared__ float s_mstar[G], s_fac[G];
-  __shared__ int s_found;
+  __shared__ unsigned long long s_key[kDecWarps];
+  __shared__ int s_li[kDecWarps];
+  __shared__ float s_fac[G];
 
   const T* k_new = k_in + (size_t)sl * D;
   const T* v_new = v_in + (size_t)sl * D;
@@ -139,9 +160,9 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
     }
   }
   // ---- per-row metadata
-  for (int li = tid; li < cnt; li += kDecThreads) {
-    const int gi = r0 + li;
-    if (COMPRESS) {
+  if (COMPRESS) {
+    for (int li = tid; li < cnt; li += kDecThreads) {
+      const int gi = r0 + li;
       ps[li] = gi < n_old ? a.pos[row0 + gi] : a.t;
       sc[li] = gi < n_old ? a.score[row0 + gi] : 0.f;
       if (gi < n_old) rn[li] = a.rnorm[row0 + gi];                  // the new row's norm is computed in the K pass
@@ -160,7 +181,7 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
     for (int u = 0; u < U; ++u) {
       const int li = li0 + u * NGRP;
       if (li < cnt) {
-        if (li < a.res_rows) ks[(size_t)li * LPR + lig] = kv[u];
+        if (COMPRESS && li < a.res_rows) ks[(size_t)li * LPR + lig] = kv[u];
         float f[EPV];
         Elem<T>::unpack(kv[u], f);
         float dot[G];
@@ -231,7 +252,11 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       for (int w = 0; w < kDecWarps; ++w) t += s_red[w][g];
       l_loc[g] = t;
     }
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+      if (tid == g) { xch->m[g] = m_loc[g]; xch->l[g] = l_loc[g]; }
   }
+  cluster_arrive();                                                  // #1 (max, sum) published; completes during the V pass
   // ---- 2. V pass: un-normalised outputs
   {
     float acc[G][EPV];
@@ -283,132 +308,112 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       for (int w = 0; w < kDecWarps; ++w) t += red[(size_t)w * G * D + i];
       xch->acc[i / D][i % D] = t;
     }
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-      if (tid == g) { xch->m[g] = m_loc[g]; xch->l[g] = l_loc[g]; }
   }
-  cluster.sync();                                                    // #1 partial softmax published
-  // ---- 3. combine across the cluster
+  cluster_wait();                                                    // #1
+  // ---- 3. global softmax normaliser from the peers' (max, sum)
+  float m_star[G], l_star[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) {
-    if (tid == g) {
-      float ms = -INFINITY;
-      for (int r = 0; r < C; ++r) ms = fmaxf(ms, cluster.map_shared_rank(xch, r)->m[g]);
-      float ls = 0.f;
-      for (int r = 0; r < C; ++r) {
-        const Xch* x = cluster.map_shared_rank(xch, r);
-        ls += x->l[g] * exp2f(x->m[g] - ms);
+    float ms = -INFINITY;
+    for (int r = 0; r < C; ++r) ms = fmaxf(ms, cluster.map_shared_rank(xch, r)->m[g]);
+    float ls = 0.f;
+    for (int r = 0; r < C; ++r) {
+      const Xch* x = cluster.map_shared_rank(xch, r);
+      ls += x->l[g] * exp2f(x->m[g] - ms);
+    }
+    m_star[g] = ms; l_star[g] = ls;
+  }
+  const bool evict = COMPRESS && (n > S);
+  unsigned long long my_min = ~0ull; int my_min_li = -1;
+  if (COMPRESS) {
+    // accumulated attention (Eq. 6 case 2): add this step's probabilities, summed over the G heads;
+    // victim candidate: lowest score outside sinks and window, ties -> latest position
+    float fac[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) fac[g] = exp2f(m_loc[g] - m_star[g]) / l_star[g];
+    for (int li = tid; li < cnt; li += kDecThreads) {
+      float p = 0.f;
+#pragma unroll
+      for (int g = 0; g < G; ++g) p = fmaf(pl[(size_t)g * a.chunk_cap + li], fac[g], p);
+      const float s_new = sc[li] + p;
+      sc[li] = s_new;
+      const int pz = ps[li];
+      if (evict && pz >= Tn && pz <= a.t - M) {
+        const unsigned long long key = ((unsigned long long)float_ord(s_new) << 32) | (uint32_t)(0x7fffffff - pz);
+        if (key < my_min) { my_min = key; my_min_li = li; }
       }
-      s_mstar[g] = ms;
-      s_fac[g] = exp2f(m_loc[g] - ms) / ls;                          // turns local p into a probability
+    }
+    if (evict) block_arg_extreme<true>(my_min, my_min_li, s_key, s_li, &xch->cand_min, &xch->cand_min_li);
+  }
+  cluster_arrive();                                                  // #2 partial outputs (and victim candidates) published
+  const int new_rank = n_old / chunk;                                // CTA that holds the new token's row
+  const int new_li = n_old - new_rank * chunk;
+  if (COMPRESS) {
+    // score write-back overlaps the barrier; the victim's row is overwritten by the new token at the very end
+    for (int li = tid; li < cnt; li += kDecThreads) {
+      const int gi = r0 + li;
+      if (gi < n_old || !evict) a.score[row0 + gi] = sc[li];
     }
   }
-  __syncthreads();
+  cluster_wait();                                                    // #2
   if (rank == 0) {
     for (int i = tid; i < G * D; i += kDecThreads) {
       const int g = i / D, dd = i % D;
-      float num = 0.f, ls = 0.f;
+      float num = 0.f;
       for (int r = 0; r < C; ++r) {
         const Xch* x = cluster.map_shared_rank(xch, r);
-        const float w = exp2f(x->m[g] - s_mstar[g]);
-        num = fmaf(x->acc[g][dd], w, num);
-        ls = fmaf(x->l[g], w, ls);
+        num = fmaf(x->acc[g][dd], exp2f(x->m[g] - m_star[g]), num);
       }
-      out[((size_t)sl * G + g) * D + dd] = Elem<T>::from_float(num / ls);
+      out[((size_t)sl * G + g) * D + dd] = Elem<T>::from_float(num / l_star[g]);
     }
   }
-  if (!COMPRESS) {
-    // append the new token's row to the cache and leave
-    if (n_old >= r0 && n_old < r0 + chunk && grp == 0) {
-      *reinterpret_cast<uint4*>(kpool + (row0 + n_old) * D + lig * EPV) = ld_global_v4(k_new + lig * EPV);
-      *reinterpret_cast<uint4*>(vpool + (row0 + n_old) * D + lig * EPV) = ld_global_v4(v_new + lig * EPV);
-    }
-    cluster.sync();                                                  // peers may still read our exchange area
-    return;
-  }
-  // accumulated attention (Eq. 6 case 2): add this step's probabilities, summed over the G heads
-  for (int li = tid; li < cnt; li += kDecThreads) {
-    float p = 0.f;
-#pragma unroll
-    for (int g = 0; g < G; ++g) p = fmaf(pl[(size_t)g * a.chunk_cap + li], s_fac[g], p);
-    sc[li] += p;
-  }
-  __syncthreads();
-  const int new_rank = n_old / chunk;                                // CTA that holds the new token's row
-  const int new_li = n_old - new_rank * chunk;
-  if (n <= S) {
-    // cache not full yet: plain append
-    for (int li = tid; li < cnt; li += kDecThreads) {
-      const int gi = r0 + li;
-      a.score[row0 + gi] = sc[li];
-      if (gi == n_old) { a.pos[row0 + gi] = a.t; a.rnorm[row0 + gi] = rn[li]; }
-    }
+  if (!evict) {
+    // append the new token's row (cache not full, or uncompressed mode)
     if (rank == new_rank && grp == 0) {
-      *reinterpret_cast<uint4*>(kpool + (row0 + n_old) * D + lig * EPV) = newkv[lig];
-      *reinterpret_cast<uint4*>(vpool + (row0 + n_old) * D + lig * EPV) = newkv[LPR + lig];
+      if (COMPRESS) {
+        *reinterpret_cast<uint4*>(kpool + (row0 + n_old) * D + lig * EPV) = newkv[lig];
+        *reinterpret_cast<uint4*>(vpool + (row0 + n_old) * D + lig * EPV) = newkv[LPR + lig];
+        if (lig == 0) { a.pos[row0 + n_old] = a.t; a.rnorm[row0 + n_old] = rn[new_li]; }
+      } else {
+        *reinterpret_cast<uint4*>(kpool + (row0 + n_old) * D + lig * EPV) = ld_global_v4(k_new + lig * EPV);
+        *reinterpret_cast<uint4*>(vpool + (row0 + n_old) * D + lig * EPV) = ld_global_v4(v_new + lig * EPV);
+      }
     }
-    if (rank == 0 && tid == 0) {
+    if (COMPRESS && rank == 0 && tid == 0) {
       a.len[sidx] = n;
       atomicAdd(&a.counters[kCntDecodeSteps], 1ull);
     }
-    cluster.sync();
+    cluster_arrive();                                                // peers may still read our exchange area
+    cluster_wait();
     return;
   }
-  // ---- 4. victim: lowest score outside sinks and window; ties -> latest position
-  {
-    unsigned long long best = ~0ull;
-    for (int li = tid; li < cnt; li += kDecThreads) {
-      const int p = ps[li];
-      if (p >= Tn && p <= a.t - M) {
-        const unsigned long long key = ((unsigned long long)float_ord(sc[li]) << 32) | (uint32_t)(0x7fffffff - p);
-        best = key < best ? key : best;
-      }
-    }
-    best = warp_min_u64(best);
-    if (lane == 0) s_red64[warp] = best;
-    if (tid == 0) s_found = -1;
-    __syncthreads();
-    if (tid == 0) {
-      unsigned long long t = s_red64[0];
-      for (int w = 1; w < kDecWarps; ++w) t = s_red64[w] < t ? s_red64[w] : t;
-      xch->cand_min = t;
-    }
-  }
-  cluster.sync();                                                    // #2 victim candidates published
-  unsigned long long kmin = ~0ull; int vic_rank = -1;
+  // ---- 4. victim (Eq. 7-8)
+  unsigned long long kmin = ~0ull; int vic_rank = 0, vic_li = 0;
   for (int r = 0; r < C; ++r) {
-    const unsigned long long t = cluster.map_shared_rank(xch, r)->cand_min;
-    if (t < kmin) { kmin = t; vic_rank = r; }
+    const Xch* x = cluster.map_shared_rank(xch, r);
+    const unsigned long long t = x->cand_min;
+    if (t < kmin) { kmin = t; vic_rank = r; vic_li = x->cand_min_li; }
   }
   if (kmin == ~0ull) {
     // nothing may be evicted (S_l < T + M): report, drop the new token, keep the cache as it is
     if (rank == 0 && tid == 0) report_error(a.status, D2O_ERR_STATE, 0xDEC00000u | (uint32_t)(sl & 0xfffff));
-    for (int li = tid; li < cnt; li += kDecThreads)
-      if (r0 + li < n_old) a.score[row0 + r0 + li] = sc[li];
-    cluster.sync();
+    cluster_arrive();
+    cluster_wait();
     return;
   }
-  const int vic_pos = 0x7fffffff - (int)(uint32_t)(kmin & 0xffffffffu);
-  if (rank == vic_rank) {
-    for (int li = tid; li < cnt; li += kDecThreads)
-      if (ps[li] == vic_pos) s_found = li;
-    __syncthreads();
-    const int li = s_found;
-    if (grp == 0) {
-      xch->vic_k[lig] = li < a.res_rows ? ks[(size_t)li * LPR + lig] : ld_global_v4(k_src(li) + lig * EPV);
-      xch->vic_v[lig] = ld_global_v4(v_src(li) + lig * EPV);
-    }
-    if (tid == 0) { xch->vic_rn = rn[li]; xch->vic_gi = r0 + li; }
-  }
-  cluster.sync();                                                    // #3 victim row published
-  const Xch* xv = cluster.map_shared_rank(xch, vic_rank);
-  const int vic_gi = xv->vic_gi;
-  const float vic_rn = xv->vic_rn;
+  const int vic_gi = vic_rank * chunk + vic_li;
   float kvic[EPV];
-  Elem<T>::unpack(xv->vic_k[lig], kvic);
+  float vic_rn;
+  {
+    const uint4* pks = cluster.map_shared_rank(ks, vic_rank);
+    const uint4 kv = vic_li < a.res_rows ? pks[(size_t)vic_li * LPR + lig]
+                                         : ld_global_v4((vic_gi < n_old ? kpool + (row0 + vic_gi) * D : k_new) + lig * EPV);
+    Elem<T>::unpack(kv, kvic);
+    vic_rn = cluster.map_shared_rank(rn, vic_rank)[vic_li];
+  }
   // ---- 5. cosine similarity of the victim with every other row (Eq. 9), arg-max, ties -> earliest position
   {
-    unsigned long long best = 0ull;
+    unsigned long long best = 0ull; int best_li = -1;
     for (int li = grp; li < cnt; li += NGRP) {
       if (r0 + li == vic_gi) continue;
       float f[EPV];
@@ -420,26 +425,19 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       s = group_sum<LPR>(s, gmask);
       const float u = s * vic_rn * rn[li];
       const unsigned long long key = ((unsigned long long)float_ord(u) << 32) | (uint32_t)(0x7fffffff - ps[li]);
-      best = key > best ? key : best;
+      if (key > best) { best = key; best_li = li; }
     }
-    best = warp_max_u64(best);
-    if (lane == 0) s_red64[warp] = best;
-    if (tid == 0) s_found = -1;
-    __syncthreads();
-    if (tid == 0) {
-      unsigned long long t = s_red64[0];
-      for (int w = 1; w < kDecWarps; ++w) t = s_red64[w] > t ? s_red64[w] : t;
-      xch->cand_max = t;
-    }
+    block_arg_extreme<false>(best, best_li, s_key, s_li, &xch->cand_max, &xch->cand_max_li);
   }
-  cluster.sync();                                                    // #4 neighbour candidates published
-  unsigned long long kmax = 0ull; int nn_rank = 0;
+  cluster_arrive();                                                  // #3 neighbour candidates published
+  cluster_wait();
+  unsigned long long kmax = 0ull; int nn_rank = 0, nn_li = 0;
   for (int r = 0; r < C; ++r) {
-    const unsigned long long t = cluster.map_shared_rank(xch, r)->cand_max;
-    if (t > kmax) { kmax = t; nn_rank = r; }
+    const Xch* x = cluster.map_shared_rank(xch, r);
+    const unsigned long long t = x->cand_max;
+    if (t > kmax) { kmax = t; nn_rank = r; nn_li = x->cand_max_li; }
   }
   const float mx = ord_float((uint32_t)(kmax >> 32));
-  const int nn_pos = 0x7fffffff - (int)(uint32_t)(kmax & 0xffffffffu);
   // ---- 6. EMA threshold (Eq. 10) and merge (Eq. 11-12)
   const float tau_new = a.beta * mx + (1.0f - a.beta) * tau_old;
   const float thr = isnan(a.tau_override) ? tau_new : a.tau_override;
@@ -450,57 +448,47 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
     atomicAdd(&a.counters[kCntEvictions], 1ull);
     atomicAdd(&a.counters[merge ? kCntMerges : kCntDiscards], 1ull);
   }
-  if (merge && rank == nn_rank) {
-    for (int li = tid; li < cnt; li += kDecThreads)
-      if (ps[li] == nn_pos && r0 + li != vic_gi) s_found = li;
-    __syncthreads();
-    const int lj = s_found;
-    if (grp == 0) {
-      const bool is_new = (r0 + lj == n_old);
-      const float ew = expf(mx);
-      const float w_e = ew / (ew + kEuler), w_c = kEuler / (ew + kEuler);
-      float fk[EPV], fv[EPV], vv[EPV];
-      const uint4 kcur = is_new ? newkv[lig]
-                                : (lj < a.res_rows ? ks[(size_t)lj * LPR + lig] : ld_global_v4(k_src(lj) + lig * EPV));
-      Elem<T>::unpack(kcur, fk);
-      Elem<T>::unpack(is_new ? newkv[LPR + lig] : ld_global_v4(v_src(lj) + lig * EPV), fv);
-      Elem<T>::unpack(xv->vic_v[lig], vv);
+  if (merge && rank == nn_rank && grp == 0) {
+    const int lj = nn_li;
+    const bool is_new = (r0 + lj == n_old);
+    const float ew = expf(mx);
+    const float w_e = ew / (ew + kEuler), w_c = kEuler / (ew + kEuler);
+    float fk[EPV], fv[EPV], vv[EPV];
+    const uint4 kcur = is_new ? newkv[lig]
+                              : (lj < a.res_rows ? ks[(size_t)lj * LPR + lig] : ld_global_v4(k_src(lj) + lig * EPV));
+    Elem<T>::unpack(kcur, fk);
+    Elem<T>::unpack(is_new ? newkv[LPR + lig] : ld_global_v4(v_src(lj) + lig * EPV), fv);
+    // the victim's value row is still in place: its slot is overwritten only after the last barrier
+    Elem<T>::unpack(ld_global_v4((vic_gi < n_old ? vpool + (row0 + vic_gi) * D : v_new) + lig * EPV), vv);
 #pragma unroll
-      for (int e = 0; e < EPV; ++e) { fk[e] = w_c * fk[e] + w_e * kvic[e]; fv[e] = w_c * fv[e] + w_e * vv[e]; }
-      const uint4 kn = Elem<T>::pack(fk), vn = Elem<T>::pack(fv);
-      Elem<T>::unpack(kn, fk);                                       // norm of what is stored
-      float ss = 0.f;
+    for (int e = 0; e < EPV; ++e) { fk[e] = w_c * fk[e] + w_e * kvic[e]; fv[e] = w_c * fv[e] + w_e * vv[e]; }
+    const uint4 kn = Elem<T>::pack(fk), vn = Elem<T>::pack(fv);
+    Elem<T>::unpack(kn, fk);                                         // norm of what is stored
+    float ss = 0.f;
 #pragma unroll
-      for (int e = 0; e < EPV; ++e) ss = fmaf(fk[e], fk[e], ss);
-      ss = group_sum<LPR>(ss, gmask);
-      const float rnew = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
-      if (is_new) { newkv[lig] = kn; newkv[LPR + lig] = vn; }
-      else {
-        *reinterpret_cast<uint4*>(kpool + (row0 + r0 + lj) * D + lig * EPV) = kn;
-        *reinterpret_cast<uint4*>(vpool + (row0 + r0 + lj) * D + lig * EPV) = vn;
-        if (lig == 0) a.rnorm[row0 + r0 + lj] = rnew;
-      }
-      if (lig == 0) rn[lj] = rnew;
+    for (int e = 0; e < EPV; ++e) ss = fmaf(fk[e], fk[e], ss);
+    ss = group_sum<LPR>(ss, gmask);
+    const float rnew = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+    if (is_new) { newkv[lig] = kn; newkv[LPR + lig] = vn; }
+    else {
+      *reinterpret_cast<uint4*>(kpool + (row0 + r0 + lj) * D + lig * EPV) = kn;
+      *reinterpret_cast<uint4*>(vpool + (row0 + r0 + lj) * D + lig * EPV) = vn;
+      if (lig == 0) a.rnorm[row0 + r0 + lj] = rnew;
     }
-    __syncthreads();
+    if (lig == 0) rn[lj] = rnew;
   }
-  // ---- 7. write back scores; the new token takes the victim's row
-  for (int li = tid; li < cnt; li += kDecThreads) {
-    const int gi = r0 + li;
-    if (gi < n_old && gi != vic_gi) a.score[row0 + gi] = sc[li];
-  }
-  if (rank == new_rank && vic_gi != n_old) {
-    if (grp == 0) {
-      *reinterpret_cast<uint4*>(kpool + (row0 + vic_gi) * D + lig * EPV) = newkv[lig];
-      *reinterpret_cast<uint4*>(vpool + (row0 + vic_gi) * D + lig * EPV) = newkv[LPR + lig];
-    }
-    if (tid == 0) {
+  cluster_arrive();                                                  // #4 all reads of peer memory and of the victim's row are done
+  cluster_wait();
+  // ---- 7. the new token takes the victim's row
+  if (rank == new_rank && vic_gi != n_old && grp == 0) {
+    *reinterpret_cast<uint4*>(kpool + (row0 + vic_gi) * D + lig * EPV) = newkv[lig];
+    *reinterpret_cast<uint4*>(vpool + (row0 + vic_gi) * D + lig * EPV) = newkv[LPR + lig];
+    if (lig == 0) {
       a.pos[row0 + vic_gi] = a.t;
       a.score[row0 + vic_gi] = sc[new_li];
       a.rnorm[row0 + vic_gi] = rn[new_li];
     }
   }
-  cluster.sync();                                                    // #5 nobody reads our shared memory any more
 }
 
 // ------------------------------------------------------------------------------------ launch
@@ -508,7 +496,7 @@ template <typename T, int D, int G, bool COMPRESS>
 static cudaError_t launch_one(const DecodeArgs& a, int n_slices, int C, const void* q, const void* k, const void* v,
                               void* out, void* kpool, void* vpool, cudaStream_t st) {
   constexpr int LPR = D * sizeof(T) / 16;
-  const size_t smem = sizeof(Exchange<G, D, T>) + (size_t)kDecWarps * G * D * 4 + (size_t)(G + 3) * a.chunk_cap * 4 +
+  const size_t smem = sizeof(Exchange<G, D>) + (size_t)kDecWarps * G * D * 4 + (size_t)(G + 3) * a.chunk_cap * 4 +
                       (size_t)2 * LPR * 16 + (size_t)a.res_rows * LPR * 16;
   auto kern = decode_kernel<T, D, G, COMPRESS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -556,13 +544,13 @@ static bool plan(int max_rows, int row_bytes, int G, int D, int want_cluster, bo
   const int budget = 200 * 1024;
   int C = want_cluster;
   if (C == 0) {
-    // smallest cluster that keeps all K rows resident in <= ~100 KB per CTA (two CTAs per SM), but enough CTAs
+    // smallest cluster that keeps all K rows resident in <= ~72 KB per CTA (three CTAs per SM), but enough CTAs
     // to cover the machine when there are few slices
     C = 1;
     while (C < kMaxCluster) {
       const int chunk = (((max_rows + C - 1) / C) + 7) & ~7;
       const long need = fixed + (long)chunk * ((G + 3) * 4 + (resident ? row_bytes : 0));
-      if (need <= 100 * 1024 && (long)n_slices * C >= 2 * 148) break;
+      if (need <= 72 * 1024 && (long)n_slices * C >= 2 * 148) break;
       C *= 2;
     }
   }
@@ -599,8 +587,8 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     }
   const int n_slices = (l1 - l0) * B * g.n_kv_heads;
   int C, chunk_cap, res_rows;
-  if (!plan(max_rows, g.d_head * c->elem_size, c->group, g.d_head, c->decode_cluster, true, n_slices, &C, &chunk_cap,
-            &res_rows)) {
+  if (!plan(max_rows, g.d_head * c->elem_size, c->group, g.d_head, c->decode_cluster, !c->decode_nonresident, n_slices,
+            &C, &chunk_cap, &res_rows)) {
     *why = D2O_ERR_UNSUPPORTED;
     return cudaSuccess;
   }

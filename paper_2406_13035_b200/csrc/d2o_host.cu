@@ -333,10 +333,11 @@ extern "C" d2o_status d2o_get_stats(d2o_ctx* c, d2o_stats* out, void* stream) {
 }
 
 extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_cluster, int32_t reserved) {
-  (void)reserved;
   if (!c) return D2O_ERR_INVALID_ARG;
+  if (reserved < 0 || reserved > 1) return D2O_ERR_INVALID_ARG;
   if (decode_cluster != 0 && decode_cluster != 1 && decode_cluster != 2 && decode_cluster != 4 && decode_cluster != 8)
     return D2O_ERR_INVALID_ARG;
   c->decode_cluster = decode_cluster;
+  c->decode_nonresident = reserved;
   return D2O_OK;
 }

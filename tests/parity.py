@@ -245,8 +245,16 @@ def _compare_state(rep, got, st, dtype, tag):
     gpos = got["pos"].numpy().astype(np.int64)
     order = np.argsort(gpos, kind="stable")
     assert np.array_equal(gpos[order], st.pos), f"{tag}: cache positions differ"
-    rep.err(f"{tag}_K", close(got["K"].double().numpy()[order], st.K, dtype))
-    rep.err(f"{tag}_V", close(got["V"].double().numpy()[order], st.V, dtype))
+    Kg, Vg = got["K"].double().numpy()[order], got["V"].double().numpy()[order]
+    eK, eV = close(Kg, st.K, dtype), close(Vg, st.V, dtype)
+    rep.err(f"{tag}_K", eK)
+    rep.err(f"{tag}_V", eV)
+    if eK <= 1.0 and eV <= 1.0:
+        # storage-follow: a merged value that sits on a rounding boundary of the cache dtype may round
+        # either way (float32 vs float64 arithmetic).  The flip is within tolerance, but one 16-bit ulp in a
+        # key moves later logits by ~1e-3, so the oracle continues from the rows the GPU actually stored.
+        rep.storage_flips = getattr(rep, "storage_flips", 0) + int((Kg != st.K).sum() + (Vg != st.V).sum())
+        st.K, st.V = Kg.copy(), Vg.copy()
     sc = got["score"].double().numpy()[order]
     rep.err(f"{tag}_score_rel", np.max(np.abs(sc - st.score) / np.maximum(np.abs(st.score), 1e-6)))
     # the cached inverse norms belong to the stored keys
@@ -302,6 +310,7 @@ def _check_decode_slice(rep, ctx, orc, wl, l, b, h, q, k, v, out, t, tabs, tie_r
     orc.slices[key] = st
     rep.err("out", close(out[b, h * G:(h + 1) * G], o, wl.dtype))
     _compare_state(rep, got, st, wl.dtype, "decode")
+    orc.slices[key] = st
     rep.err("tau_abs", abs(got["tau"] - st.tau))
     if log.evicted:
         rep.merges += int(log.merged)
