@@ -40,8 +40,8 @@ def parse():
     ap.add_argument("--config", default="cfg1")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the config's decode steps")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--cluster", type=int, default=0, help="CTAs per cluster of the decode kernel (0 = auto)")
-    ap.add_argument("--nonresident", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0, help="stages of the decode kernel's ring (0 = auto)")
+    ap.add_argument("--no-l2-hints", action="store_true", help="decode kernel: copies without L2 eviction hints")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers-per-call", type=int, default=0)
@@ -128,8 +128,8 @@ def run_ours(args, wl, rank, world, device):
                         n_sink=wl.n_sink, window=wl.window, nm_ratio=wl.nm_ratio, beta=wl.beta,
                         density_temp=wl.density_temp, min_budget=wl.min_budget)
     ctx = B.D2OContext(cfg, device)
-    if args.cluster or args.nonresident:
-        ctx.d2o_set_tuning(args.cluster, args.nonresident)
+    if args.stages or args.no_l2_hints:
+        ctx.d2o_set_tuning(args.stages, 0 if args.no_l2_hints else 1)
     # every rank works on its own sequences: same shapes, rank-dependent seed (weak scaling, no exchange)
     import dataclasses
     wl_r = dataclasses.replace(wl, seed=wl.seed + 7919 * rank)
@@ -243,7 +243,7 @@ def run_ours(args, wl, rank, world, device):
         "config": {"workload": f"{wl.name}: L={wl.n_layers} Hq={wl.n_q_heads} Hkv={wl.n_kv_heads} d={wl.d_head} "
                                f"B={wl.batch} P={wl.prompt_len} rho={wl.rho} decode_steps={nd}",
                    "l2": "decode working set (K_c+V_c of all layers) exceeds the 126 MB L2; prompt tensors exceed it too",
-                   "layers_per_decode_call": lpc, "decode_cluster": args.cluster or "auto",
+                   "layers_per_decode_call": lpc, "decode_ring_stages": args.stages or "auto",
                    "sequences_per_gpu": wl.batch, "parallelism": "replicas (independent sequences per GPU)"},
         "decode_steps_per_s_per_gpu": round(steps_per_s, 2), "decode_us_per_step": round(decode_ms * 1e3 / nd, 2),
         "stats_ms": round(stats_ms, 3), "budgets_ms": round(budget_ms, 3), "prefill_compress_ms": round(compress_ms, 3),

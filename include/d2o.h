@@ -73,14 +73,15 @@ typedef struct {
 typedef struct d2o_ctx d2o_ctx;
 
 /* Device pointers into `state` for inspection / checkpointing.  Per-layer fields refer to the
- * layer passed to d2o_get_view().  Slices are ordered (b, kv_head); slice (b, h) of the layer
- * owns rows [row_off + (b*Hkv + h)... see fields.  All DEVICE. */
+ * layer passed to d2o_get_view().  The cache rows of slice (b, layer, h) are
+ * [row_off[b, layer] + h * stride, ... + len), stride = S_l rounded up to a multiple of 8.
+ * All DEVICE. */
 typedef struct {
   const float*   colsum;     /* [B, Hq, P]   column sums of the prompt attention (Eq. 4)      */
   const double*  density;    /* [B, L, Hq]   F_v per sequence, layer, query head (all layers) */
   const int32_t* budgets;    /* [B, L]       S_l (all layers)                                  */
   const int32_t* windows;    /* [B, L]       M_l (all layers)                                  */
-  const int64_t* row_off;    /* [B, L]       first cache row of (b, layer); slice (b,h) starts at row_off + h*S_l */
+  const int64_t* row_off;    /* [B, L]       first cache row of (b, layer); slice (b,h) starts at row_off + h*roundup8(S_l) */
   void*          k_cache;    /* base of the K pool, rows of d_head elements (all layers)      */
   void*          v_cache;    /* base of the V pool                                             */
   int32_t*       pos;        /* [rows]       original position of each cache row (pool-wide)  */
@@ -174,9 +175,11 @@ d2o_status d2o_get_view(d2o_ctx* ctx, int32_t layer, d2o_view* out);
 /* Copies the counters to HOST memory; synchronises `stream`. */
 d2o_status d2o_get_stats(d2o_ctx* ctx, d2o_stats* out_host, void* stream);
 
-/* Launch-shape knobs for measurements (0 = automatic): CTAs per cluster of the decode kernel;
- * reserved = 1 makes the decode kernel re-read keys from L2 instead of keeping them in shared memory. */
-d2o_status d2o_set_tuning(d2o_ctx* ctx, int32_t decode_cluster, int32_t reserved);
+/* Knobs of the decode kernel for measurements: stages of its shared-memory ring (0 = automatic,
+ * else 2..12, 16 KB each; a depth that does not fit in shared memory makes the next
+ * d2o_decode_step return D2O_ERR_UNSUPPORTED) and whether its copies carry L2 eviction hints
+ * (1 = yes, the default; 0 = no). */
+d2o_status d2o_set_tuning(d2o_ctx* ctx, int32_t decode_stages, int32_t decode_l2_hints);
 
 #ifdef __cplusplus
 }

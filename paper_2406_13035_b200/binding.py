@@ -190,8 +190,8 @@ class D2OContext:
         _check(self.lib.d2o_decode_step_host(self.handle, l0, l1, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream()),
                "d2o_decode_step_host")
 
-    def d2o_set_tuning(self, decode_cluster: int = 0, nonresident: int = 0):
-        _check(self.lib.d2o_set_tuning(self.handle, decode_cluster, nonresident), "d2o_set_tuning")
+    def d2o_set_tuning(self, decode_stages: int = 0, decode_l2_hints: int = 1):
+        _check(self.lib.d2o_set_tuning(self.handle, decode_stages, decode_l2_hints), "d2o_set_tuning")
 
     def d2o_get_stats(self) -> D2OStats:
         s = D2OStats()
@@ -241,7 +241,7 @@ class D2OContext:
         v = self._view(layer)
         bud, win, off = tables if tables is not None else self.tables()
         S = int(bud[b, layer])
-        r0 = int(off[b, layer]) + h * S
+        r0 = int(off[b, layer]) + h * ((S + 7) // 8 * 8)      # slices start at multiples of 8 rows
         esz = 4 if c.dtype == D2O_F32 else 2
         rows = v.pool_rows
         sidx = (layer * c.batch + b) * c.n_kv_heads + h

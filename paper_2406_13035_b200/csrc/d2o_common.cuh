@@ -118,6 +118,10 @@ __device__ __forceinline__ float ord_float(uint32_t o) {
   return __uint_as_float(u);
 }
 
+// Cache rows of one slice (sequence, layer, KV head) start at a multiple of 8 rows, so that the 4-byte
+// per-row arrays (pos, score, rnorm) of a slice start on a 32-byte boundary (bulk copies need 16).
+__host__ __device__ __forceinline__ int slice_stride(int S) { return (S + 7) & ~7; }
+
 // device-side anomaly report: first writer wins
 __device__ __forceinline__ void report_error(uint32_t* status_word, uint32_t code, uint32_t detail) {
   if (atomicCAS(status_word, 0u, code) == 0u) status_word[1] = detail;
@@ -157,8 +161,8 @@ struct d2o_ctx {
   uint8_t* layer_fed;          // [L] stats seen
   uint8_t* layer_compressed;   // [L]
   int32_t* layer_steps;        // [L] decode steps taken
-  int decode_cluster;          // tuning: 0 = auto
-  int decode_nonresident;      // tuning: 1 = do not keep K rows in shared memory (re-read from L2)
+  int decode_stages;           // tuning: stages of the decode kernel's ring, 0 = auto
+  int decode_l2_hints;         // tuning: 1 = the decode kernel's copies carry L2 eviction hints
 };
 
 namespace d2o {
@@ -176,6 +180,9 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
 cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int capacity, int len, void* kc, void* vc,
                                const void* q, const void* k, const void* v, void* out, cudaStream_t st,
                                d2o_status* why);
+
+// largest number of rows (cache + the new token) of one slice the decode kernel can keep resident
+int decode_max_rows(int row_bytes, int group, int d_head);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -1,35 +1,34 @@
 // Token generation (Section 3, Eq. 2-3; Section 4.2, Eq. 6-12): one fused kernel per decode step.
 //
-// One thread-block cluster handles one slice = (layer, sequence, KV head) with its G query heads.
-// The slice's cache rows are split evenly over the CTAs of the cluster.  Each CTA
-//   1. streams its K rows once from HBM (128-bit loads), keeps them in shared memory, and
-//      computes the G logit vectors; the new token's key is row `len`;
-//   2. publishes its softmax (max, sum), then streams its V rows once and accumulates
-//      un-normalised outputs while the cluster barrier completes in the background;
-//   3. turns its probabilities into accumulated scores (Eq. 6 case 2) and publishes its lowest
-//      score outside the T sinks and the M most recent positions (Eq. 7-8: the victim candidate);
-//      rank 0 combines the partial outputs;
-//   4. reads the victim's key from its owner's shared memory (distributed shared memory) and takes
-//      the cosine similarity with its own resident rows (Eq. 9); publishes its best neighbour;
-//   5. tau_t = beta*max(U) + (1-beta)*tau_{t-1} (Eq. 10); at or above it the owner of the nearest
-//      neighbour merges the victim into it with weights e^u/(e^u+e), e/(e^u+e) (Eq. 11-12);
-//   6. the new token takes the victim's row.
-// HBM traffic per step is one pass over K_c and V_c plus a few rows.  Cluster barriers are split
-// into arrive / wait so that their latency overlaps the work that does not depend on the peers.
-// The same kernel with COMPRESS=false is the uncompressed decode attention (steps 1-3 and an
-// append), used as the comparison kernel.
-#include <cooperative_groups.h>
+// One CTA handles one slice = (layer, sequence, KV head) with its G query heads, and streams the
+// slice's cache rows through a ring of shared-memory stages filled by bulk asynchronous copies
+// (cp.async.bulk, completion on mbarriers).  A producer warp runs ahead of eight consumer warps by
+// the depth of the ring, across the boundaries of the passes, so the reductions between two passes
+// do not drain the memory pipeline:
+//
+//   pass K   keys once from HBM: logits of the G heads (plus the new token's row from the inputs)
+//            -> softmax normaliser -> AttnScore += probabilities (Eq. 6 case 2)
+//            -> victim = lowest score outside the T sinks and the M most recent positions (Eq. 7-8)
+//   pass K'  keys again, now served by L2 (the first pass asks L2 to keep them, the later passes
+//            ask it to drop what they touch): cosine of the victim with every other row (Eq. 9)
+//            -> nearest neighbour, tau_t (Eq. 10), merge decision, merged key row (Eq. 11-12)
+//   pass V   values once from HBM: outputs (Eq. 3); the value rows of the victim and of the
+//            neighbour are picked out of the stream for the merge (Eq. 11)
+//   then     merged value row, the new token takes the victim's row.
+// Pass K' is skipped while the cache is not full.  Everything that needs the whole slice is a
+// block-wide reduction inside one CTA; there is no inter-CTA communication.
 #include <math.h>
 
 #include "d2o_common.cuh"
 
-namespace cg = cooperative_groups;
-
 namespace d2o {
 
-constexpr int kDecThreads = 256;
-constexpr int kDecWarps = kDecThreads / 32;
-constexpr int kMaxCluster = 8;
+constexpr int kConsWarps = 8;                           // consumer warps
+constexpr int kConsThreads = kConsWarps * 32;
+constexpr int kDecThreads = kConsThreads + 32;          // + one producer warp
+constexpr int kStageBytes = 4 * kConsThreads * 16;      // every consumer thread reads four 16-byte vectors per stage
+constexpr int kMaxStages = 12;
+constexpr unsigned long long kWaitNs = 1000000000ull;   // an mbarrier wait gives up after 1 s
 
 struct DecodeArgs {
   const int32_t* budgets; const int32_t* windows; const int64_t* row_off;   // [B, L]
@@ -38,114 +37,203 @@ struct DecodeArgs {
   unsigned long long* counters; uint32_t* status;
   int L, l0, B, Hkv, T, t;          // t = position of the token generated in this step
   float beta, tau_override;
-  int chunk_cap;                    // rows per CTA the shared-memory arrays are sized for
-  int res_rows;                     // K rows per CTA kept resident in shared memory
-  // uncompressed mode
-  int full_capacity, full_len;
+  int row_cap;                      // rows the per-row shared-memory arrays are sized for (multiple of 8)
+  int stages;                       // stages of the ring
+  int l2_hints;                     // 1: pass K asks L2 to keep its lines, later passes to drop theirs
 };
 
-template <int G, int D>
-struct alignas(16) Exchange {        // the part of shared memory that peer CTAs read
-  float m[G];
-  float l[G];
-  float acc[G][D];
-  unsigned long long cand_min;       // victim candidate of this CTA: (score bits, 0x7fffffff - pos)
-  unsigned long long cand_max;       // neighbour candidate: (ordered similarity bits, 0x7fffffff - pos)
-  int cand_min_li, cand_max_li;      // their local row indices
-  int pad[2];
-};
+// ----------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long global_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsThreads) : "memory"); }
 
-__device__ __forceinline__ void cluster_arrive() { __syncwarp(); asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { __syncwarp(); asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: returns false (and the caller reports D2O_ERR_TIMEOUT) if the phase has not completed in time.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (!mbar_try_wait(bar, parity)) {
+    if (global_ns() - t0 > kWaitNs) return false;
+  }
+  return true;
+}
+// global -> this CTA's shared memory, 16-byte aligned on both sides, size a multiple of 16
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s_hint(void* dst, const void* src, uint32_t bytes, unsigned long long* bar,
+                                              unsigned long long policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
 
-// Block-wide extremum of a 64-bit key with the local row index of the winner (keys are unique per row).
+// Extremum over the consumer warps of a 64-bit key with the row index of the winner (keys are unique per row).
+// The result is valid in s_out_key / s_out_li after the next consumer_sync().
 template <bool MIN>
 __device__ __forceinline__ void block_arg_extreme(unsigned long long key, int li, unsigned long long* s_key,
-                                                   int* s_li, unsigned long long* out_key, int* out_li) {
+                                                   int* s_li, unsigned long long* s_out_key, int* s_out_li) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned long long w = MIN ? warp_min_u64(key) : warp_max_u64(key);
   const unsigned vote = __ballot_sync(0xffffffffu, key == w);
   const int src = __ffs(vote) - 1;
   const int wli = __shfl_sync(0xffffffffu, li, src);
   if (lane == 0) { s_key[warp] = w; s_li[warp] = wli; }
-  __syncthreads();
+  consumer_sync();
   if (threadIdx.x == 0) {
     unsigned long long b = s_key[0]; int bl = s_li[0];
-    for (int i = 1; i < kDecWarps; ++i) {
+    for (int i = 1; i < kConsWarps; ++i) {
       const bool better = MIN ? (s_key[i] < b) : (s_key[i] > b);
       if (better) { b = s_key[i]; bl = s_li[i]; }
     }
-    *out_key = b; *out_li = bl;
+    *s_out_key = b; *s_out_li = bl;
   }
 }
 
-template <typename T, int D, int G, bool COMPRESS>
+// Sums four values, each spread over the LPR lanes of a row group, with 3 + log2(LPR/4) shuffles instead of
+// 4*log2(LPR): lanes trade halves of the batch first.  Lane `lig` returns the total of value lig / (LPR/4).
+// All 32 lanes of the warp must call it.
+template <int LPR>
+__device__ __forceinline__ float reduce4(float s0, float s1, float s2, float s3, int lig) {
+  const bool hi = (lig & (LPR / 2)) != 0;
+  float k0 = hi ? s2 : s0, k1 = hi ? s3 : s1;
+  const float t0 = hi ? s0 : s2, t1 = hi ? s1 : s3;
+  k0 += __shfl_xor_sync(0xffffffffu, t0, LPR / 2);
+  k1 += __shfl_xor_sync(0xffffffffu, t1, LPR / 2);
+  const bool hi2 = (lig & (LPR / 4)) != 0;
+  float k = hi2 ? k1 : k0;
+  const float t = hi2 ? k0 : k1;
+  k += __shfl_xor_sync(0xffffffffu, t, LPR / 4);
+#pragma unroll
+  for (int o = LPR / 8; o > 0; o >>= 1) k += __shfl_xor_sync(0xffffffffu, k, o);
+  return k;
+}
+
+template <typename T, int D, int G>
 __global__ void __launch_bounds__(kDecThreads, (G <= 2 ? 3 : 2))
 decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_in, const T* __restrict__ v_in,
               T* __restrict__ out, T* __restrict__ kpool, T* __restrict__ vpool) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;                  // lanes that share one row (16-byte segment each)
-  constexpr int NGRP = kDecThreads / LPR;       // rows in flight per CTA iteration
-  using Xch = Exchange<G, D>;
+  constexpr int NGRP = kConsThreads / LPR;      // row groups of the consumers
+  constexpr int SR = 4 * NGRP;                  // rows per stage: four per consumer thread
+  constexpr int QL = LPR / 4;                   // lanes that end up with the same row total after reduce4
+  constexpr int ROWB = D * (int)sizeof(T);      // bytes per row
 
-  cg::cluster_group cluster = cg::this_cluster();
-  const int C = (int)cluster.num_blocks();
-  const int rank = (int)cluster.block_rank();
-  const int sl = blockIdx.x / C;                // slice index within the launch
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int grp = tid / LPR, lig = tid % LPR;
-  const unsigned gmask = group_mask<LPR>();
-
-  // ---- slice parameters
-  int S, M, n_old, sidx = 0;
-  int64_t row0;
-  if (COMPRESS) {
-    const int per_layer = a.B * a.Hkv;
-    const int layer = a.l0 + sl / per_layer;
-    const int bh = sl % per_layer;
-    const int b = bh / a.Hkv, h = bh % a.Hkv;
-    S = a.budgets[b * a.L + layer];
-    M = a.windows[b * a.L + layer];
-    row0 = a.row_off[b * a.L + layer] + (int64_t)h * S;
-    sidx = (layer * a.B + b) * a.Hkv + h;
-    n_old = a.len[sidx];
-  } else {
-    S = a.full_capacity; M = 0;
-    row0 = (int64_t)sl * a.full_capacity;
-    n_old = a.full_len;
-  }
-  const int n = n_old + 1;                                         // rows attended: cache + the new token
-  const int chunk = (((n + C - 1) / C) + 7) & ~7;
-  const int r0 = rank * chunk;
-  const int cnt = max(0, min(n, r0 + chunk) - r0);                 // rows of this CTA
-  const float tau_old = COMPRESS ? a.tau[sidx] : 0.f;
-  const int Tn = a.T < S ? a.T : S;
-
-  // ---- shared memory carve-up (identical in every CTA of the cluster, so peers can address it)
-  extern __shared__ __align__(16) unsigned char dsm[];
-  Xch* xch = reinterpret_cast<Xch*>(dsm);
-  float* red = reinterpret_cast<float*>(dsm + sizeof(Xch));        // [warps][G][D]
-  float* pl = red + kDecWarps * G * D;                              // [G][chunk_cap] logits -> probabilities
-  float* sc = pl + (size_t)G * a.chunk_cap;                         // [chunk_cap] scores
-  float* rn = sc + a.chunk_cap;                                     // [chunk_cap] inverse key norms
-  int* ps = reinterpret_cast<int*>(rn + a.chunk_cap);               // [chunk_cap] positions
-  uint4* newkv = reinterpret_cast<uint4*>(ps + a.chunk_cap);        // [2][LPR] staging of the new token's row
-  uint4* ks = newkv + 2 * LPR;                                      // [res_rows][LPR]
-  __shared__ float s_red[kDecWarps][G];
-  __shared__ unsigned long long s_key[kDecWarps];
-  __shared__ int s_li[kDecWarps];
-  __shared__ float s_fac[G];
-
+  const int sl = blockIdx.x;                    // slice index within the launch
   const T* k_new = k_in + (size_t)sl * D;
   const T* v_new = v_in + (size_t)sl * D;
-  auto k_src = [&](int li) -> const T* {       // global source of local row li
-    const int gi = r0 + li;
-    return gi < n_old ? kpool + (row0 + gi) * D : k_new;
-  };
-  auto v_src = [&](int li) -> const T* {
-    const int gi = r0 + li;
-    return gi < n_old ? vpool + (row0 + gi) * D : v_new;
-  };
+
+  // ---- slice parameters
+  const int per_layer = a.B * a.Hkv;
+  const int layer = a.l0 + sl / per_layer;
+  const int bh = sl % per_layer;
+  const int b = bh / a.Hkv, h = bh % a.Hkv;
+  const int S = a.budgets[b * a.L + layer];
+  const int M = a.windows[b * a.L + layer];
+  const int64_t row0 = a.row_off[b * a.L + layer] + (int64_t)h * slice_stride(S);
+  const int sidx = (layer * a.B + b) * a.Hkv + h;
+  const int n_old = a.len[sidx];
+  const float tau_old = a.tau[sidx];
+  const int n = n_old + 1;                                         // rows attended: cache + the new token
+  const int Tn = a.T < S ? a.T : S;
+  const bool evict = n > S;
+  const int n_st = (n + SR - 1) / SR;                              // stages per pass
+  const int NS = a.stages;
+
+  // ---- shared memory
+  extern __shared__ __align__(128) unsigned char dsm[];
+  uint4* ring = reinterpret_cast<uint4*>(dsm);                       // [stages][SR][LPR]
+  float* red = reinterpret_cast<float*>(dsm);                        // [warps][G][D], aliases the ring once it is drained
+  float* pl = reinterpret_cast<float*>(dsm + (size_t)NS * kStageBytes);   // [G][row_cap] logits -> probabilities
+  float* sc = pl + (size_t)G * a.row_cap;                            // [row_cap] scores
+  float* rn = sc + a.row_cap;                                        // [row_cap] inverse key norms
+  int* ps = reinterpret_cast<int*>(rn + a.row_cap);                  // [row_cap] positions
+  uint4* stash = reinterpret_cast<uint4*>(ps + a.row_cap);           // [2][LPR] value rows of the victim / the neighbour
+  __shared__ unsigned long long s_full[kMaxStages], s_empty[kMaxStages], s_meta;
+  __shared__ float s_red[2][kConsWarps][G];
+  __shared__ unsigned long long s_key[kConsWarps], s_best_key;
+  __shared__ int s_li[kConsWarps], s_best_li;
+  __shared__ int s_timeout;
+
+  if (tid == 0) {
+    // once an anomaly has been recorded (by this or an earlier launch) no wait is attempted any more
+    s_timeout = *reinterpret_cast<volatile uint32_t*>(a.status) != 0u;
+    mbar_init(&s_meta, 1);
+    for (int s = 0; s < NS; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kConsWarps); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  // =========================================================================== producer warp
+  if (warp == kConsWarps) {
+    if (lane == 0) {
+      unsigned long long keep = 0, drop = 0;
+      if (a.l2_hints) {
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
+      }
+      // positions / scores / inverse norms of the cache rows (4 rows = 16 bytes granularity: up to 3 entries
+      // past n_old are read from the slice's padding and overwritten below)
+      const int np4 = (n_old + 3) & ~3;
+      if (np4 > 0) {
+        mbar_expect_tx(&s_meta, (uint32_t)(3 * np4 * 4));
+        bulk_g2s(ps, a.pos + row0, (uint32_t)(np4 * 4), &s_meta);
+        bulk_g2s(sc, a.score + row0, (uint32_t)(np4 * 4), &s_meta);
+        bulk_g2s(rn, a.rnorm + row0, (uint32_t)(np4 * 4), &s_meta);
+      } else {
+        mbar_arrive(&s_meta);
+      }
+      const int n_pass = evict ? 3 : 2;
+      int q = 0;
+      for (int p = 0; p < n_pass; ++p) {
+        const bool is_v = (p == n_pass - 1);
+        const T* pool = is_v ? vpool : kpool;
+        const T* fresh = is_v ? v_new : k_new;
+        const bool hint = a.l2_hints != 0;
+        const unsigned long long pol = (p == 0 && evict) ? keep : drop;
+        for (int s = 0; s < n_st; ++s, ++q) {
+          const int slot = q % NS;
+          if (q >= NS && !s_timeout && !mbar_wait(&s_empty[slot], (uint32_t)(((q / NS) - 1) & 1))) s_timeout = 2;
+          const int a0 = s * SR, a1 = min(n, a0 + SR);
+          const int np = max(0, min(a1, n_old) - a0);                // cache rows of the stage
+          const bool nw = n_old >= a0 && n_old < a1;                 // the new token's row falls into the stage
+          uint4* dst = ring + (size_t)slot * SR * LPR;
+          mbar_expect_tx(&s_full[slot], (uint32_t)((np + (nw ? 1 : 0)) * ROWB));
+          if (np > 0) {
+            if (hint) bulk_g2s_hint(dst, pool + (row0 + a0) * D, (uint32_t)(np * ROWB), &s_full[slot], pol);
+            else bulk_g2s(dst, pool + (row0 + a0) * D, (uint32_t)(np * ROWB), &s_full[slot]);
+          }
+          if (nw) bulk_g2s(dst + (size_t)(n_old - a0) * LPR, fresh, (uint32_t)ROWB, &s_full[slot]);
+        }
+      }
+    }
+    return;
+  }
+
+  // =========================================================================== consumer warps
+  const int grp = tid / LPR, lig = tid % LPR;
+  const unsigned gmask = group_mask<LPR>();
+  int q = 0;                                                         // running stage counter across the passes
 
   // ---- query fragments, pre-scaled by log2(e)/sqrt(d)
   float qf[G][EPV];
@@ -159,133 +247,232 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       for (int e = 0; e < EPV; ++e) qf[g][e] = f[e] * mul;
     }
   }
-  // ---- per-row metadata
-  if (COMPRESS) {
-    for (int li = tid; li < cnt; li += kDecThreads) {
-      const int gi = r0 + li;
-      ps[li] = gi < n_old ? a.pos[row0 + gi] : a.t;
-      sc[li] = gi < n_old ? a.score[row0 + gi] : 0.f;
-      if (gi < n_old) rn[li] = a.rnorm[row0 + gi];                  // the new row's norm is computed in the K pass
+  // the new token's rows, kept by the first row group
+  uint4 knew = make_uint4(0, 0, 0, 0), vnew = make_uint4(0, 0, 0, 0);
+  if (grp == 0) { knew = ld_global_v4(k_new + lig * EPV); vnew = ld_global_v4(v_new + lig * EPV); }
+
+  // ---- pass K: logits
+  float mloc[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) mloc[g] = -INFINITY;
+  for (int s = 0; s < n_st; ++s, ++q) {
+    const int slot = q % NS;
+    if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+    const uint4* st = ring + (size_t)slot * SR * LPR;
+    float dot[G][4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int lr = u * NGRP + grp;
+      float f[EPV];
+      Elem<T>::unpack(s * SR + lr < n ? st[(size_t)lr * LPR + lig] : make_uint4(0, 0, 0, 0), f);
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float x = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) x = fmaf(qf[g][e], f[e], x);
+        dot[g][u] = x;
+      }
     }
-  }
-  // ---- 1. K pass: logits, keep rows in shared memory
-  constexpr int U = 4;
-  for (int li0 = grp; li0 < cnt; li0 += NGRP * U) {
-    uint4 kv[U];
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&s_empty[slot]);
+    const int li = s * SR + (lig / QL) * NGRP + grp;                 // the row whose total this lane receives
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int li = li0 + u * NGRP;
-      if (li < cnt) kv[u] = ld_stream_v4(k_src(li) + lig * EPV);
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int li = li0 + u * NGRP;
-      if (li < cnt) {
-        if (COMPRESS && li < a.res_rows) ks[(size_t)li * LPR + lig] = kv[u];
-        float f[EPV];
-        Elem<T>::unpack(kv[u], f);
-        float dot[G];
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-          float s = 0.f;
-#pragma unroll
-          for (int e = 0; e < EPV; ++e) s = fmaf(qf[g][e], f[e], s);
-          dot[g] = s;
-        }
-#pragma unroll
-        for (int g = 0; g < G; ++g) dot[g] = group_sum<LPR>(dot[g], gmask);
-        if (lig == 0) {
-#pragma unroll
-          for (int g = 0; g < G; ++g) pl[(size_t)g * a.chunk_cap + li] = dot[g];
-        }
-        if (COMPRESS && r0 + li == n_old) {                         // the new token: its norm and a staging copy
-          float ss = 0.f;
-#pragma unroll
-          for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
-          ss = group_sum<LPR>(ss, gmask);
-          if (lig == 0) rn[li] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
-          newkv[lig] = kv[u];
-        }
+    for (int g = 0; g < G; ++g) {
+      const float r = reduce4<LPR>(dot[g][0], dot[g][1], dot[g][2], dot[g][3], lig);
+      if (li < n) {
+        mloc[g] = fmaxf(mloc[g], r);
+        if (lig % QL == 0) pl[(size_t)g * a.row_cap + li] = r;
       }
     }
   }
-  __syncthreads();
-  // ---- local softmax statistics per query head
-  float m_loc[G], l_loc[G];
+  // ---- softmax normaliser, probabilities, accumulated attention (Eq. 6 case 2), victim candidate
+  if (!s_timeout && !mbar_wait(&s_meta, 0)) s_timeout = 2;
+  if (warp == 0) {
+    // the new token's metadata; its inverse norm from the row as stored
+    float f[EPV];
+    Elem<T>::unpack(knew, f);
+    float ss = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
+    ss = warp_sum(ss);                                               // lanes >= LPR hold zeros
+    if (lane == 0) { ps[n_old] = a.t; sc[n_old] = 0.f; rn[n_old] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f; }
+  }
+  float m_all[G], inv_l[G];
   {
-    float mx[G];
 #pragma unroll
-    for (int g = 0; g < G; ++g) mx[g] = -INFINITY;
-    for (int li = tid; li < cnt; li += kDecThreads) {
-#pragma unroll
-      for (int g = 0; g < G; ++g) mx[g] = fmaxf(mx[g], pl[(size_t)g * a.chunk_cap + li]);
-    }
-#pragma unroll
-    for (int g = 0; g < G; ++g) { mx[g] = warp_max(mx[g]); if (lane == 0) s_red[warp][g] = mx[g]; }
-    __syncthreads();
+    for (int g = 0; g < G; ++g) { const float w = warp_max(mloc[g]); if (lane == 0) s_red[0][warp][g] = w; }
+    consumer_sync();                                                 // logits, maxima and the new token's metadata
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      float t = s_red[0][g];
+      float t = s_red[0][0][g];
 #pragma unroll
-      for (int w = 1; w < kDecWarps; ++w) t = fmaxf(t, s_red[w][g]);
-      m_loc[g] = t;
+      for (int w = 1; w < kConsWarps; ++w) t = fmaxf(t, s_red[0][w][g]);
+      m_all[g] = t;
     }
-    __syncthreads();
     float sum[G];
 #pragma unroll
     for (int g = 0; g < G; ++g) sum[g] = 0.f;
-    for (int li = tid; li < cnt; li += kDecThreads) {
+    for (int li = tid; li < n; li += kConsThreads) {
 #pragma unroll
       for (int g = 0; g < G; ++g) {
-        const float p = exp2f(pl[(size_t)g * a.chunk_cap + li] - m_loc[g]);
-        pl[(size_t)g * a.chunk_cap + li] = p;
+        const float p = exp2f(pl[(size_t)g * a.row_cap + li] - m_all[g]);
+        pl[(size_t)g * a.row_cap + li] = p;
         sum[g] += p;
       }
     }
 #pragma unroll
-    for (int g = 0; g < G; ++g) { sum[g] = warp_sum(sum[g]); if (lane == 0) s_red[warp][g] = sum[g]; }
-    __syncthreads();
+    for (int g = 0; g < G; ++g) { const float w = warp_sum(sum[g]); if (lane == 0) s_red[1][warp][g] = w; }
+    consumer_sync();
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       float t = 0.f;
 #pragma unroll
-      for (int w = 0; w < kDecWarps; ++w) t += s_red[w][g];
-      l_loc[g] = t;
+      for (int w = 0; w < kConsWarps; ++w) t += s_red[1][w][g];
+      inv_l[g] = 1.0f / t;
     }
+    unsigned long long my_min = ~0ull; int my_min_li = -1;
+    for (int li = tid; li < n; li += kConsThreads) {                 // each thread revisits the rows it normalised
+      float p = 0.f;
 #pragma unroll
-    for (int g = 0; g < G; ++g)
-      if (tid == g) { xch->m[g] = m_loc[g]; xch->l[g] = l_loc[g]; }
+      for (int g = 0; g < G; ++g) p = fmaf(pl[(size_t)g * a.row_cap + li], inv_l[g], p);
+      const float s_new = sc[li] + p;
+      sc[li] = s_new;
+      if (li < n_old || !evict) a.score[row0 + li] = s_new;          // the new token's score is placed with its row
+      const int pz = ps[li];
+      if (evict && pz >= Tn && pz <= a.t - M) {                      // lowest score, ties -> latest position
+        const unsigned long long key = ((unsigned long long)float_ord(s_new) << 32) | (uint32_t)(0x7fffffff - pz);
+        if (key < my_min) { my_min = key; my_min_li = li; }
+      }
+    }
+    if (evict) block_arg_extreme<true>(my_min, my_min_li, s_key, s_li, &s_best_key, &s_best_li);
+    consumer_sync();
   }
-  cluster_arrive();                                                  // #1 (max, sum) published; completes during the V pass
-  // ---- 2. V pass: un-normalised outputs
+  // ---- victim (Eq. 7-8), pass K': cosine with every other row (Eq. 9), tau_t (Eq. 10), merged key (Eq. 11-12)
+  int vic_li = -1, nn_li = -1;
+  bool merge = false, nn_is_new = false;
+  float w_e = 0.f, w_c = 1.f, rn_slot = 0.f;
+  uint4 kslot = knew;                                                // what goes into the victim's key row
+  if (evict) {
+    vic_li = s_best_li;
+    if (s_best_key == ~0ull) {
+      // nothing may be evicted (S_l < T + M): report, drop the new token, keep the cache as it is.  The producer
+      // still delivers two passes; they are drained without being used.
+      if (tid == 0) report_error(a.status, D2O_ERR_STATE, 0xDEC00000u | (uint32_t)(sl & 0xfffff));
+      for (int s = 0; s < 2 * n_st; ++s, ++q) {
+        const int slot = q % NS;
+        if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_empty[slot]);
+      }
+      return;
+    }
+    const float vic_rn = rn[vic_li];
+    float kvic[EPV];
+    Elem<T>::unpack(ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) + lig * EPV), kvic);
+    unsigned long long best = 0ull; int best_li = -1;
+    for (int s = 0; s < n_st; ++s, ++q) {
+      const int slot = q % NS;
+      if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+      const uint4* st = ring + (size_t)slot * SR * LPR;
+      float dot[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int lr = u * NGRP + grp;
+        float f[EPV];
+        Elem<T>::unpack(s * SR + lr < n ? st[(size_t)lr * LPR + lig] : make_uint4(0, 0, 0, 0), f);
+        float x = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], f[e], x);
+        dot[u] = x;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[slot]);
+      const float r = reduce4<LPR>(dot[0], dot[1], dot[2], dot[3], lig);
+      const int li = s * SR + (lig / QL) * NGRP + grp;
+      if (li < n && lig % QL == 0 && li != vic_li) {                 // max similarity, ties -> earliest position
+        const float u = r * vic_rn * rn[li];
+        const unsigned long long key = ((unsigned long long)float_ord(u) << 32) | (uint32_t)(0x7fffffff - ps[li]);
+        if (key > best) { best = key; best_li = li; }
+      }
+    }
+    block_arg_extreme<false>(best, best_li, s_key, s_li, &s_best_key, &s_best_li);
+    consumer_sync();
+    nn_li = s_best_li;
+    const float mx = ord_float((uint32_t)(s_best_key >> 32));
+    const float tau_new = a.beta * mx + (1.0f - a.beta) * tau_old;
+    const float thr = isnan(a.tau_override) ? tau_new : a.tau_override;
+    merge = mx >= thr;
+    nn_is_new = (nn_li == n_old);
+    const float ew = expf(mx);
+    w_e = ew / (ew + kEuler); w_c = kEuler / (ew + kEuler);
+    if (tid == 0) {
+      a.tau[sidx] = tau_new;
+      atomicAdd(&a.counters[kCntDecodeSteps], 1ull);
+      atomicAdd(&a.counters[kCntEvictions], 1ull);
+      atomicAdd(&a.counters[merge ? kCntMerges : kCntDiscards], 1ull);
+    }
+    rn_slot = rn[n_old];
+    if (warp == 0 && lane < LPR) {
+      // keys are not read any more in this launch: merged key row in place, the new token's key into the victim's row
+      if (merge) {
+        float fk[EPV];
+        Elem<T>::unpack(nn_is_new ? knew : ld_global_v4(kpool + (row0 + nn_li) * D + lane * EPV), fk);
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) fk[e] = w_c * fk[e] + w_e * kvic[e];
+        const uint4 kn = Elem<T>::pack(fk);
+        Elem<T>::unpack(kn, fk);                                     // norm of what is stored
+        float ss = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) ss = fmaf(fk[e], fk[e], ss);
+        ss = group_sum<LPR>(ss, gmask);
+        const float rnew = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+        if (nn_is_new) { kslot = kn; rn_slot = rnew; }
+        else {
+          *reinterpret_cast<uint4*>(kpool + (row0 + nn_li) * D + lane * EPV) = kn;
+          if (lane == 0) a.rnorm[row0 + nn_li] = rnew;
+        }
+      }
+      if (vic_li != n_old) {
+        *reinterpret_cast<uint4*>(kpool + (row0 + vic_li) * D + lane * EPV) = kslot;
+        if (lane == 0) {
+          a.pos[row0 + vic_li] = a.t;
+          a.score[row0 + vic_li] = sc[n_old];
+          a.rnorm[row0 + vic_li] = rn_slot;
+        }
+      }
+    }
+  }
+  // ---- pass V: un-normalised outputs; the value rows of the victim and of the neighbour are picked out of the stream
   {
     float acc[G][EPV];
 #pragma unroll
     for (int g = 0; g < G; ++g)
 #pragma unroll
       for (int e = 0; e < EPV; ++e) acc[g][e] = 0.f;
-    for (int li0 = grp; li0 < cnt; li0 += NGRP * U) {
-      uint4 vv[U];
+    for (int s = 0; s < n_st; ++s, ++q) {
+      const int slot = q % NS;
+      if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+      const uint4* st = ring + (size_t)slot * SR * LPR;
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int li = li0 + u * NGRP;
-        if (li < cnt) vv[u] = ld_stream_v4(v_src(li) + lig * EPV);
-      }
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int li = li0 + u * NGRP;
-        if (li < cnt) {
+      for (int u = 0; u < 4; ++u) {
+        const int lr = u * NGRP + grp;
+        const int li = s * SR + lr;
+        if (li < n) {
+          const uint4 raw = st[(size_t)lr * LPR + lig];
+          if (li == vic_li) stash[lig] = raw;
+          if (li == nn_li) stash[LPR + lig] = raw;
           float f[EPV];
-          Elem<T>::unpack(vv[u], f);
+          Elem<T>::unpack(raw, f);
 #pragma unroll
           for (int g = 0; g < G; ++g) {
-            const float p = pl[(size_t)g * a.chunk_cap + li];
+            const float p = pl[(size_t)g * a.row_cap + li];
 #pragma unroll
             for (int e = 0; e < EPV; ++e) acc[g][e] = fmaf(p, f[e], acc[g][e]);
           }
-          if (COMPRESS && r0 + li == n_old) newkv[LPR + lig] = vv[u];
         }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[slot]);
     }
     // combine the row groups of a warp, then the warps
 #pragma unroll
@@ -295,272 +482,113 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
 #pragma unroll
         for (int e = 0; e < EPV; ++e) acc[g][e] += __shfl_xor_sync(0xffffffffu, acc[g][e], o);
     }
+    consumer_sync();                                                 // the ring is drained: reuse it
     if (lane < LPR) {
 #pragma unroll
       for (int g = 0; g < G; ++g)
 #pragma unroll
         for (int e = 0; e < EPV; ++e) red[((size_t)warp * G + g) * D + lane * EPV + e] = acc[g][e];
     }
-    __syncthreads();
-    for (int i = tid; i < G * D; i += kDecThreads) {
+    consumer_sync();
+    for (int i = tid; i < G * D; i += kConsThreads) {
       float t = 0.f;
 #pragma unroll
-      for (int w = 0; w < kDecWarps; ++w) t += red[(size_t)w * G * D + i];
-      xch->acc[i / D][i % D] = t;
+      for (int w = 0; w < kConsWarps; ++w) t += red[(size_t)w * G * D + i];
+      out[(size_t)sl * G * D + i] = Elem<T>::from_float(t * inv_l[i / D]);
     }
   }
-  cluster_wait();                                                    // #1
-  // ---- 3. global softmax normaliser from the peers' (max, sum)
-  float m_star[G], l_star[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    float ms = -INFINITY;
-    for (int r = 0; r < C; ++r) ms = fmaxf(ms, cluster.map_shared_rank(xch, r)->m[g]);
-    float ls = 0.f;
-    for (int r = 0; r < C; ++r) {
-      const Xch* x = cluster.map_shared_rank(xch, r);
-      ls += x->l[g] * exp2f(x->m[g] - ms);
-    }
-    m_star[g] = ms; l_star[g] = ls;
-  }
-  const bool evict = COMPRESS && (n > S);
-  unsigned long long my_min = ~0ull; int my_min_li = -1;
-  if (COMPRESS) {
-    // accumulated attention (Eq. 6 case 2): add this step's probabilities, summed over the G heads;
-    // victim candidate: lowest score outside sinks and window, ties -> latest position
-    float fac[G];
-#pragma unroll
-    for (int g = 0; g < G; ++g) fac[g] = exp2f(m_loc[g] - m_star[g]) / l_star[g];
-    for (int li = tid; li < cnt; li += kDecThreads) {
-      float p = 0.f;
-#pragma unroll
-      for (int g = 0; g < G; ++g) p = fmaf(pl[(size_t)g * a.chunk_cap + li], fac[g], p);
-      const float s_new = sc[li] + p;
-      sc[li] = s_new;
-      const int pz = ps[li];
-      if (evict && pz >= Tn && pz <= a.t - M) {
-        const unsigned long long key = ((unsigned long long)float_ord(s_new) << 32) | (uint32_t)(0x7fffffff - pz);
-        if (key < my_min) { my_min = key; my_min_li = li; }
-      }
-    }
-    if (evict) block_arg_extreme<true>(my_min, my_min_li, s_key, s_li, &xch->cand_min, &xch->cand_min_li);
-  }
-  cluster_arrive();                                                  // #2 partial outputs (and victim candidates) published
-  const int new_rank = n_old / chunk;                                // CTA that holds the new token's row
-  const int new_li = n_old - new_rank * chunk;
-  if (COMPRESS) {
-    // score write-back overlaps the barrier; the victim's row is overwritten by the new token at the very end
-    for (int li = tid; li < cnt; li += kDecThreads) {
-      const int gi = r0 + li;
-      if (gi < n_old || !evict) a.score[row0 + gi] = sc[li];
-    }
-  }
-  cluster_wait();                                                    // #2
-  if (rank == 0) {
-    for (int i = tid; i < G * D; i += kDecThreads) {
-      const int g = i / D, dd = i % D;
-      float num = 0.f;
-      for (int r = 0; r < C; ++r) {
-        const Xch* x = cluster.map_shared_rank(xch, r);
-        num = fmaf(x->acc[g][dd], exp2f(x->m[g] - m_star[g]), num);
-      }
-      out[((size_t)sl * G + g) * D + dd] = Elem<T>::from_float(num / l_star[g]);
-    }
-  }
+  if (tid == 0 && s_timeout == 2) report_error(a.status, D2O_ERR_TIMEOUT, 0xDEC10000u | (uint32_t)(sl & 0xffff));
   if (!evict) {
-    // append the new token's row (cache not full, or uncompressed mode)
-    if (rank == new_rank && grp == 0) {
-      if (COMPRESS) {
-        *reinterpret_cast<uint4*>(kpool + (row0 + n_old) * D + lig * EPV) = newkv[lig];
-        *reinterpret_cast<uint4*>(vpool + (row0 + n_old) * D + lig * EPV) = newkv[LPR + lig];
-        if (lig == 0) { a.pos[row0 + n_old] = a.t; a.rnorm[row0 + n_old] = rn[new_li]; }
-      } else {
-        *reinterpret_cast<uint4*>(kpool + (row0 + n_old) * D + lig * EPV) = ld_global_v4(k_new + lig * EPV);
-        *reinterpret_cast<uint4*>(vpool + (row0 + n_old) * D + lig * EPV) = ld_global_v4(v_new + lig * EPV);
-      }
+    // the cache is not full yet: append the new token's row
+    if (grp == 0) {
+      *reinterpret_cast<uint4*>(kpool + (row0 + n_old) * D + lig * EPV) = knew;
+      *reinterpret_cast<uint4*>(vpool + (row0 + n_old) * D + lig * EPV) = vnew;
+      if (lig == 0) { a.pos[row0 + n_old] = a.t; a.rnorm[row0 + n_old] = rn[n_old]; }
     }
-    if (COMPRESS && rank == 0 && tid == 0) {
+    if (tid == 0) {
       a.len[sidx] = n;
       atomicAdd(&a.counters[kCntDecodeSteps], 1ull);
     }
-    cluster_arrive();                                                // peers may still read our exchange area
-    cluster_wait();
     return;
   }
-  // ---- 4. victim (Eq. 7-8)
-  unsigned long long kmin = ~0ull; int vic_rank = 0, vic_li = 0;
-  for (int r = 0; r < C; ++r) {
-    const Xch* x = cluster.map_shared_rank(xch, r);
-    const unsigned long long t = x->cand_min;
-    if (t < kmin) { kmin = t; vic_rank = r; vic_li = x->cand_min_li; }
-  }
-  if (kmin == ~0ull) {
-    // nothing may be evicted (S_l < T + M): report, drop the new token, keep the cache as it is
-    if (rank == 0 && tid == 0) report_error(a.status, D2O_ERR_STATE, 0xDEC00000u | (uint32_t)(sl & 0xfffff));
-    cluster_arrive();
-    cluster_wait();
-    return;
-  }
-  const int vic_gi = vic_rank * chunk + vic_li;
-  float kvic[EPV];
-  float vic_rn;
-  {
-    const uint4* pks = cluster.map_shared_rank(ks, vic_rank);
-    const uint4 kv = vic_li < a.res_rows ? pks[(size_t)vic_li * LPR + lig]
-                                         : ld_global_v4((vic_gi < n_old ? kpool + (row0 + vic_gi) * D : k_new) + lig * EPV);
-    Elem<T>::unpack(kv, kvic);
-    vic_rn = cluster.map_shared_rank(rn, vic_rank)[vic_li];
-  }
-  // ---- 5. cosine similarity of the victim with every other row (Eq. 9), arg-max, ties -> earliest position
-  {
-    unsigned long long best = 0ull; int best_li = -1;
-    for (int li = grp; li < cnt; li += NGRP) {
-      if (r0 + li == vic_gi) continue;
-      float f[EPV];
-      const uint4 kv = li < a.res_rows ? ks[(size_t)li * LPR + lig] : ld_global_v4(k_src(li) + lig * EPV);
-      Elem<T>::unpack(kv, f);
-      float s = 0.f;
+  // ---- merged value row (Eq. 11); the new token's value takes the victim's row
+  if (warp == 0 && lane < LPR) {
+    uint4 vslot = vnew;
+    if (merge) {
+      float fv[EPV], vv[EPV];
+      Elem<T>::unpack(stash[LPR + lane], fv);                        // the neighbour's value row (the new token's if it is the neighbour)
+      Elem<T>::unpack(stash[lane], vv);                              // the victim's value row
 #pragma unroll
-      for (int e = 0; e < EPV; ++e) s = fmaf(kvic[e], f[e], s);
-      s = group_sum<LPR>(s, gmask);
-      const float u = s * vic_rn * rn[li];
-      const unsigned long long key = ((unsigned long long)float_ord(u) << 32) | (uint32_t)(0x7fffffff - ps[li]);
-      if (key > best) { best = key; best_li = li; }
+      for (int e = 0; e < EPV; ++e) fv[e] = w_c * fv[e] + w_e * vv[e];
+      const uint4 vn = Elem<T>::pack(fv);
+      if (nn_is_new) vslot = vn;
+      else *reinterpret_cast<uint4*>(vpool + (row0 + nn_li) * D + lane * EPV) = vn;
     }
-    block_arg_extreme<false>(best, best_li, s_key, s_li, &xch->cand_max, &xch->cand_max_li);
-  }
-  cluster_arrive();                                                  // #3 neighbour candidates published
-  cluster_wait();
-  unsigned long long kmax = 0ull; int nn_rank = 0, nn_li = 0;
-  for (int r = 0; r < C; ++r) {
-    const Xch* x = cluster.map_shared_rank(xch, r);
-    const unsigned long long t = x->cand_max;
-    if (t > kmax) { kmax = t; nn_rank = r; nn_li = x->cand_max_li; }
-  }
-  const float mx = ord_float((uint32_t)(kmax >> 32));
-  // ---- 6. EMA threshold (Eq. 10) and merge (Eq. 11-12)
-  const float tau_new = a.beta * mx + (1.0f - a.beta) * tau_old;
-  const float thr = isnan(a.tau_override) ? tau_new : a.tau_override;
-  const bool merge = mx >= thr;
-  if (rank == 0 && tid == 0) {
-    a.tau[sidx] = tau_new;
-    atomicAdd(&a.counters[kCntDecodeSteps], 1ull);
-    atomicAdd(&a.counters[kCntEvictions], 1ull);
-    atomicAdd(&a.counters[merge ? kCntMerges : kCntDiscards], 1ull);
-  }
-  if (merge && rank == nn_rank && grp == 0) {
-    const int lj = nn_li;
-    const bool is_new = (r0 + lj == n_old);
-    const float ew = expf(mx);
-    const float w_e = ew / (ew + kEuler), w_c = kEuler / (ew + kEuler);
-    float fk[EPV], fv[EPV], vv[EPV];
-    const uint4 kcur = is_new ? newkv[lig]
-                              : (lj < a.res_rows ? ks[(size_t)lj * LPR + lig] : ld_global_v4(k_src(lj) + lig * EPV));
-    Elem<T>::unpack(kcur, fk);
-    Elem<T>::unpack(is_new ? newkv[LPR + lig] : ld_global_v4(v_src(lj) + lig * EPV), fv);
-    // the victim's value row is still in place: its slot is overwritten only after the last barrier
-    Elem<T>::unpack(ld_global_v4((vic_gi < n_old ? vpool + (row0 + vic_gi) * D : v_new) + lig * EPV), vv);
-#pragma unroll
-    for (int e = 0; e < EPV; ++e) { fk[e] = w_c * fk[e] + w_e * kvic[e]; fv[e] = w_c * fv[e] + w_e * vv[e]; }
-    const uint4 kn = Elem<T>::pack(fk), vn = Elem<T>::pack(fv);
-    Elem<T>::unpack(kn, fk);                                         // norm of what is stored
-    float ss = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPV; ++e) ss = fmaf(fk[e], fk[e], ss);
-    ss = group_sum<LPR>(ss, gmask);
-    const float rnew = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
-    if (is_new) { newkv[lig] = kn; newkv[LPR + lig] = vn; }
-    else {
-      *reinterpret_cast<uint4*>(kpool + (row0 + r0 + lj) * D + lig * EPV) = kn;
-      *reinterpret_cast<uint4*>(vpool + (row0 + r0 + lj) * D + lig * EPV) = vn;
-      if (lig == 0) a.rnorm[row0 + r0 + lj] = rnew;
-    }
-    if (lig == 0) rn[lj] = rnew;
-  }
-  cluster_arrive();                                                  // #4 all reads of peer memory and of the victim's row are done
-  cluster_wait();
-  // ---- 7. the new token takes the victim's row
-  if (rank == new_rank && vic_gi != n_old && grp == 0) {
-    *reinterpret_cast<uint4*>(kpool + (row0 + vic_gi) * D + lig * EPV) = newkv[lig];
-    *reinterpret_cast<uint4*>(vpool + (row0 + vic_gi) * D + lig * EPV) = newkv[LPR + lig];
-    if (lig == 0) {
-      a.pos[row0 + vic_gi] = a.t;
-      a.score[row0 + vic_gi] = sc[new_li];
-      a.rnorm[row0 + vic_gi] = rn[new_li];
-    }
+    if (vic_li != n_old) *reinterpret_cast<uint4*>(vpool + (row0 + vic_li) * D + lane * EPV) = vslot;
   }
 }
 
 // ------------------------------------------------------------------------------------ launch
-template <typename T, int D, int G, bool COMPRESS>
-static cudaError_t launch_one(const DecodeArgs& a, int n_slices, int C, const void* q, const void* k, const void* v,
+static size_t smem_bytes(int row_cap, int stages, int G, int row_bytes) {
+  return (size_t)stages * kStageBytes + (size_t)(G + 3) * row_cap * 4 + 2 * (size_t)row_bytes;
+}
+
+template <typename T, int D, int G>
+static cudaError_t launch_one(const DecodeArgs& a, int n_slices, const void* q, const void* k, const void* v,
                               void* out, void* kpool, void* vpool, cudaStream_t st) {
-  constexpr int LPR = D * sizeof(T) / 16;
-  const size_t smem = sizeof(Exchange<G, D>) + (size_t)kDecWarps * G * D * 4 + (size_t)(G + 3) * a.chunk_cap * 4 +
-                      (size_t)2 * LPR * 16 + (size_t)a.res_rows * LPR * 16;
-  auto kern = decode_kernel<T, D, G, COMPRESS>;
+  const size_t smem = smem_bytes(a.row_cap, a.stages, G, D * (int)sizeof(T));
+  auto kern = decode_kernel<T, D, G>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(n_slices * C));
-  cfg.blockDim = dim3(kDecThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, a, (const T*)q, (const T*)k, (const T*)v, (T*)out, (T*)kpool, (T*)vpool);
+  kern<<<n_slices, kDecThreads, smem, st>>>(a, (const T*)q, (const T*)k, (const T*)v, (T*)out, (T*)kpool, (T*)vpool);
+  return cudaGetLastError();
 }
 
-template <typename T, int D, bool COMPRESS>
-static cudaError_t launch_g(int G, const DecodeArgs& a, int n_slices, int C, const void* q, const void* k,
+template <typename T, int D>
+static cudaError_t launch_g(int G, const DecodeArgs& a, int n_slices, const void* q, const void* k,
                             const void* v, void* out, void* kpool, void* vpool, cudaStream_t st) {
   switch (G) {
-    case 1: return launch_one<T, D, 1, COMPRESS>(a, n_slices, C, q, k, v, out, kpool, vpool, st);
-    case 2: return launch_one<T, D, 2, COMPRESS>(a, n_slices, C, q, k, v, out, kpool, vpool, st);
-    case 4: return launch_one<T, D, 4, COMPRESS>(a, n_slices, C, q, k, v, out, kpool, vpool, st);
-    default: return launch_one<T, D, 8, COMPRESS>(a, n_slices, C, q, k, v, out, kpool, vpool, st);
+    case 1: return launch_one<T, D, 1>(a, n_slices, q, k, v, out, kpool, vpool, st);
+    case 2: return launch_one<T, D, 2>(a, n_slices, q, k, v, out, kpool, vpool, st);
+    case 4: return launch_one<T, D, 4>(a, n_slices, q, k, v, out, kpool, vpool, st);
+    default: return launch_one<T, D, 8>(a, n_slices, q, k, v, out, kpool, vpool, st);
   }
 }
 
-template <bool COMPRESS>
-static cudaError_t launch_any(int dtype, int d, int G, const DecodeArgs& a, int n_slices, int C, const void* q,
-                              const void* k, const void* v, void* out, void* kpool, void* vpool, cudaStream_t st) {
-  if (dtype == D2O_F32)
-    return d == 64 ? launch_g<float, 64, COMPRESS>(G, a, n_slices, C, q, k, v, out, kpool, vpool, st)
-                   : launch_g<float, 128, COMPRESS>(G, a, n_slices, C, q, k, v, out, kpool, vpool, st);
-  if (dtype == D2O_F16)
-    return d == 64 ? launch_g<__half, 64, COMPRESS>(G, a, n_slices, C, q, k, v, out, kpool, vpool, st)
-                   : launch_g<__half, 128, COMPRESS>(G, a, n_slices, C, q, k, v, out, kpool, vpool, st);
-  return d == 64 ? launch_g<__nv_bfloat16, 64, COMPRESS>(G, a, n_slices, C, q, k, v, out, kpool, vpool, st)
-                 : launch_g<__nv_bfloat16, 128, COMPRESS>(G, a, n_slices, C, q, k, v, out, kpool, vpool, st);
-}
-
-// Picks the cluster size and the shared-memory split for `max_rows` rows per slice.
-static bool plan(int max_rows, int row_bytes, int G, int D, int want_cluster, bool resident, int n_slices, int* C_out,
-                 int* chunk_cap, int* res_rows) {
-  const int fixed = 2048 + G * D * 4 + kDecWarps * G * D * 4 + 1024;      // exchange area + reduction buffer + slack
-  const int budget = 200 * 1024;
-  int C = want_cluster;
-  if (C == 0) {
-    // smallest cluster that keeps all K rows resident in <= ~72 KB per CTA (three CTAs per SM), but enough CTAs
-    // to cover the machine when there are few slices
-    C = 1;
-    while (C < kMaxCluster) {
-      const int chunk = (((max_rows + C - 1) / C) + 7) & ~7;
-      const long need = fixed + (long)chunk * ((G + 3) * 4 + (resident ? row_bytes : 0));
-      if (need <= 72 * 1024 && (long)n_slices * C >= 2 * 148) break;
-      C *= 2;
+// Ring depth for `max_rows` rows per slice: the deepest ring that still lets the preferred number of CTAs share an SM.
+static bool plan(int max_rows, int row_bytes, int G, int D, int want_stages, int* row_cap, int* stages_out) {
+  const long sm_total = 227 * 1024;
+  const int cap = (max_rows + 7) & ~7;
+  const int min_stages = max(2, (kConsWarps * G * D * 4 + kStageBytes - 1) / kStageBytes);   // the ring doubles as `red`
+  const long fixed = (long)(G + 3) * cap * 4 + 2L * row_bytes + 2048;                         // + static shared memory
+  int stages = want_stages;
+  if (stages <= 0) {
+    // three CTAs per SM with at least three stages each if the per-row arrays allow it, else two, else one
+    stages = 0;
+    const int tiers[3] = {3, 2, 1};
+    for (int ti = (G <= 2 ? 0 : 1); ti < 3 && stages == 0; ++ti) {
+      const long room = sm_total / tiers[ti] - 1024 - fixed;
+      const int fit = (int)(room / kStageBytes);
+      if (fit >= max(3, min_stages) || (tiers[ti] == 1 && fit >= min_stages)) stages = fit;
     }
+    if (stages == 0) return false;
+    if (stages > 4) stages = 4;                                      // deeper rings only cost occupancy
+    if (stages < min_stages) stages = min_stages;
   }
-  const int chunk = (((max_rows + C - 1) / C) + 7) & ~7;
-  long meta = fixed + (long)chunk * (G + 3) * 4;
-  if (meta > budget) return false;
-  long rr = resident ? (budget - meta) / row_bytes : 0;
-  if (rr > chunk) rr = chunk;
-  *C_out = C; *chunk_cap = chunk; *res_rows = (int)rr;
+  if (stages < min_stages || stages > kMaxStages) return false;
+  if (fixed + (long)stages * kStageBytes > sm_total - 1024) return false;
+  *row_cap = cap; *stages_out = stages;
   return true;
+}
+
+int decode_max_rows(int row_bytes, int group, int d_head) {
+  int lo = 0, hi = 1 << 20;                                          // largest row count for which a plan exists
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) / 2;
+    int cap, st;
+    if (plan(mid, row_bytes, group, d_head, 0, &cap, &st)) lo = mid; else hi = mid - 1;
+  }
+  return lo;
 }
 
 cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const void* k, const void* v, void* out,
@@ -578,6 +606,7 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   a.L = L; a.l0 = l0; a.B = B; a.Hkv = g.n_kv_heads; a.T = g.n_sink;
   a.t = g.prompt_len + c->layer_steps[l0];
   a.beta = g.beta; a.tau_override = g.tau_override;
+  a.l2_hints = c->decode_l2_hints;
   int max_rows = 0;
   for (int l = l0; l < l1; ++l)
     for (int b = 0; b < B; ++b) {
@@ -586,30 +615,22 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
       max_rows = max(max_rows, len + 1);
     }
   const int n_slices = (l1 - l0) * B * g.n_kv_heads;
-  int C, chunk_cap, res_rows;
-  if (!plan(max_rows, g.d_head * c->elem_size, c->group, g.d_head, c->decode_cluster, !c->decode_nonresident, n_slices,
-            &C, &chunk_cap, &res_rows)) {
+  int row_cap, stages;
+  if (!plan(max_rows, g.d_head * c->elem_size, c->group, g.d_head, c->decode_stages, &row_cap, &stages)) {
     *why = D2O_ERR_UNSUPPORTED;
     return cudaSuccess;
   }
-  a.chunk_cap = chunk_cap; a.res_rows = res_rows;
-  return launch_any<true>(g.dtype, g.d_head, c->group, a, n_slices, C, q, k, v, out, S + c->lay.kpool,
-                          S + c->lay.vpool, st);
-}
-
-cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int capacity, int len, void* kc, void* vc,
-                               const void* q, const void* k, const void* v, void* out, cudaStream_t st,
-                               d2o_status* why) {
-  DecodeArgs a = {};
-  a.full_capacity = capacity; a.full_len = len;
-  int C, chunk_cap, res_rows;
-  const int esz = dtype == D2O_F32 ? 4 : 2;
-  if (!plan(len + 1, d * esz, group, d, 0, false, n_slices, &C, &chunk_cap, &res_rows)) {
-    *why = D2O_ERR_UNSUPPORTED;
-    return cudaSuccess;
-  }
-  a.chunk_cap = chunk_cap; a.res_rows = 0;
-  return launch_any<false>(dtype, d, group, a, n_slices, C, q, k, v, out, kc, vc, st);
+  a.row_cap = row_cap; a.stages = stages;
+  void* kpool = S + c->lay.kpool; void* vpool = S + c->lay.vpool;
+  const int G = c->group;
+  if (g.dtype == D2O_F32)
+    return g.d_head == 64 ? launch_g<float, 64>(G, a, n_slices, q, k, v, out, kpool, vpool, st)
+                          : launch_g<float, 128>(G, a, n_slices, q, k, v, out, kpool, vpool, st);
+  if (g.dtype == D2O_F16)
+    return g.d_head == 64 ? launch_g<__half, 64>(G, a, n_slices, q, k, v, out, kpool, vpool, st)
+                          : launch_g<__half, 128>(G, a, n_slices, q, k, v, out, kpool, vpool, st);
+  return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, a, n_slices, q, k, v, out, kpool, vpool, st)
+                        : launch_g<__nv_bfloat16, 128>(G, a, n_slices, q, k, v, out, kpool, vpool, st);
 }
 
 }  // namespace d2o

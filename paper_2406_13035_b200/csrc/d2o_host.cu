@@ -58,7 +58,8 @@ static d2o_status validate(const d2o_config* c, int64_t* total_budget, int* max_
   if (c->min_budget < 1 || c->min_budget < c->n_sink + 1 || c->min_budget > maxb) return D2O_ERR_INVALID_ARG;
   double tot = floor((double)c->rho * (double)c->n_layers * (double)c->prompt_len + 0.5);
   if (tot < (double)c->n_layers * c->min_budget || tot > (double)c->n_layers * maxb) return D2O_ERR_INVALID_ARG;
-  if (maxb + 1 > 8 * 8192) return D2O_ERR_UNSUPPORTED;   // decode kernel: one cluster (<= 8 CTAs) per slice
+  // decode kernel: the keys of one slice stay in the shared memory of one cluster
+  if (maxb + 1 > decode_max_rows(c->d_head * elem_size_of(c->dtype), g, c->d_head)) return D2O_ERR_UNSUPPORTED;
   *total_budget = (int64_t)tot;
   *max_budget = maxb;
   return D2O_OK;
@@ -67,7 +68,7 @@ static d2o_status validate(const d2o_config* c, int64_t* total_budget, int* max_
 static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, Layout* l, ScratchLayout* s) {
   const size_t B = c->batch, L = c->n_layers, Hq = c->n_q_heads, Hkv = c->n_kv_heads, P = c->prompt_len;
   const size_t d = c->d_head, e = elem_size_of(c->dtype);
-  const size_t rows = B * Hkv * (size_t)total_budget;
+  const size_t rows = B * Hkv * ((size_t)total_budget + 7 * L);     // every slice starts at a multiple of 8 rows
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
   l->status = take(16);
@@ -128,8 +129,9 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
   c->elem_size = elem_size_of(cfg->dtype);
   c->max_budget = maxb;
   c->total_budget = tot;
-  c->pool_rows = (int64_t)cfg->batch * cfg->n_kv_heads * tot;
+  c->pool_rows = (int64_t)cfg->batch * cfg->n_kv_heads * (tot + 7 * (int64_t)cfg->n_layers);
   c->lay = l; c->slay = s;
+  c->decode_l2_hints = 1;
   c->state = (char*)state; c->scratch = (char*)scratch;
   c->state_bytes = state_bytes; c->scratch_bytes = scratch_bytes;
   const size_t BL = (size_t)cfg->batch * cfg->n_layers;
@@ -204,7 +206,7 @@ extern "C" d2o_status d2o_layer_budgets(d2o_ctx* c, int32_t* budgets_host, void*
   CUDA_TRY(cudaStreamSynchronize(st));
   // the device computed offsets for the pool; make sure they fit what the caller gave us
   for (size_t i = 0; i < BL; ++i) {
-    int64_t end = c->h_row_off[i] + (int64_t)g.n_kv_heads * c->h_budgets[i];
+    int64_t end = c->h_row_off[i] + (int64_t)g.n_kv_heads * slice_stride(c->h_budgets[i]);
     if (c->h_budgets[i] < 1 || c->h_budgets[i] > c->max_budget || c->h_row_off[i] < 0 || end > c->pool_rows)
       return D2O_ERR_STATE;
   }
@@ -332,12 +334,11 @@ extern "C" d2o_status d2o_get_stats(d2o_ctx* c, d2o_stats* out, void* stream) {
   return D2O_OK;
 }
 
-extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_cluster, int32_t reserved) {
+extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t decode_l2_hints) {
   if (!c) return D2O_ERR_INVALID_ARG;
-  if (reserved < 0 || reserved > 1) return D2O_ERR_INVALID_ARG;
-  if (decode_cluster != 0 && decode_cluster != 1 && decode_cluster != 2 && decode_cluster != 4 && decode_cluster != 8)
-    return D2O_ERR_INVALID_ARG;
-  c->decode_cluster = decode_cluster;
-  c->decode_nonresident = reserved;
+  if (decode_stages < 0 || decode_stages > 12) return D2O_ERR_INVALID_ARG;
+  if (decode_l2_hints < 0 || decode_l2_hints > 1) return D2O_ERR_INVALID_ARG;
+  c->decode_stages = decode_stages;
+  c->decode_l2_hints = decode_l2_hints;
   return D2O_OK;
 }

@@ -71,7 +71,7 @@ select_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
   const int S = a.budgets[b * a.L + a.layer];
   const int Tn = a.T < S ? a.T : S;
   const int M = a.windows[b * a.L + a.layer];
-  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * S;
+  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
   const int sidx = (a.layer * a.B + b) * a.Hkv + h;
   float* keys = a.keys_in_smem ? reinterpret_cast<float*>(sel_smem) : a.keys_spill + (size_t)slice * P;
   // group score: sum over the G query heads of this KV head, fixed order (Eq. 6 case 1)
@@ -193,7 +193,7 @@ similarity_kernel(SimArgs a, const T* __restrict__ K, const T* __restrict__ kpoo
   const int Le = a.P - S;
   const int i0 = blockIdx.x * kSimTile;
   if (Le <= 0 || i0 >= Le) return;
-  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * S;
+  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
   const T* Ks = K + (size_t)slice * a.P * D;
   const int32_t* ev = a.evict_idx + (size_t)slice * a.P;
   constexpr int EPV = Elem<T>::kPerVec;
@@ -401,7 +401,7 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   const int32_t* start = a.seg_start + (size_t)slice * a.seg_stride;
   const int s0 = start[j], s1 = start[j + 1];
   if (s1 == s0) return;                              // nothing merged: the row stays bit-identical
-  const int64_t row = a.row_off[b * a.L + a.layer] + (int64_t)h * S + j;
+  const int64_t row = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S) + j;
   const int32_t* items = a.seg_items + (size_t)slice * a.P;
   const int32_t* ev = a.evict_idx + (size_t)slice * a.P;
   const float* mx = a.evict_mx + (size_t)slice * a.P;

@@ -314,7 +314,7 @@ __global__ void budget_kernel(const double* __restrict__ density, int B, int L, 
   if (threadIdx.x == 0 && row_off) {                       // cache rows laid out layer-major, then sequence
     long long o = 0;
     for (int l = 0; l < L; ++l)
-      for (int b = 0; b < B; ++b) { row_off[b * L + l] = o; o += (long long)Hkv * budgets[b * L + l]; }
+      for (int b = 0; b < B; ++b) { row_off[b * L + l] = o; o += (long long)Hkv * slice_stride(budgets[b * L + l]); }
   }
 }
 
