@@ -43,7 +43,8 @@ typedef enum {
   D2O_ERR_WORKSPACE = 3,   /* state or scratch too small / misaligned */
   D2O_ERR_STATE = 4,       /* call out of order (e.g. compress before budgets) */
   D2O_ERR_CUDA = 5,        /* a CUDA runtime call failed; see d2o_last_cuda_error() */
-  D2O_ERR_TIMEOUT = 6
+  D2O_ERR_TIMEOUT = 6,
+  D2O_ERR_TOO_LARGE = 7    /* problem exceeds the fixed capacity of an allocation-free entry point */
 } d2o_status;
 
 typedef enum { D2O_F32 = 0, D2O_F16 = 1, D2O_BF16 = 2 } d2o_dtype;
@@ -170,6 +171,34 @@ d2o_status d2o_full_decode_step(int32_t dtype, int32_t d_head, int32_t n_slices,
                                 int32_t capacity, int32_t len, void* k_cache, void* v_cache,
                                 const void* q, const void* k, const void* v, void* out,
                                 void* stream);
+
+/* Allocation-free variant of d2o_layer_stats (the paper has no counterpart: this entry point
+ * exists for callers that cannot allocate device memory).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits, for example inside a serving
+ * process whose memory pool has already claimed the whole device, in a plugin that is handed
+ * tensors but no allocator, or between the steps of a latency-critical loop where an allocation
+ * would synchronise the device.  d2o_layer_stats needs a scratch buffer for the softmax row
+ * normalisers of the prompt attention; here that buffer is a fixed array of
+ * D2O_STATIC_LSE_FLOATS floats (4 MiB) that is part of the library image, so every GPU that
+ * loads the library carries it until the process exits.  No context, no workspace: the caller
+ * passes the inputs and the outputs only.
+ *
+ *   Q DEVICE [B, Hq, P, d], K DEVICE [B, Hkv, P, d] in `dtype`;
+ *   colsum DEVICE float [B, Hq, P] (out: column sums of the causal prompt attention, Eq. 4);
+ *   density DEVICE double [B, Hq] (out: F_v = Var(colsum) per query head).
+ *
+ * Limit: batch * n_q_heads * prompt_len <= D2O_STATIC_LSE_FLOATS, else D2O_ERR_TOO_LARGE and
+ * nothing is launched.  The call neither allocates nor frees device memory.
+ * The first call on each device looks up the device address of the array (one runtime query,
+ * made with that device current); make that first call outside of any stream capture.
+ * All calls share the one array: it is fully rewritten by each call before it is read, so
+ * nothing needs clearing, but two calls whose work overlaps on the GPU (different streams)
+ * race on it.  Asynchronous on `stream` like the other calls. */
+#define D2O_STATIC_LSE_FLOATS (1u << 20)
+d2o_status d2o_layer_stats_static(int32_t dtype, int32_t d_head, int32_t batch, int32_t n_q_heads,
+                                  int32_t n_kv_heads, int32_t prompt_len, const void* Q, const void* K,
+                                  float* colsum, double* density, void* stream);
 
 d2o_status d2o_get_view(d2o_ctx* ctx, int32_t layer, d2o_view* out);
 /* Copies the counters to HOST memory; synchronises `stream`. */

@@ -25,8 +25,9 @@ EXPORTS = [
     "d2o_status_string", "d2o_last_cuda_error", "d2o_workspace_size", "d2o_create", "d2o_destroy",
     "d2o_layer_stats", "d2o_layer_budgets", "d2o_budgets_from_density", "d2o_prefill_compress",
     "d2o_decode_step", "d2o_decode_step_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
-    "d2o_set_tuning",
+    "d2o_set_tuning", "d2o_layer_stats_static",
 ]
+STATIC_LSE_FLOATS = 1 << 20      # D2O_STATIC_LSE_FLOATS of include/d2o.h
 
 
 class D2OConfig(C.Structure):
@@ -89,6 +90,7 @@ def load_library() -> C.CDLL:
     lib.d2o_get_view.argtypes = [vp, i32, C.POINTER(D2OView)]
     lib.d2o_get_stats.argtypes = [vp, C.POINTER(D2OStats), vp]
     lib.d2o_set_tuning.argtypes = [vp, i32, i32]
+    lib.d2o_layer_stats_static.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("d2o_status_string", "d2o_last_cuda_error", "d2o_destroy"):
             getattr(lib, name).restype = C.c_int
@@ -294,3 +296,21 @@ def d2o_full_decode_step(k_cache: torch.Tensor, v_cache: torch.Tensor, length: i
     _check(lib.d2o_full_decode_step(DTYPE_CODE[k_cache.dtype], d, n_slices, G, capacity, length, _ptr(k_cache),
                                     _ptr(v_cache), _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream()),
            "d2o_full_decode_step")
+
+
+def d2o_layer_stats_static(Q: torch.Tensor, K: torch.Tensor, colsum: torch.Tensor, density: torch.Tensor):
+    """Allocation-free column sums and densities of one layer's prompt attention.
+
+    For callers that must not allocate device memory while the library works (a serving process
+    whose pool owns the whole GPU, a plugin without an allocator): the library's only scratch is
+    a fixed 4 MiB array inside its own image.  The caller provides every tensor, outputs included:
+    Q [B, Hq, P, d], K [B, Hkv, P, d], colsum float32 [B, Hq, P], density float64 [B, Hq].
+    Raises D2OError (status 7) if B * Hq * P exceeds STATIC_LSE_FLOATS.  Calls that overlap on the
+    GPU share the scratch array and race; make the first call on a device outside stream capture."""
+    lib = load_library()
+    B, Hq, P, d = Q.shape
+    Hkv = K.shape[1]
+    assert colsum.dtype == torch.float32 and tuple(colsum.shape) == (B, Hq, P)
+    assert density.dtype == torch.float64 and tuple(density.shape) == (B, Hq)
+    _check(lib.d2o_layer_stats_static(DTYPE_CODE[Q.dtype], d, B, Hq, Hkv, P, _ptr(Q), _ptr(K), _ptr(colsum),
+                                      _ptr(density), _stream()), "d2o_layer_stats_static")

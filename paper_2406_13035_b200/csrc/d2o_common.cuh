@@ -184,6 +184,9 @@ cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int ca
 // largest number of rows (cache + the new token) of one slice the decode kernel can keep resident
 int decode_max_rows(int row_bytes, int group, int d_head);
 
+// remembers the text of a failed CUDA runtime call for d2o_last_cuda_error(); returns D2O_ERR_CUDA
+d2o_status record_cuda_error(cudaError_t e, const char* where);
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace d2o

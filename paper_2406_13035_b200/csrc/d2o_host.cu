@@ -12,8 +12,11 @@ using namespace d2o;
 static thread_local char g_cuda_err[256] = "";
 
 static d2o_status cuda_fail(cudaError_t e, const char* where) {
-  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", where, cudaGetErrorString(e));
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%.160s: %.80s", where, cudaGetErrorString(e));
   return D2O_ERR_CUDA;
+}
+namespace d2o {
+d2o_status record_cuda_error(cudaError_t e, const char* where) { return cuda_fail(e, where); }
 }
 #define CUDA_TRY(expr)                                   \
   do {                                                   \
@@ -30,6 +33,7 @@ extern "C" const char* d2o_status_string(d2o_status s) {
     case D2O_ERR_STATE: return "call out of order";
     case D2O_ERR_CUDA: return "CUDA runtime error";
     case D2O_ERR_TIMEOUT: return "device-side wait ran out";
+    case D2O_ERR_TOO_LARGE: return "problem exceeds the fixed capacity of the allocation-free entry point";
   }
   return "unknown status";
 }

@@ -371,4 +371,69 @@ cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, 
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------ allocation-free variant
+// Scratch for the row normalisers of d2o_layer_stats_static: part of the library image, one copy per GPU.
+static __device__ __align__(256) float g_static_lse[D2O_STATIC_LSE_FLOATS];
+constexpr int kMaxDevices = 64;
+static float* g_static_lse_addr[kMaxDevices];        // device address of g_static_lse, per device (host-side cache)
+
+template <typename T, int D>
+static cudaError_t run_stats_static(const void* Q, const void* K, float* lse_buf, float* colsum, double* density, int B,
+                                    int Hq, int group, int P, cudaStream_t st) {
+  const int nT = (P + kTile - 1) / kTile;
+  dim3 grid(nT, B * Hq);
+  const size_t sm = (size_t)2 * D * kTile * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(lse_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+  if (e != cudaSuccess) return e;
+  lse_kernel<T, D><<<grid, kStatThreads, sm, st>>>((const T*)Q, (const T*)K, lse_buf, P, Hq, group);
+  const size_t sm2 = sm + kTile * sizeof(float) + 16 * kTile * sizeof(double);
+  e = cudaFuncSetAttribute(colsum_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
+  if (e != cudaSuccess) return e;
+  colsum_kernel<T, D><<<grid, kStatThreads, sm2, st>>>((const T*)Q, (const T*)K, lse_buf, colsum, P, Hq, group);
+  density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, 1, 0);
+  return cudaGetLastError();
+}
+
 }  // namespace d2o
+
+extern "C" d2o_status d2o_layer_stats_static(int32_t dtype, int32_t d_head, int32_t batch, int32_t n_q_heads,
+                                             int32_t n_kv_heads, int32_t prompt_len, const void* Q, const void* K,
+                                             float* colsum, double* density, void* stream) {
+  using namespace d2o;
+  if (dtype != D2O_F32 && dtype != D2O_F16 && dtype != D2O_BF16) return D2O_ERR_UNSUPPORTED;
+  if (d_head != 64 && d_head != 128) return D2O_ERR_UNSUPPORTED;
+  if (batch < 1 || n_q_heads < 1 || n_kv_heads < 1 || prompt_len < 1 || n_q_heads % n_kv_heads != 0)
+    return D2O_ERR_INVALID_ARG;
+  auto aligned16 = [](const void* p) { return p && (((uintptr_t)p & 15) == 0); };
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(colsum) || !density || ((uintptr_t)density & 7)) return D2O_ERR_INVALID_ARG;
+  if ((unsigned long long)batch * n_q_heads * prompt_len > (unsigned long long)D2O_STATIC_LSE_FLOATS)
+    return D2O_ERR_TOO_LARGE;
+  // set-up, once per device: in host code `g_static_lse` is only a handle, the kernels need its device address
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return record_cuda_error(e, "cudaGetDevice");
+  if (dev < 0 || dev >= kMaxDevices) return D2O_ERR_UNSUPPORTED;
+  float* lse_buf = __atomic_load_n(&g_static_lse_addr[dev], __ATOMIC_ACQUIRE);
+  if (!lse_buf) {
+    e = cudaGetSymbolAddress((void**)&lse_buf, g_static_lse);
+    if (e != cudaSuccess || !lse_buf) return record_cuda_error(e, "cudaGetSymbolAddress(g_static_lse)");
+    __atomic_store_n(&g_static_lse_addr[dev], lse_buf, __ATOMIC_RELEASE);     // every thread would store the same value
+  }
+  const int group = n_q_heads / n_kv_heads;
+  cudaStream_t st = (cudaStream_t)stream;
+  switch (dtype) {
+    case D2O_F32:
+      e = d_head == 64 ? run_stats_static<float, 64>(Q, K, lse_buf, colsum, density, batch, n_q_heads, group, prompt_len, st)
+                       : run_stats_static<float, 128>(Q, K, lse_buf, colsum, density, batch, n_q_heads, group, prompt_len, st);
+      break;
+    case D2O_F16:
+      e = d_head == 64 ? run_stats_static<__half, 64>(Q, K, lse_buf, colsum, density, batch, n_q_heads, group, prompt_len, st)
+                       : run_stats_static<__half, 128>(Q, K, lse_buf, colsum, density, batch, n_q_heads, group, prompt_len, st);
+      break;
+    default:
+      e = d_head == 64 ? run_stats_static<__nv_bfloat16, 64>(Q, K, lse_buf, colsum, density, batch, n_q_heads, group, prompt_len, st)
+                       : run_stats_static<__nv_bfloat16, 128>(Q, K, lse_buf, colsum, density, batch, n_q_heads, group, prompt_len, st);
+  }
+  if (e != cudaSuccess) return record_cuda_error(e, "d2o_layer_stats_static launch");
+  return D2O_OK;
+}
