@@ -42,6 +42,7 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--stages", type=int, default=0, help="stages of the decode kernel's ring (0 = auto)")
     ap.add_argument("--no-l2-hints", action="store_true", help="decode kernel: copies without L2 eviction hints")
+    ap.add_argument("--ffma-similarity", action="store_true", help="prompt-stage similarity on the FFMA kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers-per-call", type=int, default=0)
@@ -126,10 +127,10 @@ def run_ours(args, wl, rank, world, device):
     cfg = B.make_config(n_layers=wl.n_layers, batch=wl.batch, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
                         d_head=wl.d_head, dtype=wl.dtype, prompt_len=wl.prompt_len, max_new_tokens=nd, rho=wl.rho,
                         n_sink=wl.n_sink, window=wl.window, nm_ratio=wl.nm_ratio, beta=wl.beta,
-                        density_temp=wl.density_temp, min_budget=wl.min_budget)
+                        density_temp=wl.density_temp, min_budget=wl.min_budget, max_budget=wl.max_budget)
     ctx = B.D2OContext(cfg, device)
-    if args.stages or args.no_l2_hints:
-        ctx.d2o_set_tuning(args.stages, 0 if args.no_l2_hints else 1)
+    if args.stages or args.no_l2_hints or args.ffma_similarity:
+        ctx.d2o_set_tuning(args.stages, 0 if args.no_l2_hints else 1, 1 if args.ffma_similarity else 0)
     # every rank works on its own sequences: same shapes, rank-dependent seed (weak scaling, no exchange)
     import dataclasses
     wl_r = dataclasses.replace(wl, seed=wl.seed + 7919 * rank)

@@ -136,7 +136,7 @@ struct Layout {            // byte offsets into `state`
   size_t status, counters, density, budgets, windows, row_off, len, tau, colsum, pos, score, rnorm, kpool, vpool, end;
 };
 struct ScratchLayout {     // byte offsets into `scratch`
-  size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, stage_q, stage_k, stage_v, stage_out, end;
+  size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, part_key, stage_q, stage_k, stage_v, stage_out, end;
 };
 
 }  // namespace d2o
@@ -163,6 +163,7 @@ struct d2o_ctx {
   int32_t* layer_steps;        // [L] decode steps taken
   int decode_stages;           // tuning: stages of the decode kernel's ring, 0 = auto
   int decode_l2_hints;         // tuning: 1 = the decode kernel's copies carry L2 eviction hints
+  int similarity_path;         // tuning: 0 = tensor cores for 16-bit keys, 1 = FFMA kernel for every dtype
 };
 
 namespace d2o {
@@ -181,7 +182,10 @@ cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int ca
                                const void* q, const void* k, const void* v, void* out, cudaStream_t st,
                                d2o_status* why);
 
-// largest number of rows (cache + the new token) of one slice the decode kernel can keep resident
+// tensor-core similarity + nearest neighbour for 16-bit keys (d2o_sim_tc.cu); fills evict_mx / evict_nn
+cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int max_S, cudaStream_t st);
+size_t sim_tc_part_key_bytes(const d2o_config* cfg, int max_budget);
+// largest number of rows (cache + the new token) of one slice the decode kernel can handle
 int decode_max_rows(int row_bytes, int group, int d_head);
 
 // remembers the text of a failed CUDA runtime call for d2o_last_cuda_error(); returns D2O_ERR_CUDA

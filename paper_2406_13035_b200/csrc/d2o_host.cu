@@ -97,6 +97,7 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   s->evict_nn = take(B * Hkv * P * 4);
   s->seg_start = take(B * Hkv * ((size_t)max_budget + 2) * 4);
   s->seg_items = take(B * Hkv * P * 4);
+  s->part_key = take(c->dtype == D2O_F32 ? 0 : sim_tc_part_key_bytes(c, max_budget));
   s->stage_q = take(L * B * Hq * d * e);
   s->stage_k = take(L * B * Hkv * d * e);
   s->stage_v = take(L * B * Hkv * d * e);
@@ -338,11 +339,14 @@ extern "C" d2o_status d2o_get_stats(d2o_ctx* c, d2o_stats* out, void* stream) {
   return D2O_OK;
 }
 
-extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t decode_l2_hints) {
+extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t decode_l2_hints,
+                                     int32_t similarity_path) {
   if (!c) return D2O_ERR_INVALID_ARG;
   if (decode_stages < 0 || decode_stages > 12) return D2O_ERR_INVALID_ARG;
   if (decode_l2_hints < 0 || decode_l2_hints > 1) return D2O_ERR_INVALID_ARG;
+  if (similarity_path < 0 || similarity_path > 1) return D2O_ERR_INVALID_ARG;
   c->decode_stages = decode_stages;
   c->decode_l2_hints = decode_l2_hints;
+  c->similarity_path = similarity_path;
   return D2O_OK;
 }

@@ -486,8 +486,13 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   const size_t sim_sm = ((size_t)2 * D * kSimTile + 2 * kSimTile) * sizeof(float);
   e = cudaFuncSetAttribute(similarity_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sim_sm);
   if (e != cudaSuccess) return e;
-  dim3 sgrid((maxLe + kSimTile - 1) / kSimTile, n_slices);
-  similarity_kernel<T, D><<<sgrid, kSimThreads, sim_sm, st>>>(ma, (const T*)K, kpool);
+  if (sizeof(T) == 2 && c->similarity_path == 0) {
+    e = launch_similarity_tc(c, layer, K, maxS, st);
+    if (e != cudaSuccess) return e;
+  } else {
+    dim3 sgrid((maxLe + kSimTile - 1) / kSimTile, n_slices);
+    similarity_kernel<T, D><<<sgrid, kSimThreads, sim_sm, st>>>(ma, (const T*)K, kpool);
+  }
 
   SegArgs ga;
   ga.budgets = sa.budgets; ga.evict_mx = ma.evict_mx; ga.evict_nn = ma.evict_nn;

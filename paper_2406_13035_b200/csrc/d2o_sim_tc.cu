@@ -1,0 +1,434 @@
+// Nearest-neighbour matching at the prompt stage (Section 4.2, Eq. 9) for 16-bit keys on the
+// 5th-generation tensor cores: U = K_e K_c^T as tcgen05.mma (kind::f16, fp32 accumulators in tensor
+// memory), fused with the scaling by the inverse key norms and the row max / arg-max.
+//
+// The evicted keys are most of the prompt (80 - 95 % at the cache ratios of interest), in prompt
+// order.  Instead of gathering them, the kernel multiplies ALL prompt rows of a slice with the
+// retained keys and lets the consumer pick the evicted positions: the A operand is then a plain
+// tiled TMA load of 128 consecutive prompt rows, and the few retained rows among them cost
+// S/P extra work.
+//
+// One CTA = (slice, chunk of up to 512 retained rows, range of 128-row prompt tiles).
+//   warp 0      TMA producer: the retained chunk once (B operand, stays in shared memory), then the
+//               prompt tiles through a 2-stage ring (A operand); 128-byte swizzled K-major tiles
+//   warp 1      allocates tensor memory, issues tcgen05.mma: 128 x 256 x 16 per instruction, d/16 per job,
+//               accumulators double-buffered in 2 x 256 tensor-memory columns
+//   warps 2-9   epilogue: tcgen05.ld of the accumulators, times 1/|k_c| per column, running max and
+//               arg-max per row (ties -> lowest slot); two warps share a row (column halves)
+// Output: for every prompt position of the tile range and this chunk, the packed key
+// (ordered max_j k_i.k_j/|k_j|, 0x7fffffff - slot).  neighbour_reduce_kernel takes the maximum over
+// the chunks at the evicted positions and multiplies by 1/|k_i|.
+#include <cuda.h>
+#include <math.h>
+
+#include "d2o_common.cuh"
+
+namespace d2o {
+
+constexpr int kTcThreads = 320;             // 10 warps
+constexpr int kTcEpiWarps = 8;
+constexpr int kTileM = 128;                 // prompt rows per A tile
+constexpr int kTileN = 256;                 // retained rows per MMA
+constexpr int kChunkN = 512;                // retained rows resident per CTA
+constexpr int kAStages = 2;
+constexpr unsigned long long kTcWaitNs = 1000000000ull;
+
+struct SimTcArgs {
+  const int32_t* budgets; const int64_t* row_off;
+  const float* rnorm;                       // pool-wide 1/|k_c|
+  unsigned long long* part_key;             // [slices][n_chunks_max][P]
+  uint32_t* status;
+  int L, layer, Hkv, P, n_chunks_max, tiles_per_cta;
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+namespace tc {
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long global_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait; false = the phase did not complete within kTcWaitNs.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (!mbar_try_wait(bar, parity)) {
+    if (global_ns() - t0 > kTcWaitNs) return false;
+  }
+  return true;
+}
+// 2-D tiled TMA load into this CTA's shared memory; x = innermost coordinate (elements), y = row
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot_in_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot_in_smem)), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x N x 16, issued by one thread
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// the mbarrier receives one arrival when all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void mma_commit(unsigned long long* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base lane + t), columns c .. c+31
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled, in 8-row groups
+// of 1024 bytes: start address, leading offset 16 B (unused for this layout), stride offset 1024 B, version 1,
+// layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+}  // namespace tc
+
+// Instruction descriptor of kind::f16: fp32 accumulators, A and B of type `fmt` (0 = fp16, 1 = bf16), both K-major,
+// N in units of 8 at bit 17, M in units of 16 at bit 24.
+__host__ __device__ constexpr uint32_t make_idesc(uint32_t fmt, uint32_t M, uint32_t N) {
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+template <int D, int FMT>
+__global__ void __launch_bounds__(kTcThreads, 1)
+sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_pool) {
+  constexpr int KB = D / 64;                                 // 64-element (128-byte) blocks along d
+  constexpr int A_BLOCK = kTileM * 128;                      // bytes of one A k-block
+  constexpr int A_STAGE = KB * A_BLOCK;
+  constexpr int B_BLOCK = kChunkN * 128;                     // bytes of one B k-block (all chunk rows)
+  constexpr uint32_t IDESC = make_idesc(FMT, kTileM, kTileN);
+
+  extern __shared__ __align__(1024) unsigned char tc_smem[];
+  unsigned char* sB = tc_smem;                               // [KB][kChunkN rows][128 B]
+  unsigned char* sA = tc_smem + KB * B_BLOCK;                // [kAStages][KB][128 rows][128 B]
+  float* s_rn = reinterpret_cast<float*>(sA + kAStages * A_STAGE);                 // [kChunkN] 1/|k_c| of the chunk
+  unsigned long long* s_pair = reinterpret_cast<unsigned long long*>(s_rn + kChunkN);   // [128] keys of the upper column half
+  __shared__ unsigned long long b_full, a_full[kAStages], a_empty[kAStages], tm_full[2], tm_empty[2];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int slice = blockIdx.z;
+  const int nc = blockIdx.y;
+  const int b = slice / a.Hkv, h = slice % a.Hkv;
+  const int S = a.budgets[b * a.L + a.layer];
+  const int c0 = nc * kChunkN;                               // first retained slot of the chunk
+  if (c0 >= S || a.P - S <= 0) return;                       // uniform for the CTA: nothing to do
+  const int n_cols = min(kChunkN, S - c0);
+  const int n_nt = (n_cols + kTileN - 1) / kTileN;           // MMA column tiles in this chunk (1 or 2)
+  const int n_tiles_all = (a.P + kTileM - 1) / kTileM;
+  const int t0 = blockIdx.x * a.tiles_per_cta;
+  const int t1 = min(n_tiles_all, t0 + a.tiles_per_cta);
+  if (t0 >= t1) return;
+  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
+  if ((tc::smem_u32(tc_smem) & 1023u) != 0u) {               // swizzled tiles need 1024-byte aligned shared memory
+    if (tid == 0) report_error(a.status, D2O_ERR_STATE, 0x51C10000u);
+    return;
+  }
+
+  if (tid == 0) {
+    s_fail = 0;
+    tc::mbar_init(&b_full, 1);
+    for (int s = 0; s < kAStages; ++s) { tc::mbar_init(&a_full[s], 1); tc::mbar_init(&a_empty[s], 1); }
+    for (int i = 0; i < 2; ++i) { tc::mbar_init(&tm_full[i], 1); tc::mbar_init(&tm_empty[i], kTcEpiWarps); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {                                           // 512 columns: two 128 x 256 fp32 accumulators
+    tc::tmem_alloc(&s_tmem, 512);
+    tc::tmem_relinquish();
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tmem_base = s_tmem;
+
+  if (warp == 0) {
+    // ======================================================================= TMA producer
+    if (lane == 0) {
+      const int rows_b = n_nt * kTileN;                      // rows past the slice's S are other slices' rows: never used
+      tc::mbar_expect_tx(&b_full, (uint32_t)(KB * rows_b * 128));
+      for (int kb = 0; kb < KB; ++kb)
+        for (int j = 0; j < n_nt; ++j)
+          tc::tma_load_2d(sB + kb * B_BLOCK + j * kTileN * 128, &map_pool, kb * 64, (int)(row0 + c0 + j * kTileN), &b_full);
+      int it = 0;
+      for (int t = t0; t < t1; ++t, ++it) {
+        const int s = it % kAStages;
+        if (it >= kAStages && !s_fail && !tc::mbar_wait(&a_empty[s], (uint32_t)(((it / kAStages) - 1) & 1))) s_fail = 1;
+        tc::mbar_expect_tx(&a_full[s], (uint32_t)A_STAGE);
+        for (int kb = 0; kb < KB; ++kb)
+          tc::tma_load_2d(sA + s * A_STAGE + kb * A_BLOCK, &map_k, kb * 64, slice * a.P + t * kTileM, &a_full[s]);
+      }
+    }
+  } else if (warp == 1) {
+    // ======================================================================= MMA issuer
+    if (lane == 0) {
+      if (!tc::mbar_wait(&b_full, 0)) s_fail = 1;
+      int it = 0, job = 0;
+      for (int t = t0; t < t1; ++t, ++it) {
+        const int s = it % kAStages;
+        if (!s_fail && !tc::mbar_wait(&a_full[s], (uint32_t)((it / kAStages) & 1))) s_fail = 1;
+        for (int j = 0; j < n_nt; ++j, ++job) {
+          const int buf = job & 1;
+          // the epilogue must have drained this accumulator (the first use of each buffer passes at once)
+          if (!s_fail && !tc::mbar_wait(&tm_empty[buf], (uint32_t)(((job >> 1) & 1) ^ 1))) s_fail = 1;
+          tc::fence_after_sync();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kTileN);
+#pragma unroll
+          for (int kb = 0; kb < KB; ++kb) {
+            const uint64_t adesc = tc::smem_desc_sw128(tc::smem_u32(sA + s * A_STAGE + kb * A_BLOCK));
+            const uint64_t bdesc = tc::smem_desc_sw128(tc::smem_u32(sB + kb * B_BLOCK + j * kTileN * 128));
+#pragma unroll
+            for (int k = 0; k < 4; ++k)                      // 16 elements = 32 bytes along K per instruction
+              tc::mma_f16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), IDESC, (kb | k) != 0 ? 1u : 0u);
+          }
+          tc::mma_commit(&tm_full[buf]);
+        }
+        tc::mma_commit(&a_empty[s]);                         // the stage is free once its MMAs have read it
+      }
+    }
+  } else {
+    // ======================================================================= epilogue warps
+    const int e = warp - 2;
+    const int quarter = warp & 3;                            // tensor-memory lanes this warp may read: 32*quarter ..
+    const int half = e >> 2;                                 // columns [128*half, 128*half + 128) of every 256-wide tile
+    const int row = quarter * 32 + lane;                     // row of the A tile owned by this thread
+    for (int i = tid - 64; i < kChunkN; i += kTcEpiWarps * 32)
+      s_rn[i] = i < n_cols ? a.rnorm[row0 + c0 + i] : 0.f;
+    asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
+    unsigned long long* out_keys = a.part_key + ((size_t)slice * a.n_chunks_max + nc) * a.P;
+    int job = 0;
+    for (int t = t0; t < t1; ++t) {
+      float best = -INFINITY; int best_col = 0x7fffffff;
+      for (int j = 0; j < n_nt; ++j, ++job) {
+        const int buf = job & 1;
+        if (!s_fail && !tc::mbar_wait(&tm_full[buf], (uint32_t)((job >> 1) & 1))) s_fail = 1;
+        tc::fence_after_sync();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kTileN + half * 128);
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          const int cl0 = j * kTileN + half * 128 + cb * 32;  // first chunk-local column of the block
+          if (cl0 >= n_cols) break;
+          float v[32];
+          tc::tmem_ld32(taddr + (uint32_t)(cb * 32), v);
+          float tb = -INFINITY; int ti = 0;
+          if (cl0 + 32 <= n_cols) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float x = v[i] * s_rn[cl0 + i];
+              if (x > tb) { tb = x; ti = i; }
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float x = v[i] * s_rn[cl0 + i];
+              if (cl0 + i < n_cols && x > tb) { tb = x; ti = i; }
+            }
+          }
+          if (tb > best) { best = tb; best_col = c0 + cl0 + ti; }   // ascending columns: the first maximum stays
+        }
+        tc::fence_before_sync();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&tm_empty[buf]);
+      }
+      // (ordered value, inverted slot): larger is better, ties go to the lower slot; -0 counts as +0
+      if (best == 0.f) best = 0.f;
+      const unsigned long long key = best > -INFINITY
+          ? (((unsigned long long)float_ord(best) << 32) | (uint32_t)(0x7fffffff - best_col)) : 0ull;
+      if (half == 1) s_pair[row] = key;
+      asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
+      if (half == 0) {
+        const unsigned long long other = s_pair[row];
+        const int pos = t * kTileM + row;
+        if (pos < a.P) out_keys[pos] = other > key ? other : key;
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
+    }
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc::fence_after_sync();
+    tc::tmem_dealloc(tmem_base, 512);
+  }
+  if (tid == 0 && s_fail) report_error(a.status, D2O_ERR_TIMEOUT, 0x51C00000u | (uint32_t)(blockIdx.z & 0xfffff));
+}
+
+// mx_i = 1/|k_i| * max over the chunks of the partial maxima, nn_i = its slot, for the evicted positions.
+struct NnReduceArgs {
+  const int32_t* budgets;
+  const int32_t* evict_idx;
+  const unsigned long long* part_key;
+  float* evict_mx; int32_t* evict_nn;
+  int L, layer, Hkv, P, n_chunks_max;
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K) {
+  constexpr int EPV = Elem<T>::kPerVec;
+  constexpr int LPR = D / EPV;
+  const int slice = blockIdx.y;
+  const int b = slice / a.Hkv;
+  const int S = a.budgets[b * a.L + a.layer];
+  const int Le = a.P - S;
+  const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
+  const int i = blockIdx.x * (blockDim.x / LPR) + grp;
+  if (i >= Le) return;
+  const int pos = a.evict_idx[(size_t)slice * a.P + i];
+  float f[EPV];
+  Elem<T>::unpack(ld_global_v4(K + ((size_t)slice * a.P + pos) * D + lig * EPV), f);
+  float ss = 0.f;
+#pragma unroll
+  for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
+  ss = group_sum<LPR>(ss, group_mask<LPR>());
+  if (lig == 0) {
+    const int n_chunks = (S + kChunkN - 1) / kChunkN;
+    unsigned long long key = 0ull;
+    for (int c = 0; c < n_chunks; ++c) {
+      const unsigned long long k2 = a.part_key[((size_t)slice * a.n_chunks_max + c) * a.P + pos];
+      key = k2 > key ? k2 : key;
+    }
+    const float rn = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+    a.evict_mx[(size_t)slice * a.P + i] = ord_float((uint32_t)(key >> 32)) * rn;
+    a.evict_nn[(size_t)slice * a.P + i] = 0x7fffffff - (int)(uint32_t)(key & 0xffffffffu);
+  }
+}
+
+// ------------------------------------------------------------------------------------ host side
+// The driver's tensor-map encoder, looked up through the runtime so that the library has no link-time dependency
+// on the driver (it must load, and reject calls with status codes, on machines without one).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+static bool encode_2d(CUtensorMap* map, int dtype, const void* base, uint64_t rows, int d, int box_rows) {
+  EncodeTiledFn encode = encode_tiled_fn();
+  if (!encode) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1u, 1u};
+  const CUtensorMapDataType dt = dtype == D2O_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  return encode(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+size_t sim_tc_part_key_bytes(const d2o_config* cfg, int max_budget) {
+  const size_t chunks = ((size_t)max_budget + kChunkN - 1) / kChunkN;
+  return (size_t)cfg->batch * cfg->n_kv_heads * chunks * cfg->prompt_len * 8;
+}
+
+// Returns cudaErrorNotSupported if the tensor maps cannot be built.
+cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int max_S, cudaStream_t st) {
+  const d2o_config& g = c->cfg;
+  const int B = g.batch, Hkv = g.n_kv_heads, P = g.prompt_len, D = g.d_head;
+  const int n_slices = B * Hkv;
+  char* S = c->state; char* X = c->scratch;
+  CUtensorMap map_k, map_pool;
+  if (!encode_2d(&map_k, g.dtype, K, (uint64_t)n_slices * P, D, kTileM)) return cudaErrorNotSupported;
+  if (!encode_2d(&map_pool, g.dtype, S + c->lay.kpool, (uint64_t)c->pool_rows, D, kTileN)) return cudaErrorNotSupported;
+  const int n_chunks_max = (c->max_budget + kChunkN - 1) / kChunkN;
+  const int n_chunks = (max_S + kChunkN - 1) / kChunkN;
+  const int n_tiles = (P + kTileM - 1) / kTileM;
+  // enough CTAs for about three per SM, but at least four tiles each so that the resident chunk is amortised
+  int splits = (3 * 148 + n_slices * n_chunks - 1) / (n_slices * n_chunks);
+  splits = max(1, min(splits, (n_tiles + 3) / 4));
+  const int tiles_per_cta = (n_tiles + splits - 1) / splits;
+  splits = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
+
+  SimTcArgs a;
+  a.budgets = (const int32_t*)(S + c->lay.budgets); a.row_off = (const int64_t*)(S + c->lay.row_off);
+  a.rnorm = (const float*)(S + c->lay.rnorm);
+  a.part_key = (unsigned long long*)(X + c->slay.part_key);
+  a.status = (uint32_t*)(S + c->lay.status);
+  a.L = g.n_layers; a.layer = layer; a.Hkv = Hkv; a.P = P; a.n_chunks_max = n_chunks_max; a.tiles_per_cta = tiles_per_cta;
+  const int KB = D / 64;
+  const size_t smem = (size_t)KB * kChunkN * 128 + (size_t)kAStages * KB * kTileM * 128 + kChunkN * 4 + kTileM * 8;
+  dim3 grid(splits, n_chunks, n_slices);
+  const int fmt = g.dtype == D2O_F16 ? 0 : 1;
+  cudaError_t e;
+#define D2O_LAUNCH_TC(DD, FF)                                                                                     \
+  do {                                                                                                            \
+    e = cudaFuncSetAttribute(sim_tc_kernel<DD, FF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
+    if (e != cudaSuccess) return e;                                                                               \
+    sim_tc_kernel<DD, FF><<<grid, kTcThreads, smem, st>>>(a, map_k, map_pool);                                    \
+  } while (0)
+  if (D == 128) { if (fmt == 0) D2O_LAUNCH_TC(128, 0); else D2O_LAUNCH_TC(128, 1); }
+  else          { if (fmt == 0) D2O_LAUNCH_TC(64, 0); else D2O_LAUNCH_TC(64, 1); }
+#undef D2O_LAUNCH_TC
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+
+  NnReduceArgs r;
+  r.budgets = a.budgets; r.evict_idx = (const int32_t*)(X + c->slay.evict_idx); r.part_key = a.part_key;
+  r.evict_mx = (float*)(X + c->slay.evict_mx); r.evict_nn = (int32_t*)(X + c->slay.evict_nn);
+  r.L = g.n_layers; r.layer = layer; r.Hkv = Hkv; r.P = P; r.n_chunks_max = n_chunks_max;
+  int minS = P;
+  for (int bb = 0; bb < B; ++bb) minS = min(minS, c->h_budgets[bb * g.n_layers + layer]);
+  const int maxLe = P - minS;
+  if (maxLe <= 0) return cudaSuccess;
+  const int lpr = D * 2 / 16;
+  dim3 rgrid((maxLe + 256 / lpr - 1) / (256 / lpr), n_slices);
+  if (g.dtype == D2O_F16) {
+    if (D == 128) neighbour_reduce_kernel<__half, 128><<<rgrid, 256, 0, st>>>(r, (const __half*)K);
+    else neighbour_reduce_kernel<__half, 64><<<rgrid, 256, 0, st>>>(r, (const __half*)K);
+  } else {
+    if (D == 128) neighbour_reduce_kernel<__nv_bfloat16, 128><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K);
+    else neighbour_reduce_kernel<__nv_bfloat16, 64><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace d2o

@@ -58,6 +58,7 @@ class Workload:
     beta: float = 0.7
     density_temp: float = 1.0
     min_budget: int = 8
+    max_budget: int = 0       # upper clamp of S_l; 0 = prompt length
     rank: int = 8
     heavy_frac: float = 0.05
     temp_first: float = 1.0   # softmax temperature of layer 0
@@ -83,7 +84,7 @@ class Workload:
         return dataclasses.replace(
             self, name=name or (self.name + "_twin"), n_layers=n_layers,
             prompt_len=self.prompt_len // prompt_div, batch=min(self.batch, batch),
-            decode_steps=steps, window=window)
+            decode_steps=steps, window=window, max_budget=self.max_budget // prompt_div)
 
 
 # The five configurations named by the benchmark definition.  ``density_temp``
@@ -100,11 +101,11 @@ CONFIGS: Dict[str, Workload] = {
     "cfg2": Workload("cfg2", batch=16, n_layers=32, n_q_heads=32, n_kv_heads=8, d_head=128,
                      dtype="bf16", prompt_len=8192, decode_steps=512, rho=0.10, window=64,
                      beta=0.7, rank=16, heavy_frac=0.02, temp_first=1.0, temp_last=0.25,
-                     density_temp=8000.0, seed=2406132),
+                     density_temp=8000.0, max_budget=4096, seed=2406132),
     "cfg3": Workload("cfg3", batch=4, n_layers=32, n_q_heads=32, n_kv_heads=8, d_head=128,
                      dtype="bf16", prompt_len=32768, decode_steps=256, rho=0.05,
                      beta=0.7, rank=8, heavy_frac=0.05, temp_first=1.0, temp_last=0.25,
-                     density_temp=32000.0, seed=2406133),
+                     density_temp=32000.0, max_budget=6144, seed=2406133),
     "cfg4": Workload("cfg4", batch=8, n_layers=32, n_q_heads=32, n_kv_heads=32, d_head=128,
                      dtype="f16", prompt_len=2048, decode_steps=1024, rho=0.20,
                      beta=0.7, rank=8, heavy_frac=0.05, temp_first=1.0, temp_last=0.25,

@@ -67,7 +67,7 @@ def make_ctx(wl: W.Workload, device="cuda:0", **over) -> B.D2OContext:
     kw = dict(n_layers=wl.n_layers, batch=wl.batch, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
               d_head=wl.d_head, dtype=wl.dtype, prompt_len=wl.prompt_len, max_new_tokens=wl.decode_steps,
               rho=wl.rho, n_sink=wl.n_sink, window=wl.window, nm_ratio=wl.nm_ratio, beta=wl.beta,
-              density_temp=wl.density_temp, min_budget=wl.min_budget)
+              density_temp=wl.density_temp, min_budget=wl.min_budget, max_budget=wl.max_budget)
     kw.update(over)
     return B.D2OContext(B.make_config(**kw), device)
 
@@ -85,14 +85,15 @@ def make_oracle(wl: W.Workload, cfg: B.D2OConfig) -> O.OracleStack:
 def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int, int, int]]] = None,
                steps: Optional[int] = None, tie_rtol: float = TIE_RTOL, ctx_over: Optional[dict] = None,
                layers_per_call: Optional[int] = None, decode_stages: int = 0, decode_l2_hints: int = 1,
+               similarity_path: int = 0,
                check_stats_all: Optional[bool] = None) -> Report:
     """`slices`: (layer, b, kv_head) triples checked against the oracle (None = all).
     The GPU always runs the whole workload."""
     rep = Report()
     ctx = make_ctx(wl, device, **(ctx_over or {}))
     cfg = ctx.cfg
-    if decode_stages or not decode_l2_hints:
-        ctx.d2o_set_tuning(decode_stages, decode_l2_hints)
+    if decode_stages or not decode_l2_hints or similarity_path:
+        ctx.d2o_set_tuning(decode_stages, decode_l2_hints, similarity_path)
     orc = make_oracle(wl, cfg)
     L, Bn, Hq, Hkv, G, P = wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.group, wl.prompt_len
     all_slices = [(l, b, h) for l in range(L) for b in range(Bn) for h in range(Hkv)]

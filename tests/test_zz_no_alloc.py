@@ -36,7 +36,8 @@ def test_static_scratch_entry_matches_regular_entry(cuda_device, name, P):
     from paper_2406_13035_b200 import build
     build.build_library()
     B.load_library()
-    base = dataclasses.replace(W.CONFIGS[name], n_layers=1, batch=2, prompt_len=P, decode_steps=1, window=8)
+    base = dataclasses.replace(W.CONFIGS[name], n_layers=1, batch=2, prompt_len=P, decode_steps=1, window=8,
+                               max_budget=0)
     for call in range(2):                               # the second call reuses the scratch of the first
         wl = dataclasses.replace(base, seed=base.seed + call)
         Q, K, _ = W.LayerStream(wl, 0, "cuda:0").prompt()
