@@ -46,6 +46,7 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers-per-call", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling captures)")
     return ap.parse_args()
 
 
@@ -341,6 +342,9 @@ def run_reference(args, wl):
 def main():
     args = parse()
     wl = W.CONFIGS[args.config] if args.config in W.CONFIGS else W.twin(args.config.replace("_twin", ""))
+    if args.layers:
+        import dataclasses
+        wl = dataclasses.replace(wl, n_layers=args.layers, name=f"{wl.name}[{args.layers} layers]")
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":

@@ -8,13 +8,15 @@
 // tiled TMA load of 128 consecutive prompt rows, and the few retained rows among them cost
 // S/P extra work.
 //
-// One CTA = (slice, chunk of up to 512 retained rows, range of 128-row prompt tiles).
+// One CTA = (slice, chunk of up to 448 retained rows, range of 128-row prompt tiles).
 //   warp 0      TMA producer: the retained chunk once (B operand, stays in shared memory), then the
-//               prompt tiles through a 2-stage ring (A operand); 128-byte swizzled K-major tiles
+//               prompt tiles through a 3-stage ring (A operand); 128-byte swizzled K-major tiles
 //   warp 1      allocates tensor memory, issues tcgen05.mma: 128 x 256 x 16 per instruction, d/16 per job,
 //               accumulators double-buffered in 2 x 256 tensor-memory columns
-//   warps 2-9   epilogue: tcgen05.ld of the accumulators, times 1/|k_c| per column, running max and
-//               arg-max per row (ties -> lowest slot); two warps share a row (column halves)
+//   warps 2-17  epilogue: tcgen05.ld of the accumulators, times 1/|k_c| per column, running max and
+//               arg-max per row (ties -> lowest slot); four warps share a row (quarters of the column blocks);
+//               the scan is bound by instruction issue (about five per accumulator element), which is
+//               why it gets sixteen warps
 // Output: for every prompt position of the tile range and this chunk, the packed key
 // (ordered max_j k_i.k_j/|k_j|, 0x7fffffff - slot).  neighbour_reduce_kernel takes the maximum over
 // the chunks at the evicted positions and multiplies by 1/|k_i|.
@@ -25,12 +27,13 @@
 
 namespace d2o {
 
-constexpr int kTcThreads = 320;             // 10 warps
-constexpr int kTcEpiWarps = 8;
+constexpr int kTcEpiWarps = 16;             // four per quarter of the tensor-memory lanes
+constexpr int kTcThreads = (2 + kTcEpiWarps) * 32;
 constexpr int kTileM = 128;                 // prompt rows per A tile
 constexpr int kTileN = 256;                 // retained rows per MMA
-constexpr int kChunkN = 512;                // retained rows resident per CTA
-constexpr int kAStages = 2;
+constexpr int kChunkN = 448;                // retained rows resident per CTA (112 KB for d = 128)
+constexpr int kBBoxRows = 64;               // rows per TMA box of the B operand
+constexpr int kAStages = 3;                 // 3 x 32 KB of prompt tiles in flight
 constexpr unsigned long long kTcWaitNs = 1000000000ull;
 
 struct SimTcArgs {
@@ -98,9 +101,9 @@ __device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_
 __device__ __forceinline__ void mma_commit(unsigned long long* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base lane + t), columns c .. c+31
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
-  uint32_t r[32];
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base lane + t), columns c .. c+31.
+// The registers are valid only after tmem_ld_wait(), which names them so that no use can move above it.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -110,9 +113,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :: "memory");
 }
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled, in 8-row groups
 // of 1024 bytes: start address, leading offset 16 B (unused for this layout), stride offset 1024 B, version 1,
@@ -128,6 +136,52 @@ __host__ __device__ constexpr uint32_t make_idesc(uint32_t fmt, uint32_t M, uint
   return (1u << 4) | (fmt << 7) | (fmt << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
+// Retained rows per chunk for a slice of S rows: ceil(S / kChunkN) chunks of equal size, rounded up to the MMA's
+// column granularity.
+__host__ __device__ __forceinline__ int chunk_columns(int S) {
+  const int n_chunks = (S + kChunkN - 1) / kChunkN;
+  return (((S + n_chunks - 1) / n_chunks) + 15) & ~15;
+}
+
+// One block of 32 accumulator columns of one row: times 1/|k_c| per column, maximum and its column (the lowest
+// on ties), merged into the row's running (best, best_col).  cl0 = chunk-local column of the block.
+__device__ __forceinline__ void scan_block(const uint32_t (&r)[32], const float* s_rn, int cl0, int n_cols, int c0,
+                                           float& best, int& best_col) {
+  // four interleaved running maxima (columns i mod 4) keep the compare chains short
+  float tb[4]; int ti[4];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) { tb[w] = -INFINITY; ti[w] = w; }
+  const float4* rn4 = reinterpret_cast<const float4*>(s_rn + cl0);
+  if (cl0 + 32 <= n_cols) {
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4) {
+      const float4 q = rn4[i4];
+      const float rv[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float x = __uint_as_float(r[i4 * 4 + w]) * rv[w];
+        if (x > tb[w]) { tb[w] = x; ti[w] = i4 * 4 + w; }
+      }
+    }
+  } else {                                                        // columns past the chunk hold other slices' rows
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4) {
+      const float4 q = rn4[i4];
+      const float rv[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float x = __uint_as_float(r[i4 * 4 + w]) * rv[w];
+        if (cl0 + i4 * 4 + w < n_cols && x > tb[w]) { tb[w] = x; ti[w] = i4 * 4 + w; }
+      }
+    }
+  }
+  // larger value wins, equal values go to the lower column
+#pragma unroll
+  for (int w = 1; w < 4; ++w)
+    if (tb[w] > tb[0] || (tb[w] == tb[0] && ti[w] < ti[0])) { tb[0] = tb[w]; ti[0] = ti[w]; }
+  if (tb[0] > best) { best = tb[0]; best_col = c0 + cl0 + ti[0]; }   // ascending blocks: the first maximum stays
+}
+
 template <int D, int FMT>
 __global__ void __launch_bounds__(kTcThreads, 1)
 sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_pool) {
@@ -135,13 +189,12 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
   constexpr int A_BLOCK = kTileM * 128;                      // bytes of one A k-block
   constexpr int A_STAGE = KB * A_BLOCK;
   constexpr int B_BLOCK = kChunkN * 128;                     // bytes of one B k-block (all chunk rows)
-  constexpr uint32_t IDESC = make_idesc(FMT, kTileM, kTileN);
 
   extern __shared__ __align__(1024) unsigned char tc_smem[];
   unsigned char* sB = tc_smem;                               // [KB][kChunkN rows][128 B]
   unsigned char* sA = tc_smem + KB * B_BLOCK;                // [kAStages][KB][128 rows][128 B]
   float* s_rn = reinterpret_cast<float*>(sA + kAStages * A_STAGE);                 // [kChunkN] 1/|k_c| of the chunk
-  unsigned long long* s_pair = reinterpret_cast<unsigned long long*>(s_rn + kChunkN);   // [128] keys of the upper column half
+  unsigned long long* s_pair = reinterpret_cast<unsigned long long*>(s_rn + kChunkN);   // [3][128] keys of the other column quarters
   __shared__ unsigned long long b_full, a_full[kAStages], a_empty[kAStages], tm_full[2], tm_empty[2];
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
@@ -151,10 +204,12 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
   const int nc = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int S = a.budgets[b * a.L + a.layer];
-  const int c0 = nc * kChunkN;                               // first retained slot of the chunk
+  const int chunk_cols = chunk_columns(S);                   // the retained rows are split evenly over the chunks
+  const int c0 = nc * chunk_cols;                            // first retained slot of the chunk
   if (c0 >= S || a.P - S <= 0) return;                       // uniform for the CTA: nothing to do
-  const int n_cols = min(kChunkN, S - c0);
+  const int n_cols = min(chunk_cols, S - c0);
   const int n_nt = (n_cols + kTileN - 1) / kTileN;           // MMA column tiles in this chunk (1 or 2)
+  const int n_last = (n_cols - (n_nt - 1) * kTileN + 15) & ~15;   // columns of the last tile's MMA (multiple of 16)
   const int n_tiles_all = (a.P + kTileM - 1) / kTileM;
   const int t0 = blockIdx.x * a.tiles_per_cta;
   const int t1 = min(n_tiles_all, t0 + a.tiles_per_cta);
@@ -185,11 +240,11 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
   if (warp == 0) {
     // ======================================================================= TMA producer
     if (lane == 0) {
-      const int rows_b = n_nt * kTileN;                      // rows past the slice's S are other slices' rows: never used
-      tc::mbar_expect_tx(&b_full, (uint32_t)(KB * rows_b * 128));
+      const int n_box = (n_cols + kBBoxRows - 1) / kBBoxRows;    // rows past the slice's S are other slices' rows: never used
+      tc::mbar_expect_tx(&b_full, (uint32_t)(KB * n_box * kBBoxRows * 128));
       for (int kb = 0; kb < KB; ++kb)
-        for (int j = 0; j < n_nt; ++j)
-          tc::tma_load_2d(sB + kb * B_BLOCK + j * kTileN * 128, &map_pool, kb * 64, (int)(row0 + c0 + j * kTileN), &b_full);
+        for (int j = 0; j < n_box; ++j)
+          tc::tma_load_2d(sB + kb * B_BLOCK + j * kBBoxRows * 128, &map_pool, kb * 64, (int)(row0 + c0 + j * kBBoxRows), &b_full);
       int it = 0;
       for (int t = t0; t < t1; ++t, ++it) {
         const int s = it % kAStages;
@@ -213,13 +268,14 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
           if (!s_fail && !tc::mbar_wait(&tm_empty[buf], (uint32_t)(((job >> 1) & 1) ^ 1))) s_fail = 1;
           tc::fence_after_sync();
           const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kTileN);
+          const uint32_t idesc = make_idesc(FMT, kTileM, j == n_nt - 1 ? (uint32_t)n_last : (uint32_t)kTileN);
 #pragma unroll
           for (int kb = 0; kb < KB; ++kb) {
             const uint64_t adesc = tc::smem_desc_sw128(tc::smem_u32(sA + s * A_STAGE + kb * A_BLOCK));
             const uint64_t bdesc = tc::smem_desc_sw128(tc::smem_u32(sB + kb * B_BLOCK + j * kTileN * 128));
 #pragma unroll
             for (int k = 0; k < 4; ++k)                      // 16 elements = 32 bytes along K per instruction
-              tc::mma_f16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), IDESC, (kb | k) != 0 ? 1u : 0u);
+              tc::mma_f16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
           }
           tc::mma_commit(&tm_full[buf]);
         }
@@ -230,58 +286,74 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
     // ======================================================================= epilogue warps
     const int e = warp - 2;
     const int quarter = warp & 3;                            // tensor-memory lanes this warp may read: 32*quarter ..
-    const int half = e >> 2;                                 // columns [128*half, 128*half + 128) of every 256-wide tile
+    const int part = e >> 2;                                 // which quarter of a tile's column blocks this warp scans
     const int row = quarter * 32 + lane;                     // row of the A tile owned by this thread
     for (int i = tid - 64; i < kChunkN; i += kTcEpiWarps * 32)
       s_rn[i] = i < n_cols ? a.rnorm[row0 + c0 + i] : 0.f;
     asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
     unsigned long long* out_keys = a.part_key + ((size_t)slice * a.n_chunks_max + nc) * a.P;
-    int job = 0;
-    for (int t = t0; t < t1; ++t) {
-      float best = -INFINITY; int best_col = 0x7fffffff;
-      for (int j = 0; j < n_nt; ++j, ++job) {
-        const int buf = job & 1;
-        if (!s_fail && !tc::mbar_wait(&tm_full[buf], (uint32_t)((job >> 1) & 1))) s_fail = 1;
-        tc::fence_after_sync();
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kTileN + half * 128);
+    // The (at most eight) 32-column blocks of a job that hold retained rows are dealt to the four warps of a row,
+    // at most two each (slots 0 and 1).  Loads run one block ahead of the scan, across job boundaries: the first
+    // block of the next job is requested before the second block of this job is scanned.
+    auto blocks_of = [&](int j, int& blk0, int& n_blk) {
+      const int n_blk_all = (min(kTileN, n_cols - j * kTileN) + 31) / 32;
+      const int per = (n_blk_all + 3) / 4;
+      blk0 = part * per;
+      n_blk = max(0, min(per, n_blk_all - blk0));
+    };
+    const int n_jobs = (t1 - t0) * n_nt;
+    uint32_t ra[32], rb[32];
+    {
+      int blk0, n_blk;
+      blocks_of(0, blk0, n_blk);
+      if (!s_fail && !tc::mbar_wait(&tm_full[0], 0u)) s_fail = 1;
+      tc::fence_after_sync();
+      if (n_blk > 0) tc::tmem_ld32_issue(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(blk0 * 32), ra);
+    }
+    float best = -INFINITY; int best_col = 0x7fffffff;
 #pragma unroll 1
-        for (int cb = 0; cb < 4; ++cb) {
-          const int cl0 = j * kTileN + half * 128 + cb * 32;  // first chunk-local column of the block
-          if (cl0 >= n_cols) break;
-          float v[32];
-          tc::tmem_ld32(taddr + (uint32_t)(cb * 32), v);
-          float tb = -INFINITY; int ti = 0;
-          if (cl0 + 32 <= n_cols) {
+    for (int job = 0; job < n_jobs; ++job) {
+      const int t = t0 + job / n_nt, j = job % n_nt;
+      const int buf = job & 1;
+      int blk0, n_blk;
+      blocks_of(j, blk0, n_blk);
+      const int col0 = j * kTileN + blk0 * 32;                // chunk-local column of this warp's first block
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kTileN + blk0 * 32);
+      if (n_blk > 0) tc::tmem_ld_wait(ra);
+      if (n_blk > 1) tc::tmem_ld32_issue(taddr + 32u, rb);
+      if (n_blk > 0) scan_block(ra, s_rn, col0, n_cols, c0, best, best_col);
+      if (n_blk > 1) tc::tmem_ld_wait(rb);
+      // every load of this job has landed in registers: hand the accumulator back to the MMA warp
+      tc::fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&tm_empty[buf]);
+      if (job + 1 < n_jobs) {
+        const int nj = (job + 1) % n_nt;
+        int nblk0, nn_blk;
+        blocks_of(nj, nblk0, nn_blk);
+        if (!s_fail && !tc::mbar_wait(&tm_full[buf ^ 1], (uint32_t)(((job + 1) >> 1) & 1))) s_fail = 1;
+        tc::fence_after_sync();
+        if (nn_blk > 0)
+          tc::tmem_ld32_issue(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf ^ 1) * kTileN + nblk0 * 32), ra);
+      }
+      if (n_blk > 1) scan_block(rb, s_rn, col0 + 32, n_cols, c0, best, best_col);
+      if (j == n_nt - 1) {
+        // (ordered value, inverted slot): larger is better, ties go to the lower slot; -0 counts as +0
+        if (best == 0.f) best = 0.f;
+        const unsigned long long key = best > -INFINITY
+            ? (((unsigned long long)float_ord(best) << 32) | (uint32_t)(0x7fffffff - best_col)) : 0ull;
+        if (part > 0) s_pair[(part - 1) * kTileM + row] = key;
+        asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
+        if (part == 0) {
+          unsigned long long k = key;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float x = v[i] * s_rn[cl0 + i];
-              if (x > tb) { tb = x; ti = i; }
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float x = v[i] * s_rn[cl0 + i];
-              if (cl0 + i < n_cols && x > tb) { tb = x; ti = i; }
-            }
-          }
-          if (tb > best) { best = tb; best_col = c0 + cl0 + ti; }   // ascending columns: the first maximum stays
+          for (int o = 0; o < 3; ++o) { const unsigned long long other = s_pair[o * kTileM + row]; k = other > k ? other : k; }
+          const int pos = t * kTileM + row;
+          if (pos < a.P) out_keys[pos] = k;
         }
-        tc::fence_before_sync();
-        __syncwarp();
-        if (lane == 0) tc::mbar_arrive(&tm_empty[buf]);
+        asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
+        best = -INFINITY; best_col = 0x7fffffff;
       }
-      // (ordered value, inverted slot): larger is better, ties go to the lower slot; -0 counts as +0
-      if (best == 0.f) best = 0.f;
-      const unsigned long long key = best > -INFINITY
-          ? (((unsigned long long)float_ord(best) << 32) | (uint32_t)(0x7fffffff - best_col)) : 0ull;
-      if (half == 1) s_pair[row] = key;
-      asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
-      if (half == 0) {
-        const unsigned long long other = s_pair[row];
-        const int pos = t * kTileM + row;
-        if (pos < a.P) out_keys[pos] = other > key ? other : key;
-      }
-      asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
     }
   }
   tc::fence_before_sync();
@@ -378,13 +450,21 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   char* S = c->state; char* X = c->scratch;
   CUtensorMap map_k, map_pool;
   if (!encode_2d(&map_k, g.dtype, K, (uint64_t)n_slices * P, D, kTileM)) return cudaErrorNotSupported;
-  if (!encode_2d(&map_pool, g.dtype, S + c->lay.kpool, (uint64_t)c->pool_rows, D, kTileN)) return cudaErrorNotSupported;
+  if (!encode_2d(&map_pool, g.dtype, S + c->lay.kpool, (uint64_t)c->pool_rows, D, kBBoxRows)) return cudaErrorNotSupported;
   const int n_chunks_max = (c->max_budget + kChunkN - 1) / kChunkN;
   const int n_chunks = (max_S + kChunkN - 1) / kChunkN;
   const int n_tiles = (P + kTileM - 1) / kTileM;
-  // enough CTAs for about three per SM, but at least four tiles each so that the resident chunk is amortised
-  int splits = (3 * 148 + n_slices * n_chunks - 1) / (n_slices * n_chunks);
-  splits = max(1, min(splits, (n_tiles + 3) / 4));
+  // One CTA per SM at a time.  Split the prompt tiles so that the waves are full: cost of a split count =
+  // waves x (start-up of a CTA + its tiles), in units of one tile's work.
+  int sms = 148;
+  { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+  int splits = 1; double best_cost = 1e30;
+  for (int sp = 1; sp <= n_tiles; ++sp) {
+    const int tpc = (n_tiles + sp - 1) / sp;
+    const int ctas = ((n_tiles + tpc - 1) / tpc) * n_chunks * n_slices;
+    const double cost = (double)((ctas + sms - 1) / sms) * (3.0 + tpc);
+    if (cost < best_cost - 1e-9) { best_cost = cost; splits = sp; }
+  }
   const int tiles_per_cta = (n_tiles + splits - 1) / splits;
   splits = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
 
@@ -395,7 +475,7 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   a.status = (uint32_t*)(S + c->lay.status);
   a.L = g.n_layers; a.layer = layer; a.Hkv = Hkv; a.P = P; a.n_chunks_max = n_chunks_max; a.tiles_per_cta = tiles_per_cta;
   const int KB = D / 64;
-  const size_t smem = (size_t)KB * kChunkN * 128 + (size_t)kAStages * KB * kTileM * 128 + kChunkN * 4 + kTileM * 8;
+  const size_t smem = (size_t)KB * kChunkN * 128 + (size_t)kAStages * KB * kTileM * 128 + kChunkN * 4 + 3 * kTileM * 8;
   dim3 grid(splits, n_chunks, n_slices);
   const int fmt = g.dtype == D2O_F16 ? 0 : 1;
   cudaError_t e;
