@@ -10,7 +10,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libd2o.so")
-SOURCES = ["d2o_host.cu", "d2o_stats.cu", "d2o_prefill.cu", "d2o_decode.cu", "d2o_full_decode.cu", "d2o_sim_tc.cu"]
+SOURCES = ["d2o_host.cu", "d2o_stats.cu", "d2o_prefill.cu", "d2o_decode.cu", "d2o_full_decode.cu", "d2o_sim_tc.cu", "d2o_colsum_tc.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

@@ -164,6 +164,7 @@ struct d2o_ctx {
   int decode_stages;           // tuning: stages of the decode kernel's ring, 0 = auto
   int decode_l2_hints;         // tuning: 1 = the decode kernel's copies carry L2 eviction hints
   int similarity_path;         // tuning: 0 = tensor cores for 16-bit keys, 1 = FFMA kernel for every dtype
+  int stats_path;              // tuning: 0 = tensor cores for the column sums of 16-bit Q/K, 1 = FFMA kernels
 };
 
 namespace d2o {
@@ -185,6 +186,10 @@ cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int ca
 // tensor-core similarity + nearest neighbour for 16-bit keys (d2o_sim_tc.cu); fills evict_mx / evict_nn
 cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int max_S, cudaStream_t st);
 size_t sim_tc_part_key_bytes(const d2o_config* cfg, int max_budget);
+// tensor-core column sums of the prompt attention for 16-bit Q/K (d2o_colsum_tc.cu)
+bool colsum_tc_supported(const d2o_config* cfg);
+cudaError_t launch_colsum_tc(const d2o_ctx* c, const void* Q, const void* K, const float* lse_in, float* colsum,
+                             cudaStream_t st);
 // largest number of rows (cache + the new token) of one slice the decode kernel can handle
 int decode_max_rows(int row_bytes, int group, int d_head);
 

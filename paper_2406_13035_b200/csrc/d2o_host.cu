@@ -340,13 +340,14 @@ extern "C" d2o_status d2o_get_stats(d2o_ctx* c, d2o_stats* out, void* stream) {
 }
 
 extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t decode_l2_hints,
-                                     int32_t similarity_path) {
+                                     int32_t similarity_path, int32_t stats_path) {
   if (!c) return D2O_ERR_INVALID_ARG;
   if (decode_stages < 0 || decode_stages > 12) return D2O_ERR_INVALID_ARG;
   if (decode_l2_hints < 0 || decode_l2_hints > 1) return D2O_ERR_INVALID_ARG;
-  if (similarity_path < 0 || similarity_path > 1) return D2O_ERR_INVALID_ARG;
+  if (similarity_path < 0 || similarity_path > 1 || stats_path < 0 || stats_path > 1) return D2O_ERR_INVALID_ARG;
   c->decode_stages = decode_stages;
   c->decode_l2_hints = decode_l2_hints;
   c->similarity_path = similarity_path;
+  c->stats_path = stats_path;
   return D2O_OK;
 }

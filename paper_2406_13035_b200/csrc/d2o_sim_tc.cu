@@ -24,6 +24,7 @@
 #include <math.h>
 
 #include "d2o_common.cuh"
+#include "d2o_tc.cuh"
 
 namespace d2o {
 
@@ -34,7 +35,6 @@ constexpr int kTileN = 256;                 // retained rows per MMA
 constexpr int kChunkN = 448;                // retained rows resident per CTA (112 KB for d = 128)
 constexpr int kBBoxRows = 64;               // rows per TMA box of the B operand
 constexpr int kAStages = 3;                 // 3 x 32 KB of prompt tiles in flight
-constexpr unsigned long long kTcWaitNs = 1000000000ull;
 
 struct SimTcArgs {
   const int32_t* budgets; const int64_t* row_off;
@@ -43,98 +43,6 @@ struct SimTcArgs {
   uint32_t* status;
   int L, layer, Hkv, P, n_chunks_max, tiles_per_cta;
 };
-
-// ----------------------------------------------------------------------------- PTX wrappers
-namespace tc {
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long global_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait; false = the phase did not complete within kTcWaitNs.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  while (!mbar_try_wait(bar, parity)) {
-    if (global_ns() - t0 > kTcWaitNs) return false;
-  }
-  return true;
-}
-// 2-D tiled TMA load into this CTA's shared memory; x = innermost coordinate (elements), y = row
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-               ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t* slot_in_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot_in_smem)), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// D[tmem] (+)= A[smem] * B[smem]^T, 128 x N x 16, issued by one thread
-__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// the mbarrier receives one arrival when all MMAs issued so far by this thread have completed
-__device__ __forceinline__ void mma_commit(unsigned long long* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base lane + t), columns c .. c+31.
-// The registers are valid only after tmem_ld_wait(), which names them so that no use can move above it.
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-      :: "memory");
-}
-// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled, in 8-row groups
-// of 1024 bytes: start address, leading offset 16 B (unused for this layout), stride offset 1024 B, version 1,
-// layout type 2 (128-byte swizzle).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-  return (uint64_t)((saddr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-}  // namespace tc
-
-// Instruction descriptor of kind::f16: fp32 accumulators, A and B of type `fmt` (0 = fp16, 1 = bf16), both K-major,
-// N in units of 8 at bit 17, M in units of 16 at bit 24.
-__host__ __device__ constexpr uint32_t make_idesc(uint32_t fmt, uint32_t M, uint32_t N) {
-  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
-}
 
 // Retained rows per chunk for a slice of S rows: ceil(S / kChunkN) chunks of equal size, rounded up to the MMA's
 // column granularity.
@@ -424,7 +332,7 @@ static EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-static bool encode_2d(CUtensorMap* map, int dtype, const void* base, uint64_t rows, int d, int box_rows) {
+bool encode_rows_2d(CUtensorMap* map, int dtype, const void* base, uint64_t rows, int d, int box_rows) {
   EncodeTiledFn encode = encode_tiled_fn();
   if (!encode) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
@@ -449,8 +357,8 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   const int n_slices = B * Hkv;
   char* S = c->state; char* X = c->scratch;
   CUtensorMap map_k, map_pool;
-  if (!encode_2d(&map_k, g.dtype, K, (uint64_t)n_slices * P, D, kTileM)) return cudaErrorNotSupported;
-  if (!encode_2d(&map_pool, g.dtype, S + c->lay.kpool, (uint64_t)c->pool_rows, D, kBBoxRows)) return cudaErrorNotSupported;
+  if (!encode_rows_2d(&map_k, g.dtype, K, (uint64_t)n_slices * P, D, kTileM)) return cudaErrorNotSupported;
+  if (!encode_rows_2d(&map_pool, g.dtype, S + c->lay.kpool, (uint64_t)c->pool_rows, D, kBBoxRows)) return cudaErrorNotSupported;
   const int n_chunks_max = (c->max_budget + kChunkN - 1) / kChunkN;
   const int n_chunks = (max_S + kChunkN - 1) / kChunkN;
   const int n_tiles = (P + kTileM - 1) / kTileM;

@@ -10,7 +10,7 @@
 //   density_kernel  warp-shuffle mean / variance of s per query head (double accumulation)
 //   budget_kernel   Eq. 5 with clamping and exact-sum integerisation, one thread per sequence
 // The two attention sweeps here are the generic FFMA implementation (any dtype, fp32 math);
-// 16-bit inputs take the tensor-core path in d2o_colsum_tc.cu when it is built in.
+// 16-bit inputs take the tensor-core path of d2o_colsum_tc.cu.
 #include <math.h>
 
 #include "d2o_common.cuh"
@@ -326,6 +326,12 @@ static cudaError_t run_stats(const d2o_ctx* c, int layer, const void* Q, const v
   const int nT = (P + kTile - 1) / kTile;
   float* colsum = (float*)(c->state + c->lay.colsum) + (size_t)layer * B * Hq * P;
   double* density = (double*)(c->state + c->lay.density);
+  if (c->stats_path == 0 && colsum_tc_supported(&g)) {
+    cudaError_t e = launch_colsum_tc(c, Q, K, lse_in, colsum, st);
+    if (e != cudaSuccess) return e;
+    density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, g.n_layers, layer);
+    return cudaGetLastError();
+  }
   const float* lse = lse_in;
   dim3 grid(nT, B * Hq);
   if (!lse) {
