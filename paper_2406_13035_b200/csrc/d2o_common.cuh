@@ -133,7 +133,7 @@ enum Counter { kCntDecodeSteps = 0, kCntEvictions, kCntMerges, kCntDiscards, kCn
 
 // ----------------------------------------------------------------------------- context
 struct Layout {            // byte offsets into `state`
-  size_t status, counters, density, budgets, windows, row_off, len, tau, colsum, pos, score, rnorm, kpool, vpool, end;
+  size_t status, counters, density, budgets, windows, row_off, order, len, tau, colsum, pos, score, rnorm, kpool, vpool, end;
 };
 struct ScratchLayout {     // byte offsets into `scratch`
   size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, part_key, stage_q, stage_k, stage_v, stage_out, end;
@@ -161,6 +161,7 @@ struct d2o_ctx {
   uint8_t* layer_fed;          // [L] stats seen
   uint8_t* layer_compressed;   // [L]
   int32_t* layer_steps;        // [L] decode steps taken
+  int32_t* h_order;            // [L * B] (layer * B + b) sorted by cache size, largest first (device copy in `state`)
   int decode_stages;           // tuning: stages of the decode kernel's ring, 0 = auto
   int decode_l2_hints;         // tuning: 1 = the decode kernel's copies carry L2 eviction hints
   int similarity_path;         // tuning: 0 = tensor cores for 16-bit keys, 1 = FFMA kernel for every dtype

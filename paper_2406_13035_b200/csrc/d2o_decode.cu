@@ -40,6 +40,7 @@ struct DecodeArgs {
   int row_cap;                      // rows the per-row shared-memory arrays are sized for (multiple of 8)
   int stages;                       // stages of the ring
   int l2_hints;                     // 1: pass K asks L2 to keep its lines, later passes to drop theirs
+  const int32_t* order;             // NULL: CTAs take (layer, b, h) in index order; else (layer * B + b) per group of Hkv CTAs
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -138,15 +139,21 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   constexpr int ROWB = D * (int)sizeof(T);      // bytes per row
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int sl = blockIdx.x;                    // slice index within the launch
+  // ---- which slice: in index order, or largest caches first through the order table
+  const int h = (int)blockIdx.x % a.Hkv;
+  int layer, b;
+  if (a.order) {
+    const int pair = a.order[blockIdx.x / a.Hkv];
+    layer = pair / a.B; b = pair % a.B;
+  } else {
+    layer = a.l0 + (int)blockIdx.x / (a.B * a.Hkv);
+    b = ((int)blockIdx.x / a.Hkv) % a.B;
+  }
+  const int sl = ((layer - a.l0) * a.B + b) * a.Hkv + h;     // slice index within the call's q/k/v/out
   const T* k_new = k_in + (size_t)sl * D;
   const T* v_new = v_in + (size_t)sl * D;
 
   // ---- slice parameters
-  const int per_layer = a.B * a.Hkv;
-  const int layer = a.l0 + sl / per_layer;
-  const int bh = sl % per_layer;
-  const int b = bh / a.Hkv, h = bh % a.Hkv;
   const int S = a.budgets[b * a.L + layer];
   const int M = a.windows[b * a.L + layer];
   const int64_t row0 = a.row_off[b * a.L + layer] + (int64_t)h * slice_stride(S);
@@ -555,29 +562,38 @@ static cudaError_t launch_g(int G, const DecodeArgs& a, int n_slices, const void
   }
 }
 
-// Ring depth for `max_rows` rows per slice: the deepest ring that still lets the preferred number of CTAs share an SM.
-static bool plan(int max_rows, int row_bytes, int G, int D, int want_stages, int* row_cap, int* stages_out) {
+// Ring depth for `max_rows` rows per slice when `per_sm` CTAs are to share an SM.  false if the per-row arrays leave
+// no room for a ring.  Occupancy matters more than depth: measured on the 7B-shaped stack with caches of 700 to
+// 1900 rows, three CTAs with two stages each beat two CTAs with three or four stages (108 us vs 113 us per step).
+static bool plan_tier(int max_rows, int row_bytes, int G, int D, int per_sm, int* row_cap, int* stages_out) {
   const long sm_total = 227 * 1024;
   const int cap = (max_rows + 7) & ~7;
   const int min_stages = max(2, (kConsWarps * G * D * 4 + kStageBytes - 1) / kStageBytes);   // the ring doubles as `red`
   const long fixed = (long)(G + 3) * cap * 4 + 2L * row_bytes + 2048;                         // + static shared memory
-  int stages = want_stages;
-  if (stages <= 0) {
-    // three CTAs per SM with at least three stages each if the per-row arrays allow it, else two, else one
-    stages = 0;
-    const int tiers[3] = {3, 2, 1};
-    for (int ti = (G <= 2 ? 0 : 1); ti < 3 && stages == 0; ++ti) {
-      const long room = sm_total / tiers[ti] - 1024 - fixed;
-      const int fit = (int)(room / kStageBytes);
-      if (fit >= max(3, min_stages) || (tiers[ti] == 1 && fit >= min_stages)) stages = fit;
-    }
-    if (stages == 0) return false;
-    if (stages > 4) stages = 4;                                      // deeper rings only cost occupancy
-    if (stages < min_stages) stages = min_stages;
-  }
-  if (stages < min_stages || stages > kMaxStages) return false;
-  if (fixed + (long)stages * kStageBytes > sm_total - 1024) return false;
-  *row_cap = cap; *stages_out = stages;
+  const long room = sm_total / per_sm - 1024 - fixed;
+  const int fit = room > 0 ? (int)(room / kStageBytes) : 0;
+  if (fit < min_stages) return false;
+  *row_cap = cap;
+  *stages_out = max(min_stages, min(fit, per_sm == 1 ? 6 : (per_sm == 2 ? 4 : 3)));
+  return true;
+}
+
+// Best occupancy tier (3, 2, 1 CTAs per SM; registers allow 3 only for G <= 2) that fits `max_rows`; 0 = none.
+static int best_tier(int max_rows, int row_bytes, int G, int D, int* row_cap, int* stages) {
+  for (int per_sm = (G <= 2 ? 3 : 2); per_sm >= 1; --per_sm)
+    if (plan_tier(max_rows, row_bytes, G, D, per_sm, row_cap, stages)) return per_sm;
+  return 0;
+}
+
+static bool plan(int max_rows, int row_bytes, int G, int D, int want_stages, int* row_cap, int* stages_out) {
+  if (want_stages <= 0) return best_tier(max_rows, row_bytes, G, D, row_cap, stages_out) != 0;
+  const long sm_total = 227 * 1024;
+  const int cap = (max_rows + 7) & ~7;
+  const int min_stages = max(2, (kConsWarps * G * D * 4 + kStageBytes - 1) / kStageBytes);
+  const long fixed = (long)(G + 3) * cap * 4 + 2L * row_bytes + 2048;
+  if (want_stages < min_stages || want_stages > kMaxStages) return false;
+  if (fixed + (long)want_stages * kStageBytes > sm_total - 1024) return false;
+  *row_cap = cap; *stages_out = want_stages;
   return true;
 }
 
@@ -607,30 +623,33 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   a.t = g.prompt_len + c->layer_steps[l0];
   a.beta = g.beta; a.tau_override = g.tau_override;
   a.l2_hints = c->decode_l2_hints;
+  const int G = c->group, Hkv = g.n_kv_heads;
+  const int row_bytes = g.d_head * c->elem_size;
+  void* kpool = S + c->lay.kpool; void* vpool = S + c->lay.vpool;
+  auto launch = [&](const DecodeArgs& aa, int n_slices, cudaStream_t s) -> cudaError_t {
+    if (g.dtype == D2O_F32)
+      return g.d_head == 64 ? launch_g<float, 64>(G, aa, n_slices, q, k, v, out, kpool, vpool, s)
+                            : launch_g<float, 128>(G, aa, n_slices, q, k, v, out, kpool, vpool, s);
+    if (g.dtype == D2O_F16)
+      return g.d_head == 64 ? launch_g<__half, 64>(G, aa, n_slices, q, k, v, out, kpool, vpool, s)
+                            : launch_g<__half, 128>(G, aa, n_slices, q, k, v, out, kpool, vpool, s);
+    return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, aa, n_slices, q, k, v, out, kpool, vpool, s)
+                          : launch_g<__nv_bfloat16, 128>(G, aa, n_slices, q, k, v, out, kpool, vpool, s);
+  };
+  auto rows_of = [&](int l, int b) { return min(c->h_budgets[b * L + l], g.prompt_len + c->layer_steps[l0]) + 1; };
+
   int max_rows = 0;
   for (int l = l0; l < l1; ++l)
-    for (int b = 0; b < B; ++b) {
-      const int Sl = c->h_budgets[b * L + l];
-      const int len = min(Sl, g.prompt_len + c->layer_steps[l0]);
-      max_rows = max(max_rows, len + 1);
-    }
-  const int n_slices = (l1 - l0) * B * g.n_kv_heads;
+    for (int b = 0; b < B; ++b) max_rows = max(max_rows, rows_of(l, b));
   int row_cap, stages;
-  if (!plan(max_rows, g.d_head * c->elem_size, c->group, g.d_head, c->decode_stages, &row_cap, &stages)) {
+  if (!plan(max_rows, row_bytes, G, g.d_head, c->decode_stages, &row_cap, &stages)) {
     *why = D2O_ERR_UNSUPPORTED;
     return cudaSuccess;
   }
   a.row_cap = row_cap; a.stages = stages;
-  void* kpool = S + c->lay.kpool; void* vpool = S + c->lay.vpool;
-  const int G = c->group;
-  if (g.dtype == D2O_F32)
-    return g.d_head == 64 ? launch_g<float, 64>(G, a, n_slices, q, k, v, out, kpool, vpool, st)
-                          : launch_g<float, 128>(G, a, n_slices, q, k, v, out, kpool, vpool, st);
-  if (g.dtype == D2O_F16)
-    return g.d_head == 64 ? launch_g<__half, 64>(G, a, n_slices, q, k, v, out, kpool, vpool, st)
-                          : launch_g<__half, 128>(G, a, n_slices, q, k, v, out, kpool, vpool, st);
-  return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, a, n_slices, q, k, v, out, kpool, vpool, st)
-                        : launch_g<__nv_bfloat16, 128>(G, a, n_slices, q, k, v, out, kpool, vpool, st);
+  // all layers in one call: CTAs take the slices largest cache first, so the long ones do not end up in the tail
+  a.order = (l0 == 0 && l1 == L) ? (const int32_t*)(S + c->lay.order) : nullptr;
+  return launch(a, (l1 - l0) * B * Hkv, st);
 }
 
 }  // namespace d2o

@@ -5,6 +5,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
+
 #include "d2o_common.cuh"
 
 using namespace d2o;
@@ -81,6 +83,7 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   l->budgets = take(B * L * 4);
   l->windows = take(B * L * 4);
   l->row_off = take(B * L * 8);
+  l->order = take(B * L * 4);
   l->len = take(L * B * Hkv * 4);
   l->tau = take(L * B * Hkv * 4);
   l->colsum = take(L * B * Hq * P * 4);
@@ -146,6 +149,7 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
   c->layer_fed = (uint8_t*)calloc(cfg->n_layers, 1);
   c->layer_compressed = (uint8_t*)calloc(cfg->n_layers, 1);
   c->layer_steps = (int32_t*)calloc(cfg->n_layers, 4);
+  c->h_order = (int32_t*)calloc(BL, 4);
   // bookkeeping (status, counters, density, budgets ... tau) starts at zero
   cudaError_t e = cudaMemsetAsync(c->state, 0, l.colsum, (cudaStream_t)stream);
   if (e != cudaSuccess) { d2o_destroy(c); return cuda_fail(e, "cudaMemsetAsync(state)"); }
@@ -156,7 +160,7 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
 extern "C" void d2o_destroy(d2o_ctx* c) {
   if (!c) return;
   free(c->h_budgets); free(c->h_windows); free(c->h_row_off);
-  free(c->layer_fed); free(c->layer_compressed); free(c->layer_steps);
+  free(c->layer_fed); free(c->layer_compressed); free(c->layer_steps); free(c->h_order);
   free(c);
 }
 
@@ -215,6 +219,17 @@ extern "C" d2o_status d2o_layer_budgets(d2o_ctx* c, int32_t* budgets_host, void*
     if (c->h_budgets[i] < 1 || c->h_budgets[i] > c->max_budget || c->h_row_off[i] < 0 || end > c->pool_rows)
       return D2O_ERR_STATE;
   }
+  // (layer, sequence) pairs by cache size, largest first: the decode kernel takes its slices in this order
+  for (size_t i = 0; i < BL; ++i) c->h_order[i] = (int32_t)i;                  // i = layer * B + b
+  {
+    const int Bn = g.batch, Ln = g.n_layers;
+    const int32_t* hb = c->h_budgets;
+    std::stable_sort(c->h_order, c->h_order + BL, [=](int32_t x, int32_t y) {
+      return hb[(x % Bn) * Ln + x / Bn] > hb[(y % Bn) * Ln + y / Bn];
+    });
+  }
+  CUDA_TRY(cudaMemcpyAsync(c->state + c->lay.order, c->h_order, BL * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
   c->have_budgets = true;
   if (budgets_host) memcpy(budgets_host, c->h_budgets, BL * 4);
   return D2O_OK;
