@@ -30,6 +30,7 @@ import torch  # noqa: E402
 from paper_2406_13035_b200 import workloads as W  # noqa: E402
 
 METRIC = "compressed decode steps/s (x sequences = tokens/s); prefill-compress ms; fraction of HBM roofline"
+DECODE_TRAFFIC_RATIO = 1.057      # ncu DRAM bytes / algorithmic bytes of decode_kernel, see profiles/decode_kernel_cfg1.md
 
 
 def parse():
@@ -107,6 +108,11 @@ def prepare_inputs(wl: W.Workload, device, decode_steps: int):
     return prompts, torch.stack(dq), torch.stack(dk), torch.stack(dv)
 
 
+def workload_string(wl: W.Workload, nd: int) -> str:
+    return (f"{wl.name}: L={wl.n_layers} Hq={wl.n_q_heads} Hkv={wl.n_kv_heads} d={wl.d_head} "
+            f"B={wl.batch} P={wl.prompt_len} rho={wl.rho} decode_steps={nd}")
+
+
 def algorithmic_decode_bytes(wl: W.Workload, budgets, step_lens):
     """Bytes one decode launch must move: K_c and V_c rows once, per-row score/pos/norm read (12 B) and
     score write (4 B), q/k/v in and out once."""
@@ -161,7 +167,9 @@ def run_ours(args, wl, rank, world, device):
                 ctx.d2o_decode_step(l0, l1, dq[s, l0:l1], dk[s, l0:l1], dv[s, l0:l1], dout[l0:l1])
         e[4].record()
         if timed:
-            launches["n"] += L * 3 + 1 + L * 4 + nd * ((L + lpc - 1) // lpc)
+            # stats: 2 attention sweeps + density per layer; budgets: 1; compress: select, similarity, neighbour
+            # reduce, segments, merge per layer (the fp32 path has one kernel fewer); decode: 1 per call
+            launches["n"] += L * 3 + 1 + L * (4 if wl.dtype == "f32" else 5) + nd * ((L + lpc - 1) // lpc)
         return e, budgets
 
     def sync_all():
@@ -209,11 +217,30 @@ def run_ours(args, wl, rank, world, device):
         peaks = json.load(open(pk_path))
     peak = float(peaks.get("hbm_gbs", 6650.0))
     achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
+    # DRAM traffic per launch: dram__bytes_read + dram__bytes_write of one decode_kernel launch under ncu on the
+    # 16-layer variant of this workload was 1.057 x its algorithmic bytes (profiles/decode_kernel_cfg1.md); it grows
+    # with the rows streamed, so it is scaled by the algorithmic bytes of this launch.
+    traffic = int(DECODE_TRAFFIC_RATIO * bytes_per_launch) if (wl.name.startswith("cfg1") and lpc == L) else None
     roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": round(achieved, 1), "peak": peak,
                 "unit": "GB/s", "frac": round(achieved / peak, 4),
                 "peak_source": "measured" if "hbm_gbs" in peaks else "fallback",
                 "algorithmic_bytes_per_launch": int(bytes_per_launch), "avg_launch_us": round(launch_ms * 1e3, 2),
-                "traffic": None}
+                "traffic": traffic}
+    # the two tensor-core phases, for context: algorithmic flops of the phase / its duration (the phase also holds
+    # the small kernels around the contraction, so these are lower bounds for the contraction kernels themselves)
+    tpeak = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    Le = P - budgets.double()                                     # evicted rows per (sequence, layer)
+    sim_flops = float((2.0 * Le * budgets.double() * wl.d_head).sum()) * wl.n_kv_heads
+    attn_flops = 2.0 * wl.batch * wl.n_q_heads * L * float(P) * P * wl.d_head      # two causal sweeps of P^2 d
+    tensor_phases = None
+    if wl.dtype != "f32":
+        tensor_phases = [
+            {"phase": "d2o_layer_stats (attn_tc_kernel x 2 sweeps + density)", "bound": "tensor",
+             "achieved": round(attn_flops / (stats_ms * 1e-3) / 1e12, 1), "peak": tpeak, "unit": "TFLOP/s",
+             "frac": round(attn_flops / (stats_ms * 1e-3) / 1e12 / tpeak, 4)},
+            {"phase": "d2o_prefill_compress (select, sim_tc_kernel, reduce, segments, merge)", "bound": "tensor",
+             "achieved": round(sim_flops / (compress_ms * 1e-3) / 1e12, 1), "peak": tpeak, "unit": "TFLOP/s",
+             "frac": round(sim_flops / (compress_ms * 1e-3) / 1e12 / tpeak, 4)}]
     # end to end: the decode loop through the host-buffer entry point
     e2e = None
     if not args.no_e2e:
@@ -244,8 +271,7 @@ def run_ours(args, wl, rank, world, device):
         "metric": METRIC, "value": round(world * wl.batch * steps_per_s, 2), "unit": "token-steps/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(pass_ms, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-        "config": {"workload": f"{wl.name}: L={wl.n_layers} Hq={wl.n_q_heads} Hkv={wl.n_kv_heads} d={wl.d_head} "
-                               f"B={wl.batch} P={wl.prompt_len} rho={wl.rho} decode_steps={nd}",
+        "config": {"workload": workload_string(wl, nd),
                    "l2": "decode working set (K_c+V_c of all layers) exceeds the 126 MB L2; prompt tensors exceed it too",
                    "layers_per_decode_call": lpc, "decode_ring_stages": args.stages or "auto",
                    "sequences_per_gpu": wl.batch, "parallelism": "replicas (independent sequences per GPU)"},
@@ -254,7 +280,7 @@ def run_ours(args, wl, rank, world, device):
         "decode_ms": round(decode_ms, 3), "wall_s": round(t_wall, 3),
         "budgets_min_max": [int(budgets.min()), int(budgets.max())],
         "merges_discards": [int(st.merges), int(st.discards)],
-        "roofline": roofline, "e2e": e2e, "gpu_launches": launches["n"], "clocks": clocks,
+        "roofline": roofline, "tensor_phases": tensor_phases, "e2e": e2e, "gpu_launches": launches["n"], "clocks": clocks,
     }
     ctx.close()
     return res
@@ -263,8 +289,8 @@ def run_ours(args, wl, rank, world, device):
 # --------------------------------------------------------------------------------------- CPU oracle leg
 def oracle_sample(wl: W.Workload, n_slices: int, n_steps: int, threads: int = 1):
     """Times the oracle on `n_slices` slices of layer 0 of the workload: column sums of their query heads,
-    compression, `n_steps` decode steps.  Returns (seconds for the prompt stage, seconds per decode step of one
-    slice)."""
+    compression at the uniform budget rho * P, `n_steps` decode steps.  Returns (seconds for the prompt stage per
+    slice, seconds per decode step of one slice, slices)."""
     import numpy as np
     from oracle import d2o_oracle as O
     from threadpoolctl import threadpool_limits
@@ -273,38 +299,30 @@ def oracle_sample(wl: W.Workload, n_slices: int, n_steps: int, threads: int = 1)
     G = wl.group
     picks = [(0, h) for h in range(min(n_slices, wl.n_kv_heads))]
     dec = [s.decode() for _ in range(n_steps)]
+
+    class PerHead:
+        """[b, h] -> float64 [P, d] of one head, converted on demand."""
+
+        def __init__(self, t):
+            self.t = t
+
+        def __getitem__(self, i):
+            return self.t[i].double().numpy()
+
     with threadpool_limits(limits=threads):
         orc = O.OracleStack(n_layers=1, batch=wl.batch, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
                             d_head=wl.d_head, dtype=wl.dtype, prompt_len=wl.prompt_len, rho=wl.rho, n_sink=wl.n_sink,
                             window=wl.window, nm_ratio=wl.nm_ratio, beta=wl.beta, min_budget=wl.min_budget)
         t0 = time.perf_counter()
         heads = [(b, h * G + g) for b, h in picks for g in range(G)]
-        Q64 = {(b, hq): Q[b, hq].double().numpy() for b, hq in heads}
-        K64 = {(b, h): K[b, h].double().numpy() for b, h in picks}
-        V64 = {(b, h): V[b, h].double().numpy() for b, h in picks}
-
-        class Idx:
-            def __init__(self, d): self.d = d
-            def __getitem__(self, i): return self.d[i]
-        orc.layer_stats(0, Idx(Q64), Idx({(b, hq): K64[(b, hq // G)] for b, hq in heads}) if False else _KQ(K64, G),
-                        heads)
+        orc.layer_stats(0, PerHead(Q), PerHead(K), heads)
         orc.budgets = np.full((wl.batch, 1), int(round(wl.rho * wl.prompt_len)), dtype=np.int64)
-        orc.prefill_compress(0, Idx(K64), Idx(V64), picks)
+        orc.prefill_compress(0, PerHead(K), PerHead(V), picks)
         t1 = time.perf_counter()
         for i, (q, k, v) in enumerate(dec):
             orc.decode_step(0, q.double().numpy(), k.double().numpy(), v.double().numpy(), wl.prompt_len + i, picks)
         t2 = time.perf_counter()
     return (t1 - t0) / len(picks), (t2 - t1) / (len(picks) * max(1, n_steps)), len(picks)
-
-
-class _KQ:
-    """K indexed by (b, kv head) for OracleStack.layer_stats."""
-
-    def __init__(self, d, G):
-        self.d, self.G = d, G
-
-    def __getitem__(self, i):
-        return self.d[i]
 
 
 def cpu_baseline(wl: W.Workload, n_slices=2, n_steps=32):
@@ -335,7 +353,7 @@ def run_reference(args, wl):
     return {"impl": "reference", "metric": METRIC, "value": value, "unit": "token-steps/s", "n_gpus": 1,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(wall / max(1, args.steps) * 1e3, 2),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"{wl.name} (bounded sample)"},
+            "config": {"workload": workload_string(wl, args.decode_steps or wl.decode_steps)},
             "prompt_stage_s_per_slice": round(prompt_s, 3),
             "cpu_baseline": {"value": value, "unit": "token-steps/s", "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "token-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
