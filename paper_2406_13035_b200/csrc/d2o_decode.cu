@@ -170,12 +170,12 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   extern __shared__ __align__(128) unsigned char dsm[];
   uint4* ring = reinterpret_cast<uint4*>(dsm);                       // [stages][SR][LPR]
   float* red = reinterpret_cast<float*>(dsm);                        // [warps][G][D], aliases the ring once it is drained
-  float* pl = reinterpret_cast<float*>(dsm + (size_t)NS * kStageBytes);   // [G][row_cap] logits -> probabilities
-  float* sc = pl + (size_t)G * a.row_cap;                            // [row_cap] scores
-  float* rn = sc + a.row_cap;                                        // [row_cap] inverse key norms
-  int* ps = reinterpret_cast<int*>(rn + a.row_cap);                  // [row_cap] positions
-  uint4* stash = reinterpret_cast<uint4*>(ps + a.row_cap);           // [2][LPR] value rows of the victim / the neighbour
-  __shared__ unsigned long long s_full[kMaxStages], s_empty[kMaxStages], s_meta;
+  float* meta_rn = reinterpret_cast<float*>(dsm + (size_t)NS * kStageBytes);   // [stages][SR] 1/|k| of a pass-K' stage's rows
+  int* meta_ps = reinterpret_cast<int*>(meta_rn + (size_t)NS * SR);  // [stages][SR] positions of a pass-K' stage's rows
+  float* pl = reinterpret_cast<float*>(meta_ps + (size_t)NS * SR);   // [G][row_cap] logits -> probabilities
+  uint4* stash = reinterpret_cast<uint4*>(pl + (size_t)G * a.row_cap);   // [2][LPR] value rows of the victim / the neighbour
+  __shared__ unsigned long long s_full[kMaxStages], s_empty[kMaxStages];
+  __shared__ float s_new_rn, s_new_score;                            // inverse key norm and accumulated score of the new token
   __shared__ float s_red[2][kConsWarps][G];
   __shared__ unsigned long long s_key[kConsWarps], s_best_key;
   __shared__ int s_li[kConsWarps], s_best_li;
@@ -184,7 +184,6 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   if (tid == 0) {
     // once an anomaly has been recorded (by this or an earlier launch) no wait is attempted any more
     s_timeout = *reinterpret_cast<volatile uint32_t*>(a.status) != 0u;
-    mbar_init(&s_meta, 1);
     for (int s = 0; s < NS; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kConsWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -198,17 +197,6 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       if (a.l2_hints) {
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
-      }
-      // positions / scores / inverse norms of the cache rows (4 rows = 16 bytes granularity: up to 3 entries
-      // past n_old are read from the slice's padding and overwritten below)
-      const int np4 = (n_old + 3) & ~3;
-      if (np4 > 0) {
-        mbar_expect_tx(&s_meta, (uint32_t)(3 * np4 * 4));
-        bulk_g2s(ps, a.pos + row0, (uint32_t)(np4 * 4), &s_meta);
-        bulk_g2s(sc, a.score + row0, (uint32_t)(np4 * 4), &s_meta);
-        bulk_g2s(rn, a.rnorm + row0, (uint32_t)(np4 * 4), &s_meta);
-      } else {
-        mbar_arrive(&s_meta);
       }
       const int n_pass = evict ? 3 : 2;
       int q = 0;
@@ -225,7 +213,15 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
           const int np = max(0, min(a1, n_old) - a0);                // cache rows of the stage
           const bool nw = n_old >= a0 && n_old < a1;                 // the new token's row falls into the stage
           uint4* dst = ring + (size_t)slot * SR * LPR;
-          mbar_expect_tx(&s_full[slot], (uint32_t)((np + (nw ? 1 : 0)) * ROWB));
+          // pass K' also needs 1/|k| and the position of its rows (16-byte granules: up to 3 entries past n_old
+          // come from the slice's padding and are never used)
+          const bool with_meta = evict && p == 1 && np > 0;
+          const int np4 = (np + 3) & ~3;
+          mbar_expect_tx(&s_full[slot], (uint32_t)((np + (nw ? 1 : 0)) * ROWB + (with_meta ? 2 * np4 * 4 : 0)));
+          if (with_meta) {
+            bulk_g2s(meta_rn + (size_t)slot * SR, a.rnorm + row0 + a0, (uint32_t)(np4 * 4), &s_full[slot]);
+            bulk_g2s(meta_ps + (size_t)slot * SR, a.pos + row0 + a0, (uint32_t)(np4 * 4), &s_full[slot]);
+          }
           if (np > 0) {
             if (hint) bulk_g2s_hint(dst, pool + (row0 + a0) * D, (uint32_t)(np * ROWB), &s_full[slot], pol);
             else bulk_g2s(dst, pool + (row0 + a0) * D, (uint32_t)(np * ROWB), &s_full[slot]);
@@ -293,7 +289,6 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
     }
   }
   // ---- softmax normaliser, probabilities, accumulated attention (Eq. 6 case 2), victim candidate
-  if (!s_timeout && !mbar_wait(&s_meta, 0)) s_timeout = 2;
   if (warp == 0) {
     // the new token's metadata; its inverse norm from the row as stored
     float f[EPV];
@@ -302,7 +297,7 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
 #pragma unroll
     for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
     ss = warp_sum(ss);                                               // lanes >= LPR hold zeros
-    if (lane == 0) { ps[n_old] = a.t; sc[n_old] = 0.f; rn[n_old] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f; }
+    if (lane == 0) s_new_rn = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
   }
   float m_all[G], inv_l[G];
   {
@@ -342,10 +337,10 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       float p = 0.f;
 #pragma unroll
       for (int g = 0; g < G; ++g) p = fmaf(pl[(size_t)g * a.row_cap + li], inv_l[g], p);
-      const float s_new = sc[li] + p;
-      sc[li] = s_new;
+      const float s_new = (li < n_old ? a.score[row0 + li] : 0.f) + p;
       if (li < n_old || !evict) a.score[row0 + li] = s_new;          // the new token's score is placed with its row
-      const int pz = ps[li];
+      else s_new_score = s_new;
+      const int pz = li < n_old ? a.pos[row0 + li] : a.t;
       if (evict && pz >= Tn && pz <= a.t - M) {                      // lowest score, ties -> latest position
         const unsigned long long key = ((unsigned long long)float_ord(s_new) << 32) | (uint32_t)(0x7fffffff - pz);
         if (key < my_min) { my_min = key; my_min_li = li; }
@@ -373,7 +368,7 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       }
       return;
     }
-    const float vic_rn = rn[vic_li];
+    const float vic_rn = vic_li < n_old ? a.rnorm[row0 + vic_li] : s_new_rn;
     float kvic[EPV];
     Elem<T>::unpack(ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) + lig * EPV), kvic);
     unsigned long long best = 0ull; int best_li = -1;
@@ -392,13 +387,17 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
         for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], f[e], x);
         dot[u] = x;
       }
+      // the row whose total this lane receives; its 1/|k| and position leave the stage before the stage is released
+      const int li = s * SR + (lig / QL) * NGRP + grp;
+      const bool mine = li < n && lig % QL == 0 && li != vic_li;
+      float rn_li = s_new_rn; int ps_li = a.t;
+      if (mine && li < n_old) { rn_li = meta_rn[(size_t)slot * SR + (li - s * SR)]; ps_li = meta_ps[(size_t)slot * SR + (li - s * SR)]; }
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_empty[slot]);
       const float r = reduce4<LPR>(dot[0], dot[1], dot[2], dot[3], lig);
-      const int li = s * SR + (lig / QL) * NGRP + grp;
-      if (li < n && lig % QL == 0 && li != vic_li) {                 // max similarity, ties -> earliest position
-        const float u = r * vic_rn * rn[li];
-        const unsigned long long key = ((unsigned long long)float_ord(u) << 32) | (uint32_t)(0x7fffffff - ps[li]);
+      if (mine) {                                                    // max similarity, ties -> earliest position
+        const float u = r * vic_rn * rn_li;
+        const unsigned long long key = ((unsigned long long)float_ord(u) << 32) | (uint32_t)(0x7fffffff - ps_li);
         if (key > best) { best = key; best_li = li; }
       }
     }
@@ -418,7 +417,7 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       atomicAdd(&a.counters[kCntEvictions], 1ull);
       atomicAdd(&a.counters[merge ? kCntMerges : kCntDiscards], 1ull);
     }
-    rn_slot = rn[n_old];
+    rn_slot = s_new_rn;
     if (warp == 0 && lane < LPR) {
       // keys are not read any more in this launch: merged key row in place, the new token's key into the victim's row
       if (merge) {
@@ -443,7 +442,7 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
         *reinterpret_cast<uint4*>(kpool + (row0 + vic_li) * D + lane * EPV) = kslot;
         if (lane == 0) {
           a.pos[row0 + vic_li] = a.t;
-          a.score[row0 + vic_li] = sc[n_old];
+          a.score[row0 + vic_li] = s_new_score;
           a.rnorm[row0 + vic_li] = rn_slot;
         }
       }
@@ -510,7 +509,7 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
     if (grp == 0) {
       *reinterpret_cast<uint4*>(kpool + (row0 + n_old) * D + lig * EPV) = knew;
       *reinterpret_cast<uint4*>(vpool + (row0 + n_old) * D + lig * EPV) = vnew;
-      if (lig == 0) { a.pos[row0 + n_old] = a.t; a.rnorm[row0 + n_old] = rn[n_old]; }
+      if (lig == 0) { a.pos[row0 + n_old] = a.t; a.rnorm[row0 + n_old] = s_new_rn; }
     }
     if (tid == 0) {
       a.len[sidx] = n;
@@ -536,8 +535,10 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
 }
 
 // ------------------------------------------------------------------------------------ launch
+// ring stages (each with the 1/|k| and position slots of its rows), probabilities, stash
+static size_t stage_bytes(int row_bytes) { return (size_t)kStageBytes + 2 * (size_t)(kStageBytes / row_bytes) * 4; }
 static size_t smem_bytes(int row_cap, int stages, int G, int row_bytes) {
-  return (size_t)stages * kStageBytes + (size_t)(G + 3) * row_cap * 4 + 2 * (size_t)row_bytes;
+  return (size_t)stages * stage_bytes(row_bytes) + (size_t)G * row_cap * 4 + 2 * (size_t)row_bytes;
 }
 
 template <typename T, int D, int G>
@@ -569,9 +570,9 @@ static bool plan_tier(int max_rows, int row_bytes, int G, int D, int per_sm, int
   const long sm_total = 227 * 1024;
   const int cap = (max_rows + 7) & ~7;
   const int min_stages = max(2, (kConsWarps * G * D * 4 + kStageBytes - 1) / kStageBytes);   // the ring doubles as `red`
-  const long fixed = (long)(G + 3) * cap * 4 + 2L * row_bytes + 2048;                         // + static shared memory
+  const long fixed = (long)G * cap * 4 + 2L * row_bytes + 2048;                               // + static shared memory
   const long room = sm_total / per_sm - 1024 - fixed;
-  const int fit = room > 0 ? (int)(room / kStageBytes) : 0;
+  const int fit = room > 0 ? (int)(room / (long)stage_bytes(row_bytes)) : 0;
   if (fit < min_stages) return false;
   *row_cap = cap;
   *stages_out = max(min_stages, min(fit, per_sm == 1 ? 6 : (per_sm == 2 ? 4 : 3)));
@@ -590,9 +591,9 @@ static bool plan(int max_rows, int row_bytes, int G, int D, int want_stages, int
   const long sm_total = 227 * 1024;
   const int cap = (max_rows + 7) & ~7;
   const int min_stages = max(2, (kConsWarps * G * D * 4 + kStageBytes - 1) / kStageBytes);
-  const long fixed = (long)(G + 3) * cap * 4 + 2L * row_bytes + 2048;
+  const long fixed = (long)G * cap * 4 + 2L * row_bytes + 2048;
   if (want_stages < min_stages || want_stages > kMaxStages) return false;
-  if (fixed + (long)want_stages * kStageBytes > sm_total - 1024) return false;
+  if (fixed + (long)want_stages * (long)stage_bytes(row_bytes) > sm_total - 1024) return false;
   *row_cap = cap; *stages_out = want_stages;
   return true;
 }
