@@ -19,6 +19,8 @@
 // block-wide reduction inside one CTA; there is no inter-CTA communication.
 #include <math.h>
 
+#include <cuda/std/type_traits>
+
 #include "d2o_common.cuh"
 
 namespace d2o {
@@ -125,6 +127,39 @@ __device__ __forceinline__ float reduce4(float s0, float s1, float s2, float s3,
 #pragma unroll
   for (int o = LPR / 8; o > 0; o >>= 1) k += __shfl_xor_sync(0xffffffffu, k, o);
   return k;
+}
+
+// One warp-level tensor-core step for the logits of 16 rows against up to 8 heads: acc (16 x 8, fp32) += A (16 rows x
+// 16 elements of d, from the row-major stage) * B (16 elements x 8 heads, the queries).  Both operands take their
+// 16-byte pieces from the same offsets of their rows, so the order of the elements inside a step is free and a
+// thread's piece is one contiguous vector load.
+template <typename T>
+__device__ __forceinline__ void mma_16x8x16(float (&acc)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                            uint32_t b0, uint32_t b1) {
+  if constexpr (sizeof(T) == 2 && !cuda::std::is_same<T, __nv_bfloat16>::value) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  } else {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  }
+}
+
+// Dot products of the 16 rows [lr0, lr0 + 16) of a stage with the (up to 8) vectors whose fragments are in `qb`
+// (one 16-byte piece per 32 elements of d and thread: vector gid = lane / 4, piece tig = lane % 4).
+// acc[0], acc[1] = row lr0 + gid against vectors 2 tig, 2 tig + 1; acc[2], acc[3] = row lr0 + gid + 8.
+template <typename T, int D>
+__device__ __forceinline__ void tile_dots(const uint4* st, int lr0, const uint4 (&qb)[D / 32], float (&acc)[4]) {
+  constexpr int LPR = D * (int)sizeof(T) / 16;
+  const int gid = (threadIdx.x & 31) >> 2, tig = threadIdx.x & 3;
+  acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+#pragma unroll
+  for (int kk = 0; kk < D / 32; ++kk) {
+    const uint4 A0 = st[(size_t)(lr0 + gid) * LPR + kk * 4 + tig];
+    const uint4 A1 = st[(size_t)(lr0 + gid + 8) * LPR + kk * 4 + tig];
+    mma_16x8x16<T>(acc, A0.x, A1.x, A0.y, A1.y, qb[kk].x, qb[kk].y);
+    mma_16x8x16<T>(acc, A0.z, A1.z, A0.w, A1.w, qb[kk].z, qb[kk].w);
+  }
 }
 
 template <typename T, int D, int G>
@@ -238,16 +273,26 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   const unsigned gmask = group_mask<LPR>();
   int q = 0;                                                         // running stage counter across the passes
 
-  // ---- query fragments, pre-scaled by log2(e)/sqrt(d)
-  float qf[G][EPV];
-  {
-    const float mul = (D == 64 ? 0.125f : 0.08838834764831845f) * kLog2e;
+  // 16-bit rows and several heads per KV head: logits and cosines on mma.sync (with one head the FMA loops are
+  // as fast and use all eight warps).  The value pass stays on FMAs: its operand would need transposing loads,
+  // which conflict eight ways on the row-major stages (measured: slower than the FMA loop).
+  constexpr bool kTensor = sizeof(T) == 2 && G >= 2;
+  const float qscale = (D == 64 ? 0.125f : 0.08838834764831845f) * kLog2e;   // log2(e)/sqrt(d)
+  const int gid = lane >> 2, tig = lane & 3;
+  // ---- query fragments: fp32, pre-scaled (FMA path) or raw 16-bit pieces of query `gid` (tensor path)
+  float qf[kTensor ? 1 : G][EPV];
+  uint4 qb[D / 32];
+  if constexpr (kTensor) {
+#pragma unroll
+    for (int kk = 0; kk < D / 32; ++kk)
+      qb[kk] = gid < G ? ld_global_v4(q_in + ((size_t)sl * G + gid) * D + kk * 32 + tig * 8) : make_uint4(0, 0, 0, 0);
+  } else {
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       float f[EPV];
       Elem<T>::unpack(ld_global_v4(q_in + ((size_t)sl * G + g) * D + lig * EPV), f);
 #pragma unroll
-      for (int e = 0; e < EPV; ++e) qf[g][e] = f[e] * mul;
+      for (int e = 0; e < EPV; ++e) qf[g][e] = f[e] * qscale;
     }
   }
   // the new token's rows, kept by the first row group
@@ -258,33 +303,68 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   float mloc[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) mloc[g] = -INFINITY;
-  for (int s = 0; s < n_st; ++s, ++q) {
-    const int slot = q % NS;
-    if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
-    const uint4* st = ring + (size_t)slot * SR * LPR;
-    float dot[G][4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int lr = u * NGRP + grp;
-      float f[EPV];
-      Elem<T>::unpack(s * SR + lr < n ? st[(size_t)lr * LPR + lig] : make_uint4(0, 0, 0, 0), f);
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float x = 0.f;
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) x = fmaf(qf[g][e], f[e], x);
-        dot[g][u] = x;
+  if constexpr (kTensor) {
+    // warp w takes rows [16 w, 16 w + 16) of a stage (a stage has SR / 16 such tiles; the other warps only
+    // hand the stage back); thread (gid, tig) ends up with rows gid, gid + 8 against heads 2 tig, 2 tig + 1
+    float mm0 = -INFINITY, mm1 = -INFINITY;
+    for (int s = 0; s < n_st; ++s, ++q) {
+      const int slot = q % NS;
+      if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+      const uint4* st = ring + (size_t)slot * SR * LPR;
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      if (warp * 16 < SR && s * SR + warp * 16 < n) tile_dots<T, D>(st, warp * 16, qb, acc);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[slot]);
+      if (warp * 16 < SR && 2 * tig < G) {
+        const int li0 = s * SR + warp * 16 + gid, li1 = li0 + 8;
+        const float x00 = acc[0] * qscale, x01 = acc[1] * qscale, x10 = acc[2] * qscale, x11 = acc[3] * qscale;
+        if (li0 < n) {
+          pl[(size_t)(2 * tig) * a.row_cap + li0] = x00; mm0 = fmaxf(mm0, x00);
+          if (2 * tig + 1 < G) { pl[(size_t)(2 * tig + 1) * a.row_cap + li0] = x01; mm1 = fmaxf(mm1, x01); }
+        }
+        if (li1 < n) {
+          pl[(size_t)(2 * tig) * a.row_cap + li1] = x10; mm0 = fmaxf(mm0, x10);
+          if (2 * tig + 1 < G) { pl[(size_t)(2 * tig + 1) * a.row_cap + li1] = x11; mm1 = fmaxf(mm1, x11); }
+        }
       }
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&s_empty[slot]);
-    const int li = s * SR + (lig / QL) * NGRP + grp;                 // the row whose total this lane receives
+    // maxima over the rows (lanes with the same tig), then every lane gets every head's maximum
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      const float r = reduce4<LPR>(dot[g][0], dot[g][1], dot[g][2], dot[g][3], lig);
-      if (li < n) {
-        mloc[g] = fmaxf(mloc[g], r);
-        if (lig % QL == 0) pl[(size_t)g * a.row_cap + li] = r;
+    for (int o = 4; o < 32; o <<= 1) {
+      mm0 = fmaxf(mm0, __shfl_xor_sync(0xffffffffu, mm0, o));
+      mm1 = fmaxf(mm1, __shfl_xor_sync(0xffffffffu, mm1, o));
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) mloc[g] = __shfl_sync(0xffffffffu, (g & 1) ? mm1 : mm0, g >> 1);
+  } else {
+    for (int s = 0; s < n_st; ++s, ++q) {
+      const int slot = q % NS;
+      if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+      const uint4* st = ring + (size_t)slot * SR * LPR;
+      float dot[G][4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int lr = u * NGRP + grp;
+        float f[EPV];
+        Elem<T>::unpack(s * SR + lr < n ? st[(size_t)lr * LPR + lig] : make_uint4(0, 0, 0, 0), f);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          float x = 0.f;
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) x = fmaf(qf[g][e], f[e], x);
+          dot[g][u] = x;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[slot]);
+      const int li = s * SR + (lig / QL) * NGRP + grp;               // the row whose total this lane receives
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float r = reduce4<LPR>(dot[g][0], dot[g][1], dot[g][2], dot[g][3], lig);
+        if (li < n) {
+          mloc[g] = fmaxf(mloc[g], r);
+          if (lig % QL == 0) pl[(size_t)g * a.row_cap + li] = r;
+        }
       }
     }
   }
@@ -372,33 +452,66 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
     float kvic[EPV];
     Elem<T>::unpack(ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) + lig * EPV), kvic);
     unsigned long long best = 0ull; int best_li = -1;
-    for (int s = 0; s < n_st; ++s, ++q) {
-      const int slot = q % NS;
-      if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
-      const uint4* st = ring + (size_t)slot * SR * LPR;
-      float dot[4];
+    if constexpr (kTensor) {
+      // the victim's key as the only vector of the B operand: lanes with tig = 0 receive the dot products
+      uint4 vb[D / 32];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int lr = u * NGRP + grp;
-        float f[EPV];
-        Elem<T>::unpack(s * SR + lr < n ? st[(size_t)lr * LPR + lig] : make_uint4(0, 0, 0, 0), f);
-        float x = 0.f;
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], f[e], x);
-        dot[u] = x;
+      for (int kk = 0; kk < D / 32; ++kk)
+        vb[kk] = gid == 0 ? ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) + kk * 32 + tig * 8)
+                          : make_uint4(0, 0, 0, 0);
+      for (int s = 0; s < n_st; ++s, ++q) {
+        const int slot = q % NS;
+        if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+        const uint4* st = ring + (size_t)slot * SR * LPR;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const bool active = warp * 16 < SR && s * SR + warp * 16 < n;
+        if (active) tile_dots<T, D>(st, warp * 16, vb, acc);
+        // 1/|k| and position of this thread's two rows leave the stage before the stage is released
+        const int lr0 = warp * 16 + gid, li0 = s * SR + lr0, li1 = li0 + 8;
+        const bool m0 = active && tig == 0 && li0 < n && li0 != vic_li, m1 = active && tig == 0 && li1 < n && li1 != vic_li;
+        float rn0 = s_new_rn, rn1 = s_new_rn; int ps0 = a.t, ps1 = a.t;
+        if (m0 && li0 < n_old) { rn0 = meta_rn[(size_t)slot * SR + lr0]; ps0 = meta_ps[(size_t)slot * SR + lr0]; }
+        if (m1 && li1 < n_old) { rn1 = meta_rn[(size_t)slot * SR + lr0 + 8]; ps1 = meta_ps[(size_t)slot * SR + lr0 + 8]; }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_empty[slot]);
+        if (m0) {                                                    // max similarity, ties -> earliest position
+          const unsigned long long key = ((unsigned long long)float_ord(acc[0] * vic_rn * rn0) << 32) | (uint32_t)(0x7fffffff - ps0);
+          if (key > best) { best = key; best_li = li0; }
+        }
+        if (m1) {
+          const unsigned long long key = ((unsigned long long)float_ord(acc[2] * vic_rn * rn1) << 32) | (uint32_t)(0x7fffffff - ps1);
+          if (key > best) { best = key; best_li = li1; }
+        }
       }
-      // the row whose total this lane receives; its 1/|k| and position leave the stage before the stage is released
-      const int li = s * SR + (lig / QL) * NGRP + grp;
-      const bool mine = li < n && lig % QL == 0 && li != vic_li;
-      float rn_li = s_new_rn; int ps_li = a.t;
-      if (mine && li < n_old) { rn_li = meta_rn[(size_t)slot * SR + (li - s * SR)]; ps_li = meta_ps[(size_t)slot * SR + (li - s * SR)]; }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&s_empty[slot]);
-      const float r = reduce4<LPR>(dot[0], dot[1], dot[2], dot[3], lig);
-      if (mine) {                                                    // max similarity, ties -> earliest position
-        const float u = r * vic_rn * rn_li;
-        const unsigned long long key = ((unsigned long long)float_ord(u) << 32) | (uint32_t)(0x7fffffff - ps_li);
-        if (key > best) { best = key; best_li = li; }
+    } else {
+    for (int s = 0; s < n_st; ++s, ++q) {
+        const int slot = q % NS;
+        if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+        const uint4* st = ring + (size_t)slot * SR * LPR;
+        float dot[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int lr = u * NGRP + grp;
+          float f[EPV];
+          Elem<T>::unpack(s * SR + lr < n ? st[(size_t)lr * LPR + lig] : make_uint4(0, 0, 0, 0), f);
+          float x = 0.f;
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], f[e], x);
+          dot[u] = x;
+        }
+        // the row whose total this lane receives; its 1/|k| and position leave the stage before the stage is released
+        const int li = s * SR + (lig / QL) * NGRP + grp;
+        const bool mine = li < n && lig % QL == 0 && li != vic_li;
+        float rn_li = s_new_rn; int ps_li = a.t;
+        if (mine && li < n_old) { rn_li = meta_rn[(size_t)slot * SR + (li - s * SR)]; ps_li = meta_ps[(size_t)slot * SR + (li - s * SR)]; }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_empty[slot]);
+        const float r = reduce4<LPR>(dot[0], dot[1], dot[2], dot[3], lig);
+        if (mine) {                                                    // max similarity, ties -> earliest position
+          const float u = r * vic_rn * rn_li;
+          const unsigned long long key = ((unsigned long long)float_ord(u) << 32) | (uint32_t)(0x7fffffff - ps_li);
+          if (key > best) { best = key; best_li = li; }
+        }
       }
     }
     block_arg_extreme<false>(best, best_li, s_key, s_li, &s_best_key, &s_best_li);
