@@ -36,7 +36,7 @@ DECODE_TRAFFIC_RATIO = 1.035      # ncu DRAM bytes / algorithmic bytes of decode
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="cfg1")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the config's decode steps")
@@ -325,7 +325,7 @@ def oracle_sample(wl: W.Workload, n_slices: int, n_steps: int, threads: int = 1)
     return (t1 - t0) / len(picks), (t2 - t1) / (len(picks) * max(1, n_steps)), len(picks)
 
 
-def cpu_baseline(wl: W.Workload, n_slices=2, n_steps=32):
+def cpu_baseline(wl: W.Workload, n_slices=16, n_steps=128):
     prompt_s, step_s, n = oracle_sample(wl, n_slices, n_steps)
     total_slices = wl.n_layers * wl.batch * wl.n_kv_heads
     return {"value": round(wl.batch / (step_s * total_slices), 4), "unit": "token-steps/s", "cores": 1,
