@@ -325,7 +325,11 @@ def oracle_sample(wl: W.Workload, n_slices: int, n_steps: int, threads: int = 1)
     return (t1 - t0) / len(picks), (t2 - t1) / (len(picks) * max(1, n_steps)), len(picks)
 
 
-def cpu_baseline(wl: W.Workload, n_slices=16, n_steps=128):
+def cpu_baseline(wl: W.Workload, n_slices=0, n_steps=128):
+    if n_slices <= 0:
+        # about 10 s of prompt-stage oracle work: one query head of 4096 positions costs about a quarter second
+        per_slice = 0.25 * wl.group * (wl.prompt_len / 4096.0) ** 2
+        n_slices = max(1, min(16, int(8.0 / per_slice)))
     prompt_s, step_s, n = oracle_sample(wl, n_slices, n_steps)
     total_slices = wl.n_layers * wl.batch * wl.n_kv_heads
     return {"value": round(wl.batch / (step_s * total_slices), 4), "unit": "token-steps/s", "cores": 1,
