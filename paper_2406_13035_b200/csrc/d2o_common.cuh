@@ -163,6 +163,7 @@ struct d2o_ctx {
   int32_t* layer_steps;        // [L] decode steps taken
   int32_t* h_order;            // [L * B] (layer * B + b) sorted by cache size, largest first (device copy in `state`)
   int decode_stages;           // tuning: stages of the decode kernel's ring, 0 = auto
+  int decode_warps;            // tuning: consumer warps per decode CTA (4, 8, 16), 0 = auto
   int decode_l2_hints;         // tuning: 1 = the decode kernel's copies carry L2 eviction hints
   int similarity_path;         // tuning: 0 = tensor cores for 16-bit keys, 1 = FFMA kernel for every dtype
   int stats_path;              // tuning: 0 = tensor cores for the column sums of 16-bit Q/K, 1 = FFMA kernels

@@ -355,7 +355,7 @@ extern "C" d2o_status d2o_get_stats(d2o_ctx* c, d2o_stats* out, void* stream) {
 }
 
 extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t decode_l2_hints,
-                                     int32_t similarity_path, int32_t stats_path) {
+                                     int32_t similarity_path, int32_t stats_path, int32_t decode_warps) {
   if (!c) return D2O_ERR_INVALID_ARG;
   if (decode_stages < 0 || decode_stages > 12) return D2O_ERR_INVALID_ARG;
   if (decode_l2_hints < 0 || decode_l2_hints > 1) return D2O_ERR_INVALID_ARG;
@@ -363,6 +363,8 @@ extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t 
   c->decode_stages = decode_stages;
   c->decode_l2_hints = decode_l2_hints;
   c->similarity_path = similarity_path;
+  if (decode_warps != 0 && decode_warps != 4 && decode_warps != 8 && decode_warps != 16) return D2O_ERR_INVALID_ARG;
   c->stats_path = stats_path;
+  c->decode_warps = decode_warps;
   return D2O_OK;
 }

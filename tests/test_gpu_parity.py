@@ -51,6 +51,13 @@ def test_ring_depths_agree(stages, hints):
     assert_report(rep, wl.dtype)
 
 
+@pytest.mark.parametrize("name,warps", [("cfg1", 4), ("cfg4", 4), ("cfg2", 16), ("cfg3", 16)])
+def test_decode_cta_sizes_agree(name, warps):
+    wl = W.twin(name)
+    rep = run_parity(wl, decode_warps=warps, steps=8)
+    assert_report(rep, wl.dtype)
+
+
 def test_layer_by_layer_calls_match():
     wl = W.twin("cfg1")
     rep = run_parity(wl, layers_per_call=1, steps=6)
