@@ -46,6 +46,7 @@ def parse():
     ap.add_argument("--no-l2-hints", action="store_true", help="decode kernel: copies without L2 eviction hints")
     ap.add_argument("--ffma-similarity", action="store_true", help="prompt-stage similarity on the FFMA kernel")
     ap.add_argument("--ffma-stats", action="store_true", help="column sums of the prompt attention on the FFMA kernels")
+    ap.add_argument("--full-cache", action="store_true", help="also time the uncompressed decode-attention kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers-per-call", type=int, default=0)
@@ -107,6 +108,21 @@ def prepare_inputs(wl: W.Workload, device, decode_steps: int):
         qs, ks, vs = zip(*[s.decode() for s in streams])
         dq.append(torch.stack(qs)); dk.append(torch.stack(ks)); dv.append(torch.stack(vs))
     return prompts, torch.stack(dq), torch.stack(dk), torch.stack(dv)
+
+
+def max_over_ranks(values, world: int, device):
+    """Element-wise maximum of a list of per-rank timings over all ranks (the replicas share no data path: this is
+    the only exchange).  Returns the list unchanged for a single rank."""
+    if world <= 1:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_rate(per_gpu_units: float, world: int, ms: float) -> float:
+    """Units all ranks processed per second, given the slowest rank's time."""
+    return world * per_gpu_units / (ms * 1e-3)
 
 
 def workload_string(wl: W.Workload, nd: int) -> str:
@@ -199,10 +215,8 @@ def run_ours(args, wl, rank, world, device):
     pass_ms = stats_ms + budget_ms + compress_ms + decode_ms
     budgets = passes[-1][1]
     # max over ranks
-    if world > 1:
-        t = torch.tensor([stats_ms, budget_ms, compress_ms, decode_ms, pass_ms], device=device, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        stats_ms, budget_ms, compress_ms, decode_ms, pass_ms = t.tolist()
+    stats_ms, budget_ms, compress_ms, decode_ms, pass_ms = max_over_ranks(
+        [stats_ms, budget_ms, compress_ms, decode_ms, pass_ms], world, device)
     steps_per_s = nd / (decode_ms * 1e-3)
     # roofline of the dominant kernel (decode): algorithmic bytes per launch / average launch duration
     P = wl.prompt_len
@@ -258,18 +272,45 @@ def run_ours(args, wl, rank, world, device):
         e1.record()
         sync_all()
         ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=device, dtype=torch.float64)
-            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-            ms = float(t.item())
-        e2e = {"value": round(world * wl.batch * n_e2e / (ms * 1e-3), 2), "unit": "token-steps/s",
+        ms = max_over_ranks([ms], world, device)[0]
+        e2e = {"value": round(whole_job_rate(wl.batch * n_e2e, world, ms), 2), "unit": "token-steps/s",
                "h2d_bytes_per_step": int(hq[0].numel() * hq.element_size() + 2 * hk[0].numel() * hk.element_size()),
                "d2h_bytes_per_step": int(ho.numel() * ho.element_size()), "steps": n_e2e}
+    # the uncompressed comparison: decode attention over the full cache of prompt + generated tokens, all layers per call
+    full = None
+    if args.full_cache or wl.name.startswith("cfg4"):
+        n_sl = L * wl.batch * wl.n_kv_heads
+        nf = min(nd, 32)
+        cap = P + nf
+        g = torch.Generator(device=device).manual_seed(wl.seed + 99)
+        kc = torch.randn(n_sl, cap, wl.d_head, generator=g, device=device).to(dq.dtype)
+        vc = torch.randn(n_sl, cap, wl.d_head, generator=g, device=device).to(dq.dtype)
+        fq = dq[:nf].reshape(nf, n_sl, wl.group, wl.d_head).contiguous()
+        fk = dk[:nf].reshape(nf, n_sl, wl.d_head).contiguous()
+        fv = dv[:nf].reshape(nf, n_sl, wl.d_head).contiguous()
+        fo = torch.empty_like(fq[0])
+        for s in range(min(3, nf)):
+            B.d2o_full_decode_step(kc, vc, P + s, fq[s], fk[s], fv[s], fo)
+        sync_all()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for s in range(nf):
+            B.d2o_full_decode_step(kc, vc, P + s, fq[s], fk[s], fv[s], fo)
+        e1.record()
+        sync_all()
+        fms = max_over_ranks([e0.elapsed_time(e1)], world, device)[0]
+        esz = 4 if wl.dtype == "f32" else 2
+        fbytes = n_sl * (P + (nf - 1) / 2.0 + 1) * 2 * wl.d_head * esz
+        full = {"kernel": "full_decode_kernel", "us_per_step": round(fms * 1e3 / nf, 2), "steps": nf,
+                "cache_rows": [P, P + nf], "achieved_GBps": round(fbytes / (fms * 1e-3 / nf) / 1e9, 1),
+                "frac_of_hbm_peak": round(fbytes / (fms * 1e-3 / nf) / 1e9 / peak, 4),
+                "compressed_over_full_speedup": round((fms / nf) / (decode_ms / nd), 2)}
+        del kc, vc
     st = ctx.d2o_get_stats()
     if st.error_word != 0:
         raise RuntimeError(f"device error word {st.error_word} ({st.error_detail:#x})")
     res = {
-        "metric": METRIC, "value": round(world * wl.batch * steps_per_s, 2), "unit": "token-steps/s",
+        "metric": METRIC, "value": round(whole_job_rate(wl.batch * nd, world, decode_ms), 2), "unit": "token-steps/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(pass_ms, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
         "config": {"workload": workload_string(wl, nd),
@@ -281,7 +322,7 @@ def run_ours(args, wl, rank, world, device):
         "decode_ms": round(decode_ms, 3), "wall_s": round(t_wall, 3),
         "budgets_min_max": [int(budgets.min()), int(budgets.max())],
         "merges_discards": [int(st.merges), int(st.discards)],
-        "roofline": roofline, "tensor_phases": tensor_phases, "e2e": e2e, "gpu_launches": launches["n"], "clocks": clocks,
+        "roofline": roofline, "tensor_phases": tensor_phases, "full_cache_decode": full, "e2e": e2e, "gpu_launches": launches["n"], "clocks": clocks,
     }
     ctx.close()
     return res
