@@ -43,6 +43,8 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--stages", type=int, default=0, help="stages of the decode kernel's ring (0 = auto)")
     ap.add_argument("--decode-warps", type=int, default=0, help="consumer warps per decode CTA (0 = auto)")
+    ap.add_argument("--smem-rows", type=int, default=0,
+                    help="decode kernel: rows of a slice with their logits in shared memory (0 = auto)")
     ap.add_argument("--no-l2-hints", action="store_true", help="decode kernel: copies without L2 eviction hints")
     ap.add_argument("--ffma-similarity", action="store_true", help="prompt-stage similarity on the FFMA kernel")
     ap.add_argument("--ffma-stats", action="store_true", help="column sums of the prompt attention on the FFMA kernels")
@@ -154,9 +156,10 @@ def run_ours(args, wl, rank, world, device):
                         n_sink=wl.n_sink, window=wl.window, nm_ratio=wl.nm_ratio, beta=wl.beta,
                         density_temp=wl.density_temp, min_budget=wl.min_budget, max_budget=wl.max_budget)
     ctx = B.D2OContext(cfg, device)
-    if args.stages or args.no_l2_hints or args.ffma_similarity or args.ffma_stats or args.decode_warps:
+    if (args.stages or args.no_l2_hints or args.ffma_similarity or args.ffma_stats or args.decode_warps
+            or args.smem_rows):
         ctx.d2o_set_tuning(args.stages, 0 if args.no_l2_hints else 1, 1 if args.ffma_similarity else 0,
-                           1 if args.ffma_stats else 0, args.decode_warps)
+                           1 if args.ffma_stats else 0, args.decode_warps, args.smem_rows)
     # every rank works on its own sequences: same shapes, rank-dependent seed (weak scaling, no exchange)
     import dataclasses
     wl_r = dataclasses.replace(wl, seed=wl.seed + 7919 * rank)

@@ -210,9 +210,12 @@ d2o_status d2o_get_stats(d2o_ctx* ctx, d2o_stats* out_host, void* stream);
  * (1 = yes, the default; 0 = no); similarity_path 0 = tensor-core kernel for fp16/bf16 keys at the
  * prompt stage (default), 1 = the FFMA kernel for every dtype; stats_path likewise for the column
  * sums of d2o_layer_stats; decode_warps = consumer warps per CTA of the decode kernel (0 = automatic,
- * 4 or 8 with one or two query heads per KV head, 8 or 16 with four or eight). */
+ * 4 or 8 with one or two query heads per KV head, 8 or 16 with four or eight); decode_smem_rows =
+ * rows of a slice whose logits the decode kernel keeps in shared memory, the rest going through an
+ * L2-resident array of the scratch buffer (0 = automatic, else >= 8). */
 d2o_status d2o_set_tuning(d2o_ctx* ctx, int32_t decode_stages, int32_t decode_l2_hints,
-                          int32_t similarity_path, int32_t stats_path, int32_t decode_warps);
+                          int32_t similarity_path, int32_t stats_path, int32_t decode_warps,
+                          int32_t decode_smem_rows);
 
 #ifdef __cplusplus
 }

@@ -136,7 +136,7 @@ struct Layout {            // byte offsets into `state`
   size_t status, counters, density, budgets, windows, row_off, order, len, tau, colsum, pos, score, rnorm, kpool, vpool, end;
 };
 struct ScratchLayout {     // byte offsets into `scratch`
-  size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, part_key, stage_q, stage_k, stage_v, stage_out, end;
+  size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, part_key, pl_spill, stage_q, stage_k, stage_v, stage_out, end;
 };
 
 }  // namespace d2o
@@ -164,6 +164,7 @@ struct d2o_ctx {
   int32_t* h_order;            // [L * B] (layer * B + b) sorted by cache size, largest first (device copy in `state`)
   int decode_stages;           // tuning: stages of the decode kernel's ring, 0 = auto
   int decode_warps;            // tuning: consumer warps per decode CTA (4, 8, 16), 0 = auto
+  int decode_smem_rows;        // tuning: rows of a slice with their logits in shared memory, 0 = auto
   int decode_l2_hints;         // tuning: 1 = the decode kernel's copies carry L2 eviction hints
   int similarity_path;         // tuning: 0 = tensor cores for 16-bit keys, 1 = FFMA kernel for every dtype
   int stats_path;              // tuning: 0 = tensor cores for the column sums of 16-bit Q/K, 1 = FFMA kernels

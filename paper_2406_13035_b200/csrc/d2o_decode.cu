@@ -22,6 +22,7 @@
 #include <cuda/std/type_traits>
 
 #include "d2o_common.cuh"
+#include "d2o_tc.cuh"
 
 namespace d2o {
 
@@ -32,6 +33,7 @@ namespace d2o {
 __host__ __device__ constexpr int stage_bytes_of(int cw) { return 4 * cw * 32 * 16; }
 constexpr int kMaxStages = 12;
 constexpr unsigned long long kWaitNs = 1000000000ull;   // an mbarrier wait gives up after 1 s
+constexpr uint32_t kSuspendNs = 4000u;                  // a waiting thread may stay suspended this long before it looks again
 
 struct DecodeArgs {
   const int32_t* budgets; const int32_t* windows; const int64_t* row_off;   // [B, L]
@@ -40,7 +42,8 @@ struct DecodeArgs {
   unsigned long long* counters; uint32_t* status;
   int L, l0, B, Hkv, T, t;          // t = position of the token generated in this step
   float beta, tau_override;
-  int row_cap;                      // rows the per-row shared-memory arrays are sized for (multiple of 8)
+  int row_cap;                      // rows of a slice whose logits / probabilities live in shared memory (multiple of 8)
+  float* spill;                     // the same for rows >= row_cap: [(row0 + 8 slice) G + g (stride(S) + 8) + row], stays in L2
   int stages;                       // stages of the ring
   int l2_hints;                     // 1: pass K asks L2 to keep its lines, later passes to drop theirs
   const int32_t* order;             // NULL: CTAs take (layer, b, h) in index order; else (layer * B + b) per group of Hkv CTAs
@@ -65,9 +68,9 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
   return ok != 0;
 }
 // Bounded wait: returns false (and the caller reports D2O_ERR_TIMEOUT) if the phase has not completed in time.
@@ -78,6 +81,20 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
     if (global_ns() - t0 > kWaitNs) return false;
   }
   return true;
+}
+// Wait for a stage in the kernel's loops: one probe when the phase is already complete (the common case); otherwise
+// poll until it completes, another thread has recorded a timeout, or this one does.
+__device__ __forceinline__ void stage_wait(unsigned long long* bar, uint32_t parity, volatile int* timeout) {
+  if (mbar_try_wait(bar, parity)) return;
+  const unsigned long long t0 = global_ns();
+  while (*timeout == 0) {
+    if (mbar_try_wait(bar, parity)) return;
+    if (global_ns() - t0 > kWaitNs) { *timeout = 2; return; }
+  }
+}
+// next slot of the ring; the parity flips on wrap-around
+__device__ __forceinline__ void ring_next(int& slot, uint32_t& ph, int stages) {
+  if (++slot == stages) { slot = 0; ph ^= 1u; }
 }
 // global -> this CTA's shared memory, 16-byte aligned on both sides, size a multiple of 16
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
@@ -147,6 +164,28 @@ __device__ __forceinline__ void mma_16x8x16(float (&acc)[4], uint32_t a0, uint32
   }
 }
 
+// (hi, lo) 16-bit pairs of two fp32 weights, hi + lo carrying 16 (bf16) or 22 (fp16) significant bits: x -> low half
+template <typename T>
+__device__ __forceinline__ void split_pair(float x, float y, uint32_t& hi, uint32_t& lo) {
+  if constexpr (cuda::std::is_same<T, __nv_bfloat16>::value) {
+    // hi = the upper 16 bits (the subtraction is then exact), lo = the remainder rounded
+    const uint32_t xb = __float_as_uint(x) & 0xffff0000u, yb = __float_as_uint(y) & 0xffff0000u;
+    hi = (xb >> 16) | yb;
+    const __nv_bfloat162 l = __floats2bfloat162_rn(x - __uint_as_float(xb), y - __uint_as_float(yb));
+    lo = *reinterpret_cast<const uint32_t*>(&l);
+  } else {
+    const __half xh = __float2half_rn(x), yh = __float2half_rn(y);
+    const __half2 h = __halves2half2(xh, yh);
+    const __half2 l = __halves2half2(__float2half_rn(x - __half2float(xh)), __float2half_rn(y - __half2float(yh)));
+    hi = *reinterpret_cast<const uint32_t*>(&h); lo = *reinterpret_cast<const uint32_t*>(&l);
+  }
+}
+// four 8x8 16-bit matrices, transposed on the way into registers (value rows become the A operand's columns)
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t saddr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(saddr) : "memory");
+}
+
 // Dot products of the 16 rows [lr0, lr0 + 16) of a stage with the (up to 8) vectors whose fragments are in `qb`
 // (one 16-byte piece per 32 elements of d and thread: vector gid = lane / 4, piece tig = lane % 4).
 // acc[0], acc[1] = row lr0 + gid against vectors 2 tig, 2 tig + 1; acc[2], acc[3] = row lr0 + gid + 8.
@@ -154,20 +193,32 @@ template <typename T, int D>
 __device__ __forceinline__ void tile_dots(const uint4* st, int lr0, const uint4 (&qb)[D / 32], float (&acc)[4]) {
   constexpr int LPR = D * (int)sizeof(T) / 16;
   const int gid = (threadIdx.x & 31) >> 2, tig = threadIdx.x & 3;
-  acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+  // one accumulator per 16 elements of d: the steps do not wait for one another (a chain of D / 16 dependent
+  // tensor-core steps per stage is what a warp's time would otherwise go to)
+  float part[D / 16][4];
 #pragma unroll
   for (int kk = 0; kk < D / 32; ++kk) {
     const uint4 A0 = st[(size_t)(lr0 + gid) * LPR + kk * 4 + tig];
     const uint4 A1 = st[(size_t)(lr0 + gid + 8) * LPR + kk * 4 + tig];
-    mma_16x8x16<T>(acc, A0.x, A1.x, A0.y, A1.y, qb[kk].x, qb[kk].y);
-    mma_16x8x16<T>(acc, A0.z, A1.z, A0.w, A1.w, qb[kk].z, qb[kk].w);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) part[2 * kk][e] = part[2 * kk + 1][e] = 0.f;
+    mma_16x8x16<T>(part[2 * kk], A0.x, A1.x, A0.y, A1.y, qb[kk].x, qb[kk].y);
+    mma_16x8x16<T>(part[2 * kk + 1], A0.z, A1.z, A0.w, A1.w, qb[kk].z, qb[kk].w);
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < D / 16; ++i) t += part[i][e];
+    acc[e] = t;
   }
 }
 
 template <typename T, int D, int G, int CW>
 __global__ void __launch_bounds__((CW + 1) * 32, (CW == 4 ? (G <= 2 ? 6 : 4) : (CW == 8 ? (G <= 2 ? 4 : 2) : 1)))
-decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_in, const T* __restrict__ v_in,
-              T* __restrict__ out, T* __restrict__ kpool, T* __restrict__ vpool) {
+decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* __restrict__ q_in,
+              const T* __restrict__ k_in, const T* __restrict__ v_in, T* __restrict__ out, T* __restrict__ kpool,
+              T* __restrict__ vpool) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;                  // lanes that share one row (16-byte segment each)
   constexpr int kConsWarps = CW, kConsThreads = CW * 32, kStageBytes = stage_bytes_of(CW);
@@ -176,6 +227,11 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   constexpr int QL = LPR / 4;                   // lanes that end up with the same row total after reduce4
   constexpr int ROWB = D * (int)sizeof(T);      // bytes per row
 
+  // 16-bit rows and several heads per KV head: logits, cosines and outputs on mma.sync (with one head the FMA loops
+  // are as fast and use every warp).  The value stages then arrive through a tiled tensor map with the 128-byte
+  // swizzle, because the value pass reads them with transposing matrix loads, which would conflict eight ways on
+  // row-major 256-byte rows.
+  constexpr bool kTensor = sizeof(T) == 2 && G >= 2;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // ---- which slice: in index order, or largest caches first through the order table
   const int h = (int)blockIdx.x % a.Hkv;
@@ -205,19 +261,31 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   const int NS = a.stages;
 
   // ---- shared memory
-  extern __shared__ __align__(128) unsigned char dsm[];
+  extern __shared__ __align__(1024) unsigned char dsm[];
   uint4* ring = reinterpret_cast<uint4*>(dsm);                       // [stages][SR][LPR]
   float* red = reinterpret_cast<float*>(dsm);                        // [warps][G][D], aliases the ring once it is drained
   float* meta_rn = reinterpret_cast<float*>(dsm + (size_t)NS * kStageBytes);   // [stages][SR] 1/|k| of a pass-K' stage's rows
   int* meta_ps = reinterpret_cast<int*>(meta_rn + (size_t)NS * SR);  // [stages][SR] positions of a pass-K' stage's rows
   float* pl = reinterpret_cast<float*>(meta_ps + (size_t)NS * SR);   // [G][row_cap] logits -> probabilities
   uint4* stash = reinterpret_cast<uint4*>(pl + (size_t)G * a.row_cap);   // [2][LPR] value rows of the victim / the neighbour
+  // rows beyond row_cap (slices much longer than most): same array in global memory, which the CTA rewrites every
+  // step and which therefore stays in L2; 16 bytes per row against the 768 streamed for its key and value
+  float* const pl_far = a.spill + (size_t)(row0 + 8 * (int64_t)sidx) * G;
+  const int far_stride = slice_stride(S) + 8;
+  auto pl_get = [&](int g, int li) -> float {
+    if (li < a.row_cap) return pl[(size_t)g * a.row_cap + li];
+    return pl_far[(size_t)g * far_stride + li];
+  };
+  auto pl_put = [&](int g, int li, float x) {
+    if (li < a.row_cap) pl[(size_t)g * a.row_cap + li] = x;
+    else pl_far[(size_t)g * far_stride + li] = x;
+  };
   __shared__ unsigned long long s_full[kMaxStages], s_empty[kMaxStages];
   __shared__ float s_new_rn, s_new_score;                            // inverse key norm and accumulated score of the new token
   __shared__ float s_red[2][kConsWarps][G];
   __shared__ unsigned long long s_key[kConsWarps], s_best_key;
   __shared__ int s_li[kConsWarps], s_best_li;
-  __shared__ int s_timeout;
+  __shared__ volatile int s_timeout;
 
   if (tid == 0) {
     // once an anomaly has been recorded (by this or an earlier launch) no wait is attempted any more
@@ -237,20 +305,30 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
       }
       const int n_pass = evict ? 3 : 2;
-      int q = 0;
+      int slot = 0, q = 0;
+      uint32_t ph = 1;                                               // parity of the previous use of a slot
       for (int p = 0; p < n_pass; ++p) {
         const bool is_v = (p == n_pass - 1);
         const T* pool = is_v ? vpool : kpool;
         const T* fresh = is_v ? v_new : k_new;
         const bool hint = a.l2_hints != 0;
         const unsigned long long pol = (p == 0 && evict) ? keep : drop;
-        for (int s = 0; s < n_st; ++s, ++q) {
-          const int slot = q % NS;
-          if (q >= NS && !s_timeout && !mbar_wait(&s_empty[slot], (uint32_t)(((q / NS) - 1) & 1))) s_timeout = 2;
+        for (int s = 0; s < n_st; ++s, ++q, ring_next(slot, ph, NS)) {
+          if (q >= NS) stage_wait(&s_empty[slot], ph, &s_timeout);
           const int a0 = s * SR, a1 = min(n, a0 + SR);
           const int np = max(0, min(a1, n_old) - a0);                // cache rows of the stage
           const bool nw = n_old >= a0 && n_old < a1;                 // the new token's row falls into the stage
           uint4* dst = ring + (size_t)slot * SR * LPR;
+          if (kTensor && is_v) {
+            // swizzled [d half][SR rows][128 B]; the box always has SR rows (what lies past the cache rows is zeroed
+            // by the consumers); the new token's value row is added from the inputs at the end
+            mbar_expect_tx(&s_full[slot], (uint32_t)(SR * ROWB));
+#pragma unroll
+            for (int hf = 0; hf < ROWB / 128; ++hf)
+              tc::tma_load_2d(reinterpret_cast<unsigned char*>(dst) + (size_t)hf * SR * 128, &map_v, hf * 64, (int)(row0 + a0),
+                              &s_full[slot]);
+            continue;
+          }
           // pass K' also needs 1/|k| and the position of its rows (16-byte granules: up to 3 entries past n_old
           // come from the slice's padding and are never used)
           const bool with_meta = evict && p == 1 && np > 0;
@@ -274,12 +352,9 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
   // =========================================================================== consumer warps
   const int grp = tid / LPR, lig = tid % LPR;
   const unsigned gmask = group_mask<LPR>();
-  int q = 0;                                                         // running stage counter across the passes
+  int slot = 0;                                                      // ring position and parity, running across the passes
+  uint32_t ph = 0;
 
-  // 16-bit rows and several heads per KV head: logits and cosines on mma.sync (with one head the FMA loops are
-  // as fast and use all eight warps).  The value pass stays on FMAs: its operand would need transposing loads,
-  // which conflict eight ways on the row-major stages (measured: slower than the FMA loop).
-  constexpr bool kTensor = sizeof(T) == 2 && G >= 2;
   const float qscale = (D == 64 ? 0.125f : 0.08838834764831845f) * kLog2e;   // log2(e)/sqrt(d)
   const int gid = lane >> 2, tig = lane & 3;
   // ---- query fragments: fp32, pre-scaled (FMA path) or raw 16-bit pieces of query `gid` (tensor path)
@@ -307,27 +382,45 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
 #pragma unroll
   for (int g = 0; g < G; ++g) mloc[g] = -INFINITY;
   if constexpr (kTensor) {
-    // warp w takes rows [16 w, 16 w + 16) of a stage (a stage has SR / 16 such tiles; the other warps only
-    // hand the stage back); thread (gid, tig) ends up with rows gid, gid + 8 against heads 2 tig, 2 tig + 1
+    // a stage has SR / 16 tiles of 16 rows, half as many as there are warps: the lower half of the warps takes the
+    // even stages, the upper half the odd ones (the others only hand the stage back), so that two stages are worked
+    // on at a time; thread (gid, tig) ends up with rows gid, gid + 8 of its tile against heads 2 tig, 2 tig + 1
     float mm0 = -INFINITY, mm1 = -INFINITY;
-    for (int s = 0; s < n_st; ++s, ++q) {
-      const int slot = q % NS;
-      if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+    const int n_plain = min(n, a.row_cap);                           // rows whose logits go to shared memory unchecked
+    constexpr int kTiles = SR / 16;
+    // this warp's tile in the even / the odd stages (-1: none), and where its logits go
+    const int tile_even = warp < kTiles ? warp : -1, tile_odd = warp >= kTiles && warp < 2 * kTiles ? warp - kTiles : -1;
+    float* const pl_mine = pl + (size_t)(2 * tig) * a.row_cap + gid;
+    for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
+      stage_wait(&s_full[slot], ph, &s_timeout);
       const uint4* st = ring + (size_t)slot * SR * LPR;
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
-      if (warp * 16 < SR && s * SR + warp * 16 < n) tile_dots<T, D>(st, warp * 16, qb, acc);
+      const int tile = (s & 1) ? tile_odd : tile_even;
+      const int lt = s * SR + tile * 16;                             // first row of the tile
+      const bool mine = tile >= 0 && lt < n;
+      if (mine) tile_dots<T, D>(st, tile * 16, qb, acc);
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_empty[slot]);
-      if (warp * 16 < SR && 2 * tig < G) {
-        const int li0 = s * SR + warp * 16 + gid, li1 = li0 + 8;
+      if (mine && 2 * tig < G) {
+        const int li0 = lt + gid, li1 = li0 + 8;
         const float x00 = acc[0] * qscale, x01 = acc[1] * qscale, x10 = acc[2] * qscale, x11 = acc[3] * qscale;
+        if (lt + 16 <= n_plain) {
+          float* p = pl_mine + lt;
+          p[0] = x00; p[8] = x10;
+          mm0 = fmaxf(mm0, fmaxf(x00, x10));
+          if (G > 1) {
+            p[a.row_cap] = x01; p[a.row_cap + 8] = x11;
+            mm1 = fmaxf(mm1, fmaxf(x01, x11));
+          }
+          continue;
+        }
         if (li0 < n) {
-          pl[(size_t)(2 * tig) * a.row_cap + li0] = x00; mm0 = fmaxf(mm0, x00);
-          if (2 * tig + 1 < G) { pl[(size_t)(2 * tig + 1) * a.row_cap + li0] = x01; mm1 = fmaxf(mm1, x01); }
+          pl_put(2 * tig, li0, x00); mm0 = fmaxf(mm0, x00);
+          if (2 * tig + 1 < G) { pl_put(2 * tig + 1, li0, x01); mm1 = fmaxf(mm1, x01); }
         }
         if (li1 < n) {
-          pl[(size_t)(2 * tig) * a.row_cap + li1] = x10; mm0 = fmaxf(mm0, x10);
-          if (2 * tig + 1 < G) { pl[(size_t)(2 * tig + 1) * a.row_cap + li1] = x11; mm1 = fmaxf(mm1, x11); }
+          pl_put(2 * tig, li1, x10); mm0 = fmaxf(mm0, x10);
+          if (2 * tig + 1 < G) { pl_put(2 * tig + 1, li1, x11); mm1 = fmaxf(mm1, x11); }
         }
       }
     }
@@ -340,9 +433,8 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
 #pragma unroll
     for (int g = 0; g < G; ++g) mloc[g] = __shfl_sync(0xffffffffu, (g & 1) ? mm1 : mm0, g >> 1);
   } else {
-    for (int s = 0; s < n_st; ++s, ++q) {
-      const int slot = q % NS;
-      if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+    for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
+      stage_wait(&s_full[slot], ph, &s_timeout);
       const uint4* st = ring + (size_t)slot * SR * LPR;
       float dot[G][4];
 #pragma unroll
@@ -366,7 +458,7 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
         const float r = reduce4<LPR>(dot[g][0], dot[g][1], dot[g][2], dot[g][3], lig);
         if (li < n) {
           mloc[g] = fmaxf(mloc[g], r);
-          if (lig % QL == 0) pl[(size_t)g * a.row_cap + li] = r;
+          if (lig % QL == 0) pl_put(g, li, r);
         }
       }
     }
@@ -397,11 +489,24 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
     float sum[G];
 #pragma unroll
     for (int g = 0; g < G; ++g) sum[g] = 0.f;
-    for (int li = tid; li < n; li += kConsThreads) {
+    // cache rows with their logits in shared memory go four at a time; the last few, the new token and the rows
+    // whose logits are in global memory one by one
+    const int n_vec = (min(n_old, a.row_cap) / 4) * 4;
+    for (int li = tid * 4; li < n_vec; li += kConsThreads * 4) {
 #pragma unroll
       for (int g = 0; g < G; ++g) {
-        const float p = exp2f(pl[(size_t)g * a.row_cap + li] - m_all[g]);
-        pl[(size_t)g * a.row_cap + li] = p;
+        float4* p4 = reinterpret_cast<float4*>(pl + (size_t)g * a.row_cap + li);
+        float4 x = *p4;
+        x.x = exp2f(x.x - m_all[g]); x.y = exp2f(x.y - m_all[g]); x.z = exp2f(x.z - m_all[g]); x.w = exp2f(x.w - m_all[g]);
+        *p4 = x;
+        sum[g] += (x.x + x.y) + (x.z + x.w);
+      }
+    }
+    for (int li = n_vec + tid; li < n; li += kConsThreads) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float p = exp2f(pl_get(g, li) - m_all[g]);
+        pl_put(g, li, p);
         sum[g] += p;
       }
     }
@@ -416,10 +521,35 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       inv_l[g] = 1.0f / t;
     }
     unsigned long long my_min = ~0ull; int my_min_li = -1;
-    for (int li = tid; li < n; li += kConsThreads) {                 // each thread revisits the rows it normalised
+    for (int li = tid * 4; li < n_vec; li += kConsThreads * 4) {
+      float4 p = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float4 x = *reinterpret_cast<const float4*>(pl + (size_t)g * a.row_cap + li);
+        p.x = fmaf(x.x, inv_l[g], p.x); p.y = fmaf(x.y, inv_l[g], p.y);
+        p.z = fmaf(x.z, inv_l[g], p.z); p.w = fmaf(x.w, inv_l[g], p.w);
+      }
+      float4* sc = reinterpret_cast<float4*>(a.score + row0 + li);
+      float4 sn = *sc;
+      sn.x += p.x; sn.y += p.y; sn.z += p.z; sn.w += p.w;
+      *sc = sn;
+      if (evict) {                                                   // lowest score, ties -> latest position
+        const int4 pz = *reinterpret_cast<const int4*>(a.pos + row0 + li);
+        const float sv[4] = {sn.x, sn.y, sn.z, sn.w};
+        const int pv[4] = {pz.x, pz.y, pz.z, pz.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (pv[j] >= Tn && pv[j] <= a.t - M) {
+            const unsigned long long key = ((unsigned long long)float_ord(sv[j]) << 32) | (uint32_t)(0x7fffffff - pv[j]);
+            if (key < my_min) { my_min = key; my_min_li = li + j; }
+          }
+        }
+      }
+    }
+    for (int li = n_vec + tid; li < n; li += kConsThreads) {
       float p = 0.f;
 #pragma unroll
-      for (int g = 0; g < G; ++g) p = fmaf(pl[(size_t)g * a.row_cap + li], inv_l[g], p);
+      for (int g = 0; g < G; ++g) p = fmaf(pl_get(g, li), inv_l[g], p);
       const float s_new = (li < n_old ? a.score[row0 + li] : 0.f) + p;
       if (li < n_old || !evict) a.score[row0 + li] = s_new;          // the new token's score is placed with its row
       else s_new_score = s_new;
@@ -443,9 +573,8 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       // nothing may be evicted (S_l < T + M): report, drop the new token, keep the cache as it is.  The producer
       // still delivers two passes; they are drained without being used.
       if (tid == 0) report_error(a.status, D2O_ERR_STATE, 0xDEC00000u | (uint32_t)(sl & 0xfffff));
-      for (int s = 0; s < 2 * n_st; ++s, ++q) {
-        const int slot = q % NS;
-        if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+      for (int s = 0; s < 2 * n_st; ++s, ring_next(slot, ph, NS)) {
+        stage_wait(&s_full[slot], ph, &s_timeout);
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_empty[slot]);
       }
@@ -462,15 +591,15 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
       for (int kk = 0; kk < D / 32; ++kk)
         vb[kk] = gid == 0 ? ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) + kk * 32 + tig * 8)
                           : make_uint4(0, 0, 0, 0);
-      for (int s = 0; s < n_st; ++s, ++q) {
-        const int slot = q % NS;
-        if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+      for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
+        stage_wait(&s_full[slot], ph, &s_timeout);
         const uint4* st = ring + (size_t)slot * SR * LPR;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        const bool active = warp * 16 < SR && s * SR + warp * 16 < n;
-        if (active) tile_dots<T, D>(st, warp * 16, vb, acc);
+        const int tile = warp - (s & 1) * (SR / 16);
+        const bool active = tile >= 0 && tile < SR / 16 && s * SR + tile * 16 < n;
+        if (active) tile_dots<T, D>(st, tile * 16, vb, acc);
         // 1/|k| and position of this thread's two rows leave the stage before the stage is released
-        const int lr0 = warp * 16 + gid, li0 = s * SR + lr0, li1 = li0 + 8;
+        const int lr0 = tile * 16 + gid, li0 = s * SR + lr0, li1 = li0 + 8;
         const bool m0 = active && tig == 0 && li0 < n && li0 != vic_li, m1 = active && tig == 0 && li1 < n && li1 != vic_li;
         float rn0 = s_new_rn, rn1 = s_new_rn; int ps0 = a.t, ps1 = a.t;
         if (m0 && li0 < n_old) { rn0 = meta_rn[(size_t)slot * SR + lr0]; ps0 = meta_ps[(size_t)slot * SR + lr0]; }
@@ -487,9 +616,8 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
         }
       }
     } else {
-    for (int s = 0; s < n_st; ++s, ++q) {
-        const int slot = q % NS;
-        if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+    for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
+        stage_wait(&s_full[slot], ph, &s_timeout);
         const uint4* st = ring + (size_t)slot * SR * LPR;
         float dot[4];
 #pragma unroll
@@ -565,15 +693,112 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
     }
   }
   // ---- pass V: un-normalised outputs; the value rows of the victim and of the neighbour are picked out of the stream
-  {
+  if constexpr (kTensor) {
+    // out^T (d x heads) = V^T (d x rows) P (rows x heads) on mma.sync.  A stage holds NH = ROWB / 128 column halves
+    // of SR rows x 128 bytes, each swizzled (16-byte chunk c of row r sits at chunk c ^ (r & 7)).  Warp w takes the
+    // 16 rows rt = w / NH of half hf = w % NH: four 16 x 16 tiles of V^T, read with transposing matrix loads; the
+    // weights are split into two 16-bit terms so that the products keep fp32-like accuracy.  The new token is not in
+    // the stream: its term is added in the final reduction.
+    constexpr int NH = ROWB / 128;
+    const int hf = warp % NH, rt = warp / NH;
+    float acc[4][4];
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[mt][e] = 0.f;
+    // per-lane constants: byte offsets of the four transposing loads inside a stage, the weights of head gid
+    // (lanes with gid >= G read head 0: their columns of the product are never used)
+    const int krow = (lane & 7) + ((lane >> 4) & 1) * 8;             // this lane's row of the 16 x 16 tile for ldmatrix
+    const uint32_t tile_off = (uint32_t)(hf * SR * 128 + rt * 16 * 128);
+    uint32_t ld_off[4];
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
+      ld_off[mt] = tile_off + (uint32_t)(krow * 128 + (((mt * 2 + ((lane >> 3) & 1)) ^ (lane & 7)) << 4));
+    const uint32_t ring_u32 = smem_u32(ring);
+    const int gw = gid < G ? gid : 0;
+    const float* wrow = pl + (size_t)gw * a.row_cap + rt * 16 + 2 * tig;
+    const int n_fast = min(n_old, a.row_cap);                       // rows with nothing special about them
+    const int vic_row = vic_li < n_old ? vic_li : -64, nn_row = nn_li < n_old ? nn_li : -64;
+    int li0 = rt * 16;                                               // first row of this warp's tile
+    for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS), li0 += SR, wrow += SR) {
+      stage_wait(&s_full[slot], ph, &s_timeout);
+      const uint32_t stage_u32 = ring_u32 + (uint32_t)slot * (uint32_t)kStageBytes;
+      if (li0 < n_old) {
+        uint32_t bh0, bl0, bh1, bl1;
+        if (li0 + 16 <= n_fast) {
+          const float2 w0 = *reinterpret_cast<const float2*>(wrow), w1 = *reinterpret_cast<const float2*>(wrow + 8);
+          split_pair<T>(w0.x, w0.y, bh0, bl0);
+          split_pair<T>(w1.x, w1.y, bh1, bl1);
+        } else {
+          // the last rows of the cache, or rows whose weights are in global memory
+          uint4* tile = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(ring) + (size_t)slot * kStageBytes + tile_off);
+          if (li0 + 16 > n_old) {
+            // rows past the cache (the slice's padding, the next slice, or nothing at all) count as zero
+            for (int i = lane; i < 16 * 8; i += 32)
+              if (li0 + (i >> 3) >= n_old) tile[i] = make_uint4(0, 0, 0, 0);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+          }
+          const int r0 = li0 + 2 * tig;
+          float2 w0, w1;
+          w0.x = r0 < n_old ? pl_get(gw, r0) : 0.f;
+          w0.y = r0 + 1 < n_old ? pl_get(gw, r0 + 1) : 0.f;
+          w1.x = r0 + 8 < n_old ? pl_get(gw, r0 + 8) : 0.f;
+          w1.y = r0 + 9 < n_old ? pl_get(gw, r0 + 9) : 0.f;
+          split_pair<T>(w0.x, w0.y, bh0, bl0);
+          split_pair<T>(w1.x, w1.y, bh1, bl1);
+        }
+        if ((unsigned)(vic_row - li0) < 16u || (unsigned)(nn_row - li0) < 16u) {
+          const uint4* tile = reinterpret_cast<const uint4*>(reinterpret_cast<unsigned char*>(ring) + (size_t)slot * kStageBytes + tile_off);
+          if ((unsigned)(vic_row - li0) < 16u && lane < 8) {
+            const int r = vic_row - li0;
+            stash[hf * 8 + lane] = tile[r * 8 + (lane ^ (r & 7))];
+          }
+          if ((unsigned)(nn_row - li0) < 16u && lane < 8) {
+            const int r = nn_row - li0;
+            stash[LPR + hf * 8 + lane] = tile[r * 8 + (lane ^ (r & 7))];
+          }
+        }
+        uint32_t fa[4][4];
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt) ldmatrix_x4_trans(stage_u32 + ld_off[mt], fa[mt][0], fa[mt][1], fa[mt][2], fa[mt][3]);
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt) mma_16x8x16<T>(acc[mt], fa[mt][0], fa[mt][1], fa[mt][2], fa[mt][3], bh0, bh1);
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt) mma_16x8x16<T>(acc[mt], fa[mt][0], fa[mt][1], fa[mt][2], fa[mt][3], bl0, bl1);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[slot]);
+    }
+    // a victim or neighbour that is the new token itself
+    if (grp == 0) {
+      if (vic_li == n_old) stash[lig] = vnew;
+      if (nn_li == n_old) stash[LPR + lig] = vnew;
+    }
+    consumer_sync<CW>();                                                 // the ring is drained: reuse it
+    // red[rt][g][d]; acc[mt] = (d = hf 64 + mt 16 + gid, + 8) x (heads 2 tig, 2 tig + 1)
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int g = 2 * tig + (e & 1), dd = hf * 64 + mt * 16 + gid + (e >> 1) * 8;
+        if (g < G) red[((size_t)rt * G + g) * D + dd] = acc[mt][e];
+      }
+    consumer_sync<CW>();
+    for (int i = tid; i < G * D; i += kConsThreads) {
+      float t = pl_get(i / D, n_old) * Elem<T>::to_float(v_new[i % D]);
+#pragma unroll
+      for (int w = 0; w < kConsWarps / NH; ++w) t += red[(size_t)w * G * D + i];
+      out[(size_t)sl * G * D + i] = Elem<T>::from_float(t * inv_l[i / D]);
+    }
+  } else {
     float acc[G][EPV];
 #pragma unroll
     for (int g = 0; g < G; ++g)
 #pragma unroll
       for (int e = 0; e < EPV; ++e) acc[g][e] = 0.f;
-    for (int s = 0; s < n_st; ++s, ++q) {
-      const int slot = q % NS;
-      if (!s_timeout && !mbar_wait(&s_full[slot], (uint32_t)((q / NS) & 1))) s_timeout = 2;
+    for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
+      stage_wait(&s_full[slot], ph, &s_timeout);
       const uint4* st = ring + (size_t)slot * SR * LPR;
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -587,7 +812,7 @@ decode_kernel(DecodeArgs a, const T* __restrict__ q_in, const T* __restrict__ k_
           Elem<T>::unpack(raw, f);
 #pragma unroll
           for (int g = 0; g < G; ++g) {
-            const float p = pl[(size_t)g * a.row_cap + li];
+            const float p = pl_get(g, li);
 #pragma unroll
             for (int e = 0; e < EPV; ++e) acc[g][e] = fmaf(p, f[e], acc[g][e]);
           }
@@ -659,29 +884,31 @@ static size_t smem_bytes(int cw, int row_cap, int stages, int G, int row_bytes) 
 }
 
 template <typename T, int D, int G, int CW>
-static cudaError_t launch_one(const DecodeArgs& a, int n_slices, const void* q, const void* k, const void* v,
-                              void* out, void* kpool, void* vpool, cudaStream_t st) {
+static cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& map_v, int n_slices, const void* q, const void* k,
+                              const void* v, void* out, void* kpool, void* vpool, cudaStream_t st) {
   const size_t smem = smem_bytes(CW, a.row_cap, a.stages, G, D * (int)sizeof(T));
   auto kern = decode_kernel<T, D, G, CW>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<n_slices, (CW + 1) * 32, smem, st>>>(a, (const T*)q, (const T*)k, (const T*)v, (T*)out, (T*)kpool, (T*)vpool);
+  kern<<<n_slices, (CW + 1) * 32, smem, st>>>(a, map_v, (const T*)q, (const T*)k, (const T*)v, (T*)out, (T*)kpool, (T*)vpool);
   return cudaGetLastError();
 }
 
 // G = 1, 2: 4 or 8 consumer warps; G = 4, 8: 8 or 16
 template <typename T, int D>
-static cudaError_t launch_g(int G, int cw, const DecodeArgs& a, int n_slices, const void* q, const void* k,
-                            const void* v, void* out, void* kpool, void* vpool, cudaStream_t st) {
+static cudaError_t launch_g(int G, int cw, const DecodeArgs& a, const CUtensorMap& map_v, int n_slices, const void* q,
+                            const void* k, const void* v, void* out, void* kpool, void* vpool, cudaStream_t st) {
   switch (G) {
-    case 1: return cw == 4 ? launch_one<T, D, 1, 4>(a, n_slices, q, k, v, out, kpool, vpool, st)
-                           : launch_one<T, D, 1, 8>(a, n_slices, q, k, v, out, kpool, vpool, st);
-    case 2: return cw == 4 ? launch_one<T, D, 2, 4>(a, n_slices, q, k, v, out, kpool, vpool, st)
-                           : launch_one<T, D, 2, 8>(a, n_slices, q, k, v, out, kpool, vpool, st);
-    case 4: return cw == 16 ? launch_one<T, D, 4, 16>(a, n_slices, q, k, v, out, kpool, vpool, st)
-                            : launch_one<T, D, 4, 8>(a, n_slices, q, k, v, out, kpool, vpool, st);
-    default: return cw == 16 ? launch_one<T, D, 8, 16>(a, n_slices, q, k, v, out, kpool, vpool, st)
-                             : launch_one<T, D, 8, 8>(a, n_slices, q, k, v, out, kpool, vpool, st);
+    case 1: return cw == 4 ? launch_one<T, D, 1, 4>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                           : launch_one<T, D, 1, 8>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    case 2: return cw == 4 ? launch_one<T, D, 2, 4>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                           : launch_one<T, D, 2, 8>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    case 4: return cw == 16 ? launch_one<T, D, 4, 16>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                 : cw == 4 ? launch_one<T, D, 4, 4>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                           : launch_one<T, D, 4, 8>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    default: return cw == 16 ? launch_one<T, D, 8, 16>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                  : cw == 4 ? launch_one<T, D, 8, 4>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                            : launch_one<T, D, 8, 8>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
   }
 }
 
@@ -691,9 +918,9 @@ static int max_per_sm(int cw, int G) { return cw == 4 ? (G <= 2 ? 6 : 4) : (cw =
 // Ring depth for `max_rows` rows per slice when `per_sm` CTAs are to share an SM.  false if the per-row arrays leave
 // no room for a ring.  Occupancy matters more than depth: measured on the 7B-shaped stack with caches of 700 to
 // 1900 rows, three CTAs with two stages each beat two CTAs with three or four stages (108 us vs 113 us per step).
-static bool plan_tier(int cw, int max_rows, int row_bytes, int G, int D, int per_sm, int* row_cap, int* stages_out) {
+static bool plan_tier(int cw, int smem_rows, int row_bytes, int G, int D, int per_sm, int* row_cap, int* stages_out) {
   const long sm_total = 227 * 1024;
-  const int cap = (max_rows + 7) & ~7;
+  const int cap = (smem_rows + 7) & ~7;
   const int min_stages = max(2, (cw * G * D * 4 + stage_bytes_of(cw) - 1) / stage_bytes_of(cw));   // the ring doubles as `red`
   const long fixed = (long)G * cap * 4 + 2L * row_bytes + 2048;                               // + static shared memory
   const long room = sm_total / per_sm - 1024 - fixed;
@@ -705,16 +932,16 @@ static bool plan_tier(int cw, int max_rows, int row_bytes, int G, int D, int per
 }
 
 // Best occupancy tier that fits `max_rows`; 0 = none.
-static int best_tier(int cw, int max_rows, int row_bytes, int G, int D, int* row_cap, int* stages) {
+static int best_tier(int cw, int smem_rows, int row_bytes, int G, int D, int* row_cap, int* stages) {
   for (int per_sm = max_per_sm(cw, G); per_sm >= 1; --per_sm)
-    if (plan_tier(cw, max_rows, row_bytes, G, D, per_sm, row_cap, stages)) return per_sm;
+    if (plan_tier(cw, smem_rows, row_bytes, G, D, per_sm, row_cap, stages)) return per_sm;
   return 0;
 }
 
-static bool plan(int cw, int max_rows, int row_bytes, int G, int D, int want_stages, int* row_cap, int* stages_out) {
-  if (want_stages <= 0) return best_tier(cw, max_rows, row_bytes, G, D, row_cap, stages_out) != 0;
+static bool plan(int cw, int smem_rows, int row_bytes, int G, int D, int want_stages, int* row_cap, int* stages_out) {
+  if (want_stages <= 0) return best_tier(cw, smem_rows, row_bytes, G, D, row_cap, stages_out) != 0;
   const long sm_total = 227 * 1024;
-  const int cap = (max_rows + 7) & ~7;
+  const int cap = (smem_rows + 7) & ~7;
   const int min_stages = max(2, (cw * G * D * 4 + stage_bytes_of(cw) - 1) / stage_bytes_of(cw));
   const long fixed = (long)G * cap * 4 + 2L * row_bytes + 2048;
   if (want_stages < min_stages || want_stages > kMaxStages) return false;
@@ -723,14 +950,18 @@ static bool plan(int cw, int max_rows, int row_bytes, int G, int D, int want_sta
   return true;
 }
 
+// Rows of a slice whose logits stay in shared memory: all of them while that takes 16 KB or less; else enough for
+// slices a quarter longer than the mean (the budgets of Eq. 5 give a few layers several times the mean, and sizing
+// the array for those would cost every CTA its ring depth or the SM a resident CTA).
+static int smem_rows_for(int max_rows, double mean_rows, int G) {
+  const int free_rows = 16 * 1024 / (4 * G);
+  if (max_rows <= free_rows) return max_rows;
+  return min(max_rows, max(free_rows, (int)(1.25 * mean_rows)));
+}
+
 int decode_max_rows(int row_bytes, int group, int d_head) {
-  int lo = 0, hi = 1 << 20;                                          // largest row count for which a plan exists
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) / 2;
-    int cap, st;
-    if (plan(8, mid, row_bytes, group, d_head, 0, &cap, &st)) lo = mid; else hi = mid - 1;
-  }
-  return lo;
+  (void)row_bytes; (void)group; (void)d_head;
+  return 1 << 24;                                                    // rows beyond the shared-memory array go through L2
 }
 
 cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const void* k, const void* v, void* out,
@@ -772,23 +1003,36 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     if (G <= 2 && n_slices >= 8 * 148 * 4 && max_rows <= 1536) cw = 4;
     if (G >= 4 && n_slices <= 148 * 8 && max_rows > 2.0 * mean_rows) cw = 16;
   }
-  if ((G <= 2 && cw == 16) || (G >= 4 && cw == 4)) cw = 8;
+  if (G <= 2 && cw == 16) cw = 8;
   int row_cap, stages;
-  if (!plan(cw, max_rows, row_bytes, G, g.d_head, c->decode_stages, &row_cap, &stages)) {
+  int smem_rows = smem_rows_for(max_rows, (double)sum_rows / ((l1 - l0) * B), G);
+  if (c->decode_smem_rows > 0) smem_rows = min(max_rows, c->decode_smem_rows);
+  if (!plan(cw, smem_rows, row_bytes, G, g.d_head, c->decode_stages, &row_cap, &stages)) {
     *why = D2O_ERR_UNSUPPORTED;
     return cudaSuccess;
   }
   a.row_cap = row_cap; a.stages = stages;
+  a.spill = (float*)(c->scratch + c->slay.pl_spill);
   // all layers in one call: CTAs take the slices largest cache first, so the long ones do not end up in the tail
   a.order = (l0 == 0 && l1 == L) ? (const int32_t*)(S + c->lay.order) : nullptr;
+  // 16-bit caches with grouped queries read the value rows through a tensor map (swizzled stages)
+  CUtensorMap map_v;
+  memset(&map_v, 0, sizeof(map_v));
+  if (c->elem_size == 2 && G >= 2) {
+    const int box_rows = stage_bytes_of(cw) / row_bytes;
+    if (c->pool_rows >= (1ll << 31) || !encode_rows_2d(&map_v, g.dtype, vpool, (uint64_t)c->pool_rows, g.d_head, box_rows)) {
+      *why = D2O_ERR_UNSUPPORTED;
+      return cudaSuccess;
+    }
+  }
   if (g.dtype == D2O_F32)
-    return g.d_head == 64 ? launch_g<float, 64>(G, cw, a, n_slices, q, k, v, out, kpool, vpool, st)
-                          : launch_g<float, 128>(G, cw, a, n_slices, q, k, v, out, kpool, vpool, st);
+    return g.d_head == 64 ? launch_g<float, 64>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                          : launch_g<float, 128>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
   if (g.dtype == D2O_F16)
-    return g.d_head == 64 ? launch_g<__half, 64>(G, cw, a, n_slices, q, k, v, out, kpool, vpool, st)
-                          : launch_g<__half, 128>(G, cw, a, n_slices, q, k, v, out, kpool, vpool, st);
-  return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, cw, a, n_slices, q, k, v, out, kpool, vpool, st)
-                        : launch_g<__nv_bfloat16, 128>(G, cw, a, n_slices, q, k, v, out, kpool, vpool, st);
+    return g.d_head == 64 ? launch_g<__half, 64>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                          : launch_g<__half, 128>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+  return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                        : launch_g<__nv_bfloat16, 128>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
 }
 
 }  // namespace d2o

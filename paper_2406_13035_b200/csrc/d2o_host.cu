@@ -64,7 +64,7 @@ static d2o_status validate(const d2o_config* c, int64_t* total_budget, int* max_
   if (c->min_budget < 1 || c->min_budget < c->n_sink + 1 || c->min_budget > maxb) return D2O_ERR_INVALID_ARG;
   double tot = floor((double)c->rho * (double)c->n_layers * (double)c->prompt_len + 0.5);
   if (tot < (double)c->n_layers * c->min_budget || tot > (double)c->n_layers * maxb) return D2O_ERR_INVALID_ARG;
-  // decode kernel: the keys of one slice stay in the shared memory of one cluster
+  // decode kernel: per-row arrays of one slice
   if (maxb + 1 > decode_max_rows(c->d_head * elem_size_of(c->dtype), g, c->d_head)) return D2O_ERR_UNSUPPORTED;
   *total_budget = (int64_t)tot;
   *max_budget = maxb;
@@ -101,6 +101,7 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   s->seg_start = take(B * Hkv * ((size_t)max_budget + 2) * 4);
   s->seg_items = take(B * Hkv * P * 4);
   s->part_key = take(c->dtype == D2O_F32 ? 0 : sim_tc_part_key_bytes(c, max_budget));
+  s->pl_spill = take((rows + 8 * L * B * Hkv) * (Hq / Hkv) * 4);
   s->stage_q = take(L * B * Hq * d * e);
   s->stage_k = take(L * B * Hkv * d * e);
   s->stage_v = take(L * B * Hkv * d * e);
@@ -355,7 +356,8 @@ extern "C" d2o_status d2o_get_stats(d2o_ctx* c, d2o_stats* out, void* stream) {
 }
 
 extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t decode_l2_hints,
-                                     int32_t similarity_path, int32_t stats_path, int32_t decode_warps) {
+                                     int32_t similarity_path, int32_t stats_path, int32_t decode_warps,
+                                     int32_t decode_smem_rows) {
   if (!c) return D2O_ERR_INVALID_ARG;
   if (decode_stages < 0 || decode_stages > 12) return D2O_ERR_INVALID_ARG;
   if (decode_l2_hints < 0 || decode_l2_hints > 1) return D2O_ERR_INVALID_ARG;
@@ -364,7 +366,9 @@ extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t 
   c->decode_l2_hints = decode_l2_hints;
   c->similarity_path = similarity_path;
   if (decode_warps != 0 && decode_warps != 4 && decode_warps != 8 && decode_warps != 16) return D2O_ERR_INVALID_ARG;
+  if (decode_smem_rows != 0 && decode_smem_rows < 8) return D2O_ERR_INVALID_ARG;
   c->stats_path = stats_path;
   c->decode_warps = decode_warps;
+  c->decode_smem_rows = decode_smem_rows;
   return D2O_OK;
 }

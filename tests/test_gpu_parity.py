@@ -58,6 +58,14 @@ def test_decode_cta_sizes_agree(name, warps):
     assert_report(rep, wl.dtype)
 
 
+@pytest.mark.parametrize("name,rows", [("cfg1", 64), ("cfg2", 40), ("cfg3", 128), ("cfg0", 8)])
+def test_logits_beyond_shared_memory_agree(name, rows):
+    # most rows of every slice keep their logits in the L2-resident array instead of shared memory
+    wl = W.CONFIGS[name] if name == "cfg0" else W.twin(name)
+    rep = run_parity(wl, decode_smem_rows=rows, steps=8)
+    assert_report(rep, wl.dtype)
+
+
 def test_layer_by_layer_calls_match():
     wl = W.twin("cfg1")
     rep = run_parity(wl, layers_per_call=1, steps=6)
