@@ -107,6 +107,13 @@ __device__ __forceinline__ void bulk_g2s_hint(void* dst, const void* src, uint32
                ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
 }
 
+// 2-D tiled load with an L2 eviction-priority hint; x = innermost coordinate (elements), y = row
+__device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar,
+                                                 unsigned long long policy) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+               ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+
 // Extremum over the consumer warps of a 64-bit key with the row index of the winner (keys are unique per row).
 // The result is valid in s_out_key / s_out_li after the next consumer_sync().
 template <bool MIN, int CW>
@@ -186,24 +193,27 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t saddr, uint32_t& r0, 
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(saddr) : "memory");
 }
 
-// Dot products of the 16 rows [lr0, lr0 + 16) of a stage with the (up to 8) vectors whose fragments are in `qb`
-// (one 16-byte piece per 32 elements of d and thread: vector gid = lane / 4, piece tig = lane % 4).
-// acc[0], acc[1] = row lr0 + gid against vectors 2 tig, 2 tig + 1; acc[2], acc[3] = row lr0 + gid + 8.
-template <typename T, int D>
-__device__ __forceinline__ void tile_dots(const uint4* st, int lr0, const uint4 (&qb)[D / 32], float (&acc)[4]) {
-  constexpr int LPR = D * (int)sizeof(T) / 16;
+// Dot products of the 16 rows of tile `tile` of a swizzled stage ([d half][SR rows][128 bytes], 16-byte chunk c of
+// row r at chunk c ^ (r & 7)) with the (up to 8) vectors whose fragments are in `qb`.  Thread (gid, tig) reads chunk
+// 2 tig + (j & 1) of half j / 2 of rows gid and gid + 8 in step j: with the swizzle the eight lanes of a quarter-warp
+// hit eight different bank groups.  The order of the elements inside a step is free as long as both operands agree,
+// so a thread's piece is one vector load; `qb[j]` holds the same chunk of vector gid.
+// acc[0], acc[1] = row gid of the tile against vectors 2 tig, 2 tig + 1; acc[2], acc[3] = row gid + 8.
+template <typename T, int D, int SR>
+__device__ __forceinline__ void tile_dots(const unsigned char* stage, int tile, const uint4 (&qb)[D / 32], float (&acc)[4]) {
   const int gid = (threadIdx.x & 31) >> 2, tig = threadIdx.x & 3;
-  // one accumulator per 16 elements of d: the steps do not wait for one another (a chain of D / 16 dependent
-  // tensor-core steps per stage is what a warp's time would otherwise go to)
+  // one accumulator per 16 elements of d: the steps do not wait for one another
   float part[D / 16][4];
 #pragma unroll
-  for (int kk = 0; kk < D / 32; ++kk) {
-    const uint4 A0 = st[(size_t)(lr0 + gid) * LPR + kk * 4 + tig];
-    const uint4 A1 = st[(size_t)(lr0 + gid + 8) * LPR + kk * 4 + tig];
+  for (int j = 0; j < D / 32; ++j) {
+    const unsigned char* row = stage + (size_t)(j >> 1) * SR * 128 + (size_t)(tile * 16 + gid) * 128 +
+                               (((2 * tig + (j & 1)) ^ gid) << 4);
+    const uint4 A0 = *reinterpret_cast<const uint4*>(row);
+    const uint4 A1 = *reinterpret_cast<const uint4*>(row + 8 * 128);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) part[2 * kk][e] = part[2 * kk + 1][e] = 0.f;
-    mma_16x8x16<T>(part[2 * kk], A0.x, A1.x, A0.y, A1.y, qb[kk].x, qb[kk].y);
-    mma_16x8x16<T>(part[2 * kk + 1], A0.z, A1.z, A0.w, A1.w, qb[kk].z, qb[kk].w);
+    for (int e = 0; e < 4; ++e) part[2 * j][e] = part[2 * j + 1][e] = 0.f;
+    mma_16x8x16<T>(part[2 * j], A0.x, A1.x, A0.y, A1.y, qb[j].x, qb[j].y);
+    mma_16x8x16<T>(part[2 * j + 1], A0.z, A1.z, A0.w, A1.w, qb[j].z, qb[j].w);
   }
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
@@ -216,7 +226,8 @@ __device__ __forceinline__ void tile_dots(const uint4* st, int lr0, const uint4 
 
 template <typename T, int D, int G, int CW>
 __global__ void __launch_bounds__((CW + 1) * 32, (CW == 4 ? (G <= 2 ? 6 : 4) : (CW == 8 ? (G <= 2 ? 4 : 2) : 1)))
-decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* __restrict__ q_in,
+decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+              const T* __restrict__ q_in,
               const T* __restrict__ k_in, const T* __restrict__ v_in, T* __restrict__ out, T* __restrict__ kpool,
               T* __restrict__ vpool) {
   constexpr int EPV = Elem<T>::kPerVec;
@@ -319,20 +330,28 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* 
           const int np = max(0, min(a1, n_old) - a0);                // cache rows of the stage
           const bool nw = n_old >= a0 && n_old < a1;                 // the new token's row falls into the stage
           uint4* dst = ring + (size_t)slot * SR * LPR;
-          if (kTensor && is_v) {
-            // swizzled [d half][SR rows][128 B]; the box always has SR rows (what lies past the cache rows is zeroed
-            // by the consumers); the new token's value row is added from the inputs at the end
-            mbar_expect_tx(&s_full[slot], (uint32_t)(SR * ROWB));
-#pragma unroll
-            for (int hf = 0; hf < ROWB / 128; ++hf)
-              tc::tma_load_2d(reinterpret_cast<unsigned char*>(dst) + (size_t)hf * SR * 128, &map_v, hf * 64, (int)(row0 + a0),
-                              &s_full[slot]);
-            continue;
-          }
           // pass K' also needs 1/|k| and the position of its rows (16-byte granules: up to 3 entries past n_old
           // come from the slice's padding and are never used)
           const bool with_meta = evict && p == 1 && np > 0;
           const int np4 = (np + 3) & ~3;
+          if (kTensor) {
+            // swizzled [d half][SR rows][128 B]; the box always has SR rows (what lies past the cache rows is never
+            // used, or zeroed by the consumers); the new token's rows are not in the stream: its logits, its cosine
+            // and its term of the output are added from the inputs
+            mbar_expect_tx(&s_full[slot], (uint32_t)(SR * ROWB + (with_meta ? 2 * np4 * 4 : 0)));
+            if (with_meta) {
+              bulk_g2s(meta_rn + (size_t)slot * SR, a.rnorm + row0 + a0, (uint32_t)(np4 * 4), &s_full[slot]);
+              bulk_g2s(meta_ps + (size_t)slot * SR, a.pos + row0 + a0, (uint32_t)(np4 * 4), &s_full[slot]);
+            }
+            const CUtensorMap* map = is_v ? &map_v : &map_k;
+#pragma unroll
+            for (int hf = 0; hf < ROWB / 128; ++hf) {
+              void* to = reinterpret_cast<unsigned char*>(dst) + (size_t)hf * SR * 128;
+              if (hint) tma_load_2d_hint(to, map, hf * 64, (int)(row0 + a0), &s_full[slot], pol);
+              else tc::tma_load_2d(to, map, hf * 64, (int)(row0 + a0), &s_full[slot]);
+            }
+            continue;
+          }
           mbar_expect_tx(&s_full[slot], (uint32_t)((np + (nw ? 1 : 0)) * ROWB + (with_meta ? 2 * np4 * 4 : 0)));
           if (with_meta) {
             bulk_g2s(meta_rn + (size_t)slot * SR, a.rnorm + row0 + a0, (uint32_t)(np4 * 4), &s_full[slot]);
@@ -350,6 +369,11 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* 
   }
 
   // =========================================================================== consumer warps
+  // the accumulated scores and positions of the rows are needed right after pass K: ask L2 for their lines now
+  for (int i = tid * 32; i < n_old; i += kConsThreads * 32) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.score + row0 + i));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.pos + row0 + i));
+  }
   const int grp = tid / LPR, lig = tid % LPR;
   const unsigned gmask = group_mask<LPR>();
   int slot = 0;                                                      // ring position and parity, running across the passes
@@ -362,8 +386,9 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* 
   uint4 qb[D / 32];
   if constexpr (kTensor) {
 #pragma unroll
-    for (int kk = 0; kk < D / 32; ++kk)
-      qb[kk] = gid < G ? ld_global_v4(q_in + ((size_t)sl * G + gid) * D + kk * 32 + tig * 8) : make_uint4(0, 0, 0, 0);
+    for (int j = 0; j < D / 32; ++j)
+      qb[j] = gid < G ? ld_global_v4(q_in + ((size_t)sl * G + gid) * D + ((j >> 1) * 8 + 2 * tig + (j & 1)) * 8)
+                      : make_uint4(0, 0, 0, 0);
   } else {
 #pragma unroll
     for (int g = 0; g < G; ++g) {
@@ -386,19 +411,19 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* 
     // even stages, the upper half the odd ones (the others only hand the stage back), so that two stages are worked
     // on at a time; thread (gid, tig) ends up with rows gid, gid + 8 of its tile against heads 2 tig, 2 tig + 1
     float mm0 = -INFINITY, mm1 = -INFINITY;
-    const int n_plain = min(n, a.row_cap);                           // rows whose logits go to shared memory unchecked
+    const int n_plain = min(n_old, a.row_cap);                       // rows whose logits go to shared memory unchecked
     constexpr int kTiles = SR / 16;
     // this warp's tile in the even / the odd stages (-1: none), and where its logits go
     const int tile_even = warp < kTiles ? warp : -1, tile_odd = warp >= kTiles && warp < 2 * kTiles ? warp - kTiles : -1;
     float* const pl_mine = pl + (size_t)(2 * tig) * a.row_cap + gid;
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
       stage_wait(&s_full[slot], ph, &s_timeout);
-      const uint4* st = ring + (size_t)slot * SR * LPR;
+      const unsigned char* st = reinterpret_cast<const unsigned char*>(ring) + (size_t)slot * kStageBytes;
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
       const int tile = (s & 1) ? tile_odd : tile_even;
       const int lt = s * SR + tile * 16;                             // first row of the tile
-      const bool mine = tile >= 0 && lt < n;
-      if (mine) tile_dots<T, D>(st, tile * 16, qb, acc);
+      const bool mine = tile >= 0 && lt < n_old;
+      if (mine) tile_dots<T, D, SR>(st, tile, qb, acc);
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_empty[slot]);
       if (mine && 2 * tig < G) {
@@ -414,11 +439,11 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* 
           }
           continue;
         }
-        if (li0 < n) {
+        if (li0 < n_old) {
           pl_put(2 * tig, li0, x00); mm0 = fmaxf(mm0, x00);
           if (2 * tig + 1 < G) { pl_put(2 * tig + 1, li0, x01); mm1 = fmaxf(mm1, x01); }
         }
-        if (li1 < n) {
+        if (li1 < n_old) {
           pl_put(2 * tig, li1, x10); mm0 = fmaxf(mm0, x10);
           if (2 * tig + 1 < G) { pl_put(2 * tig + 1, li1, x11); mm1 = fmaxf(mm1, x11); }
         }
@@ -432,6 +457,22 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* 
     }
 #pragma unroll
     for (int g = 0; g < G; ++g) mloc[g] = __shfl_sync(0xffffffffu, (g & 1) ? mm1 : mm0, g >> 1);
+    if (warp == 0) {
+      // the new token's logits: its key row is held by the first LPR lanes
+      float kf[EPV];
+      Elem<T>::unpack(knew, kf);
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float qv[EPV];
+        Elem<T>::unpack(lane < LPR ? ld_global_v4(q_in + ((size_t)sl * G + g) * D + lane * EPV) : make_uint4(0, 0, 0, 0), qv);
+        float x = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) x = fmaf(qv[e], kf[e], x);
+        x = warp_sum(x) * qscale;
+        if (lane == 0) pl_put(g, n_old, x);
+        mloc[g] = fmaxf(mloc[g], x);
+      }
+    }
   } else {
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
       stage_wait(&s_full[slot], ph, &s_timeout);
@@ -588,22 +629,23 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* 
       // the victim's key as the only vector of the B operand: lanes with tig = 0 receive the dot products
       uint4 vb[D / 32];
 #pragma unroll
-      for (int kk = 0; kk < D / 32; ++kk)
-        vb[kk] = gid == 0 ? ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) + kk * 32 + tig * 8)
-                          : make_uint4(0, 0, 0, 0);
+      for (int j = 0; j < D / 32; ++j)
+        vb[j] = gid == 0 ? ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) +
+                                        ((j >> 1) * 8 + 2 * tig + (j & 1)) * 8)
+                         : make_uint4(0, 0, 0, 0);
       for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
         stage_wait(&s_full[slot], ph, &s_timeout);
-        const uint4* st = ring + (size_t)slot * SR * LPR;
+        const unsigned char* st = reinterpret_cast<const unsigned char*>(ring) + (size_t)slot * kStageBytes;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         const int tile = warp - (s & 1) * (SR / 16);
-        const bool active = tile >= 0 && tile < SR / 16 && s * SR + tile * 16 < n;
-        if (active) tile_dots<T, D>(st, tile * 16, vb, acc);
+        const bool active = tile >= 0 && tile < SR / 16 && s * SR + tile * 16 < n_old;
+        if (active) tile_dots<T, D, SR>(st, tile, vb, acc);
         // 1/|k| and position of this thread's two rows leave the stage before the stage is released
         const int lr0 = tile * 16 + gid, li0 = s * SR + lr0, li1 = li0 + 8;
-        const bool m0 = active && tig == 0 && li0 < n && li0 != vic_li, m1 = active && tig == 0 && li1 < n && li1 != vic_li;
-        float rn0 = s_new_rn, rn1 = s_new_rn; int ps0 = a.t, ps1 = a.t;
-        if (m0 && li0 < n_old) { rn0 = meta_rn[(size_t)slot * SR + lr0]; ps0 = meta_ps[(size_t)slot * SR + lr0]; }
-        if (m1 && li1 < n_old) { rn1 = meta_rn[(size_t)slot * SR + lr0 + 8]; ps1 = meta_ps[(size_t)slot * SR + lr0 + 8]; }
+        const bool m0 = active && tig == 0 && li0 < n_old && li0 != vic_li, m1 = active && tig == 0 && li1 < n_old && li1 != vic_li;
+        float rn0 = 0.f, rn1 = 0.f; int ps0 = 0, ps1 = 0;
+        if (m0) { rn0 = meta_rn[(size_t)slot * SR + lr0]; ps0 = meta_ps[(size_t)slot * SR + lr0]; }
+        if (m1) { rn1 = meta_rn[(size_t)slot * SR + lr0 + 8]; ps1 = meta_ps[(size_t)slot * SR + lr0 + 8]; }
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_empty[slot]);
         if (m0) {                                                    // max similarity, ties -> earliest position
@@ -614,6 +656,19 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_v, const T* 
           const unsigned long long key = ((unsigned long long)float_ord(acc[2] * vic_rn * rn1) << 32) | (uint32_t)(0x7fffffff - ps1);
           if (key > best) { best = key; best_li = li1; }
         }
+      }
+      if (warp == 0 && vic_li != n_old) {
+        // the new token as a merge target: its key row is held by the first LPR lanes
+        float kf[EPV];
+        Elem<T>::unpack(knew, kf);
+        float x = 0.f;
+        if (lane < LPR) {
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], kf[e], x);
+        }
+        x = warp_sum(x);
+        const unsigned long long key = ((unsigned long long)float_ord(x * vic_rn * s_new_rn) << 32) | (uint32_t)(0x7fffffff - a.t);
+        if (lane == 0 && key > best) { best = key; best_li = n_old; }
       }
     } else {
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
@@ -884,31 +939,31 @@ static size_t smem_bytes(int cw, int row_cap, int stages, int G, int row_bytes) 
 }
 
 template <typename T, int D, int G, int CW>
-static cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& map_v, int n_slices, const void* q, const void* k,
+static cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v, int n_slices, const void* q, const void* k,
                               const void* v, void* out, void* kpool, void* vpool, cudaStream_t st) {
   const size_t smem = smem_bytes(CW, a.row_cap, a.stages, G, D * (int)sizeof(T));
   auto kern = decode_kernel<T, D, G, CW>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<n_slices, (CW + 1) * 32, smem, st>>>(a, map_v, (const T*)q, (const T*)k, (const T*)v, (T*)out, (T*)kpool, (T*)vpool);
+  kern<<<n_slices, (CW + 1) * 32, smem, st>>>(a, map_k, map_v, (const T*)q, (const T*)k, (const T*)v, (T*)out, (T*)kpool, (T*)vpool);
   return cudaGetLastError();
 }
 
 // G = 1, 2: 4 or 8 consumer warps; G = 4, 8: 8 or 16
 template <typename T, int D>
-static cudaError_t launch_g(int G, int cw, const DecodeArgs& a, const CUtensorMap& map_v, int n_slices, const void* q,
+static cudaError_t launch_g(int G, int cw, const DecodeArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v, int n_slices, const void* q,
                             const void* k, const void* v, void* out, void* kpool, void* vpool, cudaStream_t st) {
   switch (G) {
-    case 1: return cw == 4 ? launch_one<T, D, 1, 4>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                           : launch_one<T, D, 1, 8>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
-    case 2: return cw == 4 ? launch_one<T, D, 2, 4>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                           : launch_one<T, D, 2, 8>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
-    case 4: return cw == 16 ? launch_one<T, D, 4, 16>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                 : cw == 4 ? launch_one<T, D, 4, 4>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                           : launch_one<T, D, 4, 8>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
-    default: return cw == 16 ? launch_one<T, D, 8, 16>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                  : cw == 4 ? launch_one<T, D, 8, 4>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                            : launch_one<T, D, 8, 8>(a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    case 1: return cw == 4 ? launch_one<T, D, 1, 4>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                           : launch_one<T, D, 1, 8>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    case 2: return cw == 4 ? launch_one<T, D, 2, 4>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                           : launch_one<T, D, 2, 8>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    case 4: return cw == 16 ? launch_one<T, D, 4, 16>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                 : cw == 4 ? launch_one<T, D, 4, 4>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                           : launch_one<T, D, 4, 8>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    default: return cw == 16 ? launch_one<T, D, 8, 16>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                  : cw == 4 ? launch_one<T, D, 8, 4>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                            : launch_one<T, D, 8, 8>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
   }
 }
 
@@ -951,12 +1006,12 @@ static bool plan(int cw, int smem_rows, int row_bytes, int G, int D, int want_st
 }
 
 // Rows of a slice whose logits stay in shared memory: all of them while that takes 16 KB or less; else enough for
-// slices a quarter longer than the mean (the budgets of Eq. 5 give a few layers several times the mean, and sizing
+// slices twice as long as the mean (the budgets of Eq. 5 give a few layers several times the mean, and sizing
 // the array for those would cost every CTA its ring depth or the SM a resident CTA).
 static int smem_rows_for(int max_rows, double mean_rows, int G) {
   const int free_rows = 16 * 1024 / (4 * G);
   if (max_rows <= free_rows) return max_rows;
-  return min(max_rows, max(free_rows, (int)(1.25 * mean_rows)));
+  return min(max_rows, max(free_rows, (int)(2.0 * mean_rows)));
 }
 
 int decode_max_rows(int row_bytes, int group, int d_head) {
@@ -1016,23 +1071,25 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   // all layers in one call: CTAs take the slices largest cache first, so the long ones do not end up in the tail
   a.order = (l0 == 0 && l1 == L) ? (const int32_t*)(S + c->lay.order) : nullptr;
   // 16-bit caches with grouped queries read the value rows through a tensor map (swizzled stages)
-  CUtensorMap map_v;
+  CUtensorMap map_k, map_v;
+  memset(&map_k, 0, sizeof(map_k));
   memset(&map_v, 0, sizeof(map_v));
   if (c->elem_size == 2 && G >= 2) {
     const int box_rows = stage_bytes_of(cw) / row_bytes;
-    if (c->pool_rows >= (1ll << 31) || !encode_rows_2d(&map_v, g.dtype, vpool, (uint64_t)c->pool_rows, g.d_head, box_rows)) {
+    if (c->pool_rows >= (1ll << 31) || !encode_rows_2d(&map_k, g.dtype, kpool, (uint64_t)c->pool_rows, g.d_head, box_rows) ||
+        !encode_rows_2d(&map_v, g.dtype, vpool, (uint64_t)c->pool_rows, g.d_head, box_rows)) {
       *why = D2O_ERR_UNSUPPORTED;
       return cudaSuccess;
     }
   }
   if (g.dtype == D2O_F32)
-    return g.d_head == 64 ? launch_g<float, 64>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                          : launch_g<float, 128>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    return g.d_head == 64 ? launch_g<float, 64>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                          : launch_g<float, 128>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
   if (g.dtype == D2O_F16)
-    return g.d_head == 64 ? launch_g<__half, 64>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                          : launch_g<__half, 128>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
-  return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                        : launch_g<__nv_bfloat16, 128>(G, cw, a, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    return g.d_head == 64 ? launch_g<__half, 64>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                          : launch_g<__half, 128>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+  return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
+                        : launch_g<__nv_bfloat16, 128>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
 }
 
 }  // namespace d2o
