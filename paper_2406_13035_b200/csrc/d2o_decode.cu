@@ -159,6 +159,18 @@ __device__ __forceinline__ float reduce4(float s0, float s1, float s2, float s3,
 // 16 elements of d, from the row-major stage) * B (16 elements x 8 heads, the queries).  Both operands take their
 // 16-byte pieces from the same offsets of their rows, so the order of the elements inside a step is free and a
 // thread's piece is one contiguous vector load.
+// the same step with a zero accumulator on input: d = a * b
+template <typename T>
+__device__ __forceinline__ void mma_16x8x16_zero(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                 uint32_t b0, uint32_t b1) {
+  if constexpr (sizeof(T) == 2 && !cuda::std::is_same<T, __nv_bfloat16>::value) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+  } else {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+  }
+}
 template <typename T>
 __device__ __forceinline__ void mma_16x8x16(float (&acc)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                             uint32_t b0, uint32_t b1) {
@@ -202,18 +214,21 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t saddr, uint32_t& r0, 
 template <typename T, int D, int SR>
 __device__ __forceinline__ void tile_dots(const unsigned char* stage, int tile, const uint4 (&qb)[D / 32], float (&acc)[4]) {
   const int gid = (threadIdx.x & 31) >> 2, tig = threadIdx.x & 3;
-  // one accumulator per 16 elements of d: the steps do not wait for one another
-  float part[D / 16][4];
+  // all fragments first, then one tensor-core step per 16 elements of d, each into its own accumulator: neither
+  // the loads nor the steps wait for one another
+  uint4 A0[D / 32], A1[D / 32];
 #pragma unroll
   for (int j = 0; j < D / 32; ++j) {
     const unsigned char* row = stage + (size_t)(j >> 1) * SR * 128 + (size_t)(tile * 16 + gid) * 128 +
                                (((2 * tig + (j & 1)) ^ gid) << 4);
-    const uint4 A0 = *reinterpret_cast<const uint4*>(row);
-    const uint4 A1 = *reinterpret_cast<const uint4*>(row + 8 * 128);
+    A0[j] = *reinterpret_cast<const uint4*>(row);
+    A1[j] = *reinterpret_cast<const uint4*>(row + 8 * 128);
+  }
+  float part[D / 16][4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) part[2 * j][e] = part[2 * j + 1][e] = 0.f;
-    mma_16x8x16<T>(part[2 * j], A0.x, A1.x, A0.y, A1.y, qb[j].x, qb[j].y);
-    mma_16x8x16<T>(part[2 * j + 1], A0.z, A1.z, A0.w, A1.w, qb[j].z, qb[j].w);
+  for (int j = 0; j < D / 32; ++j) {
+    mma_16x8x16_zero<T>(part[2 * j], A0[j].x, A1[j].x, A0[j].y, A1[j].y, qb[j].x, qb[j].y);
+    mma_16x8x16_zero<T>(part[2 * j + 1], A0[j].z, A1[j].z, A0[j].w, A1[j].w, qb[j].z, qb[j].w);
   }
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
@@ -225,7 +240,7 @@ __device__ __forceinline__ void tile_dots(const unsigned char* stage, int tile, 
 }
 
 template <typename T, int D, int G, int CW>
-__global__ void __launch_bounds__((CW + 1) * 32, (CW == 4 ? (G <= 2 ? 6 : 4) : (CW == 8 ? (G <= 2 ? 4 : 2) : 1)))
+__global__ void __launch_bounds__((CW + 1) * 32, (CW == 4 ? (G <= 2 ? 7 : 4) : (CW == 8 ? (G <= 2 ? 4 : 2) : 1)))
 decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const T* __restrict__ q_in,
               const T* __restrict__ k_in, const T* __restrict__ v_in, T* __restrict__ out, T* __restrict__ kpool,
@@ -968,7 +983,7 @@ static cudaError_t launch_g(int G, int cw, const DecodeArgs& a, const CUtensorMa
 }
 
 // CTAs per SM the registers allow (mirrors the kernel's __launch_bounds__)
-static int max_per_sm(int cw, int G) { return cw == 4 ? (G <= 2 ? 6 : 4) : (cw == 8 ? (G <= 2 ? 4 : 2) : 1); }
+static int max_per_sm(int cw, int G) { return cw == 4 ? (G <= 2 ? 7 : 4) : (cw == 8 ? (G <= 2 ? 4 : 2) : 1); }
 
 // Ring depth for `max_rows` rows per slice when `per_sm` CTAs are to share an SM.  false if the per-row arrays leave
 // no room for a ring.  Occupancy matters more than depth: measured on the 7B-shaped stack with caches of 700 to
@@ -1047,7 +1062,7 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
       sum_rows += r;
     }
   const int n_slices = (l1 - l0) * B * Hkv;
-  // Consumer warps per CTA.  One head per KV head and enough small slices for six and more CTAs on every SM:
+  // Consumer warps per CTA.  One head per KV head and enough small slices for seven and more CTAs on every SM:
   // four warps (measured on the serving-shaped config, 8192 slices of ~410 rows: 350 vs 370 us per step).
   // Grouped queries with slices several times the mean and few of them: sixteen warps, one CTA per SM, so that the
   // longest slice streams twice as fast.  Otherwise eight.
