@@ -33,6 +33,7 @@ namespace d2o {
 __host__ __device__ constexpr int stage_bytes_of(int cw) { return 4 * cw * 32 * 16; }
 constexpr int kMaxStages = 12;
 constexpr unsigned long long kWaitNs = 1000000000ull;   // an mbarrier wait gives up after 1 s
+constexpr int kTensorMinG = 2;                          // query heads per KV head from which the tensor-core path is used
 constexpr uint32_t kSuspendNs = 4000u;                  // a waiting thread may stay suspended this long before it looks again
 
 struct DecodeArgs {
@@ -239,8 +240,16 @@ __device__ __forceinline__ void tile_dots(const unsigned char* stage, int tile, 
   }
 }
 
+// 16-bit caches take the tensor-core path (more registers per thread, fewer instructions per row)
+__host__ __device__ constexpr bool tensor_path(int elem_size, int G) { return elem_size == 2 && G >= kTensorMinG; }
+// CTAs per SM the kernel is compiled for
+__host__ __device__ constexpr int ctas_per_sm(int cw, int G, int elem_size) {
+  const bool t = tensor_path(elem_size, G);
+  return cw == 4 ? (G <= 2 ? (t ? 5 : 7) : 4) : (cw == 8 ? (G <= 2 ? (t ? 3 : 4) : 2) : 1);
+}
+
 template <typename T, int D, int G, int CW>
-__global__ void __launch_bounds__((CW + 1) * 32, (CW == 4 ? (G <= 2 ? 7 : 4) : (CW == 8 ? (G <= 2 ? 4 : 2) : 1)))
+__global__ void __launch_bounds__((CW + 1) * 32, ctas_per_sm(CW, G, (int)sizeof(T)))
 decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const T* __restrict__ q_in,
               const T* __restrict__ k_in, const T* __restrict__ v_in, T* __restrict__ out, T* __restrict__ kpool,
@@ -257,7 +266,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   // are as fast and use every warp).  The value stages then arrive through a tiled tensor map with the 128-byte
   // swizzle, because the value pass reads them with transposing matrix loads, which would conflict eight ways on
   // row-major 256-byte rows.
-  constexpr bool kTensor = sizeof(T) == 2 && G >= 2;
+  constexpr bool kTensor = tensor_path((int)sizeof(T), G);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // ---- which slice: in index order, or largest caches first through the order table
   const int h = (int)blockIdx.x % a.Hkv;
@@ -983,7 +992,7 @@ static cudaError_t launch_g(int G, int cw, const DecodeArgs& a, const CUtensorMa
 }
 
 // CTAs per SM the registers allow (mirrors the kernel's __launch_bounds__)
-static int max_per_sm(int cw, int G) { return cw == 4 ? (G <= 2 ? 7 : 4) : (cw == 8 ? (G <= 2 ? 4 : 2) : 1); }
+static int max_per_sm(int cw, int G, int elem_size) { return ctas_per_sm(cw, G, elem_size); }
 
 // Ring depth for `max_rows` rows per slice when `per_sm` CTAs are to share an SM.  false if the per-row arrays leave
 // no room for a ring.  Occupancy matters more than depth: measured on the 7B-shaped stack with caches of 700 to
@@ -1003,7 +1012,7 @@ static bool plan_tier(int cw, int smem_rows, int row_bytes, int G, int D, int pe
 
 // Best occupancy tier that fits `max_rows`; 0 = none.
 static int best_tier(int cw, int smem_rows, int row_bytes, int G, int D, int* row_cap, int* stages) {
-  for (int per_sm = max_per_sm(cw, G); per_sm >= 1; --per_sm)
+  for (int per_sm = max_per_sm(cw, G, row_bytes / D); per_sm >= 1; --per_sm)
     if (plan_tier(cw, smem_rows, row_bytes, G, D, per_sm, row_cap, stages)) return per_sm;
   return 0;
 }
@@ -1089,7 +1098,7 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   CUtensorMap map_k, map_v;
   memset(&map_k, 0, sizeof(map_k));
   memset(&map_v, 0, sizeof(map_v));
-  if (c->elem_size == 2 && G >= 2) {
+  if (tensor_path(c->elem_size, G)) {
     const int box_rows = stage_bytes_of(cw) / row_bytes;
     if (c->pool_rows >= (1ll << 31) || !encode_rows_2d(&map_k, g.dtype, kpool, (uint64_t)c->pool_rows, g.d_head, box_rows) ||
         !encode_rows_2d(&map_v, g.dtype, vpool, (uint64_t)c->pool_rows, g.d_head, box_rows)) {
