@@ -100,6 +100,7 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   s->evict_nn = take(B * Hkv * P * 4);
   s->seg_start = take(B * Hkv * ((size_t)max_budget + 2) * 4);
   s->seg_items = take(B * Hkv * P * 4);
+  s->seg_tmp = take(B * Hkv * P * 4);
   s->part_key = take(c->dtype == D2O_F32 ? 0 : sim_tc_part_key_bytes(c, max_budget));
   s->pl_spill = take((rows + 8 * L * B * Hkv) * (Hq / Hkv) * 4);
   s->stage_q = take(L * B * Hq * d * e);

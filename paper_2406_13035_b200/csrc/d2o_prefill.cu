@@ -295,7 +295,7 @@ similarity_kernel(SimArgs a, const T* __restrict__ K, const T* __restrict__ kpoo
 struct SegArgs {
   const int32_t* budgets;
   const float* evict_mx; const int32_t* evict_nn;
-  int32_t* seg_start; int32_t* seg_items; float* tau;
+  int32_t* seg_start; int32_t* seg_items; int32_t* seg_tmp; float* tau;
   unsigned long long* counters;
   int L, layer, B, Hkv, P, seg_stride;
   float tau_override;
@@ -303,7 +303,7 @@ struct SegArgs {
 
 __global__ void __launch_bounds__(1024)
 segment_kernel(SegArgs a) {
-  extern __shared__ __align__(16) int seg_smem[];       // [S + 1] counts / cursors
+  extern __shared__ __align__(16) int seg_smem[];       // [max(S + 1, 32 * 64)] counts / cursors, then radix histograms
   __shared__ double part[32];
   __shared__ float s_thr;
   __shared__ int warp_tot[32];
@@ -356,23 +356,68 @@ segment_kernel(SegArgs a) {
     __syncthreads();
   }
   if (threadIdx.x == 0) atomicAdd(&a.counters[kCntPrefillMerged], (unsigned long long)run);
-  // ordered fill by one warp: evicted tokens are visited in ascending index, lanes that share a
-  // target are ranked with match_any, so every list is in ascending position
-  if (warp == 0) {
-    for (int base = 0; base < Le; base += 32) {
-      const int i = base + lane;
-      const bool on = i < Le && mx[i] >= thr;
-      const int j = on ? nn[i] : -1 - lane;               // distinct dummies for idle lanes
-      const unsigned peers = __match_any_sync(0xffffffffu, j);
-      if (on) {
+  // Ordered fill: the passing evicted tokens sorted by (neighbour, index), so that every segment lists its tokens in
+  // ascending position.  Stable least-significant-digit radix sort on the neighbour slot, 6 bits per pass; each
+  // warp owns a contiguous chunk of the source, counts its digits, and after a scan over (digit, warp) scatters its
+  // chunk in order (lanes with the same digit are ranked with match_any).
+  if (run == 0) return;
+  int* hist = reinterpret_cast<int*>(seg_smem);         // [32 warps][64 digits]; the cursors are not needed any more
+  int32_t* tmp = a.seg_tmp + (size_t)slice * a.P;
+  int bits = 0;
+  while ((S >> bits) != 0) ++bits;                      // slots are < S
+  const int passes = (bits + 5) / 6;
+  const int n_warps = (int)(blockDim.x >> 5);
+  for (int p = 0; p < passes; ++p) {
+    // the last pass must land in `items`
+    int32_t* dst = ((passes - 1 - p) & 1) ? tmp : items;
+    const int32_t* src = dst == items ? tmp : items;    // unused in pass 0 (the source is the index range itself)
+    const int n_src = p == 0 ? Le : run;
+    const int chunk = (((n_src + n_warps - 1) / n_warps) + 31) & ~31;
+    const int c0 = warp * chunk, c1 = min(n_src, c0 + chunk);
+    const int shift = 6 * p;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_warps * 64; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    for (int base = c0; base < c1; base += 32) {
+      const int k = base + lane;
+      int item = -1;
+      if (k < c1) {
+        if (p == 0) { if (mx[k] >= thr) item = k; }
+        else item = src[k];
+      }
+      if (item >= 0) atomicAdd(&hist[warp * 64 + ((nn[item] >> shift) & 63)], 1);
+    }
+    __syncthreads();
+    // exclusive scan in (digit, warp) order: 64 * n_warps entries, two per thread
+    {
+      const int e0 = 2 * threadIdx.x, e1 = e0 + 1;
+      const int total_e = 64 * n_warps;
+      const int v0 = e0 < total_e ? hist[(e0 % n_warps) * 64 + e0 / n_warps] : 0;
+      const int v1 = e1 < total_e ? hist[(e1 % n_warps) * 64 + e1 / n_warps] : 0;
+      const int ex = block_exclusive_scan(v0 + v1, warp_tot, &s_total);
+      if (e0 < total_e) hist[(e0 % n_warps) * 64 + e0 / n_warps] = ex;
+      if (e1 < total_e) hist[(e1 % n_warps) * 64 + e1 / n_warps] = ex + v0;
+    }
+    __syncthreads();
+    for (int base = c0; base < c1; base += 32) {
+      const int k = base + lane;
+      int item = -1;
+      if (k < c1) {
+        if (p == 0) { if (mx[k] >= thr) item = k; }
+        else item = src[k];
+      }
+      const int dgt = item >= 0 ? ((nn[item] >> shift) & 63) : 64 + lane;   // distinct dummies for idle lanes
+      const unsigned peers = __match_any_sync(0xffffffffu, dgt);
+      if (item >= 0) {
         const int rank = __popc(peers & ((1u << lane) - 1u));
-        const int cur = seg_smem[j];
-        items[cur + rank] = i;
+        const int cur = hist[warp * 64 + dgt];
+        dst[cur + rank] = item;
         __syncwarp(peers);
-        if (rank == 0) seg_smem[j] = cur + __popc(peers);
+        if (rank == 0) hist[warp * 64 + dgt] = cur + __popc(peers);
       }
       __syncwarp();
     }
+    __threadfence_block();
   }
 }
 
@@ -497,10 +542,12 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   SegArgs ga;
   ga.budgets = sa.budgets; ga.evict_mx = ma.evict_mx; ga.evict_nn = ma.evict_nn;
   ga.seg_start = (int32_t*)(X + c->slay.seg_start); ga.seg_items = (int32_t*)(X + c->slay.seg_items);
+  ga.seg_tmp = (int32_t*)(X + c->slay.seg_tmp);
   ga.tau = sa.tau; ga.counters = sa.counters;
   ga.L = L; ga.layer = layer; ga.B = B; ga.Hkv = Hkv; ga.P = P; ga.seg_stride = seg_stride;
   ga.tau_override = g.tau_override;
-  const size_t seg_sm = (size_t)(maxS + 1) * sizeof(int);
+  // counts / cursors per retained slot, later the radix histograms (32 warps x 64 digits)
+  const size_t seg_sm = (size_t)max(maxS + 1, 32 * 64) * sizeof(int);
   e = cudaFuncSetAttribute(segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)(seg_sm > 48 * 1024 ? seg_sm : 48 * 1024));
   if (e != cudaSuccess) return e;
