@@ -45,6 +45,8 @@ def parse():
     ap.add_argument("--decode-warps", type=int, default=0, help="consumer warps per decode CTA (0 = auto)")
     ap.add_argument("--smem-rows", type=int, default=0,
                     help="decode kernel: rows of a slice with their logits in shared memory (0 = auto)")
+    ap.add_argument("--long-pairs", type=int, default=0,
+                    help="decode: (layer, sequence) pairs in the long-slice launch (0 = auto, -1 = never)")
     ap.add_argument("--no-l2-hints", action="store_true", help="decode kernel: copies without L2 eviction hints")
     ap.add_argument("--ffma-similarity", action="store_true", help="prompt-stage similarity on the FFMA kernel")
     ap.add_argument("--ffma-stats", action="store_true", help="column sums of the prompt attention on the FFMA kernels")
@@ -157,9 +159,9 @@ def run_ours(args, wl, rank, world, device):
                         density_temp=wl.density_temp, min_budget=wl.min_budget, max_budget=wl.max_budget)
     ctx = B.D2OContext(cfg, device)
     if (args.stages or args.no_l2_hints or args.ffma_similarity or args.ffma_stats or args.decode_warps
-            or args.smem_rows):
+            or args.smem_rows or args.long_pairs):
         ctx.d2o_set_tuning(args.stages, 0 if args.no_l2_hints else 1, 1 if args.ffma_similarity else 0,
-                           1 if args.ffma_stats else 0, args.decode_warps, args.smem_rows)
+                           1 if args.ffma_stats else 0, args.decode_warps, args.smem_rows, args.long_pairs)
     # every rank works on its own sequences: same shapes, rank-dependent seed (weak scaling, no exchange)
     import dataclasses
     wl_r = dataclasses.replace(wl, seed=wl.seed + 7919 * rank)
@@ -168,7 +170,7 @@ def run_ours(args, wl, rank, world, device):
     L = wl.n_layers
     lpc = args.layers_per_call or L
     ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
-    launches = {"n": 0}
+    launches = {"n": 0, "decode_seen": 0}
 
     def one_pass(timed: bool):
         e = [ev() for _ in range(5)]
@@ -186,10 +188,13 @@ def run_ours(args, wl, rank, world, device):
                 l1 = min(L, l0 + lpc)
                 ctx.d2o_decode_step(l0, l1, dq[s, l0:l1], dk[s, l0:l1], dv[s, l0:l1], dout[l0:l1])
         e[4].record()
+        # stats: 2 attention sweeps + density per layer; budgets: 1; compress: select, similarity, neighbour
+        # reduce, segments, merge per layer (the fp32 path has one kernel fewer); decode: as counted by the
+        # library (a step over all layers is one launch, or two when the longest slices get their own)
+        dl = ctx.d2o_get_stats().decode_launches
         if timed:
-            # stats: 2 attention sweeps + density per layer; budgets: 1; compress: select, similarity, neighbour
-            # reduce, segments, merge per layer (the fp32 path has one kernel fewer); decode: 1 per call
-            launches["n"] += L * 3 + 1 + L * (4 if wl.dtype == "f32" else 5) + nd * ((L + lpc - 1) // lpc)
+            launches["n"] += L * 3 + 1 + L * (4 if wl.dtype == "f32" else 5) + (dl - launches["decode_seen"])
+        launches["decode_seen"] = dl
         return e, budgets
 
     def sync_all():

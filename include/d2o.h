@@ -105,6 +105,7 @@ typedef struct {
   uint64_t prefill_merged;   /* ... of which merged                                            */
   uint32_t error_word;       /* 0 = none; else first device-side anomaly (d2o_status)         */
   uint32_t error_detail;
+  uint64_t decode_launches;  /* decode kernels launched so far (a step over all layers may take two)  */
 } d2o_stats;
 
 const char* d2o_status_string(d2o_status s);
@@ -212,10 +213,13 @@ d2o_status d2o_get_stats(d2o_ctx* ctx, d2o_stats* out_host, void* stream);
  * sums of d2o_layer_stats; decode_warps = consumer warps per CTA of the decode kernel (0 = automatic,
  * 4 or 8 with one or two query heads per KV head, 8 or 16 with four or eight); decode_smem_rows =
  * rows of a slice whose logits the decode kernel keeps in shared memory, the rest going through an
- * L2-resident array of the scratch buffer (0 = automatic, else >= 8). */
+ * L2-resident array of the scratch buffer (0 = automatic, else >= 8); decode_long_pairs = how many
+ * of the (layer, sequence) pairs with the largest budgets a decode step over all layers runs in a
+ * launch of their own with sixteen-warp CTAs, ahead of and overlapping the launch of the rest
+ * (0 = automatic, negative = never, positive = that many). */
 d2o_status d2o_set_tuning(d2o_ctx* ctx, int32_t decode_stages, int32_t decode_l2_hints,
                           int32_t similarity_path, int32_t stats_path, int32_t decode_warps,
-                          int32_t decode_smem_rows);
+                          int32_t decode_smem_rows, int32_t decode_long_pairs);
 
 #ifdef __cplusplus
 }

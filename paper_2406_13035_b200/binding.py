@@ -50,7 +50,7 @@ class D2OView(C.Structure):
 class D2OStats(C.Structure):
     _fields_ = [("decode_steps", C.c_uint64), ("evictions", C.c_uint64), ("merges", C.c_uint64),
                 ("discards", C.c_uint64), ("prefill_evicted", C.c_uint64), ("prefill_merged", C.c_uint64),
-                ("error_word", C.c_uint32), ("error_detail", C.c_uint32)]
+                ("error_word", C.c_uint32), ("error_detail", C.c_uint32), ("decode_launches", C.c_uint64)]
 
 
 class D2OError(RuntimeError):
@@ -89,7 +89,7 @@ def load_library() -> C.CDLL:
     lib.d2o_full_decode_step.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.d2o_get_view.argtypes = [vp, i32, C.POINTER(D2OView)]
     lib.d2o_get_stats.argtypes = [vp, C.POINTER(D2OStats), vp]
-    lib.d2o_set_tuning.argtypes = [vp, i32, i32, i32, i32, i32, i32]
+    lib.d2o_set_tuning.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32]
     lib.d2o_layer_stats_static.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("d2o_status_string", "d2o_last_cuda_error", "d2o_destroy"):
@@ -193,9 +193,10 @@ class D2OContext:
                "d2o_decode_step_host")
 
     def d2o_set_tuning(self, decode_stages: int = 0, decode_l2_hints: int = 1, similarity_path: int = 0,
-                       stats_path: int = 0, decode_warps: int = 0, decode_smem_rows: int = 0):
+                       stats_path: int = 0, decode_warps: int = 0, decode_smem_rows: int = 0,
+                       decode_long_pairs: int = 0):
         _check(self.lib.d2o_set_tuning(self.handle, decode_stages, decode_l2_hints, similarity_path, stats_path,
-                                       decode_warps, decode_smem_rows), "d2o_set_tuning")
+                                       decode_warps, decode_smem_rows, decode_long_pairs), "d2o_set_tuning")
 
     def d2o_get_stats(self) -> D2OStats:
         s = D2OStats()

@@ -165,6 +165,8 @@ struct d2o_ctx {
   int decode_stages;           // tuning: stages of the decode kernel's ring, 0 = auto
   int decode_warps;            // tuning: consumer warps per decode CTA (4, 8, 16), 0 = auto
   int decode_smem_rows;        // tuning: rows of a slice with their logits in shared memory, 0 = auto
+  mutable uint64_t decode_launches;   // decode kernels launched so far
+  int decode_long_pairs;       // tuning: (layer, sequence) pairs in the long-slice launch, 0 = auto, < 0 = never
   int decode_l2_hints;         // tuning: 1 = the decode kernel's copies carry L2 eviction hints
   int similarity_path;         // tuning: 0 = tensor cores for 16-bit keys, 1 = FFMA kernel for every dtype
   int stats_path;              // tuning: 0 = tensor cores for the column sums of 16-bit Q/K, 1 = FFMA kernels

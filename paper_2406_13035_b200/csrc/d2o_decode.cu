@@ -48,6 +48,7 @@ struct DecodeArgs {
   int stages;                       // stages of the ring
   int l2_hints;                     // 1: pass K asks L2 to keep its lines, later passes to drop theirs
   const int32_t* order;             // NULL: CTAs take (layer, b, h) in index order; else (layer * B + b) per group of Hkv CTAs
+  int pair_base;                    // first entry of `order` this launch works on
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -245,7 +246,7 @@ __host__ __device__ constexpr bool tensor_path(int elem_size, int G) { return el
 // CTAs per SM the kernel is compiled for
 __host__ __device__ constexpr int ctas_per_sm(int cw, int G, int elem_size) {
   const bool t = tensor_path(elem_size, G);
-  return cw == 4 ? (G <= 2 ? (t ? 5 : 7) : 4) : (cw == 8 ? (G <= 2 ? (t ? 3 : 4) : 2) : 1);
+  return cw == 4 ? (G <= 2 ? (t ? 5 : 7) : 4) : (cw == 8 ? (G <= 2 ? (t ? 3 : 4) : 2) : (G <= 2 && !t ? 2 : 1));
 }
 
 template <typename T, int D, int G, int CW>
@@ -268,11 +269,14 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   // row-major 256-byte rows.
   constexpr bool kTensor = tensor_path((int)sizeof(T), G);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // a launch that follows with programmatic stream serialisation (the short slices of the same step, which share
+  // nothing with this one) may start as soon as every CTA of this one is running
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // ---- which slice: in index order, or largest caches first through the order table
   const int h = (int)blockIdx.x % a.Hkv;
   int layer, b;
   if (a.order) {
-    const int pair = a.order[blockIdx.x / a.Hkv];
+    const int pair = a.order[a.pair_base + (int)blockIdx.x / a.Hkv];
     layer = pair / a.B; b = pair % a.B;
   } else {
     layer = a.l0 + (int)blockIdx.x / (a.B * a.Hkv);
@@ -963,33 +967,36 @@ static size_t smem_bytes(int cw, int row_cap, int stages, int G, int row_bytes) 
 }
 
 template <typename T, int D, int G, int CW>
-static cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v, int n_slices, const void* q, const void* k,
-                              const void* v, void* out, void* kpool, void* vpool, cudaStream_t st) {
+static cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v, int n_slices,
+                              const void* q, const void* k, const void* v, void* out, void* kpool, void* vpool,
+                              cudaStream_t st, bool overlap_previous) {
   const size_t smem = smem_bytes(CW, a.row_cap, a.stages, G, D * (int)sizeof(T));
   auto kern = decode_kernel<T, D, G, CW>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<n_slices, (CW + 1) * 32, smem, st>>>(a, map_k, map_v, (const T*)q, (const T*)k, (const T*)v, (T*)out, (T*)kpool, (T*)vpool);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)n_slices); cfg.blockDim = dim3((CW + 1) * 32); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = overlap_previous ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, a, map_k, map_v, (const T*)q, (const T*)k, (const T*)v, (T*)out, (T*)kpool, (T*)vpool);
 }
 
-// G = 1, 2: 4 or 8 consumer warps; G = 4, 8: 8 or 16
+// G = 1, 2: 4, 8 or 16 consumer warps; G = 4, 8: the same
+#define D2O_LAUNCH(GG, CC) launch_one<T, D, GG, CC>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap)
 template <typename T, int D>
-static cudaError_t launch_g(int G, int cw, const DecodeArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v, int n_slices, const void* q,
-                            const void* k, const void* v, void* out, void* kpool, void* vpool, cudaStream_t st) {
+static cudaError_t launch_g(int G, int cw, const DecodeArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v, int n_slices,
+                            const void* q, const void* k, const void* v, void* out, void* kpool, void* vpool,
+                            cudaStream_t st, bool overlap) {
   switch (G) {
-    case 1: return cw == 4 ? launch_one<T, D, 1, 4>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                           : launch_one<T, D, 1, 8>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
-    case 2: return cw == 4 ? launch_one<T, D, 2, 4>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                           : launch_one<T, D, 2, 8>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
-    case 4: return cw == 16 ? launch_one<T, D, 4, 16>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                 : cw == 4 ? launch_one<T, D, 4, 4>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                           : launch_one<T, D, 4, 8>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
-    default: return cw == 16 ? launch_one<T, D, 8, 16>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                  : cw == 4 ? launch_one<T, D, 8, 4>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                            : launch_one<T, D, 8, 8>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+    case 1: return cw == 16 ? D2O_LAUNCH(1, 16) : cw == 4 ? D2O_LAUNCH(1, 4) : D2O_LAUNCH(1, 8);
+    case 2: return cw == 16 ? D2O_LAUNCH(2, 16) : cw == 4 ? D2O_LAUNCH(2, 4) : D2O_LAUNCH(2, 8);
+    case 4: return cw == 16 ? D2O_LAUNCH(4, 16) : cw == 4 ? D2O_LAUNCH(4, 4) : D2O_LAUNCH(4, 8);
+    default: return cw == 16 ? D2O_LAUNCH(8, 16) : cw == 4 ? D2O_LAUNCH(8, 4) : D2O_LAUNCH(8, 8);
   }
 }
+#undef D2O_LAUNCH
 
 // CTAs per SM the registers allow (mirrors the kernel's __launch_bounds__)
 static int max_per_sm(int cw, int G, int elem_size) { return ctas_per_sm(cw, G, elem_size); }
@@ -1070,50 +1077,95 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
       max_rows = max(max_rows, r);
       sum_rows += r;
     }
-  const int n_slices = (l1 - l0) * B * Hkv;
+  // all layers in one call: CTAs take the slices largest cache first, so the long ones do not end up in the tail
+  const bool ordered = (l0 == 0 && l1 == L);
+  a.order = ordered ? (const int32_t*)(S + c->lay.order) : nullptr;
+  a.spill = (float*)(c->scratch + c->slay.pl_spill);
+  const int n_pairs = (l1 - l0) * B;
+  const double mean_rows = (double)sum_rows / n_pairs;
+  auto rows_of_pair = [&](int i) {                                    // i-th pair in launch order
+    const int pr = ordered ? c->h_order[i] : (l0 * B + i);
+    return min(c->h_budgets[(pr % B) * L + pr / B], g.prompt_len + c->layer_steps[l0]) + 1;
+  };
+
+  // A step takes at least as long as its longest slice takes in one CTA.  Where that is more than the whole step
+  // would otherwise need (few sequences, a few layers with several times the mean budget), the longest slices go
+  // into a launch of their own with sixteen consumer warps per CTA, and the rest follows in a second launch that
+  // is allowed to start while the first is still running (the two share no slice).  Estimate with rough per-row
+  // costs of an eight-warp CTA; exactness does not matter, the split only has to catch the outliers.
+  int n_long = 0;
+  if (ordered && c->decode_warps == 0 && c->decode_long_pairs == 0 && n_pairs > 1) {
+    const double fixed_us = 8.0, row_us = tensor_path(c->elem_size, G) ? 0.025 : 0.05;
+    const double slots = 148.0 * ctas_per_sm(8, G, c->elem_size);
+    double work = 0.0;
+    for (int i = 0; i < n_pairs; ++i) work += Hkv * (fixed_us + row_us * rows_of_pair(i));
+    // measured optimum: four pairs on the 7B-shaped config (FMA path), twelve on the long-context one (tensor path)
+    const double limit = (tensor_path(c->elem_size, G) ? 0.55 : 0.7) * work / slots;
+    while (n_long < n_pairs && (n_long + 1) * Hkv <= 2 * 148 && fixed_us + row_us * rows_of_pair(n_long) > limit) ++n_long;
+    if (n_long == n_pairs) n_long = 0;
+  } else if (ordered && c->decode_long_pairs > 0) {
+    n_long = min(c->decode_long_pairs, n_pairs - 1);
+  }
+
+  // one launch over the pairs [p0, p1) of the order
+  auto launch_class = [&](int p0, int p1, int cw, bool overlap) -> cudaError_t {
+    int cls_max = 0;
+    long long cls_sum = 0;
+    for (int i = p0; i < p1; ++i) { const int r = rows_of_pair(i); cls_max = max(cls_max, r); cls_sum += r; }
+    const int n_slices = (p1 - p0) * Hkv;
+    int row_cap, stages;
+    int smem_rows = smem_rows_for(cls_max, (double)cls_sum / (p1 - p0), G);
+    if (c->decode_smem_rows > 0) smem_rows = min(cls_max, c->decode_smem_rows);
+    if (!plan(cw, smem_rows, row_bytes, G, g.d_head, c->decode_stages, &row_cap, &stages)) {
+      *why = D2O_ERR_UNSUPPORTED;
+      return cudaSuccess;
+    }
+    c->decode_launches += 1;
+    DecodeArgs ac = a;
+    ac.row_cap = row_cap; ac.stages = stages; ac.pair_base = p0;
+    // 16-bit caches with grouped queries read their rows through tensor maps (swizzled stages)
+    CUtensorMap map_k, map_v;
+    memset(&map_k, 0, sizeof(map_k));
+    memset(&map_v, 0, sizeof(map_v));
+    if (tensor_path(c->elem_size, G)) {
+      const int box_rows = stage_bytes_of(cw) / row_bytes;
+      if (c->pool_rows >= (1ll << 31) || !encode_rows_2d(&map_k, g.dtype, kpool, (uint64_t)c->pool_rows, g.d_head, box_rows) ||
+          !encode_rows_2d(&map_v, g.dtype, vpool, (uint64_t)c->pool_rows, g.d_head, box_rows)) {
+        *why = D2O_ERR_UNSUPPORTED;
+        return cudaSuccess;
+      }
+    }
+    // inputs and outputs of the step are indexed by the slice's place in the call, which the kernel derives itself
+    if (g.dtype == D2O_F32)
+      return g.d_head == 64 ? launch_g<float, 64>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap)
+                            : launch_g<float, 128>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap);
+    if (g.dtype == D2O_F16)
+      return g.d_head == 64 ? launch_g<__half, 64>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap)
+                            : launch_g<__half, 128>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap);
+    return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap)
+                          : launch_g<__nv_bfloat16, 128>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap);
+  };
+
+  if (n_long > 0) {
+    cudaError_t e = launch_class(0, n_long, 16, false);
+    if (e != cudaSuccess || *why != D2O_OK) return e;
+    const int rest = (n_pairs - n_long) * Hkv;
+    int rest_max = rows_of_pair(n_long);
+    const int cw = (G <= 2 && rest >= 8 * 148 * 4 && rest_max <= 1536) ? 4 : 8;
+    return launch_class(n_long, n_pairs, cw, true);
+  }
   // Consumer warps per CTA.  One head per KV head and enough small slices for seven and more CTAs on every SM:
   // four warps (measured on the serving-shaped config, 8192 slices of ~410 rows: 350 vs 370 us per step).
   // Grouped queries with slices several times the mean and few of them: sixteen warps, one CTA per SM, so that the
   // longest slice streams twice as fast.  Otherwise eight.
+  const int n_slices = n_pairs * Hkv;
   int cw = c->decode_warps;
   if (cw == 0) {
     cw = 8;
-    const double mean_rows = (double)sum_rows / ((l1 - l0) * B);
     if (G <= 2 && n_slices >= 8 * 148 * 4 && max_rows <= 1536) cw = 4;
     if (G >= 4 && n_slices <= 148 * 8 && max_rows > 2.0 * mean_rows) cw = 16;
   }
-  if (G <= 2 && cw == 16) cw = 8;
-  int row_cap, stages;
-  int smem_rows = smem_rows_for(max_rows, (double)sum_rows / ((l1 - l0) * B), G);
-  if (c->decode_smem_rows > 0) smem_rows = min(max_rows, c->decode_smem_rows);
-  if (!plan(cw, smem_rows, row_bytes, G, g.d_head, c->decode_stages, &row_cap, &stages)) {
-    *why = D2O_ERR_UNSUPPORTED;
-    return cudaSuccess;
-  }
-  a.row_cap = row_cap; a.stages = stages;
-  a.spill = (float*)(c->scratch + c->slay.pl_spill);
-  // all layers in one call: CTAs take the slices largest cache first, so the long ones do not end up in the tail
-  a.order = (l0 == 0 && l1 == L) ? (const int32_t*)(S + c->lay.order) : nullptr;
-  // 16-bit caches with grouped queries read the value rows through a tensor map (swizzled stages)
-  CUtensorMap map_k, map_v;
-  memset(&map_k, 0, sizeof(map_k));
-  memset(&map_v, 0, sizeof(map_v));
-  if (tensor_path(c->elem_size, G)) {
-    const int box_rows = stage_bytes_of(cw) / row_bytes;
-    if (c->pool_rows >= (1ll << 31) || !encode_rows_2d(&map_k, g.dtype, kpool, (uint64_t)c->pool_rows, g.d_head, box_rows) ||
-        !encode_rows_2d(&map_v, g.dtype, vpool, (uint64_t)c->pool_rows, g.d_head, box_rows)) {
-      *why = D2O_ERR_UNSUPPORTED;
-      return cudaSuccess;
-    }
-  }
-  if (g.dtype == D2O_F32)
-    return g.d_head == 64 ? launch_g<float, 64>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                          : launch_g<float, 128>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
-  if (g.dtype == D2O_F16)
-    return g.d_head == 64 ? launch_g<__half, 64>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                          : launch_g<__half, 128>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
-  return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st)
-                        : launch_g<__nv_bfloat16, 128>(G, cw, a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st);
+  return launch_class(0, n_pairs, cw, false);
 }
 
 }  // namespace d2o

@@ -353,12 +353,13 @@ extern "C" d2o_status d2o_get_stats(d2o_ctx* c, d2o_stats* out, void* stream) {
   out->prefill_merged = cnt[kCntPrefillMerged];
   out->error_word = word[0];
   out->error_detail = word[1];
+  out->decode_launches = c->decode_launches;
   return D2O_OK;
 }
 
 extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t decode_l2_hints,
                                      int32_t similarity_path, int32_t stats_path, int32_t decode_warps,
-                                     int32_t decode_smem_rows) {
+                                     int32_t decode_smem_rows, int32_t decode_long_pairs) {
   if (!c) return D2O_ERR_INVALID_ARG;
   if (decode_stages < 0 || decode_stages > 12) return D2O_ERR_INVALID_ARG;
   if (decode_l2_hints < 0 || decode_l2_hints > 1) return D2O_ERR_INVALID_ARG;
@@ -371,5 +372,6 @@ extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t 
   c->stats_path = stats_path;
   c->decode_warps = decode_warps;
   c->decode_smem_rows = decode_smem_rows;
+  c->decode_long_pairs = decode_long_pairs;
   return D2O_OK;
 }

@@ -86,16 +86,17 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
                steps: Optional[int] = None, tie_rtol: float = TIE_RTOL, ctx_over: Optional[dict] = None,
                layers_per_call: Optional[int] = None, decode_stages: int = 0, decode_l2_hints: int = 1,
                similarity_path: int = 0, stats_path: int = 0, decode_warps: int = 0,
-               decode_smem_rows: int = 0,
+               decode_smem_rows: int = 0, decode_long_pairs: int = 0,
                check_stats_all: Optional[bool] = None) -> Report:
     """`slices`: (layer, b, kv_head) triples checked against the oracle (None = all).
     The GPU always runs the whole workload."""
     rep = Report()
     ctx = make_ctx(wl, device, **(ctx_over or {}))
     cfg = ctx.cfg
-    if decode_stages or not decode_l2_hints or similarity_path or stats_path or decode_warps or decode_smem_rows:
+    if (decode_stages or not decode_l2_hints or similarity_path or stats_path or decode_warps or decode_smem_rows
+            or decode_long_pairs):
         ctx.d2o_set_tuning(decode_stages, decode_l2_hints, similarity_path, stats_path, decode_warps,
-                           decode_smem_rows)
+                           decode_smem_rows, decode_long_pairs)
     orc = make_oracle(wl, cfg)
     L, Bn, Hq, Hkv, G, P = wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.group, wl.prompt_len
     all_slices = [(l, b, h) for l in range(L) for b in range(Bn) for h in range(Hkv)]

@@ -66,6 +66,14 @@ def test_logits_beyond_shared_memory_agree(name, rows):
     assert_report(rep, wl.dtype)
 
 
+@pytest.mark.parametrize("name,pairs", [("cfg1", 1), ("cfg2", 3), ("cfg3", 2), ("cfg4", 1), ("cfg0", 1)])
+def test_long_slice_launch_agrees(name, pairs):
+    # the pairs with the largest budgets in a sixteen-warp launch of their own, the rest overlapping it
+    wl = dataclasses.replace(W.CONFIGS[name], n_layers=2, decode_steps=8) if name == "cfg0" else W.twin(name)
+    rep = run_parity(wl, decode_long_pairs=pairs, steps=8)
+    assert_report(rep, wl.dtype)
+
+
 def test_layer_by_layer_calls_match():
     wl = W.twin("cfg1")
     rep = run_parity(wl, layers_per_call=1, steps=6)
