@@ -30,7 +30,7 @@ import torch  # noqa: E402
 from paper_2406_13035_b200 import workloads as W  # noqa: E402
 
 METRIC = "compressed decode steps/s (x sequences = tokens/s); prefill-compress ms; fraction of HBM roofline"
-DECODE_TRAFFIC_RATIO = 1.10       # ncu DRAM bytes / algorithmic bytes of decode_kernel, see profiles/decode_kernel_cfg1.md
+DECODE_TRAFFIC_RATIO = 1.11       # ncu DRAM bytes / algorithmic bytes of one decode step, see profiles/decode_kernel_cfg1.md
 
 
 def parse():
@@ -240,9 +240,9 @@ def run_ours(args, wl, rank, world, device):
         peaks = json.load(open(pk_path))
     peak = float(peaks.get("hbm_gbs", 6650.0))
     achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
-    # DRAM traffic per launch: dram__bytes_read + dram__bytes_write of one decode_kernel launch under ncu on the
-    # 16-layer variant of this workload was 1.10 x its algorithmic bytes (profiles/decode_kernel_cfg1.md); it grows
-    # with the rows streamed, so it is scaled by the algorithmic bytes of this launch.
+    # DRAM traffic per step: dram__bytes_read + dram__bytes_write of the decode_kernel launches of one step of this
+    # workload under ncu (two launches: the longest slices, then the rest) was 1.11 x the algorithmic bytes
+    # (profiles/decode_kernel_cfg1.md).
     traffic = int(DECODE_TRAFFIC_RATIO * bytes_per_launch) if (wl.name.startswith("cfg1") and lpc == L) else None
     roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": round(achieved, 1), "peak": peak,
                 "unit": "GB/s", "frac": round(achieved / peak, 4),
