@@ -249,8 +249,9 @@ __host__ __device__ constexpr int ctas_per_sm(int cw, int G, int elem_size) {
   return cw == 4 ? (G <= 2 ? (t ? 5 : 7) : 4) : (cw == 8 ? (G <= 2 ? (t ? 3 : 4) : 2) : (G <= 2 && !t ? 2 : 1));
 }
 
-template <typename T, int D, int G, int CW>
-__global__ void __launch_bounds__((CW + 1) * 32, ctas_per_sm(CW, G, (int)sizeof(T)))
+// OCC = CTAs per SM the registers are capped for (0: the table above)
+template <typename T, int D, int G, int CW, int OCC = 0>
+__global__ void __launch_bounds__((CW + 1) * 32, OCC > 0 ? OCC : ctas_per_sm(CW, G, (int)sizeof(T)))
 decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const T* __restrict__ q_in,
               const T* __restrict__ k_in, const T* __restrict__ v_in, T* __restrict__ out, T* __restrict__ kpool,
@@ -966,12 +967,12 @@ static size_t smem_bytes(int cw, int row_cap, int stages, int G, int row_bytes) 
   return (size_t)stages * stage_bytes(cw, row_bytes) + (size_t)G * row_cap * 4 + 2 * (size_t)row_bytes;
 }
 
-template <typename T, int D, int G, int CW>
+template <typename T, int D, int G, int CW, int OCC = 0>
 static cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v, int n_slices,
                               const void* q, const void* k, const void* v, void* out, void* kpool, void* vpool,
                               cudaStream_t st, bool overlap_previous) {
   const size_t smem = smem_bytes(CW, a.row_cap, a.stages, G, D * (int)sizeof(T));
-  auto kern = decode_kernel<T, D, G, CW>;
+  auto kern = decode_kernel<T, D, G, CW, OCC>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -988,7 +989,14 @@ static cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& map_k, con
 template <typename T, int D>
 static cudaError_t launch_g(int G, int cw, const DecodeArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v, int n_slices,
                             const void* q, const void* k, const void* v, void* out, void* kpool, void* vpool,
-                            cudaStream_t st, bool overlap) {
+                            cudaStream_t st, bool overlap, bool three_per_sm) {
+  // grouped queries on the tensor path with eight warps: a second build capped at 72 registers for three CTAs per SM
+  if constexpr (sizeof(T) == 2) {
+    if (three_per_sm && cw == 8 && G == 4)
+      return launch_one<T, D, 4, 8, 3>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap);
+    if (three_per_sm && cw == 8 && G == 8)
+      return launch_one<T, D, 8, 8, 3>(a, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap);
+  }
   switch (G) {
     case 1: return cw == 16 ? D2O_LAUNCH(1, 16) : cw == 4 ? D2O_LAUNCH(1, 4) : D2O_LAUNCH(1, 8);
     case 2: return cw == 16 ? D2O_LAUNCH(2, 16) : cw == 4 ? D2O_LAUNCH(2, 4) : D2O_LAUNCH(2, 8);
@@ -1018,14 +1026,14 @@ static bool plan_tier(int cw, int smem_rows, int row_bytes, int G, int D, int pe
 }
 
 // Best occupancy tier that fits `max_rows`; 0 = none.
-static int best_tier(int cw, int smem_rows, int row_bytes, int G, int D, int* row_cap, int* stages) {
-  for (int per_sm = max_per_sm(cw, G, row_bytes / D); per_sm >= 1; --per_sm)
+static int best_tier(int cw, int smem_rows, int row_bytes, int G, int D, int occ, int* row_cap, int* stages) {
+  for (int per_sm = occ > 0 ? occ : max_per_sm(cw, G, row_bytes / D); per_sm >= 1; --per_sm)
     if (plan_tier(cw, smem_rows, row_bytes, G, D, per_sm, row_cap, stages)) return per_sm;
   return 0;
 }
 
-static bool plan(int cw, int smem_rows, int row_bytes, int G, int D, int want_stages, int* row_cap, int* stages_out) {
-  if (want_stages <= 0) return best_tier(cw, smem_rows, row_bytes, G, D, row_cap, stages_out) != 0;
+static bool plan(int cw, int smem_rows, int row_bytes, int G, int D, int want_stages, int occ, int* row_cap, int* stages_out) {
+  if (want_stages <= 0) return best_tier(cw, smem_rows, row_bytes, G, D, occ, row_cap, stages_out) != 0;
   const long sm_total = 227 * 1024;
   const int cap = (smem_rows + 7) & ~7;
   const int min_stages = max(2, (cw * G * D * 4 + stage_bytes_of(cw) - 1) / stage_bytes_of(cw));
@@ -1116,7 +1124,19 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     int row_cap, stages;
     int smem_rows = smem_rows_for(cls_max, (double)cls_sum / (p1 - p0), G);
     if (c->decode_smem_rows > 0) smem_rows = min(cls_max, c->decode_smem_rows);
-    if (!plan(cw, smem_rows, row_bytes, G, g.d_head, c->decode_stages, &row_cap, &stages)) {
+    // Tensor path, eight warps, G >= 4: three CTAs per SM (a build capped at 72 registers) when three ring stages
+    // and the logits of rows up to 1.5 x the mean still fit a third of the shared memory; measured on the
+    // 8B-shaped config 382 vs 396 us per step, while with longer slices (two CTAs anyway) that build only spills.
+    bool three = false;
+    if (tensor_path(c->elem_size, G) && cw == 8 && G >= 4 && c->decode_stages == 0) {
+      const long third = 227 * 1024 / 3 - 1024 - 2L * row_bytes - 2048 - 3L * (long)stage_bytes(8, row_bytes);
+      const int rows3 = (int)(third / (4 * G)) & ~7;
+      if (rows3 >= 1.5 * (double)cls_sum / (p1 - p0) || rows3 >= cls_max) {
+        three = true;
+        if (c->decode_smem_rows == 0) smem_rows = min(smem_rows, rows3);
+      }
+    }
+    if (!plan(cw, smem_rows, row_bytes, G, g.d_head, c->decode_stages, three ? 3 : 0, &row_cap, &stages)) {
       *why = D2O_ERR_UNSUPPORTED;
       return cudaSuccess;
     }
@@ -1137,13 +1157,13 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     }
     // inputs and outputs of the step are indexed by the slice's place in the call, which the kernel derives itself
     if (g.dtype == D2O_F32)
-      return g.d_head == 64 ? launch_g<float, 64>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap)
-                            : launch_g<float, 128>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap);
+      return g.d_head == 64 ? launch_g<float, 64>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap, three)
+                            : launch_g<float, 128>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap, three);
     if (g.dtype == D2O_F16)
-      return g.d_head == 64 ? launch_g<__half, 64>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap)
-                            : launch_g<__half, 128>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap);
-    return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap)
-                          : launch_g<__nv_bfloat16, 128>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap);
+      return g.d_head == 64 ? launch_g<__half, 64>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap, three)
+                            : launch_g<__half, 128>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap, three);
+    return g.d_head == 64 ? launch_g<__nv_bfloat16, 64>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap, three)
+                          : launch_g<__nv_bfloat16, 128>(G, cw, ac, map_k, map_v, n_slices, q, k, v, out, kpool, vpool, st, overlap, three);
   };
 
   if (n_long > 0) {
