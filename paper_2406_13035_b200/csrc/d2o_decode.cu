@@ -435,6 +435,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   float mloc[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) mloc[g] = -INFINITY;
+  const int n_plain_fma = min(n, a.row_cap);                        // FMA path: rows (the new token's included) with logits in shared memory
   if constexpr (kTensor) {
     // a stage has SR / 16 tiles of 16 rows, half as many as there are warps: the lower half of the warps takes the
     // even stages, the upper half the odd ones (the others only hand the stage back), so that two stages are worked
@@ -505,13 +506,22 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   } else {
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
       stage_wait(&s_full[slot], ph, &s_timeout);
-      const uint4* st = ring + (size_t)slot * SR * LPR;
+      const uint4* st = ring + (size_t)slot * SR * LPR + (size_t)grp * LPR + lig;   // this thread's piece of row grp
+      const bool full = (s + 1) * SR <= n_plain_fma;                 // every row of the stage is a plain row
+      uint4 raw[4];
+      if (full) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) raw[u] = st[(size_t)u * NGRP * LPR];
+      } else {
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          raw[u] = s * SR + u * NGRP + grp < n ? st[(size_t)u * NGRP * LPR] : make_uint4(0, 0, 0, 0);
+      }
       float dot[G][4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int lr = u * NGRP + grp;
         float f[EPV];
-        Elem<T>::unpack(s * SR + lr < n ? st[(size_t)lr * LPR + lig] : make_uint4(0, 0, 0, 0), f);
+        Elem<T>::unpack(raw[u], f);
 #pragma unroll
         for (int g = 0; g < G; ++g) {
           float x = 0.f;
@@ -526,7 +536,10 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         const float r = reduce4<LPR>(dot[g][0], dot[g][1], dot[g][2], dot[g][3], lig);
-        if (li < n) {
+        if (full) {
+          mloc[g] = fmaxf(mloc[g], r);
+          if (lig % QL == 0) pl[(size_t)g * a.row_cap + li] = r;
+        } else if (li < n) {
           mloc[g] = fmaxf(mloc[g], r);
           if (lig % QL == 0) pl_put(g, li, r);
         }
@@ -702,13 +715,22 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     } else {
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
         stage_wait(&s_full[slot], ph, &s_timeout);
-        const uint4* st = ring + (size_t)slot * SR * LPR;
+        const uint4* st = ring + (size_t)slot * SR * LPR + (size_t)grp * LPR + lig;
+        const bool full = (s + 1) * SR <= n;
+        uint4 raw[4];
+        if (full) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) raw[u] = st[(size_t)u * NGRP * LPR];
+        } else {
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            raw[u] = s * SR + u * NGRP + grp < n ? st[(size_t)u * NGRP * LPR] : make_uint4(0, 0, 0, 0);
+        }
         float dot[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          const int lr = u * NGRP + grp;
           float f[EPV];
-          Elem<T>::unpack(s * SR + lr < n ? st[(size_t)lr * LPR + lig] : make_uint4(0, 0, 0, 0), f);
+          Elem<T>::unpack(raw[u], f);
           float x = 0.f;
 #pragma unroll
           for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], f[e], x);
@@ -883,22 +905,42 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       for (int e = 0; e < EPV; ++e) acc[g][e] = 0.f;
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
       stage_wait(&s_full[slot], ph, &s_timeout);
-      const uint4* st = ring + (size_t)slot * SR * LPR;
+      const uint4* st = ring + (size_t)slot * SR * LPR + (size_t)grp * LPR + lig;
+      const int lbase = s * SR + grp;                                // this thread's rows: lbase + u * NGRP
+      // a plain stage: all rows are cache rows with their weights in shared memory, neither victim nor neighbour
+      const bool plain = (s + 1) * SR <= n_plain_fma && (unsigned)(vic_li - s * SR) >= (unsigned)SR &&
+                         (unsigned)(nn_li - s * SR) >= (unsigned)SR;
+      if (plain) {
+        uint4 raw[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int lr = u * NGRP + grp;
-        const int li = s * SR + lr;
-        if (li < n) {
-          const uint4 raw = st[(size_t)lr * LPR + lig];
-          if (li == vic_li) stash[lig] = raw;
-          if (li == nn_li) stash[LPR + lig] = raw;
+        for (int u = 0; u < 4; ++u) raw[u] = st[(size_t)u * NGRP * LPR];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
           float f[EPV];
-          Elem<T>::unpack(raw, f);
+          Elem<T>::unpack(raw[u], f);
 #pragma unroll
           for (int g = 0; g < G; ++g) {
-            const float p = pl_get(g, li);
+            const float p = pl[(size_t)g * a.row_cap + lbase + u * NGRP];
 #pragma unroll
             for (int e = 0; e < EPV; ++e) acc[g][e] = fmaf(p, f[e], acc[g][e]);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int li = lbase + u * NGRP;
+          if (li < n) {
+            const uint4 raw = st[(size_t)u * NGRP * LPR];
+            if (li == vic_li) stash[lig] = raw;
+            if (li == nn_li) stash[LPR + lig] = raw;
+            float f[EPV];
+            Elem<T>::unpack(raw, f);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+              const float p = pl_get(g, li);
+#pragma unroll
+              for (int e = 0; e < EPV; ++e) acc[g][e] = fmaf(p, f[e], acc[g][e]);
+            }
           }
         }
       }
