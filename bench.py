@@ -172,7 +172,7 @@ def run_ours(args, wl, rank, world, device):
     ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
     launches = {"n": 0, "decode_seen": 0}
 
-    def one_pass(timed: bool):
+    def one_pass(timed: bool, step_events=None):
         e = [ev() for _ in range(5)]
         e[0].record()
         for l in range(L):
@@ -187,6 +187,8 @@ def run_ours(args, wl, rank, world, device):
             for l0 in range(0, L, lpc):
                 l1 = min(L, l0 + lpc)
                 ctx.d2o_decode_step(l0, l1, dq[s, l0:l1], dk[s, l0:l1], dv[s, l0:l1], dout[l0:l1])
+            if step_events is not None:
+                step_events[s + 1].record()
         e[4].record()
         # stats: 2 attention sweeps + density per layer; budgets: 1; compress: select, similarity, neighbour
         # reduce, segments, merge per layer (the fp32 path has one kernel fewer); decode: as counted by the
@@ -215,6 +217,14 @@ def run_ours(args, wl, rank, world, device):
     sync_all()
     t_wall = time.perf_counter() - t_wall
     clocks = sampler.stop()
+    # one more pass, outside the timed ones, with an event after every decode step: the spread of the step times
+    step_ev = [ev() for _ in range(nd + 1)]
+    extra = one_pass(False, step_ev)
+    step_ev[0] = extra[0][3]
+    torch.cuda.synchronize()
+    step_us = sorted(step_ev[i].elapsed_time(step_ev[i + 1]) * 1e3 for i in range(nd))
+    step_pct = {"p50": round(step_us[nd // 2], 2), "p99": round(step_us[min(nd - 1, (nd * 99) // 100)], 2),
+                "max": round(step_us[-1], 2)}
     seg = [[p[0][i].elapsed_time(p[0][i + 1]) for i in range(4)] for p in passes]          # ms
     stats_ms = statistics.mean(s[0] for s in seg)
     budget_ms = statistics.mean(s[1] for s in seg)
@@ -325,7 +335,7 @@ def run_ours(args, wl, rank, world, device):
                    "l2": "decode working set (K_c+V_c of all layers) exceeds the 126 MB L2; prompt tensors exceed it too",
                    "layers_per_decode_call": lpc, "decode_ring_stages": args.stages or "auto",
                    "sequences_per_gpu": wl.batch, "parallelism": "replicas (independent sequences per GPU)"},
-        "decode_steps_per_s_per_gpu": round(steps_per_s, 2), "decode_us_per_step": round(decode_ms * 1e3 / nd, 2),
+        "decode_steps_per_s_per_gpu": round(steps_per_s, 2), "decode_us_per_step": round(decode_ms * 1e3 / nd, 2), "decode_step_us_percentiles": step_pct,
         "stats_ms": round(stats_ms, 3), "budgets_ms": round(budget_ms, 3), "prefill_compress_ms": round(compress_ms, 3),
         "decode_ms": round(decode_ms, 3), "wall_s": round(t_wall, 3),
         "budgets_min_max": [int(budgets.min()), int(budgets.max())],
