@@ -17,6 +17,11 @@
 //   then     merged value row, the new token takes the victim's row.
 // Pass K' is skipped while the cache is not full.  Everything that needs the whole slice is a
 // block-wide reduction inside one CTA; there is no inter-CTA communication.
+//
+// Arithmetic: fp32 FMAs on unpacked rows (one query head per KV head, or fp32 caches), or, for 16-bit caches with
+// grouped queries, mma.sync for all three passes on stages that arrive through tiled tensor maps with the 128-byte
+// swizzle.  A decode step over all layers runs the slices largest first and, where a few slices are much longer
+// than the rest, those in a launch of their own with sixteen consumer warps (see launch_decode).
 #include <math.h>
 
 #include <cuda/std/type_traits>
@@ -74,15 +79,6 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
   return ok != 0;
-}
-// Bounded wait: returns false (and the caller reports D2O_ERR_TIMEOUT) if the phase has not completed in time.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  while (!mbar_try_wait(bar, parity)) {
-    if (global_ns() - t0 > kWaitNs) return false;
-  }
-  return true;
 }
 // Wait for a stage in the kernel's loops: one probe when the phase is already complete (the common case); otherwise
 // poll until it completes, another thread has recorded a timeout, or this one does.
