@@ -1146,7 +1146,7 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     double work = 0.0;
     for (int i = 0; i < n_pairs; ++i) work += Hkv * (fixed_us + row_us * rows_of_pair(i));
     // measured optimum: four pairs on the 7B-shaped config (FMA path), twelve on the long-context one (tensor path)
-    const double limit = (tensor_path(c->elem_size, G) ? 0.55 : 0.7) * work / slots;
+    const double limit = (tensor_path(c->elem_size, G) ? 0.55 : 0.65) * work / slots;
     while (n_long < n_pairs && (n_long + 1) * Hkv <= 2 * 148 && fixed_us + row_us * rows_of_pair(n_long) > limit) ++n_long;
     if (n_long == n_pairs) n_long = 0;
   } else if (ordered && c->decode_long_pairs > 0) {
@@ -1209,7 +1209,8 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     if (e != cudaSuccess || *why != D2O_OK) return e;
     const int rest = (n_pairs - n_long) * Hkv;
     int rest_max = rows_of_pair(n_long);
-    const int cw = (G <= 2 && rest >= 8 * 148 * 4 && rest_max <= 1536) ? 4 : 8;
+    const int cw = (c->decode_warps == 4 || c->decode_warps == 8) ? c->decode_warps
+                   : ((G <= 2 && rest >= 8 * 148 * 4 && rest_max <= 1536) ? 4 : 8);
     return launch_class(n_long, n_pairs, cw, true);
   }
   // Consumer warps per CTA.  One head per KV head and enough small slices for seven and more CTAs on every SM:
