@@ -55,6 +55,7 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers-per-call", type=int, default=0)
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling captures)")
+    ap.add_argument("--batch", type=int, default=0, help="override the number of sequences (the serving sweep of config 4)")
     return ap.parse_args()
 
 
@@ -426,6 +427,9 @@ def run_reference(args, wl):
 def main():
     args = parse()
     wl = W.CONFIGS[args.config] if args.config in W.CONFIGS else W.twin(args.config.replace("_twin", ""))
+    if args.batch:
+        import dataclasses
+        wl = dataclasses.replace(wl, batch=args.batch, name=f"{wl.name}[B={args.batch}]")
     if args.layers:
         import dataclasses
         wl = dataclasses.replace(wl, n_layers=args.layers, name=f"{wl.name}[{args.layers} layers]")
