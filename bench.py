@@ -191,12 +191,12 @@ def run_ours(args, wl, rank, world, device):
             if step_events is not None:
                 step_events[s + 1].record()
         e[4].record()
-        # stats: 2 attention sweeps + density per layer; budgets: 1; compress: select, similarity, neighbour
-        # reduce, segments, merge per layer (the fp32 path has one kernel fewer); decode: as counted by the
+        # stats: 2 attention sweeps + density per layer; budgets: 1; compress: select, gather, similarity,
+        # neighbour reduce, segments, merge per layer (the fp32 path has one kernel fewer); decode: as counted by the
         # library (a step over all layers is one launch, or two when the longest slices get their own)
         dl = ctx.d2o_get_stats().decode_launches
         if timed:
-            launches["n"] += L * 3 + 1 + L * (4 if wl.dtype == "f32" else 5) + (dl - launches["decode_seen"])
+            launches["n"] += L * 3 + 1 + L * (5 if wl.dtype == "f32" else 6) + (dl - launches["decode_seen"])
         launches["decode_seen"] = dl
         return e, budgets
 

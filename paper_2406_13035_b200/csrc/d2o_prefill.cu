@@ -4,7 +4,8 @@
 // Kernels in this file, per layer, one slice = one (sequence, KV head):
 //   select_kernel      group-summed scores, block radix select of the Top-N under the order
 //                      (score desc, position asc), ordered compaction into retained / evicted
-//                      position lists, gather of K_c, V_c, scores and inverse key norms
+//                      position lists and the retained scores
+//   gather_kernel      K_c, V_c and inverse key norms of the retained positions
 //   similarity_kernel  cosine of every evicted key with every retained key, row max / arg-max
 //                      (generic FFMA version; 16-bit inputs take the tcgen05 kernel when built in)
 //   segment_kernel     tau_0 = mean of the row maxima; threshold test; evicted tokens grouped by
@@ -145,15 +146,27 @@ select_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
     if (n_ret != n_keep) report_error(a.status, D2O_ERR_STATE, 0x5E000000u | (uint32_t)slice);
     atomicAdd(&a.counters[kCntPrefillEvicted], (unsigned long long)(P - n_keep));
   }
-  __threadfence_block();
-  __syncthreads();
-  // gather K_c, V_c and 1/|k|: one row per LPR-lane group
+}
+
+// Gather of K_c, V_c and 1/|k| for the positions select_kernel wrote: one row per LPR-lane group, 64 rows per CTA
+// (a kernel of its own so that a single sequence still fills the GPU).
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+gather_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T* __restrict__ kpool,
+              T* __restrict__ vpool) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;                   // lanes per row
+  const int slice = blockIdx.y;
+  const int b = slice / a.Hkv, h = slice % a.Hkv;
+  const int P = a.P;
+  const int S = a.budgets[b * a.L + a.layer];
+  const int n_keep = S >= P ? P : S;
+  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
   const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
   const T* Ks = K + (size_t)slice * P * D;
   const T* Vs = V + (size_t)slice * P * D;
-  for (int r = grp; r < n_keep; r += blockDim.x / LPR) {
+  const int r1 = min(n_keep, ((int)blockIdx.x + 1) * 64);
+  for (int r = blockIdx.x * 64 + grp; r < r1; r += blockDim.x / LPR) {
     const int j = a.pos[row0 + r];
     const uint4 kv = ld_global_v4(Ks + (size_t)j * D + lig * EPV);
     const uint4 vv = ld_global_v4(Vs + (size_t)j * D + lig * EPV);
@@ -518,6 +531,11 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
                                        (int)(sel_sm > 48 * 1024 ? sel_sm : 48 * 1024));
   if (e != cudaSuccess) return e;
   select_kernel<T, D><<<n_slices, kSelThreads, sel_sm, st>>>(sa, (const T*)K, (const T*)V, kpool, vpool);
+  {
+    const int keep_max = min(maxS, P);
+    dim3 ggrid((unsigned)((keep_max + 63) / 64), (unsigned)n_slices);
+    gather_kernel<T, D><<<ggrid, 256, 0, st>>>(sa, (const T*)K, (const T*)V, kpool, vpool);
+  }
 
   int minS = P;
   for (int b = 0; b < B; ++b) minS = min(minS, c->h_budgets[b * L + layer]);
