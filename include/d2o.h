@@ -159,7 +159,8 @@ d2o_status d2o_decode_step(d2o_ctx* ctx, int32_t l0, int32_t l1, const void* q, 
                            const void* v, void* out, void* stream);
 
 /* Same with HOST buffers (pinned memory recommended): copies q, k, v to the device, runs the
- * step, copies `out` back and synchronises `stream`. */
+ * step, copies `out` back and synchronises `stream`.  If q, k and v lie back to back in host
+ * memory in this order they travel in one transfer. */
 d2o_status d2o_decode_step_host(d2o_ctx* ctx, int32_t l0, int32_t l1, const void* q_host,
                                 const void* k_host, const void* v_host, void* out_host,
                                 void* stream);

@@ -284,9 +284,20 @@ extern "C" d2o_status d2o_decode_step_host(d2o_ctx* c, int32_t l0, int32_t l1, c
   char* dk = c->scratch + c->slay.stage_k;
   char* dv = c->scratch + c->slay.stage_v;
   char* dout = c->scratch + c->slay.stage_out;
-  CUDA_TRY(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s));
-  CUDA_TRY(cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, s));
-  CUDA_TRY(cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, s));
+  // q, k, v adjacent in host memory (in this order) and in the staging area: one transfer instead of three.  The
+  // runtime rejects a range that spans two separately pinned allocations before enqueuing anything; then, as for
+  // buffers that are not adjacent, three transfers.
+  const char* qh = (const char*)q_host;
+  bool merged = false;
+  if ((const char*)k_host == qh + qb && (const char*)v_host == qh + qb + kb && dk == dq + qb && dv == dk + kb) {
+    merged = cudaMemcpyAsync(dq, q_host, qb + 2 * kb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!merged) (void)cudaGetLastError();
+  }
+  if (!merged) {
+    CUDA_TRY(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s));
+    CUDA_TRY(cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, s));
+    CUDA_TRY(cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, s));
+  }
   d2o_status why = D2O_OK;
   cudaError_t e = launch_decode(c, l0, l1, dq, dk, dv, dout, s, &why);
   if (why != D2O_OK) return why;
