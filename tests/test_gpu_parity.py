@@ -109,6 +109,17 @@ def test_budget_never_reached_equals_full_attention():
     assert_report(rep, wl.dtype)
 
 
+def test_budgets_large_temperature_gives_uniform_allocation(cuda_device):
+    # gamma -> infinity: the uniform allocation of the paper's ablation (alpha_l = rho)
+    F = np.random.default_rng(3).gamma(1.0, size=(2, 16, 8)) * 500.0
+    bud, win, off, status = B.d2o_budgets_from_density(torch.tensor(F, device=cuda_device), n_kv_heads=2,
+                                                       prompt_len=2000, rho=B.f32(0.2), min_budget=1,
+                                                       density_temp=B.f32(1e30), head_reduce=0, n_sink=1, window=0,
+                                                       nm_ratio=B.f32(3.0))
+    assert int(status[0]) == 0
+    assert (bud.cpu().numpy() == 400).all()
+
+
 def test_budgets_pure_function_matches_oracle(cuda_device):
     r = np.random.default_rng(5)
     for trial in range(40):

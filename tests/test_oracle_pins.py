@@ -120,6 +120,14 @@ def test_budgets_equal_density_is_uniform():
     assert O.layer_budgets(np.array([[2.0]]), 1000, 0.3)[0] == 300  # L = 1
 
 
+def test_budgets_large_temperature_is_the_uniform_allocation():
+    # the ablation's "uniform allocation" alpha_l = rho (Section 5.4, setting 4) is the limit gamma -> infinity of
+    # exp(-F / gamma): every layer gets rho * P whatever the densities are
+    F = rng(11).gamma(1.0, size=(16, 8)) * 500.0
+    S = O.layer_budgets(F, 2000, 0.2, 1, 1e30)
+    assert (S == 400).all()
+
+
 def test_budgets_match_softmax_formula_when_unclamped():
     r = rng(7)
     L, P, rho = 12, 4096, 0.3
