@@ -68,7 +68,9 @@ typedef struct {
   float   density_temp;    /* gamma in exp(-F/gamma); 1.0 is Eq. 5 as printed               */
   int32_t min_budget;      /* lower clamp of S_l (>= n_sink + 1)                            */
   int32_t max_budget;      /* upper clamp of S_l; <= 0 means L_prompt                       */
-  int32_t head_reduce;     /* 0: w_l = sum_h exp(-F_lh/gamma) (Appendix A.5); 1: exp(-mean_h F_lh/gamma) */
+  int32_t head_reduce;     /* layer weight w_l from the per-head densities: 0: sum_h exp(-F_lh/gamma)
+                            * (Appendix A.5); 1: exp(-mean_h F_lh/gamma); reciprocal-of-variance allocation of
+                            * the ablation (Section 5.4, setting 2): 2: sum_h 1/F_lh; 3: 1/mean_h F_lh          */
 } d2o_config;
 
 typedef struct d2o_ctx d2o_ctx;

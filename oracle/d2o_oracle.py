@@ -97,6 +97,7 @@ def layer_weights(F: np.ndarray, gamma: float = 1.0, head_reduce: int = 0) -> np
     ``F`` is [L, H] (one density per layer and query head).
     head_reduce 0 (default; appendix form, Eq. for alpha_l^h): w_l = sum_h exp(-F_lh/gamma)
     head_reduce 1: w_l = exp(-mean_h(F_lh)/gamma)   (main-text form with a per-layer mean)
+    head_reduce 2, 3: w_l = sum_h 1/F_lh, 1/mean_h(F_lh)   (the ablation's reciprocal-of-variance allocation)
     ``gamma`` = 1 is the paper's formula.  The common factor exp(F_min/gamma) is taken out
     for numerical stability; it cancels in the normalisation."""
     F = np.asarray(F, dtype=np.float64)
@@ -107,7 +108,15 @@ def layer_weights(F: np.ndarray, gamma: float = 1.0, head_reduce: int = 0) -> np
     if head_reduce == 1:
         Fm = F.sum(axis=1) / F.shape[1]
         return np.exp(-(Fm - Fm.min()) / gamma)
-    raise ValueError("head_reduce must be 0 or 1")
+    # reciprocal-of-variance allocation (Section 5.4, setting 2): alpha_l proportional to 1 / F; per head (2) or on
+    # the mean over heads (3); a zero variance counts as the smallest positive one
+    tiny = 1e-300
+    if head_reduce == 2:
+        return np.minimum((1.0 / np.maximum(F, tiny)).sum(axis=1), 1e300)
+    if head_reduce == 3:
+        Fm = F.sum(axis=1) / F.shape[1]
+        return np.minimum(1.0 / np.maximum(Fm, tiny), 1e300)
+    raise ValueError("head_reduce must be 0, 1, 2 or 3")
 
 
 def layer_budgets(F: np.ndarray, P: int, rho: float, min_budget: int = 1,

@@ -58,7 +58,7 @@ static d2o_status validate(const d2o_config* c, int64_t* total_budget, int* max_
   if (c->n_sink < 0 || c->nm_ratio < 0.0f || !isfinite(c->nm_ratio)) return D2O_ERR_INVALID_ARG;
   if (!(c->beta >= 0.0f && c->beta <= 1.0f)) return D2O_ERR_INVALID_ARG;
   if (!(c->density_temp > 0.0f) || !isfinite(c->density_temp)) return D2O_ERR_INVALID_ARG;
-  if (c->head_reduce != 0 && c->head_reduce != 1) return D2O_ERR_UNSUPPORTED;
+  if (c->head_reduce < 0 || c->head_reduce > 3) return D2O_ERR_UNSUPPORTED;
   int maxb = c->max_budget > 0 ? c->max_budget : c->prompt_len;
   if (maxb > c->prompt_len + c->max_new_tokens) return D2O_ERR_INVALID_ARG;
   if (c->min_budget < 1 || c->min_budget < c->n_sink + 1 || c->min_budget > maxb) return D2O_ERR_INVALID_ARG;
@@ -186,7 +186,7 @@ extern "C" d2o_status d2o_budgets_from_density(const double* density, int32_t ba
   if (!density || !budgets || batch < 1 || n_layers < 1 || n_layers > 1024 || n_heads < 1 || n_kv_heads < 1 ||
       prompt_len < 1)
     return D2O_ERR_INVALID_ARG;
-  if (!(rho > 0.0f) || !(density_temp > 0.0f) || (head_reduce != 0 && head_reduce != 1)) return D2O_ERR_INVALID_ARG;
+  if (!(rho > 0.0f) || !(density_temp > 0.0f) || head_reduce < 0 || head_reduce > 3) return D2O_ERR_INVALID_ARG;
   if (max_budget <= 0) max_budget = prompt_len;
   if (min_budget < 1 || min_budget > max_budget) return D2O_ERR_INVALID_ARG;
   double tot = floor((double)rho * n_layers * prompt_len + 0.5);

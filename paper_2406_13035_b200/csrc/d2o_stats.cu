@@ -238,6 +238,16 @@ __global__ void budget_kernel(const double* __restrict__ density, int B, int L, 
         for (int h = 0; h < H; ++h) a = __dadd_rn(a, exp(-__ddiv_rn(__dadd_rn(F[l * H + h], -fmin), gamma)));
         w[l] = a;
       }
+    } else if (head_reduce == 2) {
+      // reciprocal of the variance, per head (a zero variance counts as the smallest positive one)
+      for (int l = 0; l < L; ++l) {
+        double a = 0.0;
+        for (int h = 0; h < H; ++h) {
+          const double f = F[l * H + h];
+          a = __dadd_rn(a, __ddiv_rn(1.0, f > 1e-300 ? f : 1e-300));
+        }
+        w[l] = a;
+      }
     } else {
       double fmin = INFINITY;
       for (int l = 0; l < L; ++l) {
@@ -246,9 +256,13 @@ __global__ void budget_kernel(const double* __restrict__ density, int B, int L, 
         x[l] = __ddiv_rn(a, (double)H);
         fmin = fmin < x[l] ? fmin : x[l];
       }
-      for (int l = 0; l < L; ++l) w[l] = exp(-__ddiv_rn(__dadd_rn(x[l], -fmin), gamma));
+      if (head_reduce == 1) {
+        for (int l = 0; l < L; ++l) w[l] = exp(-__ddiv_rn(__dadd_rn(x[l], -fmin), gamma));
+      } else {
+        for (int l = 0; l < L; ++l) w[l] = __ddiv_rn(1.0, x[l] > 1e-300 ? x[l] : 1e-300);
+      }
     }
-    for (int l = 0; l < L; ++l) w[l] = w[l] > 1e-300 ? w[l] : 1e-300;
+    for (int l = 0; l < L; ++l) w[l] = w[l] > 1e-300 ? (w[l] < 1e300 ? w[l] : 1e300) : 1e-300;
     // kinks of the piecewise-linear total(lambda), ascending (insertion sort)
     int nk = 0;
     for (int l = 0; l < L; ++l) {

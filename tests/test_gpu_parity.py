@@ -131,7 +131,7 @@ def test_budgets_pure_function_matches_oracle(cuda_device):
         F = r.gamma(1.0, size=(Bn, L, H)) * float(r.choice([0.01, 1.0, 30.0, 3000.0]))
         if L * smin > math.floor(rho * L * P + 0.5):
             continue
-        hr = int(trial % 2)
+        hr = int(trial % 4)                                          # both softmax rules and both reciprocal rules
         nm = B.f32(3.0)
         bud, win, off, status = B.d2o_budgets_from_density(torch.tensor(F, device=cuda_device), n_kv_heads=2,
                                                            prompt_len=P, rho=rho, min_budget=smin,

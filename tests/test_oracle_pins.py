@@ -128,6 +128,29 @@ def test_budgets_large_temperature_is_the_uniform_allocation():
     assert (S == 400).all()
 
 
+def test_budgets_reciprocal_of_variance_allocation():
+    # Section 5.4, setting 2: alpha_l = (1 / F_l) / sum_l (1 / F_l) * L * rho.  F = 1, 2, 4 -> shares 4/7, 2/7, 1/7
+    # of S_tot = 0.25 * 3 * 7000 = 5250
+    S = O.layer_budgets(np.array([[1.0], [2.0], [4.0]]), 7000, 0.25, 1, 1.0, 2)
+    assert S.tolist() == [3000, 1500, 750]
+    assert O.layer_budgets(np.array([[1.0], [2.0], [4.0]]), 7000, 0.25, 1, 1.0, 3).tolist() == [3000, 1500, 750]
+    # per head: w_l = sum_h 1 / F_lh; on the mean: w_l = 1 / mean_h F_lh
+    F = np.array([[1.0, 4.0], [2.0, 2.0]])                          # rule 2: w = 1.25, 1.0; rule 3: w = 0.4, 0.5
+    assert O.layer_budgets(F, 9000, 0.5, 1, 1.0, 2).tolist() == [5000, 4000]
+    assert O.layer_budgets(F, 9000, 0.5, 1, 1.0, 3).tolist() == [4000, 5000]
+    # the rule does not depend on the unit of F, nor on gamma
+    r = rng(21)
+    Fr = r.gamma(2.0, size=(12, 4)) + 0.1
+    a = O.layer_budgets(Fr, 4096, 0.3, 8, 1.0, 2)
+    assert (O.layer_budgets(Fr * 1024.0, 4096, 0.3, 8, 77.0, 2) == a).all()
+    assert a.sum() == round(0.3 * 12 * 4096)
+    w = (1.0 / Fr).sum(axis=1)
+    for i in range(12):
+        for j in range(12):
+            if w[i] > w[j]:
+                assert a[i] >= a[j] - 1
+
+
 def test_budgets_match_softmax_formula_when_unclamped():
     r = rng(7)
     L, P, rho = 12, 4096, 0.3
