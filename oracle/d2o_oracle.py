@@ -18,10 +18,14 @@ places where a storage dtype enters are the merged rows of ``K_c``/``V_c``,
 which a real cache stores in the model dtype: they are rounded (nearest-even)
 right after a merge, exactly where the cache is written.
 
-Pins (tests/test_oracle_*.py): closed forms, invariants, brute force and
+Pins (tests/test_oracle_pins.py): closed forms, invariants, brute force and
 library routines for every function below.  The end-to-end numeric values of a
 compressed run have no published reference: *parity unpinned* beyond those
 per-step pins.
+
+The functions read top to bottom as the paper's steps.  Nothing in here replays
+another implementation's choices: a harness that wants to follow a near-tie
+composes the step functions itself.
 
 Readings of points the paper leaves open are marked "Reading:" where they are
 taken.
@@ -92,7 +96,7 @@ def attention_density(s: np.ndarray) -> float:
 
 
 def layer_weights(F: np.ndarray, gamma: float = 1.0, head_reduce: int = 0) -> np.ndarray:
-    """Un-normalised inverse-variance-softmax weight of each layer.
+    """Un-normalised allocation weight of each layer.
 
     ``F`` is [L, H] (one density per layer and query head).
     head_reduce 0 (default; appendix form, Eq. for alpha_l^h): w_l = sum_h exp(-F_lh/gamma)
@@ -119,33 +123,26 @@ def layer_weights(F: np.ndarray, gamma: float = 1.0, head_reduce: int = 0) -> np
     raise ValueError("head_reduce must be 0, 1, 2 or 3")
 
 
-def layer_budgets(F: np.ndarray, P: int, rho: float, min_budget: int = 1,
-                  gamma: float = 1.0, head_reduce: int = 0, max_budget: int = 0) -> np.ndarray:
-    """Integer cache size S_l of every layer (Eq. 5; constraint sum_l S_l = S*L*rho).
+def allocate_budgets(w: np.ndarray, S_tot: int, lo: int, cap: int) -> np.ndarray:
+    """Integer sizes x_u = clip(lam * w_u, lo, cap) of allocation units (layers, or (layer, head) pairs)
+    with the single scale ``lam`` that makes them add up to ``S_tot``, then floor + largest remainder.
 
-    Unclamped, S_l = alpha_l * P with alpha_l = L*rho*w_l / sum_l w_l.
-    Reading (the paper is silent on all three):
-      * a layer cannot hold fewer than ``min_budget`` or more than ``max_budget`` tokens
-        (``P`` unless given: the prompt has no more), so
-        S_l = clip(lam * w_l, min_budget, max_budget) with the single scale ``lam`` chosen so
-        that the total is still S_tot (equal to the unclamped formula when no clamp binds);
-      * S_tot = floor(rho*L*P + 1/2);
-      * integer sizes by floor + largest remainder (ties: lower layer first)."""
-    w = layer_weights(F, gamma, head_reduce)
-    L = w.size
-    S_tot = int(math.floor(rho * L * P + 0.5))
-    cap = max_budget if max_budget > 0 else P
-    lo, hi = float(min_budget), float(cap)
-    if not (L * lo <= S_tot <= L * hi):
-        raise ValueError("global budget outside [L*min_budget, L*max_budget]")
-    w = np.maximum(w, 1e-300)        # exp underflow: keep ratios finite
+    Reading (the paper gives S_u = alpha_u * S with sum alpha_u fixed, and is silent on bounds and on
+    integer sizes): a unit cannot hold fewer than ``lo`` or more than ``cap`` tokens; the proportional
+    rule is kept for every unit that neither bound touches (equal to the unclamped formula when no
+    clamp binds); remainders go to the largest fractional parts, ties to the lower unit index."""
+    w = np.maximum(np.asarray(w, dtype=np.float64), 1e-300)        # exp underflow: keep ratios finite
+    n = w.size
+    lo_f, hi_f = float(lo), float(cap)
+    if not (n * lo_f <= S_tot <= n * hi_f):
+        raise ValueError("global budget outside [n*min_budget, n*max_budget]")
 
     def total(lam: float) -> float:
-        return float(np.clip(lam * w, lo, hi).sum())
+        return float(np.clip(lam * w, lo_f, hi_f).sum())
 
     # total(lam) is continuous, piecewise linear and non-decreasing; its kinks are where
-    # a layer leaves the lower clamp (lo/w_l) or reaches the upper one (hi/w_l).
-    kinks = np.sort(np.concatenate([lo / w, hi / w]))
+    # a unit leaves the lower clamp (lo/w_u) or reaches the upper one (cap/w_u).
+    kinks = np.sort(np.concatenate([lo_f / w, hi_f / w]))
     k = 0
     while k < kinks.size and total(kinks[k]) < S_tot:
         k += 1
@@ -156,26 +153,78 @@ def layer_budgets(F: np.ndarray, P: int, rho: float, min_budget: int = 1,
     else:
         a, b = kinks[k - 1], kinks[k]
         mid = 0.5 * (a + b)
-        free = (mid * w > lo) & (mid * w < hi)         # layers on the linear part of this segment
-        fixed = float(np.clip(mid * w, lo, hi)[~free].sum())
+        free = (mid * w > lo_f) & (mid * w < hi_f)     # units on the linear part of this segment
+        fixed = float(np.clip(mid * w, lo_f, hi_f)[~free].sum())
         wf = float(w[free].sum())
         lam = (S_tot - fixed) / wf if wf > 0.0 else b
         lam = min(max(lam, a), b)
-    x = np.clip(lam * w, lo, hi)
+    x = np.clip(lam * w, lo_f, hi_f)
     base = np.floor(x)
     rem = x - base
     S = base.astype(np.int64)
     left = S_tot - int(S.sum())
-    assert 0 <= left <= L, "largest-remainder step out of range"
-    order = sorted(range(L), key=lambda l: (-rem[l], l))
-    for l in order:
+    assert 0 <= left <= n, "largest-remainder step out of range"
+    order = sorted(range(n), key=lambda u: (-rem[u], u))
+    for u in order:
         if left == 0:
             break
-        if S[l] < cap:
-            S[l] += 1
+        if S[u] < cap:
+            S[u] += 1
             left -= 1
     assert left == 0
     return S
+
+
+def layer_budgets(F: np.ndarray, P: int, rho: float, min_budget: int = 1,
+                  gamma: float = 1.0, head_reduce: int = 0, max_budget: int = 0) -> np.ndarray:
+    """Integer cache size S_l of every layer (Eq. 5; constraint sum_l S_l = S*L*rho).
+
+    Unclamped, S_l = alpha_l * P with alpha_l = L*rho*w_l / sum_l w_l.
+    Reading: S_tot = floor(rho*L*P + 1/2); bounds ``min_budget`` and ``max_budget`` (``P`` unless
+    given: the prompt has no more) and integer sizes as in allocate_budgets."""
+    w = layer_weights(F, gamma, head_reduce)
+    L = w.size
+    S_tot = int(math.floor(rho * L * P + 0.5))
+    cap = max_budget if max_budget > 0 else P
+    return allocate_budgets(w, S_tot, min_budget, cap)
+
+
+def head_budgets(F: np.ndarray, P: int, rho: float, group: int = 1, min_budget: int = 1,
+                 gamma: float = 1.0, max_budget: int = 0) -> np.ndarray:
+    """Per-head cache sizes S_l^h = alpha_l^h * S_total of the appendix ("Cache Size Allocation Based
+    on Attention Variance"): alpha_l^h = exp(-F_lh) / sum_{l,h} exp(-F_lh), so that
+    S_l = sum_h S_l^h and alpha_l = sum_h alpha_l^h.  Returns int64 [L, Hkv].
+
+    Reading: the unit that owns cache rows is a KV head; with grouped queries its weight is the sum
+    of the weights of its ``group`` query heads (the same sum that forms its attention score), and
+    S_total = floor(rho * L * Hkv * P + 1/2) head-tokens, i.e. the same number of cache rows as the
+    per-layer rule.  Bounds and integer sizes as in allocate_budgets."""
+    F = np.asarray(F, dtype=np.float64)
+    L, H = F.shape
+    assert H % group == 0
+    Hkv = H // group
+    wq = np.exp(-(F - F.min()) / gamma)                            # [L, H]
+    w = wq.reshape(L, Hkv, group).sum(axis=2).reshape(-1)          # [L * Hkv]
+    S_tot = int(math.floor(rho * L * Hkv * P + 0.5))
+    cap = max_budget if max_budget > 0 else P
+    return allocate_budgets(w, S_tot, min_budget, cap).reshape(L, Hkv)
+
+
+def exp_decay_budgets(F: np.ndarray, P: int, min_budget: int = 1, gamma: float = 1.0,
+                      max_budget: int = 0) -> np.ndarray:
+    """The ablation's "Exponential Decay Allocation" (Section 5.4, setting 3): alpha_l = exp(-F_l),
+    S_l = alpha_l * P.  The factor is not normalised, so the total is whatever the densities give.
+
+    Reading: with several heads alpha_l is the mean over the query heads of exp(-F_lh / gamma)
+    (a fraction in (0, 1]; one head gives the printed formula); S_l = floor(alpha_l * P + 1/2)
+    clamped to [min_budget, max_budget]."""
+    F = np.asarray(F, dtype=np.float64)
+    if F.ndim == 1:
+        F = F[:, None]
+    alpha = np.exp(-F / gamma).sum(axis=1) / F.shape[1]
+    cap = max_budget if max_budget > 0 else P
+    S = np.floor(alpha * P + 0.5).astype(np.int64)
+    return np.clip(S, min_budget, cap)
 
 
 def window_size(S: int, T: int, window: int, nm_ratio: float) -> int:
@@ -239,34 +288,42 @@ def initial_threshold(mx: np.ndarray) -> float:
     return float(mx.sum() / mx.size) if mx.size else 0.0
 
 
+def merge_mask(mx: np.ndarray, tau: float) -> np.ndarray:
+    """m_i of Eq. 12 for the nearest neighbour of evicted token i: it is merged iff its best
+    similarity is not lower than the threshold ("lower than tau: permanently discarded")."""
+    return np.asarray(mx, dtype=np.float64) >= tau
+
+
 def weighted_merge(Kc: np.ndarray, Vc: np.ndarray, Ke: np.ndarray, Ve: np.ndarray,
-                   mx: np.ndarray, nn: np.ndarray, tau: float) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+                   mx: np.ndarray, nn: np.ndarray, mask: np.ndarray,
+                   policy: str = "weighted") -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
     """Eq. 11-12 for all conserved tokens at once.
 
-    m_ij = 1 iff j is i's nearest neighbour and i passed the threshold (mx_i >= tau;
-    "lower than tau: discarded").  Reading of Eq. 12: the weight of evicted token i is
+    ``mask[i]`` says whether evicted token i is merged into conserved token ``nn[i]``
+    (m_ij = 1 iff j is i's nearest neighbour and i passed the threshold, see merge_mask).
+    Reading of Eq. 12: the weight of evicted token i is
     exp(u_ij) m_ij / (sum_i' exp(u_i'j) m_i'j + e), so the weights of a conserved token
-    and of everything merged into it sum to one.  Returns (K_c', V_c', denominators)."""
+    and of everything merged into it sum to one.
+    ``policy`` "average" is the ablation's average merging ("Merge Policy"): the conserved token and
+    every token merged into it weigh the same, 1 / (1 + number merged).
+    Returns (K_c', V_c', denominators; a conserved token's own weight is e, or 1, over its denominator)."""
+    if policy not in ("weighted", "average"):
+        raise ValueError("policy must be 'weighted' or 'average'")
     Kc = np.array(Kc, dtype=np.float64)
     Vc = np.array(Vc, dtype=np.float64)
     Lc = Kc.shape[0]
-    den = np.full(Lc, E, dtype=np.float64)
-    Kn = E * Kc
-    Vn = E * Vc
-    for i in range(mx.size):
-        if mx[i] >= tau:
+    own = E if policy == "weighted" else 1.0
+    den = np.full(Lc, own, dtype=np.float64)
+    Kn = own * Kc
+    Vn = own * Vc
+    for i in range(len(mx)):
+        if mask[i]:
             j = int(nn[i])
-            w = math.exp(mx[i])
+            w = math.exp(mx[i]) if policy == "weighted" else 1.0
             den[j] += w
             Kn[j] += w * Ke[i]
             Vn[j] += w * Ve[i]
     return Kn / den[:, None], Vn / den[:, None], den
-
-
-def _merge_with_mask(Kc, Vc, Ke, Ve, mx, nn, mask):
-    """weighted_merge with an explicit mask m_i instead of the threshold test (harness replay)."""
-    passing = np.where(mask, mx, -np.inf)
-    return weighted_merge(Kc, Vc, Ke, Ve, passing, nn, -1e300)
 
 
 @dataclass
@@ -281,14 +338,24 @@ class SliceState:
     T: int
     M: int
     dtype: str
+    feature: str = "k"     # rows the similarity is computed on: keys (the method) or values (ablation)
+    policy: str = "weighted"
     log: dict = field(default_factory=dict)
 
 
+def feature_rows(K: np.ndarray, V: np.ndarray, feature: str) -> np.ndarray:
+    """Rows that enter the similarity of Eq. 9: the keys in the method ("we compute the similarity
+    matrix only on the key tokens"); the values in the ablation's "Feature choice" row V."""
+    if feature == "k":
+        return K
+    if feature == "v":
+        return V
+    raise ValueError("feature must be 'k' or 'v'")
+
+
 def prefill_compress_slice(K: np.ndarray, V: np.ndarray, score: np.ndarray, S: int, T: int, M: int,
-                           dtype: str, tau_override: float = float("nan"),
-                           force_retained: Optional[np.ndarray] = None,
-                           force_nn: Optional[np.ndarray] = None,
-                           force_merged: Optional[np.ndarray] = None) -> SliceState:
+                           dtype: str, tau_override: float = float("nan"), feature: str = "k",
+                           policy: str = "weighted") -> SliceState:
     """Prompt-stage compression of one slice: eviction (Eq. 7-8), nearest-neighbour
     matching (Eq. 9), tau_0 (Eq. 10) and weighted merging (Eq. 11-12).
 
@@ -296,40 +363,25 @@ def prefill_compress_slice(K: np.ndarray, V: np.ndarray, score: np.ndarray, S: i
     over the query heads that share this KV head (reading for grouped-query attention).
     Reading: similarities use the un-merged keys and all merges happen at once;
     every conserved slot (sinks and window included) can receive merges;
-    a conserved token keeps its own accumulated score.
-    ``force_*`` let a harness replay another implementation's choice at a near-tie: the kept
-    positions, the neighbour column of some evicted rows (-1 = keep own), the merge mask."""
+    a conserved token keeps its own accumulated score."""
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
-    retained, evicted = select_retained(score, S, T, M)
-    if force_retained is not None:
-        retained = np.array(sorted(int(j) for j in force_retained), dtype=np.int64)
-        keep = set(retained.tolist())
-        evicted = np.array([j for j in range(K.shape[0]) if j not in keep], dtype=np.int64)
+    retained, evicted = select_retained(score, S, T, M)                      # Eq. 7-8
     Kc, Vc = K[retained], V[retained]
     Ke, Ve = K[evicted], V[evicted]
-    U = cosine_matrix(Ke, Kc)
+    U = cosine_matrix(feature_rows(Ke, Ve, feature), feature_rows(Kc, Vc, feature))   # Eq. 9
     mx, nn = nearest_neighbour(U)
-    if force_nn is not None:
-        for i, j in enumerate(force_nn):
-            if j >= 0:
-                nn[i] = j
-                mx[i] = U[i, j]
-    tau0 = initial_threshold(mx)
+    tau0 = initial_threshold(mx)                                             # Eq. 10, t = 0
     thr = tau0 if math.isnan(tau_override) else tau_override
-    if force_merged is not None:
-        # a merge mask is replayed by moving the threshold out of the way row by row
-        Km, Vm, den = _merge_with_mask(Kc, Vc, Ke, Ve, mx, nn, np.asarray(force_merged, bool))
-    else:
-        Km, Vm, den = weighted_merge(Kc, Vc, Ke, Ve, mx, nn, thr)
-    touched = den > E
+    mask = merge_mask(mx, thr)
+    Km, Vm, den = weighted_merge(Kc, Vc, Ke, Ve, mx, nn, mask, policy)       # Eq. 11-12
+    touched = den > (E if policy == "weighted" else 1.0)
     Kn = np.where(touched[:, None], round_storage(Km, dtype), Kc)
     Vn = np.where(touched[:, None], round_storage(Vm, dtype), Vc)
     st = SliceState(pos=retained.copy(), K=Kn, V=Vn, score=np.asarray(score, np.float64)[retained].copy(),
-                    tau=tau0, S=S, T=T, M=M, dtype=dtype)
-    st.log = dict(retained=retained, evicted=evicted, mx=mx, nn=nn, den=den, U=U, thr=thr,
-                  merged=(np.asarray(force_merged, bool) if force_merged is not None
-                          else ((mx >= thr) if mx.size else np.zeros(0, bool))))
+                    tau=tau0, S=S, T=T, M=M, dtype=dtype, feature=feature, policy=policy)
+    st.log = dict(retained=retained, evicted=evicted, mx=mx, nn=nn, den=den, U=U, thr=thr, merged=mask,
+                  K_exact=Km, V_exact=Vm, touched=touched)
     return st
 
 
@@ -358,26 +410,14 @@ class StepLog:
     tau: float = float("nan")
     merged: bool = False
     evicted: bool = False
+    K_exact: Optional[np.ndarray] = None  # the merged rows before storage rounding
+    V_exact: Optional[np.ndarray] = None
 
 
-def decode_step_slice(st: SliceState, q: np.ndarray, k: np.ndarray, v: np.ndarray, t: int, beta: float,
-                      tau_override: float = float("nan"),
-                      force_victim_pos: Optional[int] = None,
-                      force_nn_pos: Optional[int] = None) -> Tuple[np.ndarray, StepLog]:
-    """One generated token for one slice.  ``q`` [G, d], ``k``/``v`` [d], ``t`` = position of
-    the new token.  Returns the attention outputs [G, d] (float64) and a log.
-
-    Steps: append (Eq. 2); attention over the cache incl. the new token (Eq. 3);
-    AttnScore += probabilities summed over the G query heads (Eq. 6 case 2); if the cache
-    now exceeds S: evict the lowest-scoring token outside the T sinks and the M most
-    recent positions (Eq. 7-8 keep S = T + N + M); U = cosine of the evicted key to every
-    remaining key (Eq. 9); tau_t = beta*max(U) + (1-beta)*tau_{t-1} (Eq. 10);
-    max(U) >= tau_t -> merge into the nearest neighbour with weights
-    e^{u}/(e^{u}+e), e/(e^{u}+e) (Eq. 11-12 with one evicted token), else discard.
-    Reading: victim ties -> the later position; neighbour ties -> the earlier position;
-    the threshold is updated first, then compared; the neighbour keeps its own score.
-    ``force_*`` let a harness replay another implementation's choice at a near-tie."""
-    q = np.asarray(q, dtype=np.float64).reshape(-1, k.size)
+def decode_attend(st: SliceState, q: np.ndarray, k: np.ndarray, v: np.ndarray, t: int) -> np.ndarray:
+    """Append the new token (Eq. 2), attend over the cache including it (Eq. 3), and add the
+    probabilities of the G query heads to AttnScore (Eq. 6 case 2).  Returns the outputs [G, d]."""
+    q = np.asarray(q, dtype=np.float64).reshape(-1, np.asarray(k).size)
     st.pos = np.append(st.pos, t)
     st.K = np.vstack([st.K, np.asarray(k, np.float64)[None, :]])
     st.V = np.vstack([st.V, np.asarray(v, np.float64)[None, :]])
@@ -387,44 +427,76 @@ def decode_step_slice(st: SliceState, q: np.ndarray, k: np.ndarray, v: np.ndarra
         o, p = softmax_attention(q[g], st.K, st.V)
         out[g] = o
         st.score += p
+    return out
+
+
+def victim_order(st: SliceState, t: int) -> List[int]:
+    """Rows that may be evicted at step ``t`` (outside the T sinks and the M most recent positions,
+    Eq. 7-8), worst first.  Reading: lowest score first, equal scores -> the later position first."""
+    elig = [i for i in range(st.pos.size) if st.T <= st.pos[i] <= t - st.M]
+    return sorted(elig, key=lambda i: (st.score[i], -st.pos[i]))
+
+
+def evict_row(st: SliceState, vi: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Remove row ``vi`` from the cache; returns its key and value."""
+    k_e, v_e = st.K[vi].copy(), st.V[vi].copy()
+    keep = np.arange(st.pos.size) != vi
+    st.pos, st.K, st.V, st.score = st.pos[keep], st.K[keep], st.V[keep], st.score[keep]
+    return k_e, v_e
+
+
+def neighbour_order(st: SliceState, k_e: np.ndarray, v_e: np.ndarray) -> Tuple[np.ndarray, List[int]]:
+    """U = cosine of the evicted token with every remaining row (Eq. 9, one evicted token) and the
+    rows ordered best first.  Reading: equal similarity -> the earlier position first."""
+    U = cosine_matrix(feature_rows(k_e, v_e, st.feature)[None, :], feature_rows(st.K, st.V, st.feature))[0]
+    return U, sorted(range(U.size), key=lambda j: (-U[j], st.pos[j]))
+
+
+def compensate(st: SliceState, k_e: np.ndarray, v_e: np.ndarray, nj: int, mx: float, beta: float,
+               tau_override: float, log: StepLog) -> None:
+    """tau_t = beta * Max(U_t) + (1 - beta) * tau_{t-1} (Eq. 10), then merge the evicted token into row
+    ``nj`` if mx >= tau_t, with weights e^{u}/(e^{u}+e) and e/(e^{u}+e) (Eq. 11-12 with one evicted
+    token), else discard it.  Reading: the threshold is updated first, then compared; the neighbour
+    keeps its own score; the merged rows are rounded to the cache dtype where they are stored."""
+    st.tau = beta * mx + (1.0 - beta) * st.tau
+    thr = st.tau if math.isnan(tau_override) else tau_override
+    log.mx, log.nn_pos, log.tau = mx, int(st.pos[nj]), st.tau
+    if merge_mask(np.array([mx]), thr)[0]:
+        Km, Vm, _ = weighted_merge(st.K[nj][None, :], st.V[nj][None, :], k_e[None, :], v_e[None, :],
+                                   np.array([mx]), np.array([0]), np.array([True]), st.policy)
+        log.K_exact, log.V_exact = Km[0], Vm[0]
+        st.K[nj] = round_storage(Km[0], st.dtype)
+        st.V[nj] = round_storage(Vm[0], st.dtype)
+        log.merged = True
+
+
+def decode_step_slice(st: SliceState, q: np.ndarray, k: np.ndarray, v: np.ndarray, t: int, beta: float,
+                      tau_override: float = float("nan")) -> Tuple[np.ndarray, StepLog]:
+    """One generated token for one slice.  ``q`` [G, d], ``k``/``v`` [d], ``t`` = position of
+    the new token.  Returns the attention outputs [G, d] (float64) and a log.
+
+    Steps: append, attend, accumulate (decode_attend); if the cache now exceeds S: evict the
+    lowest-scoring token outside the T sinks and the M most recent positions (victim_order,
+    evict_row); cosine of the evicted token to every remaining one (neighbour_order);
+    threshold update and merge-or-discard (compensate)."""
+    out = decode_attend(st, q, k, v, t)
     log = StepLog(tau=st.tau)
     if st.pos.size <= st.S:
         return out, log
-    # ---- eviction of one token
-    elig = [i for i in range(st.pos.size) if st.T <= st.pos[i] <= t - st.M]
-    assert elig, "no evictable slot: S < T + M"
-    ranked = sorted(elig, key=lambda i: (st.score[i], -st.pos[i]))   # lowest score, then latest position
-    vi = ranked[0]
+    ranked = victim_order(st, t)
+    assert ranked, "no evictable slot: S < T + M"
     if len(ranked) > 1:
         a, b = st.score[ranked[0]], st.score[ranked[1]]
         log.victim_gap = abs(b - a) / max(abs(a), abs(b), 1e-300)
         log.runner_up_pos = int(st.pos[ranked[1]])
-    if force_victim_pos is not None:
-        vi = int(np.nonzero(st.pos == force_victim_pos)[0][0])
-    log.victim_pos = int(st.pos[vi])
+    log.victim_pos = int(st.pos[ranked[0]])
     log.evicted = True
-    k_e, v_e = st.K[vi].copy(), st.V[vi].copy()
-    keep = np.arange(st.pos.size) != vi
-    st.pos, st.K, st.V, st.score = st.pos[keep], st.K[keep], st.V[keep], st.score[keep]
-    # ---- compensation
-    U = cosine_matrix(k_e[None, :], st.K)[0]
-    order = sorted(range(U.size), key=lambda j: (-U[j], st.pos[j]))
-    nj = order[0]
+    k_e, v_e = evict_row(st, ranked[0])
+    U, order = neighbour_order(st, k_e, v_e)
     if len(order) > 1:
         log.nn_gap = float(U[order[0]] - U[order[1]])
         log.nn_runner_pos = int(st.pos[order[1]])
-    if force_nn_pos is not None:
-        nj = int(np.nonzero(st.pos == force_nn_pos)[0][0])
-    mx = float(U[nj])
-    st.tau = beta * mx + (1.0 - beta) * st.tau
-    thr = st.tau if math.isnan(tau_override) else tau_override
-    log.mx, log.nn_pos, log.tau = mx, int(st.pos[nj]), st.tau
-    if mx >= thr:
-        w_e = math.exp(mx) / (math.exp(mx) + E)
-        w_c = E / (math.exp(mx) + E)
-        st.K[nj] = round_storage(w_c * st.K[nj] + w_e * k_e, st.dtype)
-        st.V[nj] = round_storage(w_c * st.V[nj] + w_e * v_e, st.dtype)
-        log.merged = True
+    compensate(st, k_e, v_e, order[0], float(U[order[0]]), beta, tau_override, log)
     return out, log
 
 
@@ -435,15 +507,29 @@ def full_attention_step(q: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndarr
                      for g in range(q.shape[0])])
 
 
+def group_score(colsum: np.ndarray, h: int, G: int) -> np.ndarray:
+    """AttnScore of KV head ``h`` at the prompt stage from the per-query-head column sums [Hq, P].
+    Reading (grouped-query attention; the paper does not treat it): one retained set per KV head,
+    whose score is the sum over its G query heads' attention, at the prompt stage as in decode_attend."""
+    return np.asarray(colsum, dtype=np.float64)[h * G:(h + 1) * G].sum(axis=0)
+
+
 # --------------------------------------------------------------------------------------
 # whole path for a small stack (used by the parity tests, the smoke check and the timed
 # CPU baseline).  Tensors: Q [B,Hq,P,d], K/V [B,Hkv,P,d] per layer.
 # --------------------------------------------------------------------------------------
 class OracleStack:
+    """``prompt_lens`` (one length per sequence, each <= prompt_len) makes the batch ragged: sequence b
+    uses the first prompt_lens[b] positions of its tensors, its own budgets, and its generated tokens
+    continue at position prompt_lens[b].  ``budget_rule``: "layer" (Eq. 5), "head" (per-head sizes of
+    the appendix) or "exp_decay" (Section 5.4, setting 3)."""
+
     def __init__(self, *, n_layers: int, batch: int, n_q_heads: int, n_kv_heads: int, d_head: int,
                  dtype: str, prompt_len: int, rho: float, n_sink: int, window: int, nm_ratio: float,
                  beta: float, density_temp: float = 1.0, min_budget: int = 1, head_reduce: int = 0,
-                 tau_override: float = float("nan"), max_budget: int = 0):
+                 tau_override: float = float("nan"), max_budget: int = 0, feature: str = "k",
+                 policy: str = "weighted", budget_rule: str = "layer",
+                 prompt_lens: Optional[List[int]] = None):
         self.L, self.B, self.Hq, self.Hkv, self.d = n_layers, batch, n_q_heads, n_kv_heads, d_head
         self.G = n_q_heads // n_kv_heads
         self.dtype, self.P, self.rho = dtype, prompt_len, rho
@@ -451,55 +537,71 @@ class OracleStack:
         self.gamma, self.min_budget, self.head_reduce = density_temp, min_budget, head_reduce
         self.tau_override = tau_override
         self.max_budget = max_budget
+        self.feature, self.policy, self.budget_rule = feature, policy, budget_rule
+        self.Pb = [prompt_len] * batch if prompt_lens is None else [int(p) for p in prompt_lens]
+        assert len(self.Pb) == batch and all(1 <= p <= prompt_len for p in self.Pb)
         self.colsum = np.zeros((self.L, self.B, self.Hq, self.P))
         self.F = np.zeros((self.B, self.L, self.Hq))
-        self.budgets: Optional[np.ndarray] = None          # [B, L]
+        self.budgets: Optional[np.ndarray] = None          # [B, L, Hkv]
         self.slices: dict = {}
-        self.t = prompt_len
 
     def layer_stats(self, layer: int, Q: np.ndarray, K: np.ndarray, heads: Optional[List[Tuple[int, int]]] = None):
         """Column sums and densities of one layer; ``heads`` restricts to (b, hq) pairs."""
         todo = heads if heads is not None else [(b, h) for b in range(self.B) for h in range(self.Hq)]
         for b, h in todo:
-            s = colsum_scores(Q[b, h], K[b, h // self.G])
-            self.colsum[layer, b, h] = s
+            Pb = self.Pb[b]
+            s = colsum_scores(Q[b, h][:Pb], K[b, h // self.G][:Pb])
+            self.colsum[layer, b, h, :Pb] = s
             self.F[b, layer, h] = attention_density(s)
 
     def layer_budgets(self, F: Optional[np.ndarray] = None) -> np.ndarray:
+        """Cache size of every (sequence, layer, KV head), int64 [B, L, Hkv]; the per-layer rules give
+        all KV heads of a layer the same size."""
         F = self.F if F is None else np.asarray(F, np.float64)
-        self.budgets = np.stack([layer_budgets(F[b], self.P, self.rho, self.min_budget, self.gamma,
-                                               self.head_reduce, self.max_budget) for b in range(self.B)])
-        return self.budgets
+        out = np.zeros((self.B, self.L, self.Hkv), dtype=np.int64)
+        for b in range(self.B):
+            Pb = self.Pb[b]
+            cap = self.max_budget if self.max_budget > 0 else Pb
+            if self.budget_rule == "layer":
+                out[b] = layer_budgets(F[b], Pb, self.rho, self.min_budget, self.gamma, self.head_reduce,
+                                       cap)[:, None]
+            elif self.budget_rule == "head":
+                out[b] = head_budgets(F[b], Pb, self.rho, self.G, self.min_budget, self.gamma, cap)
+            elif self.budget_rule == "exp_decay":
+                out[b] = exp_decay_budgets(F[b], Pb, self.min_budget, self.gamma, cap)[:, None]
+            else:
+                raise ValueError("budget_rule must be 'layer', 'head' or 'exp_decay'")
+        self.budgets = out
+        return out
 
-    def slice_params(self, b: int, layer: int) -> Tuple[int, int, int]:
-        S = int(self.budgets[b, layer])
+    def slice_params(self, b: int, layer: int, h: int = 0) -> Tuple[int, int, int]:
+        S = int(self.budgets[b, layer, h])
         T = min(self.T, S)
         M = window_size(S, T, self.window, self.nm_ratio)
         return S, T, M
 
     def group_score(self, layer: int, b: int, h: int) -> np.ndarray:
-        """AttnScore of one KV head at the prompt stage: the sum over its G query heads."""
-        return self.colsum[layer, b, h * self.G:(h + 1) * self.G].sum(axis=0)
+        return group_score(self.colsum[layer, b, :, :self.Pb[b]], h, self.G)
 
     def prefill_compress(self, layer: int, K: np.ndarray, V: np.ndarray,
-                         slices: Optional[List[Tuple[int, int]]] = None, force: Optional[dict] = None):
-        """``slices`` restricts to (b, kv head) pairs; ``force[(layer,b,h)]`` may hold the
-        keyword overrides of prefill_compress_slice."""
+                         slices: Optional[List[Tuple[int, int]]] = None):
+        """``slices`` restricts to (b, kv head) pairs."""
         todo = slices if slices is not None else [(b, h) for b in range(self.B) for h in range(self.Hkv)]
         for b, h in todo:
-            S, T, M = self.slice_params(b, layer)
-            kw = (force or {}).get((layer, b, h), {})
-            self.slices[(layer, b, h)] = prefill_compress_slice(K[b, h], V[b, h], self.group_score(layer, b, h),
-                                                                S, T, M, self.dtype, self.tau_override, **kw)
+            S, T, M = self.slice_params(b, layer, h)
+            Pb = self.Pb[b]
+            self.slices[(layer, b, h)] = prefill_compress_slice(K[b, h][:Pb], V[b, h][:Pb],
+                                                                self.group_score(layer, b, h), S, T, M,
+                                                                self.dtype, self.tau_override, self.feature,
+                                                                self.policy)
 
-    def decode_step(self, layer: int, q: np.ndarray, k: np.ndarray, v: np.ndarray, t: int,
-                    slices: Optional[List[Tuple[int, int]]] = None, force: Optional[dict] = None):
-        """q [B,Hq,d], k/v [B,Hkv,d] -> {(b,kvh): (out [G,d], StepLog)}."""
+    def decode_step(self, layer: int, q: np.ndarray, k: np.ndarray, v: np.ndarray, step: int,
+                    slices: Optional[List[Tuple[int, int]]] = None):
+        """Token number ``step`` (0-based) after the prompt: q [B,Hq,d], k/v [B,Hkv,d] ->
+        {(b,kvh): (out [G,d], StepLog)}; the new token of sequence b has position prompt_lens[b] + step."""
         todo = slices if slices is not None else [(b, h) for b in range(self.B) for h in range(self.Hkv)]
         res = {}
         for b, h in todo:
-            f = (force or {}).get((layer, b, h), {})
             res[(b, h)] = decode_step_slice(self.slices[(layer, b, h)], q[b, h * self.G:(h + 1) * self.G],
-                                            k[b, h], v[b, h], t, self.beta, self.tau_override,
-                                            f.get("victim"), f.get("nn"))
+                                            k[b, h], v[b, h], self.Pb[b] + step, self.beta, self.tau_override)
         return res

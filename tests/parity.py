@@ -8,8 +8,16 @@ CPU, on the same seeded tensors, and compares stage by stage:
 Where floating point decides an index (Top-N boundary, arg-min victim, arg-max neighbour,
 threshold test) the GPU decides in float32 and the oracle in float64.  A disagreement is a
 *tolerated tie* only if the oracle's own gap between the two candidates is below `tie_rtol`
-(1e-6 relative); the oracle then replays the GPU's choice ("tie-follow") so that later stages
-stay comparable, and the event is counted in the report.
+(1e-6 relative); the harness then replays the GPU's choice ("tie-follow") by composing the oracle's
+step functions itself, so that later stages stay comparable, and the event is counted in the report.
+
+Cache content: for float32 caches the oracle keeps its own trajectory over all steps and the merged
+rows are compared at the 1e-5 tolerance.  For 16-bit caches a merged value that sits on a rounding
+boundary of the cache dtype may round either way in float32 (GPU) and float64 (oracle) arithmetic; one
+16-bit ulp in a key moves later logits by ~1e-3, so after a comparison that passed the oracle continues
+from the rows the GPU stored ("storage-follow").  Every adopted element is checked: it must lie in a
+row that was merged in this very step, be the neighbouring representable value of the oracle's, and the
+oracle's unrounded value must sit within a few float32 ulps of the rounding boundary between the two.
 """
 from __future__ import annotations
 
@@ -26,6 +34,9 @@ from paper_2406_13035_b200 import binding as B
 from paper_2406_13035_b200 import workloads as W
 
 TIE_RTOL = 1e-6
+# |exact - rounding boundary| of an adopted 16-bit element, relative to the row's scale: a few float32 ulps for the
+# two-term merge of a decode step, more for a prompt-stage row that sums up to hundreds of float32 terms
+BOUNDARY_RTOL = {"decode": 4e-6, "prefill": 2e-5}
 
 
 @dataclass
@@ -37,6 +48,7 @@ class Report:
     steps: int = 0
     merges: int = 0
     discards: int = 0
+    storage_flips: int = 0
 
     def err(self, key: str, v: float):
         self.max_err[key] = max(self.max_err.get(key, 0.0), float(v))
@@ -128,9 +140,10 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
             ref = orc.F[b, l, h * G + g]
             rep.err("density_rel", abs(F_gpu[b, l, h * G + g] - ref) / max(abs(ref), 1e-12))
     # budgets: the oracle's pure function on the GPU's densities must give the GPU's integers
-    orc_b = orc.layer_budgets(F_gpu)
-    rep.ties["budget"] = int((orc_b != budgets).sum())
-    orc.budgets = budgets.copy()                       # budget-follow
+    orc_b = orc.layer_budgets(F_gpu)                   # [B, L, Hkv]
+    gpu_b = budgets[:, :, None] if budgets.ndim == 2 else budgets
+    rep.ties["budget"] = int((orc_b != gpu_b).sum())
+    orc.budgets = np.broadcast_to(gpu_b, orc_b.shape).copy()     # budget-follow
     tabs = ctx.tables()
     for b in range(Bn):
         for l in range(L):
@@ -150,7 +163,6 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
     n_steps = wl.decode_steps if steps is None else steps
     lpc = L if layers_per_call is None else layers_per_call
     for step in range(n_steps):
-        t = P + step
         qs, ks, vs = zip(*[streams[l].decode() for l in range(L)])
         q, k, v = torch.stack(qs), torch.stack(ks), torch.stack(vs)
         out = torch.empty_like(q)
@@ -160,7 +172,7 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
                                 out[l0:l1])
         qc, kc, vc, oc = np64(q), np64(k), np64(v), np64(out)
         for l, b, h in chk:
-            _check_decode_slice(rep, ctx, orc, wl, l, b, h, qc[l], kc[l], vc[l], oc[l], t, tabs, tie_rtol)
+            _check_decode_slice(rep, ctx, orc, wl, l, b, h, qc[l], kc[l], vc[l], oc[l], step, tabs, tie_rtol)
         rep.steps += 1
     st = ctx.d2o_get_stats()
     assert st.error_word == 0, f"device error word {st.error_word} detail {st.error_detail:#x}"
@@ -183,17 +195,83 @@ def _gap_rel(a: float, b: float) -> float:
     return abs(a - b) / max(abs(a), abs(b), 1e-300)
 
 
-def _check_prefill_slice(rep, ctx, orc, wl, l, b, h, K64, V64, tabs, tie_rtol):
-    G, P = wl.group, wl.prompt_len
-    got = ctx.slice_state(l, b, h, tabs)
-    S, T, M = orc.slice_params(b, l)
+def replay_prefill(orc, l, b, h, K64, V64, retained=None, nn_override=None, mask_override=None):
+    """The steps of O.prefill_compress_slice, composed here so that the GPU's choice at a near-tie (kept set,
+    neighbour of some evicted rows, merge mask) can take the place of the oracle's own.  Used only after a
+    disagreement has been shown to be a tie."""
+    S, T, M = orc.slice_params(b, l, h)
+    Pb = orc.Pb[b]
+    K, V = K64[b, h][:Pb], V64[b, h][:Pb]
     score = orc.group_score(l, b, h)
-    force = {}
+    if retained is None:
+        retained, evicted = O.select_retained(score, S, T, M)
+    else:
+        retained = np.array(sorted(int(j) for j in retained), dtype=np.int64)
+        keep = set(retained.tolist())
+        evicted = np.array([j for j in range(Pb) if j not in keep], dtype=np.int64)
+    Kc, Vc, Ke, Ve = K[retained], V[retained], K[evicted], V[evicted]
+    U = O.cosine_matrix(O.feature_rows(Ke, Ve, orc.feature), O.feature_rows(Kc, Vc, orc.feature))
+    mx, nn = O.nearest_neighbour(U)
+    if nn_override is not None:
+        for i, j in enumerate(nn_override):
+            if j >= 0:
+                nn[i] = j
+                mx[i] = U[i, j]
+    tau0 = O.initial_threshold(mx)
+    thr = tau0 if math.isnan(orc.tau_override) else orc.tau_override
+    mask = O.merge_mask(mx, thr) if mask_override is None else np.asarray(mask_override, bool)
+    Km, Vm, den = O.weighted_merge(Kc, Vc, Ke, Ve, mx, nn, mask, orc.policy)
+    touched = den > (O.E if orc.policy == "weighted" else 1.0)
+    Kn = np.where(touched[:, None], O.round_storage(Km, orc.dtype), Kc)
+    Vn = np.where(touched[:, None], O.round_storage(Vm, orc.dtype), Vc)
+    st = O.SliceState(pos=retained.copy(), K=Kn, V=Vn, score=score[retained].copy(), tau=tau0, S=S, T=T, M=M,
+                      dtype=orc.dtype, feature=orc.feature, policy=orc.policy)
+    st.log = dict(retained=retained, evicted=evicted, mx=mx, nn=nn, den=den, U=U, thr=thr, merged=mask,
+                  K_exact=Km, V_exact=Vm, touched=touched)
+    orc.slices[(l, b, h)] = st
+    return st
+
+
+def replay_decode(st, q, k, v, t, beta, tau_override, victim_pos=None, nn_pos=None):
+    """The steps of O.decode_step_slice with the GPU's victim and / or neighbour in place of the oracle's own."""
+    out = O.decode_attend(st, q, k, v, t)
+    log = O.StepLog(tau=st.tau)
+    if st.pos.size <= st.S:
+        return out, log
+    ranked = O.victim_order(st, t)
+    assert ranked
+    vi = ranked[0] if victim_pos is None else int(np.nonzero(st.pos == victim_pos)[0][0])
+    if len(ranked) > 1:
+        a, b_ = st.score[ranked[0]], st.score[ranked[1]]
+        log.victim_gap = abs(b_ - a) / max(abs(a), abs(b_), 1e-300)
+        log.runner_up_pos = int(st.pos[ranked[1]])
+    log.victim_pos, log.evicted = int(st.pos[vi]), True
+    k_e, v_e = O.evict_row(st, vi)
+    U, order = O.neighbour_order(st, k_e, v_e)
+    nj = order[0] if nn_pos is None else int(np.nonzero(st.pos == nn_pos)[0][0])
+    if len(order) > 1:
+        log.nn_gap = float(U[order[0]] - U[order[1]])
+        log.nn_runner_pos = int(st.pos[order[1]])
+    O.compensate(st, k_e, v_e, nj, float(U[nj]), beta, tau_override, log)
+    return out, log
+
+
+def _thr_tie(mx: float, thr: float, tie_rtol: float) -> bool:
+    # cosines and thresholds live on a unit scale: relative to max(|mx|, |thr|, 1)
+    return abs(mx - thr) <= tie_rtol * max(abs(mx), abs(thr), 1.0)
+
+
+def _check_prefill_slice(rep, ctx, orc, wl, l, b, h, K64, V64, tabs, tie_rtol):
+    P = orc.Pb[b]
+    got = ctx.slice_state(l, b, h, tabs)
+    S, T, M = orc.slice_params(b, l, h)
+    score = orc.group_score(l, b, h)
     orc.prefill_compress(l, K64, V64, [(b, h)])
     st = orc.slices[(l, b, h)]
     gpos = got["pos"].numpy().astype(np.int64)
     assert got["len"] == min(S, P)
     assert np.all(np.diff(gpos) > 0), "GPU retained positions must be ascending"
+    follow = {}
     if not np.array_equal(gpos, st.pos):
         # tolerated only if every swapped pair is a near-tie at the Top-N boundary
         only_gpu = sorted(set(gpos.tolist()) - set(st.pos.tolist()))
@@ -205,9 +283,8 @@ def _check_prefill_slice(rep, ctx, orc, wl, l, b, h, K64, V64, tabs, tie_rtol):
             f"retained set differs beyond a tie: layer {l} b {b} h {h}: {only_gpu} vs {only_orc}, gap {_gap_rel(lo, hi):.3e}"
         assert all(T <= j < P - M for j in only_gpu)
         rep.ties["topn"] += len(only_gpu)
-        force["force_retained"] = gpos
-        orc.prefill_compress(l, K64, V64, [(b, h)], force={(l, b, h): force})
-        st = orc.slices[(l, b, h)]
+        follow["retained"] = gpos
+        st = replay_prefill(orc, l, b, h, K64, V64, **follow)
     Le = P - min(S, P)
     if Le > 0:
         eidx, emx, enn = ctx.evict_lists(b, h, Le)
@@ -215,6 +292,7 @@ def _check_prefill_slice(rep, ctx, orc, wl, l, b, h, K64, V64, tabs, tie_rtol):
         U = st.log["U"]
         mx_o, nn_o = st.log["mx"], st.log["nn"]
         gnn = enn.numpy().astype(np.int64)
+        assert gnn.min() >= 0 and gnn.max() < min(S, P), "neighbour slot out of range"
         bad = np.nonzero(gnn != nn_o)[0]
         if bad.size:
             for i in bad:
@@ -223,9 +301,8 @@ def _check_prefill_slice(rep, ctx, orc, wl, l, b, h, K64, V64, tabs, tie_rtol):
             rep.ties["nn"] += int(bad.size)
             fnn = np.full(Le, -1, np.int64)
             fnn[bad] = gnn[bad]
-            force["force_nn"] = fnn
-            orc.prefill_compress(l, K64, V64, [(b, h)], force={(l, b, h): force})
-            st = orc.slices[(l, b, h)]
+            follow["nn_override"] = fnn
+            st = replay_prefill(orc, l, b, h, K64, V64, **follow)
             mx_o = st.log["mx"]
         rep.err("sim_abs", np.max(np.abs(emx.numpy() - mx_o)))
         rep.err("tau0_abs", abs(got["tau"] - st.tau))
@@ -236,16 +313,26 @@ def _check_prefill_slice(rep, ctx, orc, wl, l, b, h, K64, V64, tabs, tie_rtol):
         flip = np.nonzero(gmask != omask)[0]
         if flip.size:
             for i in flip:
-                assert abs(mx_o[i] - st.log["thr"]) <= 4e-6, \
+                assert _thr_tie(mx_o[i], st.log["thr"], tie_rtol), \
                     f"merge decision differs beyond a tie: row {i}: mx {mx_o[i]} thr {st.log['thr']}"
             rep.ties["mask"] += int(flip.size)
-            force["force_merged"] = gmask
-            orc.prefill_compress(l, K64, V64, [(b, h)], force={(l, b, h): force})
-            st = orc.slices[(l, b, h)]
-    _compare_state(rep, got, st, wl.dtype, "prefill")
+            follow["mask_override"] = gmask
+            st = replay_prefill(orc, l, b, h, K64, V64, **follow)
+    _compare_state(rep, got, st, wl.dtype, "prefill", st.log.get("K_exact"), st.log.get("V_exact"),
+                   st.log.get("touched"))
 
 
-def _compare_state(rep, got, st, dtype, tag):
+def _adjacent(a: np.ndarray, b: np.ndarray, dtype: str) -> np.ndarray:
+    """True where a and b (both representable in the 16-bit dtype) are neighbouring representable values."""
+    td = torch.float16 if dtype == "f16" else torch.bfloat16
+    ia = torch.tensor(a, dtype=torch.float64).to(td).view(torch.int16).to(torch.int32)
+    ib = torch.tensor(b, dtype=torch.float64).to(td).view(torch.int16).to(torch.int32)
+    return ((ia - ib).abs() == 1).numpy()
+
+
+def _compare_state(rep, got, st, dtype, tag, K_exact=None, V_exact=None, merged_rows=None):
+    """`K_exact`/`V_exact`: the oracle's unrounded merged rows ([len, d], or None when nothing was merged);
+    `merged_rows`: boolean [len], the rows written by a merge in the step just compared."""
     gpos = got["pos"].numpy().astype(np.int64)
     order = np.argsort(gpos, kind="stable")
     assert np.array_equal(gpos[order], st.pos), f"{tag}: cache positions differ"
@@ -253,39 +340,54 @@ def _compare_state(rep, got, st, dtype, tag):
     eK, eV = close(Kg, st.K, dtype), close(Vg, st.V, dtype)
     rep.err(f"{tag}_K", eK)
     rep.err(f"{tag}_V", eV)
-    if eK <= 1.0 and eV <= 1.0:
-        # storage-follow: a merged value that sits on a rounding boundary of the cache dtype may round
-        # either way (float32 vs float64 arithmetic).  The flip is within tolerance, but one 16-bit ulp in a
-        # key moves later logits by ~1e-3, so the oracle continues from the rows the GPU actually stored.
-        rep.storage_flips = getattr(rep, "storage_flips", 0) + int((Kg != st.K).sum() + (Vg != st.V).sum())
+    if dtype != "f32" and eK <= 1.0 and eV <= 1.0:
+        # storage-follow, 16-bit caches only (see the module docstring); every adopted element is checked
+        for name, G_, R_, X_ in (("K", Kg, st.K, K_exact), ("V", Vg, st.V, V_exact)):
+            diff = G_ != R_
+            if not diff.any():
+                continue
+            assert merged_rows is not None and X_ is not None, f"{tag}: {name} differs in a step without a merge"
+            rows = np.nonzero(diff.any(axis=1))[0]
+            assert np.all(np.asarray(merged_rows)[rows]), f"{tag}: {name} differs outside the merged rows {rows}"
+            assert np.all(_adjacent(G_[diff], R_[diff], dtype)), f"{tag}: adopted {name} elements are not one ulp apart"
+            mid = 0.5 * (G_ + R_)
+            scale = np.maximum(np.abs(mid), np.sqrt(np.mean(np.asarray(X_)[rows] ** 2)))
+            off = np.abs(np.asarray(X_) - mid)[diff] / scale[diff]
+            rep.err(f"{tag}_boundary_rel", float(off.max()))
+            assert off.max() <= BOUNDARY_RTOL[tag], f"{tag}: adopted {name} element {off.max():.2e} away from the rounding boundary"
+            rep.storage_flips += int(diff.sum())
         st.K, st.V = Kg.copy(), Vg.copy()
     sc = got["score"].double().numpy()[order]
     rep.err(f"{tag}_score_rel", np.max(np.abs(sc - st.score) / np.maximum(np.abs(st.score), 1e-6)))
-    # the cached inverse norms belong to the stored keys
-    Kg = got["K"].double().numpy()
-    nrm = np.sqrt((Kg * Kg).sum(axis=1))
+    # the cached inverse norms belong to the stored rows the similarity is computed on
+    Fg = O.feature_rows(got["K"].double().numpy(), got["V"].double().numpy(), st.feature)
+    nrm = np.sqrt((Fg * Fg).sum(axis=1))
     rn = got["rnorm"].double().numpy()
     ok = nrm > 0
     rep.err(f"{tag}_rnorm_rel", np.max(np.abs(rn[ok] * nrm[ok] - 1.0)) if ok.any() else 0.0)
+    assert np.all(rn[~ok] == 0.0), f"{tag}: a zero row must have inverse norm 0"
 
 
-def _check_decode_slice(rep, ctx, orc, wl, l, b, h, q, k, v, out, t, tabs, tie_rtol):
+def _check_decode_slice(rep, ctx, orc, wl, l, b, h, q, k, v, out, step, tabs, tie_rtol):
     G = wl.group
     key = (l, b, h)
+    t = orc.Pb[b] + step
     before = copy.deepcopy(orc.slices[key])
     got = ctx.slice_state(l, b, h, tabs)
     gset = set(got["pos"].tolist())
     qs, ks, vs = q[b, h * G:(h + 1) * G], k[b, h], v[b, h]
 
-    def attempt(force_victim=None, force_nn=None, tau_override=None):
+    def attempt(victim=None, nn=None, tau_override=None):
         st = copy.deepcopy(before)
-        o, log = O.decode_step_slice(st, qs, ks, vs, t, orc.beta,
-                                     orc.tau_override if tau_override is None else tau_override,
-                                     force_victim, force_nn)
+        tov = orc.tau_override if tau_override is None else tau_override
+        if victim is None and nn is None:
+            o, log = O.decode_step_slice(st, qs, ks, vs, t, orc.beta, tov)
+        else:
+            o, log = replay_decode(st, qs, ks, vs, t, orc.beta, tov, victim, nn)
         return st, o, log
 
     st, o, log = attempt()
-    fv = fn = None
+    fv = None
     if log.evicted and set(st.pos.tolist()) != gset:
         gone = sorted((set(before.pos.tolist()) | {t}) - gset)
         assert len(gone) == 1, f"GPU cache lost {gone} at t={t}"
@@ -293,28 +395,32 @@ def _check_decode_slice(rep, ctx, orc, wl, l, b, h, q, k, v, out, t, tabs, tie_r
             f"victim differs beyond a tie at t={t} slice {key}: GPU {gone[0]} oracle {log.victim_pos} gap {log.victim_gap:.3e}"
         rep.ties["victim"] += 1
         fv = gone[0]
-        st, o, log = attempt(force_victim=fv)
+        st, o, log = attempt(victim=fv)
     # merged / discarded and neighbour choice show in the cache content
     e = _state_err(got, st, wl.dtype)
     if log.evicted and e > 1.0:
         tried = False
-        if abs(log.mx - log.tau) <= 4e-6:                     # threshold tie: replay the other decision
+        if _thr_tie(log.mx, log.tau, tie_rtol):               # threshold tie: replay the other decision
             alt = float("inf") if log.merged else float("-inf")
-            st2, o2, log2 = attempt(force_victim=fv, tau_override=alt)
+            st2, o2, log2 = attempt(victim=fv, tau_override=alt)
             st2.tau = st.tau
             if _state_err(got, st2, wl.dtype) <= 1.0:
                 st, o, log, tried = st2, o2, log2, True
                 rep.ties["dec_merge"] += 1
         if not tried and log.nn_gap <= tie_rtol:              # neighbour tie
-            st2, o2, log2 = attempt(force_victim=fv, force_nn=log.nn_runner_pos)
+            st2, o2, log2 = attempt(victim=fv, nn=log.nn_runner_pos)
             if _state_err(got, st2, wl.dtype) <= 1.0:
                 st, o, log, tried = st2, o2, log2, True
                 rep.ties["dec_nn"] += 1
         assert tried, f"cache content differs at t={t} slice {key}: err {e:.3f} (mx {log.mx}, tau {log.tau}, nn_gap {log.nn_gap})"
     orc.slices[key] = st
     rep.err("out", close(out[b, h * G:(h + 1) * G], o, wl.dtype))
-    _compare_state(rep, got, st, wl.dtype, "decode")
-    orc.slices[key] = st
+    Kx = Vx = rows = None
+    if log.merged:
+        rows = st.pos == log.nn_pos
+        Kx = np.where(rows[:, None], log.K_exact[None, :], st.K)
+        Vx = np.where(rows[:, None], log.V_exact[None, :], st.V)
+    _compare_state(rep, got, st, wl.dtype, "decode", Kx, Vx, rows)
     rep.err("tau_abs", abs(got["tau"] - st.tau))
     if log.evicted:
         rep.merges += int(log.merged)
@@ -330,7 +436,8 @@ def _state_err(got, st, dtype) -> float:
                close(got["V"].double().numpy()[order], st.V, dtype))
 
 
-def assert_report(rep: Report, dtype: str, max_tie_frac: float = 0.01):
+def assert_report(rep: Report, dtype: str, max_ties: int = 0):
+    """`max_ties`: tolerated near-ties (counted and reported).  The committed configurations produce none."""
     e = rep.max_err
     assert e.get("colsum_rel", 0) < 2e-4, e
     assert e.get("density_rel", 0) < 2e-4, e
@@ -343,5 +450,4 @@ def assert_report(rep: Report, dtype: str, max_tie_frac: float = 0.01):
     assert e.get("tau_abs", 0) < 1e-5, e
     assert e.get("prefill_rnorm_rel", 0) < 1e-5 and e.get("decode_rnorm_rel", 0) < 1e-5, e
     assert rep.ties["budget"] == 0, rep.ties
-    decisions = max(1, rep.checked_slices * max(1, rep.steps))
-    assert sum(rep.ties.values()) <= max(2, max_tie_frac * decisions), rep.ties
+    assert sum(rep.ties.values()) <= max_ties, rep.ties

@@ -255,11 +255,11 @@ def test_tau0_and_merge_weights():
     tau0 = O.initial_threshold(mx)
     assert mx.min() <= tau0 <= mx.max() and abs(tau0 - np.mean(mx)) < 1e-15
     # tau = +inf: pure eviction, conserved rows unchanged bit for bit
-    Kp, Vp, den = O.weighted_merge(Kc, Vc, Ke, Ve, mx, nn, float("inf"))
+    Kp, Vp, den = O.weighted_merge(Kc, Vc, Ke, Ve, mx, nn, O.merge_mask(mx, float("inf")))
     np.testing.assert_array_equal(den, np.full(Lc, math.e))
     np.testing.assert_allclose(Kp, Kc, rtol=1e-15)
     # tau = -inf: every evicted token is counted exactly once
-    Km, Vm, den = O.weighted_merge(Kc, Vc, Ke, Ve, mx, nn, float("-inf"))
+    Km, Vm, den = O.weighted_merge(Kc, Vc, Ke, Ve, mx, nn, O.merge_mask(mx, float("-inf")))
     assert abs((den - math.e).sum() - np.exp(mx).sum()) < 1e-10
     # convexity: explicit weights reproduce the merged rows and sum to one
     for j in range(Lc):
@@ -274,7 +274,7 @@ def test_tau0_and_merge_weights():
         hi = np.maximum(Kc[j], Ke[idx].max(0)) if idx.size else Kc[j]
         assert np.all(Km[j] >= lo - 1e-12) and np.all(Km[j] <= hi + 1e-12)
     # threshold at tau0 merges exactly the rows with mx >= tau0
-    K0, V0, den0 = O.weighted_merge(Kc, Vc, Ke, Ve, mx, nn, tau0)
+    K0, V0, den0 = O.weighted_merge(Kc, Vc, Ke, Ve, mx, nn, O.merge_mask(mx, tau0))
     assert abs((den0 - math.e).sum() - np.exp(mx[mx >= tau0]).sum()) < 1e-10
 
 
@@ -283,11 +283,11 @@ def test_merge_single_victim_closed_forms():
     kc, vc = np.array([[1.0, 0, 0, 0]]), np.array([[2.0, 2, 2, 2]])
     # identical direction: u = 1 -> plain average
     K1, V1, _ = O.weighted_merge(kc, vc, np.array([[3.0, 0, 0, 0]]), np.array([[4.0, 4, 4, 4]]),
-                                 np.array([1.0]), np.array([0]), 0.0)
+                                 np.array([1.0]), np.array([0]), np.array([True]))
     np.testing.assert_allclose(K1[0], [2.0, 0, 0, 0], atol=1e-15)
     np.testing.assert_allclose(V1[0], [3.0] * 4, atol=1e-15)
     # orthogonal: u = 0 -> evicted weight 1/(1+e)
-    K2, _, _ = O.weighted_merge(kc, vc, np.array([[0.0, 5, 0, 0]]), vc, np.array([0.0]), np.array([0]), -1.0)
+    K2, _, _ = O.weighted_merge(kc, vc, np.array([[0.0, 5, 0, 0]]), vc, np.array([0.0]), np.array([0]), np.array([True]))
     w = 1.0 / (1.0 + math.e)
     np.testing.assert_allclose(K2[0], [1 - w, 5 * w, 0, 0], atol=1e-15)
 
@@ -429,3 +429,288 @@ def test_decode_merge_single_token_weights():
     np.testing.assert_allclose(st.V[row], O.round_storage((1 - w_e) * V[2] + w_e * V[1], "f32"), atol=0)
     assert st.tau == pytest.approx(0.5 * 0.6 + 0.5 * -1.0)
     assert st.pos.tolist() == [0, 2, 3]
+
+
+# ---------------------------------------------------------------- budgets with an upper clamp (Eq. 5 + bounds)
+def _bisect_budgets(w, tot, lo, cap):
+    """Independent statement of the clamped proportional rule: bisection on the monotone total."""
+    a, b = 0.0, 1.0
+    while np.clip(b * w, lo, cap).sum() < tot and b < 1e307:
+        b *= 2.0
+    for _ in range(300):
+        mid = 0.5 * (a + b)
+        if np.clip(mid * w, lo, cap).sum() < tot:
+            a = mid
+        else:
+            b = mid
+    return np.clip(b * w, lo, cap)
+
+
+def test_budgets_with_max_budget_closed_form():
+    # Eq. 5 with weights 8 : 1 : 1 (F = 0, ln 8, ln 8): unclamped shares of S_tot = 0.5 * 3 * 1000 = 1500 would be
+    # 1200, 150, 150.  A cap of 600 saturates layer 0; the other two share the remaining 900 by weight: 450 each.
+    F = np.array([[0.0], [math.log(8.0)], [math.log(8.0)]])
+    assert O.layer_budgets(F, 1000, 0.5).tolist() == [1000, 250, 250]          # cap = P binds already
+    assert O.layer_budgets(F, 1000, 0.5, max_budget=600).tolist() == [600, 450, 450]
+    assert O.layer_budgets(F, 1000, 0.5, max_budget=1200).tolist() == [1200, 150, 150]
+    # weights 4 : 2 : 1, S_tot = 700, cap 300: layer 0 saturates, the rest share 400 as 2 : 1 -> 266.67, 133.33
+    F = np.array([[0.0], [math.log(2.0)], [math.log(4.0)]])
+    S = O.layer_budgets(F, 1000, 0.7 / 3.0, max_budget=300)
+    assert S.tolist() == [300, 267, 133]
+    # both clamps at once: lower clamp 100 lifts layer 2; the middle layer takes what is left
+    S = O.layer_budgets(np.array([[0.0], [math.log(2.0)], [math.log(400.0)]]), 1000, 0.6 / 3.0, min_budget=100,
+                        max_budget=300)
+    assert S.tolist() == [300, 200, 100]
+
+
+def test_budgets_with_max_budget_sum_bounds_and_bisection():
+    r = rng(61)
+    done = 0
+    for trial in range(300):
+        L = int(r.integers(1, 40))
+        H = int(r.integers(1, 5))
+        P = int(r.integers(16, 5000))
+        rho = float(r.uniform(0.05, 0.9))
+        smin = int(r.integers(1, 8))
+        tot = math.floor(rho * L * P + 0.5)
+        mean = tot / L
+        cap = int(min(P, max(smin, math.ceil(mean * float(r.uniform(1.0, 4.0))))))
+        F = r.gamma(1.0, size=(L, H)) * float(r.choice([0.01, 1.0, 50.0, 1e4]))
+        gamma = float(r.choice([1.0, 10.0, 100.0]))
+        hr = int(trial % 4)
+        if not (L * smin <= tot <= L * cap):
+            continue
+        S = O.layer_budgets(F, P, rho, smin, gamma, hr, cap)
+        assert S.sum() == tot                                         # sum_l alpha_l = L * rho still holds
+        assert S.min() >= smin and S.max() <= cap
+        w = np.maximum(O.layer_weights(F, gamma, hr), 1e-300)
+        x = _bisect_budgets(w, tot, smin, cap)
+        assert np.all(np.abs(S - x) < 1.0 + 1e-6), (S, x)
+        for a in range(L):                                            # a larger weight never gets a smaller cache
+            for b in range(L):
+                if w[a] > w[b]:
+                    assert S[a] >= S[b] - 1
+        done += 1
+    assert done > 150
+
+
+def test_allocate_budgets_remainders_go_to_the_lower_unit():
+    # three equal units share 10: 3.33 each -> floor 3, one left over -> unit 0
+    assert O.allocate_budgets(np.ones(3), 10, 1, 10).tolist() == [4, 3, 3]
+    assert O.allocate_budgets(np.ones(3), 11, 1, 10).tolist() == [4, 4, 3]
+    # a saturated unit never takes a remainder
+    assert O.allocate_budgets(np.array([100.0, 1.0, 1.0]), 11, 1, 4).tolist() == [4, 4, 3]
+
+
+# ---------------------------------------------------------------- per-head and exponential-decay allocation
+def test_head_budgets_follow_the_appendix_formula():
+    r = rng(62)
+    L, H, P, rho = 6, 4, 3000, 0.25
+    F = r.uniform(0.0, 1.0, size=(L, H))
+    a = scipy.special.softmax(-F.reshape(-1)).reshape(L, H)        # alpha_l^h, sums to one over all (l, h)
+    S = O.head_budgets(F, P, rho)
+    tot = math.floor(rho * L * H * P + 0.5)
+    assert S.shape == (L, H) and S.sum() == tot
+    assert np.all(np.abs(S - a * tot) < 1.0)                        # S_l^h = alpha_l^h * S_total
+    # S_l = sum_h S_l^h is the per-layer rule's size times the number of heads (alpha_l = sum_h alpha_l^h)
+    Sl = O.layer_budgets(F, P, rho)
+    assert np.all(np.abs(S.sum(axis=1) - H * Sl) <= H + 1)
+    # grouped queries: a KV head's weight is the sum of its query heads' weights
+    Sg = O.head_budgets(F, P, rho, group=2)
+    ag = a.reshape(L, 2, 2).sum(axis=2)
+    totg = math.floor(rho * L * 2 * P + 0.5)
+    assert Sg.shape == (L, 2) and Sg.sum() == totg
+    assert np.all(np.abs(Sg - ag * totg) < 1.0)
+    # equal densities -> every head gets rho * P; one head, one layer -> rho * P
+    assert (O.head_budgets(np.full((3, 4), 2.5), 1000, 0.2) == 200).all()
+    assert O.head_budgets(np.array([[7.0]]), 1000, 0.3)[0, 0] == 300
+    # bounds
+    Sc = O.head_budgets(F * 50.0, P, rho, min_budget=16, max_budget=1500)
+    assert Sc.min() >= 16 and Sc.max() <= 1500 and Sc.sum() == tot
+
+
+def test_exp_decay_budgets_closed_form():
+    # alpha_l = exp(-F_l): F = 0, ln 2, ln 4 -> 1, 1/2, 1/4 of the prompt; not normalised
+    F = np.array([[0.0], [math.log(2.0)], [math.log(4.0)]])
+    assert O.exp_decay_budgets(F, 1000).tolist() == [1000, 500, 250]
+    assert O.exp_decay_budgets(F, 1000, gamma=2.0).tolist() == [1000, 707, 500]
+    assert O.exp_decay_budgets(F, 1000, min_budget=300, max_budget=800).tolist() == [800, 500, 300]
+    # several heads: the mean of the per-head factors
+    F2 = np.array([[0.0, math.log(4.0)]])
+    assert O.exp_decay_budgets(F2, 1000).tolist() == [625]
+    # monotone in the density
+    r = rng(63)
+    Fr = np.sort(r.uniform(0, 3, size=(9, 1)), axis=0)
+    assert np.all(np.diff(O.exp_decay_budgets(Fr, 4096)) <= 0)
+
+
+# ---------------------------------------------------------------- grouped-query score (reading for GQA)
+def test_group_score_is_the_sum_over_the_query_heads():
+    # Hq = 4, G = 2: KV head 0 owns query heads 0, 1; KV head 1 owns 2, 3
+    cs = np.array([[1.0, 2.0, 3.0], [10.0, 20.0, 30.0], [0.5, 0.25, 0.125], [4.0, 4.0, 4.0]])
+    assert O.group_score(cs, 0, 2).tolist() == [11.0, 22.0, 33.0]
+    assert O.group_score(cs, 1, 2).tolist() == [4.5, 4.25, 4.125]
+    assert O.group_score(cs, 2, 1).tolist() == [0.5, 0.25, 0.125]
+    # the same sum that the decode step accumulates: two query heads with known probabilities
+    d = 2
+    st = O.SliceState(pos=np.array([0]), K=np.zeros((1, d)), V=np.zeros((1, d)), score=np.array([0.0]), tau=0.0,
+                      S=8, T=0, M=1, dtype="f32")
+    O.decode_attend(st, np.zeros((2, d)), np.zeros(d), np.zeros(d), 1)   # zero logits: each head gives 1/2, 1/2
+    assert st.score.tolist() == [1.0, 1.0]
+    # and the stack uses it
+    stack = O.OracleStack(n_layers=1, batch=1, n_q_heads=4, n_kv_heads=2, d_head=2, dtype="f32", prompt_len=3,
+                          rho=1.0, n_sink=0, window=1, nm_ratio=3.0, beta=0.7)
+    stack.colsum[0, 0] = cs
+    assert stack.group_score(0, 0, 1).tolist() == [4.5, 4.25, 4.125]
+
+
+# ---------------------------------------------------------------- exact ties at decode (readings)
+def test_decode_victim_tie_goes_to_the_later_position():
+    d = 4
+    K = np.eye(4)[:3] * 1.0
+    # slots at positions 0 (sink), 1, 2 with bit-equal scores on 1 and 2; zero queries add the same 1/4 to each
+    st = O.SliceState(pos=np.array([0, 1, 2]), K=K.copy(), V=np.zeros((3, d)), score=np.array([9.0, 0.5, 0.5]),
+                      tau=5.0, S=3, T=1, M=1, dtype="f32")
+    out, log = O.decode_step_slice(st, np.zeros((1, d)), np.array([0.0, 0, 0, 1.0]), np.zeros(d), 3, 0.7)
+    assert log.evicted and log.victim_pos == 2 and log.runner_up_pos == 1 and log.victim_gap == 0.0
+    assert st.pos.tolist() == [0, 1, 3]
+    assert O.victim_order(O.SliceState(pos=np.array([0, 1, 2, 3]), K=np.zeros((4, d)), V=np.zeros((4, d)),
+                                       score=np.array([0.0, 0.5, 0.5, 0.1]), tau=0.0, S=3, T=1, M=1, dtype="f32"),
+                          3) == [2, 1]                                 # pos 0 is a sink, pos 3 is in the window
+
+
+def test_decode_neighbour_tie_goes_to_the_earlier_position():
+    d = 4
+    # victim = position 1 (lowest score); positions 0 and 2 hold the same direction (bit-equal cosine 0.6)
+    K = np.array([[0.6, 0.8, 0, 0], [1.0, 0, 0, 0], [0.6, 0.8, 0, 0]])
+    V = np.arange(12.0).reshape(3, d)
+    st = O.SliceState(pos=np.array([0, 1, 2]), K=K.copy(), V=V.copy(), score=np.array([9.0, 0.0, 1.0]),
+                      tau=-1.0, S=3, T=1, M=1, dtype="f32")
+    out, log = O.decode_step_slice(st, np.zeros((1, d)), np.array([0.0, 0, 0, 1.0]), np.zeros(d), 3, 0.5)
+    assert log.victim_pos == 1 and log.nn_pos == 0 and log.nn_runner_pos == 2 and log.nn_gap == 0.0
+    assert log.merged
+    w_e = math.exp(0.6) / (math.exp(0.6) + math.e)
+    np.testing.assert_allclose(st.K[0], O.round_storage((1 - w_e) * K[0] + w_e * K[1], "f32"), atol=0)
+    np.testing.assert_array_equal(st.K[1], K[2])                     # the later twin is untouched
+
+
+# ---------------------------------------------------------------- ablation switches (Section 5.4 tables)
+def test_average_merge_policy():
+    r = rng(64)
+    Lc, Le, d = 5, 30, 8
+    Kc, Vc = r.standard_normal((Lc, d)), r.standard_normal((Lc, d))
+    Ke, Ve = r.standard_normal((Le, d)), r.standard_normal((Le, d))
+    mx, nn = O.nearest_neighbour(O.cosine_matrix(Ke, Kc))
+    mask = O.merge_mask(mx, O.initial_threshold(mx))
+    Ka, Va, den = O.weighted_merge(Kc, Vc, Ke, Ve, mx, nn, mask, "average")
+    for j in range(Lc):
+        idx = np.nonzero((nn == j) & mask)[0]
+        assert den[j] == 1 + idx.size
+        np.testing.assert_allclose(Ka[j], (Kc[j] + Ke[idx].sum(0)) / (1 + idx.size), atol=1e-13)   # plain mean
+        np.testing.assert_allclose(Va[j], (Vc[j] + Ve[idx].sum(0)) / (1 + idx.size), atol=1e-13)
+    # one victim at decode: the plain average of the two rows, whatever the similarity
+    K = np.array([[1.0, 0, 0, 0], [0.0, 1, 0, 0], [0.0, 0.6, 0.8, 0]])
+    V = r.standard_normal((3, 4))
+    st = O.SliceState(pos=np.array([0, 1, 2]), K=K.copy(), V=V.copy(), score=np.array([9.0, 0.0, 1.0]),
+                      tau=-1.0, S=3, T=1, M=1, dtype="f32", policy="average")
+    out, log = O.decode_step_slice(st, np.zeros((1, 4)), np.array([0.0, 0, 0, 1.0]), np.ones(4), 3, 0.5)
+    assert log.merged and log.nn_pos == 2
+    row = list(st.pos).index(2)
+    np.testing.assert_allclose(st.K[row], O.round_storage(0.5 * (K[2] + K[1]), "f32"), atol=0)
+    np.testing.assert_allclose(st.V[row], O.round_storage(0.5 * (V[2] + V[1]), "f32"), atol=0)
+
+
+def test_value_feature_uses_cosine_of_the_values():
+    r = rng(65)
+    P, d, S, T, M = 48, 8, 12, 1, 3
+    Q, K, V, score = make_slice(r, P, d, 1)
+    sk = O.prefill_compress_slice(K, V, score, S, T, M, "f32", feature="k")
+    sv = O.prefill_compress_slice(K, V, score, S, T, M, "f32", feature="v")
+    np.testing.assert_array_equal(sk.pos, sv.pos)                  # eviction does not depend on the feature
+    ret, ev = sk.log["retained"], sk.log["evicted"]
+    Uv = 1.0 - scipy.spatial.distance.cdist(V[ev], V[ret], "cosine")
+    np.testing.assert_allclose(sv.log["U"], Uv, atol=1e-12)
+    np.testing.assert_array_equal(sv.log["nn"], np.argmax(Uv, axis=1))
+    assert abs(sv.tau - Uv.max(axis=1).mean()) < 1e-12
+    # swapping the roles of K and V swaps the two results
+    sw = O.prefill_compress_slice(V, K, score, S, T, M, "f32", feature="k")
+    np.testing.assert_array_equal(sw.K, sv.V)
+    np.testing.assert_array_equal(sw.V, sv.K)
+    # decode: the neighbour is the best cosine among the values
+    st = O.SliceState(pos=np.array([0, 1, 2]), K=np.eye(4)[:3].copy(),
+                      V=np.array([[0.0, 1, 0, 0], [1.0, 0, 0, 0], [0.8, 0.6, 0, 0]]),
+                      score=np.array([9.0, 0.0, 1.0]), tau=-1.0, S=3, T=1, M=1, dtype="f32", feature="v")
+    out, log = O.decode_step_slice(st, np.zeros((1, 4)), np.array([0.0, 0, 0, 1.0]), np.array([0.0, 0, 1, 0]), 3, 0.5)
+    assert log.victim_pos == 1 and log.nn_pos == 2 and log.mx == pytest.approx(0.8)
+
+
+def test_no_ema_threshold_merges_every_victim():
+    # beta = 1 ("w.o. EMA-Threshold"): tau_t equals the current maximum, so every evicted token is merged
+    r = rng(66)
+    P, d, G, S, T, M = 40, 8, 1, 12, 1, 3
+    Q, K, V, score = make_slice(r, P, d, G)
+    st = O.prefill_compress_slice(K, V, score, S, T, M, "f32")
+    for i in range(12):
+        out, log = O.decode_step_slice(st, r.standard_normal((G, d)), r.standard_normal(d), r.standard_normal(d),
+                                       P + i, 1.0)
+        assert log.evicted and log.merged and log.tau == log.mx
+    # beta = 0: the threshold never moves from tau_0
+    st = O.prefill_compress_slice(K, V, score, S, T, M, "f32")
+    tau0 = st.tau
+    for i in range(6):
+        O.decode_step_slice(st, r.standard_normal((G, d)), r.standard_normal(d), r.standard_normal(d), P + i, 0.0)
+        assert st.tau == tau0
+
+
+def test_window_only_cache_and_zero_keys():
+    # N = 0: the cache is the sinks and the window; the victim at decode is the oldest window position
+    r = rng(67)
+    P, d = 30, 4
+    Q, K, V, score = make_slice(r, P, d, 1)
+    st = O.prefill_compress_slice(K, V, score, 9, 1, 8, "f32")
+    assert st.pos.tolist() == [0] + list(range(22, 30))
+    out, log = O.decode_step_slice(st, r.standard_normal((1, d)), r.standard_normal(d), r.standard_normal(d), P, 0.7)
+    assert log.victim_pos == 22                                      # only position t - M is outside sinks and window
+    # a zero key has similarity 0 to everything and, evicted, merges with weight 1 / (1 + e) if it passes
+    K0 = K.copy()
+    K0[5] = 0.0
+    s0 = O.prefill_compress_slice(K0, V, score, 9, 1, 8, "f32")
+    i5 = list(s0.log["evicted"]).index(5)
+    assert s0.log["mx"][i5] == 0.0 and s0.log["nn"][i5] == 0
+
+
+# ---------------------------------------------------------------- ragged batch (per-sequence prompt lengths)
+def test_ragged_batch_equals_separate_sequences():
+    r = rng(68)
+    L, Hq, Hkv, d, Pmax = 2, 4, 2, 8, 40
+    lens = [40, 23]
+    Qs = [r.standard_normal((2, Hq, Pmax, d)) for _ in range(L)]
+    Ks = [r.standard_normal((2, Hkv, Pmax, d)) for _ in range(L)]
+    Vs = [r.standard_normal((2, Hkv, Pmax, d)) for _ in range(L)]
+    kw = dict(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, d_head=d, dtype="f32", rho=0.4, n_sink=1, window=0,
+              nm_ratio=3.0, beta=0.7, density_temp=4.0, min_budget=4)
+    rag = O.OracleStack(batch=2, prompt_len=Pmax, prompt_lens=lens, **kw)
+    for l in range(L):
+        rag.layer_stats(l, Qs[l], Ks[l])
+    rag.layer_budgets()
+    for l in range(L):
+        rag.prefill_compress(l, Ks[l], Vs[l])
+    dec = [(r.standard_normal((2, Hq, d)), r.standard_normal((2, Hkv, d)), r.standard_normal((2, Hkv, d)))
+           for _ in range(3)]
+    outs = [[rag.decode_step(l, *dec[s], s) for l in range(L)] for s in range(3)]
+    for b, Pb in enumerate(lens):
+        one = O.OracleStack(batch=1, prompt_len=Pb, **kw)
+        for l in range(L):
+            one.layer_stats(l, Qs[l][b:b + 1, :, :Pb], Ks[l][b:b + 1, :, :Pb])
+        one.layer_budgets()
+        np.testing.assert_array_equal(one.budgets[0], rag.budgets[b])
+        assert rag.budgets[b].sum() == Hkv * math.floor(0.4 * L * Pb + 0.5)
+        for l in range(L):
+            one.prefill_compress(l, Ks[l][b:b + 1, :, :Pb], Vs[l][b:b + 1, :, :Pb])
+        for s in range(3):
+            for l in range(L):
+                res = one.decode_step(l, dec[s][0][b:b + 1], dec[s][1][b:b + 1], dec[s][2][b:b + 1], s)
+                for h in range(Hkv):
+                    np.testing.assert_array_equal(res[(0, h)][0], outs[s][l][(b, h)][0])
+                    assert res[(0, h)][1].victim_pos == outs[s][l][(b, h)][1].victim_pos
+                    assert outs[s][l][(b, h)][1].victim_pos < Pb + s + 1
