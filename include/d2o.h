@@ -192,10 +192,19 @@ d2o_status d2o_full_decode_step(int32_t dtype, int32_t d_head, int32_t n_slices,
  *   colsum DEVICE float [B, Hq, P] (out: column sums of the causal prompt attention, Eq. 4);
  *   density DEVICE double [B, Hq] (out: F_v = Var(colsum) per query head).
  *
- * Limit: batch * n_q_heads * prompt_len <= D2O_STATIC_LSE_FLOATS, else D2O_ERR_TOO_LARGE and
- * nothing is launched.  The call neither allocates nor frees device memory.
+ * It always runs the generic kernels (fp32 arithmetic on CUDA cores, any dtype, any prompt
+ * length).  d2o_layer_stats runs the same kernels, and then returns bit-identical results, for
+ * fp32 inputs, for a prompt length that is not a multiple of 4, or with stats_path = 1; for
+ * 16-bit inputs it otherwise takes its tensor-core kernels, which are several times faster and
+ * agree with this entry point to rounding (column sums within 2e-4 relative).
+ *
+ * Limit: batch * n_q_heads * prompt_len <= D2O_STATIC_LSE_FLOATS and batch * n_q_heads <= 65535,
+ * else D2O_ERR_TOO_LARGE and nothing is launched.  The call neither allocates nor frees device
+ * memory.
  * The first call on each device looks up the device address of the array (one runtime query,
- * made with that device current); make that first call outside of any stream capture.
+ * made with that device current) and keeps it for the life of the process; make that first call
+ * outside of any stream capture.  After cudaDeviceReset() the kept address is stale: a process
+ * that resets a device must not call this entry point on it again.
  * All calls share the one array: it is fully rewritten by each call before it is read, so
  * nothing needs clearing, but two calls whose work overlaps on the GPU (different streams)
  * race on it.  Asynchronous on `stream` like the other calls. */

@@ -146,6 +146,7 @@ struct d2o_ctx {
   int group;
   int elem_size;
   int max_budget;
+  int n_sms;                   // multiprocessors of the device the context was created on
   int64_t total_budget;        // S_tot per sequence = round(rho * L * P)
   int64_t pool_rows;           // B * Hkv * S_tot
   d2o::Layout lay;
@@ -195,8 +196,6 @@ size_t sim_tc_part_key_bytes(const d2o_config* cfg, int max_budget);
 bool colsum_tc_supported(const d2o_config* cfg);
 cudaError_t launch_colsum_tc(const d2o_ctx* c, const void* Q, const void* K, const float* lse_in, float* colsum,
                              cudaStream_t st);
-// largest number of rows (cache + the new token) of one slice the decode kernel can handle
-int decode_max_rows(int row_bytes, int group, int d_head);
 
 // remembers the text of a failed CUDA runtime call for d2o_last_cuda_error(); returns D2O_ERR_CUDA
 d2o_status record_cuda_error(cudaError_t e, const char* where);

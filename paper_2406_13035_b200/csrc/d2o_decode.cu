@@ -90,6 +90,9 @@ __device__ __forceinline__ void stage_wait(unsigned long long* bar, uint32_t par
     if (global_ns() - t0 > kWaitNs) { *timeout = 2; return; }
   }
 }
+// Similarity as an ordered key: -0 (a zero-norm row times a negative dot product) must count as +0, or equal
+// similarities would not tie.
+__device__ __forceinline__ uint32_t sim_ord(float u) { return float_ord(__fadd_rn(u, 0.f)); }
 // next slot of the ring; the parity flips on wrap-around
 __device__ __forceinline__ void ring_next(int& slot, uint32_t& ph, int stages) {
   if (++slot == stages) { slot = 0; ph ^= 1u; }
@@ -265,9 +268,13 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   // swizzle, because the value pass reads them with transposing matrix loads, which would conflict eight ways on
   // row-major 256-byte rows.
   constexpr bool kTensor = tensor_path((int)sizeof(T), G);
+  constexpr int kTiles = SR / 16;                                      // 16-row tiles per stage (tensor path)
+  constexpr bool kHalfTiles = 2 * kTiles == CW;                        // half as many tiles as warps (256-byte rows)
+  static_assert(!kTensor || kTiles == CW || kHalfTiles, "tile assignment of the tensor path");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // a launch that follows with programmatic stream serialisation (the short slices of the same step, which share
-  // nothing with this one) may start as soon as every CTA of this one is running
+  // nothing with this one) may start as soon as every CTA of this one is running; its producer warps wait for this
+  // grid to finish before they exit (griddepcontrol.wait below)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // ---- which slice: in index order, or largest caches first through the order table
   const int h = (int)blockIdx.x % a.Hkv;
@@ -390,6 +397,10 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         }
       }
     }
+    // A grid launched with programmatic stream serialisation may run beside its predecessor, but it must not be
+    // complete before it: whatever the stream runs next (the next step, a copy of the outputs) is ordered behind
+    // this grid only.  Returns at once in an ordinarily launched grid.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     return;
   }
 
@@ -433,14 +444,15 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   for (int g = 0; g < G; ++g) mloc[g] = -INFINITY;
   const int n_plain_fma = min(n, a.row_cap);                        // FMA path: rows (the new token's included) with logits in shared memory
   if constexpr (kTensor) {
-    // a stage has SR / 16 tiles of 16 rows, half as many as there are warps: the lower half of the warps takes the
-    // even stages, the upper half the odd ones (the others only hand the stage back), so that two stages are worked
-    // on at a time; thread (gid, tig) ends up with rows gid, gid + 8 of its tile against heads 2 tig, 2 tig + 1
+    // a stage has SR / 16 tiles of 16 rows.  With 256-byte rows that is half as many as there are warps: the lower
+    // half of the warps takes the even stages, the upper half the odd ones (the others only hand the stage back), so
+    // that two stages are worked on at a time.  With 128-byte rows every warp has a tile in every stage.  Thread
+    // (gid, tig) ends up with rows gid, gid + 8 of its tile against heads 2 tig, 2 tig + 1
     float mm0 = -INFINITY, mm1 = -INFINITY;
     const int n_plain = min(n_old, a.row_cap);                       // rows whose logits go to shared memory unchecked
-    constexpr int kTiles = SR / 16;
     // this warp's tile in the even / the odd stages (-1: none), and where its logits go
-    const int tile_even = warp < kTiles ? warp : -1, tile_odd = warp >= kTiles && warp < 2 * kTiles ? warp - kTiles : -1;
+    const int tile_even = warp < kTiles ? warp : -1;
+    const int tile_odd = kHalfTiles ? (warp >= kTiles ? warp - kTiles : -1) : warp;
     float* const pl_mine = pl + (size_t)(2 * tig) * a.row_cap + gid;
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
       stage_wait(&s_full[slot], ph, &s_timeout);
@@ -675,8 +687,8 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         stage_wait(&s_full[slot], ph, &s_timeout);
         const unsigned char* st = reinterpret_cast<const unsigned char*>(ring) + (size_t)slot * kStageBytes;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        const int tile = warp - (s & 1) * (SR / 16);
-        const bool active = tile >= 0 && tile < SR / 16 && s * SR + tile * 16 < n_old;
+        const int tile = kHalfTiles ? warp - (s & 1) * kTiles : warp;
+        const bool active = tile >= 0 && tile < kTiles && s * SR + tile * 16 < n_old;
         if (active) tile_dots<T, D, SR>(st, tile, vb, acc);
         // 1/|k| and position of this thread's two rows leave the stage before the stage is released
         const int lr0 = tile * 16 + gid, li0 = s * SR + lr0, li1 = li0 + 8;
@@ -687,11 +699,11 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_empty[slot]);
         if (m0) {                                                    // max similarity, ties -> earliest position
-          const unsigned long long key = ((unsigned long long)float_ord(acc[0] * vic_rn * rn0) << 32) | (uint32_t)(0x7fffffff - ps0);
+          const unsigned long long key = ((unsigned long long)sim_ord(acc[0] * vic_rn * rn0) << 32) | (uint32_t)(0x7fffffff - ps0);
           if (key > best) { best = key; best_li = li0; }
         }
         if (m1) {
-          const unsigned long long key = ((unsigned long long)float_ord(acc[2] * vic_rn * rn1) << 32) | (uint32_t)(0x7fffffff - ps1);
+          const unsigned long long key = ((unsigned long long)sim_ord(acc[2] * vic_rn * rn1) << 32) | (uint32_t)(0x7fffffff - ps1);
           if (key > best) { best = key; best_li = li1; }
         }
       }
@@ -705,7 +717,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
           for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], kf[e], x);
         }
         x = warp_sum(x);
-        const unsigned long long key = ((unsigned long long)float_ord(x * vic_rn * s_new_rn) << 32) | (uint32_t)(0x7fffffff - a.t);
+        const unsigned long long key = ((unsigned long long)sim_ord(x * vic_rn * s_new_rn) << 32) | (uint32_t)(0x7fffffff - a.t);
         if (lane == 0 && key > best) { best = key; best_li = n_old; }
       }
     } else {
@@ -742,7 +754,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         const float r = reduce4<LPR>(dot[0], dot[1], dot[2], dot[3], lig);
         if (mine) {                                                    // max similarity, ties -> earliest position
           const float u = r * vic_rn * rn_li;
-          const unsigned long long key = ((unsigned long long)float_ord(u) << 32) | (uint32_t)(0x7fffffff - ps_li);
+          const unsigned long long key = ((unsigned long long)sim_ord(u) << 32) | (uint32_t)(0x7fffffff - ps_li);
           if (key > best) { best = key; best_li = li; }
         }
       }
@@ -1091,11 +1103,6 @@ static int smem_rows_for(int max_rows, double mean_rows, int G) {
   return min(max_rows, max(free_rows, (int)(2.0 * mean_rows)));
 }
 
-int decode_max_rows(int row_bytes, int group, int d_head) {
-  (void)row_bytes; (void)group; (void)d_head;
-  return 1 << 24;                                                    // rows beyond the shared-memory array go through L2
-}
-
 cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const void* k, const void* v, void* out,
                           cudaStream_t st, d2o_status* why) {
   const d2o_config& g = c->cfg;
@@ -1142,12 +1149,12 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   int n_long = 0;
   if (ordered && c->decode_warps == 0 && c->decode_long_pairs == 0 && n_pairs > 1) {
     const double fixed_us = 8.0, row_us = tensor_path(c->elem_size, G) ? 0.025 : 0.05;
-    const double slots = 148.0 * ctas_per_sm(8, G, c->elem_size);
+    const double slots = (double)c->n_sms * ctas_per_sm(8, G, c->elem_size);
     double work = 0.0;
     for (int i = 0; i < n_pairs; ++i) work += Hkv * (fixed_us + row_us * rows_of_pair(i));
     // measured optimum: four pairs on the 7B-shaped config (FMA path), twelve on the long-context one (tensor path)
     const double limit = (tensor_path(c->elem_size, G) ? 0.55 : 0.65) * work / slots;
-    while (n_long < n_pairs && (n_long + 1) * Hkv <= 2 * 148 && fixed_us + row_us * rows_of_pair(n_long) > limit) ++n_long;
+    while (n_long < n_pairs && (n_long + 1) * Hkv <= 2 * c->n_sms && fixed_us + row_us * rows_of_pair(n_long) > limit) ++n_long;
     if (n_long == n_pairs) n_long = 0;
   } else if (ordered && c->decode_long_pairs > 0) {
     n_long = min(c->decode_long_pairs, n_pairs - 1);
@@ -1210,7 +1217,7 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     const int rest = (n_pairs - n_long) * Hkv;
     int rest_max = rows_of_pair(n_long);
     const int cw = (c->decode_warps == 4 || c->decode_warps == 8) ? c->decode_warps
-                   : ((G <= 2 && rest >= 8 * 148 * 4 && rest_max <= 1536) ? 4 : 8);
+                   : ((G <= 2 && rest >= 8 * c->n_sms * 4 && rest_max <= 1536) ? 4 : 8);
     return launch_class(n_long, n_pairs, cw, true);
   }
   // Consumer warps per CTA.  One head per KV head and enough small slices for seven and more CTAs on every SM:
@@ -1221,8 +1228,8 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   int cw = c->decode_warps;
   if (cw == 0) {
     cw = 8;
-    if (G <= 2 && n_slices >= 8 * 148 * 4 && max_rows <= 1536) cw = 4;
-    if (G >= 4 && n_slices <= 148 * 8 && max_rows > 2.0 * mean_rows) cw = 16;
+    if (G <= 2 && n_slices >= 8 * c->n_sms * 4 && max_rows <= 1536) cw = 4;
+    if (G >= 4 && n_slices <= c->n_sms * 8 && max_rows > 2.0 * mean_rows) cw = 16;
   }
   return launch_class(0, n_pairs, cw, false);
 }

@@ -272,9 +272,12 @@ cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int ca
   // smallest cluster that gives the machine two waves of CTAs and keeps the logits of a CTA under 64 KB
   int C = 1;
   const int rows = len + 1;
+  int sms = 0, dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return cudaGetLastError();
   while (C < kFullMaxCluster) {
     const int chunk = (((rows + C - 1) / C) + 7) & ~7;
-    if ((long)chunk * group * 4 <= 64 * 1024 && (long)n_slices * C >= 2 * 148) break;
+    if ((long)chunk * group * 4 <= 64 * 1024 && (long)n_slices * C >= 2L * sms) break;
     C *= 2;
   }
   a.chunk_cap = (((rows + C - 1) / C) + 7) & ~7;

@@ -43,6 +43,7 @@ extern "C" const char* d2o_status_string(d2o_status s) {
 extern "C" const char* d2o_last_cuda_error(void) { return g_cuda_err; }
 
 static int elem_size_of(int dtype) { return dtype == D2O_F32 ? 4 : 2; }
+constexpr int kMaxSliceRows = 56 * 1024;      // rows of one slice (S_l + 1): 4 bytes each of the 227 KB of shared memory
 
 static d2o_status validate(const d2o_config* c, int64_t* total_budget, int* max_budget) {
   if (!c) return D2O_ERR_INVALID_ARG;
@@ -64,8 +65,8 @@ static d2o_status validate(const d2o_config* c, int64_t* total_budget, int* max_
   if (c->min_budget < 1 || c->min_budget < c->n_sink + 1 || c->min_budget > maxb) return D2O_ERR_INVALID_ARG;
   double tot = floor((double)c->rho * (double)c->n_layers * (double)c->prompt_len + 0.5);
   if (tot < (double)c->n_layers * c->min_budget || tot > (double)c->n_layers * maxb) return D2O_ERR_INVALID_ARG;
-  // decode kernel: per-row arrays of one slice
-  if (maxb + 1 > decode_max_rows(c->d_head * elem_size_of(c->dtype), g, c->d_head)) return D2O_ERR_UNSUPPORTED;
+  // the prompt-stage segment kernel keeps one counter per retained row of a slice in shared memory
+  if (maxb + 1 > kMaxSliceRows) return D2O_ERR_UNSUPPORTED;
   *total_budget = (int64_t)tot;
   *max_budget = maxb;
   return D2O_OK;
@@ -142,6 +143,16 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
   c->pool_rows = (int64_t)cfg->batch * cfg->n_kv_heads * (tot + 7 * (int64_t)cfg->n_layers);
   c->lay = l; c->slay = s;
   c->decode_l2_hints = 1;
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+      (void)cudaGetLastError();
+      free(c);
+      return D2O_ERR_CUDA;
+    }
+    c->n_sms = sms;
+  }
   c->state = (char*)state; c->scratch = (char*)scratch;
   c->state_bytes = state_bytes; c->scratch_bytes = scratch_bytes;
   const size_t BL = (size_t)cfg->batch * cfg->n_layers;

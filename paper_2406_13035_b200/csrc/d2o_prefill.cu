@@ -290,7 +290,8 @@ similarity_kernel(SimArgs a, const T* __restrict__ K, const T* __restrict__ kpoo
   // combine the 16 threads (tx) of a row: max u, ties -> lowest slot
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
-    unsigned long long key = ((unsigned long long)float_ord(best[r]) << 32) | (uint32_t)(0x7fffffff - bidx[r]);
+    // -0 (a zero-norm row) counts as +0, so that equal similarities tie
+    unsigned long long key = ((unsigned long long)float_ord(__fadd_rn(best[r], 0.f)) << 32) | (uint32_t)(0x7fffffff - bidx[r]);
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) {
       const unsigned long long t = __shfl_xor_sync(0xffffffffu, key, o);
@@ -298,8 +299,11 @@ similarity_kernel(SimArgs a, const T* __restrict__ K, const T* __restrict__ kpoo
     }
     const int i = i0 + ty * 4 + r;
     if (tx == 0 && i < Le) {
-      a.evict_mx[(size_t)slice * a.P + i] = ord_float((uint32_t)(key >> 32));
-      a.evict_nn[(size_t)slice * a.P + i] = 0x7fffffff - (int)(uint32_t)(key & 0xffffffffu);
+      // a row whose similarities are all NaN keeps the initial key: maximum -inf, neighbour 0, never merged
+      const int slot = 0x7fffffff - (int)(uint32_t)(key & 0xffffffffu);
+      const bool found = (unsigned)slot < (unsigned)S;
+      a.evict_mx[(size_t)slice * a.P + i] = found ? ord_float((uint32_t)(key >> 32)) : -INFINITY;
+      a.evict_nn[(size_t)slice * a.P + i] = found ? slot : 0;
     }
   }
 }
@@ -310,6 +314,7 @@ struct SegArgs {
   const float* evict_mx; const int32_t* evict_nn;
   int32_t* seg_start; int32_t* seg_items; int32_t* seg_tmp; float* tau;
   unsigned long long* counters;
+  uint32_t* status;
   int L, layer, B, Hkv, P, seg_stride;
   float tau_override;
 };
@@ -352,9 +357,16 @@ segment_kernel(SegArgs a) {
   for (int j = threadIdx.x; j <= S; j += blockDim.x) seg_smem[j] = 0;
   __syncthreads();
   const float thr = s_thr;
+  // An evicted token is merged iff its best similarity reaches the threshold.  A row without a finite maximum or
+  // with a neighbour outside the slice (non-finite keys) is never merged; it is reported once per slice.
+  auto merges = [&](int i) { return mx[i] >= thr && mx[i] > -INFINITY && (unsigned)nn[i] < (unsigned)S; };
+  bool bad_row = false;
   // how many evicted tokens pass the threshold for each retained slot (integer counts: order-free)
-  for (int i = threadIdx.x; i < Le; i += blockDim.x)
-    if (mx[i] >= thr) atomicAdd(&seg_smem[nn[i]], 1);
+  for (int i = threadIdx.x; i < Le; i += blockDim.x) {
+    if (merges(i)) atomicAdd(&seg_smem[nn[i]], 1);
+    else if (!(mx[i] > -INFINITY) || (unsigned)nn[i] >= (unsigned)S) bad_row = true;
+  }
+  if (bad_row) report_error(a.status, D2O_ERR_STATE, 0x5E600000u | (uint32_t)(slice & 0xfffff));
   __syncthreads();
   // exclusive scan of the counts -> segment starts
   int run = 0;
@@ -395,7 +407,7 @@ segment_kernel(SegArgs a) {
       const int k = base + lane;
       int item = -1;
       if (k < c1) {
-        if (p == 0) { if (mx[k] >= thr) item = k; }
+        if (p == 0) { if (merges(k)) item = k; }
         else item = src[k];
       }
       if (item >= 0) atomicAdd(&hist[warp * 64 + ((nn[item] >> shift) & 63)], 1);
@@ -416,7 +428,7 @@ segment_kernel(SegArgs a) {
       const int k = base + lane;
       int item = -1;
       if (k < c1) {
-        if (p == 0) { if (mx[k] >= thr) item = k; }
+        if (p == 0) { if (merges(k)) item = k; }
         else item = src[k];
       }
       const int dgt = item >= 0 ? ((nn[item] >> shift) & 63) : 64 + lane;   // distinct dummies for idle lanes
@@ -561,7 +573,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   ga.budgets = sa.budgets; ga.evict_mx = ma.evict_mx; ga.evict_nn = ma.evict_nn;
   ga.seg_start = (int32_t*)(X + c->slay.seg_start); ga.seg_items = (int32_t*)(X + c->slay.seg_items);
   ga.seg_tmp = (int32_t*)(X + c->slay.seg_tmp);
-  ga.tau = sa.tau; ga.counters = sa.counters;
+  ga.tau = sa.tau; ga.counters = sa.counters; ga.status = sa.status;
   ga.L = L; ga.layer = layer; ga.B = B; ga.Hkv = Hkv; ga.P = P; ga.seg_stride = seg_stride;
   ga.tau_override = g.tau_override;
   // counts / cursors per retained slot, later the radix histograms (32 warps x 64 digits)

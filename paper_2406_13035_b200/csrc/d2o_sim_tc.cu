@@ -309,8 +309,11 @@ neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K) {
       key = k2 > key ? k2 : key;
     }
     const float rn = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
-    a.evict_mx[(size_t)slice * a.P + i] = ord_float((uint32_t)(key >> 32)) * rn;
-    a.evict_nn[(size_t)slice * a.P + i] = 0x7fffffff - (int)(uint32_t)(key & 0xffffffffu);
+    // a row whose partial maxima are all empty (non-finite keys) gets maximum -inf, neighbour 0 and is never merged
+    const int slot = 0x7fffffff - (int)(uint32_t)(key & 0xffffffffu);
+    const bool found = key != 0ull && (unsigned)slot < (unsigned)S;
+    a.evict_mx[(size_t)slice * a.P + i] = found ? ord_float((uint32_t)(key >> 32)) * rn : -INFINITY;
+    a.evict_nn[(size_t)slice * a.P + i] = found ? slot : 0;
   }
 }
 

@@ -428,6 +428,7 @@ extern "C" d2o_status d2o_layer_stats_static(int32_t dtype, int32_t d_head, int3
   if (!aligned16(Q) || !aligned16(K) || !aligned16(colsum) || !density || ((uintptr_t)density & 7)) return D2O_ERR_INVALID_ARG;
   if ((unsigned long long)batch * n_q_heads * prompt_len > (unsigned long long)D2O_STATIC_LSE_FLOATS)
     return D2O_ERR_TOO_LARGE;
+  if ((long long)batch * n_q_heads > 65535) return D2O_ERR_TOO_LARGE;      // one grid row per (sequence, head)
   // set-up, once per device: in host code `g_static_lse` is only a handle, the kernels need its device address
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);

@@ -99,9 +99,11 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
                layers_per_call: Optional[int] = None, decode_stages: int = 0, decode_l2_hints: int = 1,
                similarity_path: int = 0, stats_path: int = 0, decode_warps: int = 0,
                decode_smem_rows: int = 0, decode_long_pairs: int = 0,
-               check_stats_all: Optional[bool] = None) -> Report:
+               check_stats_all: Optional[bool] = None, prompt_hook=None, decode_hook=None,
+               max_ties: Optional[int] = None) -> Report:
     """`slices`: (layer, b, kv_head) triples checked against the oracle (None = all).
-    The GPU always runs the whole workload."""
+    The GPU always runs the whole workload.  `prompt_hook(layer, Q, K, V)` and `decode_hook(step, q, k, v)` may
+    return edited input tensors (both sides then see the edited ones)."""
     rep = Report()
     ctx = make_ctx(wl, device, **(ctx_over or {}))
     cfg = ctx.cfg
@@ -122,6 +124,8 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
     KV = []
     for l in range(L):
         Q, K, V = streams[l].prompt()
+        if prompt_hook is not None:
+            Q, K, V = prompt_hook(l, Q, K, V)
         ctx.d2o_layer_stats(l, Q, K)
         KV.append((K, V))
         if l in chk_by_layer:
@@ -165,6 +169,8 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
     for step in range(n_steps):
         qs, ks, vs = zip(*[streams[l].decode() for l in range(L)])
         q, k, v = torch.stack(qs), torch.stack(ks), torch.stack(vs)
+        if decode_hook is not None:
+            q, k, v = decode_hook(step, q, k, v)
         out = torch.empty_like(q)
         for l0 in range(0, L, lpc):
             l1 = min(L, l0 + lpc)

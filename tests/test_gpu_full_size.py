@@ -40,6 +40,8 @@ def sample_slices(wl, n, seed):
     ("cfg2", 6, 48, None),       # Llama-3-8B-shaped GQA, batch 16, prompt 8192
     ("cfg3", 2, 32, None),       # prompt 32768
     ("cfg4", 8, 64, 8),          # serving sweep, batch 8
+    ("cfg4", 6, 48, 1),          # serving sweep, batch 1
+    ("cfg4", 6, 24, 32),         # serving sweep, batch 32
 ])
 def test_full_size_sampled_slices(name, n_slices, steps, batch):
     wl = W.CONFIGS[name]
@@ -51,4 +53,4 @@ def test_full_size_sampled_slices(name, n_slices, steps, batch):
     assert_report(rep, wl.dtype)
     assert rep.merges + rep.discards > 0
     print(name, "slices", slices, rep.max_err, rep.ties, "merges", rep.merges, "discards", rep.discards,
-          "storage flips", getattr(rep, "storage_flips", 0))
+          "storage flips", rep.storage_flips)

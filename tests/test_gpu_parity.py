@@ -101,6 +101,81 @@ def test_shape_and_hyperparameter_sweep(T, window, d, dtype, hq, hkv):
     assert_report(rep, wl.dtype)
 
 
+@pytest.mark.parametrize("dtype,d,hq,hkv,warps,smem_rows", [
+    ("f16", 128, 4, 2, 0, 0), ("f16", 128, 8, 2, 16, 0), ("f16", 128, 8, 1, 4, 0),
+    ("f16", 64, 4, 2, 4, 0), ("f16", 64, 8, 2, 8, 0), ("bf16", 64, 8, 1, 16, 0),
+    ("bf16", 64, 8, 2, 0, 0), ("f16", 64, 8, 4, 8, 96), ("bf16", 128, 8, 2, 8, 200),
+])
+def test_grouped_query_tensor_path_long_slices(dtype, d, hq, hkv, warps, smem_rows):
+    # 16-bit caches with 2, 4 or 8 query heads per KV head (the mma.sync decode path, both element types), with
+    # slices several ring stages long for every CTA size, also with most logits outside shared memory
+    wl = dataclasses.replace(W.CONFIGS["cfg0"], name="gqa", n_q_heads=hq, n_kv_heads=hkv, d_head=d, dtype=dtype,
+                             prompt_len=2048, decode_steps=6, n_sink=1, window=0, rho=0.3, n_layers=2, batch=1,
+                             density_temp=500.0, min_budget=16, beta=0.7)
+    rep = run_parity(wl, decode_warps=warps, decode_smem_rows=smem_rows)
+    assert_report(rep, wl.dtype)
+    assert rep.merges + rep.discards == rep.checked_slices * 6
+
+
+@pytest.mark.parametrize("beta", [0.0, 1.0])
+def test_ema_extremes(beta):
+    # beta = 1 is the ablation's "w.o. EMA-Threshold" (every victim merged); beta = 0 freezes tau at tau_0
+    wl = small(prompt_len=320, decode_steps=8, beta=beta)
+    rep = run_parity(wl)
+    assert_report(rep, wl.dtype)
+    if beta == 1.0:
+        assert rep.discards == 0 and rep.merges == 8 * 8
+    wl = dataclasses.replace(W.twin("cfg2"), beta=beta, decode_steps=6)
+    rep = run_parity(wl)
+    assert_report(rep, wl.dtype)
+    if beta == 1.0:
+        assert rep.discards == 0
+
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg2"])
+def test_window_and_sinks_only(name):
+    # N = 0: the cache holds the sinks and the recent window only (S = T + M for every layer)
+    base = W.CONFIGS["cfg0"] if name == "cfg0" else W.twin("cfg2")
+    P = 256
+    wl = dataclasses.replace(base, prompt_len=P, decode_steps=6, rho=0.125, window=30, n_sink=2, min_budget=32,
+                             max_budget=32, density_temp=1e30, n_layers=min(base.n_layers, 2))
+    rep = run_parity(wl)
+    assert_report(rep, wl.dtype)
+    assert rep.merges + rep.discards == rep.checked_slices * 6
+
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfg2"])
+def test_zero_norm_keys(name):
+    # a zero key has similarity 0 to everything: as an evicted prompt token, as a retained one (window), as the
+    # key of a generated token, and as the victim of a later step
+    base = W.CONFIGS["cfg0"] if name == "cfg0" else W.twin(name)
+    wl = dataclasses.replace(base, prompt_len=256, decode_steps=10, n_layers=min(base.n_layers, 2))
+
+    def prompt_hook(l, Q, K, V):
+        K = K.clone()
+        K[:, :, 7] = 0                    # low score, mid prompt: evicted
+        K[:, :, 100] = 0
+        K[:, :, 255] = 0                  # in the recent window: retained
+        return Q, K, V
+
+    def decode_hook(step, q, k, v):
+        if step in (1, 2):
+            k = k.clone()
+            k[:] = 0
+        return q, k, v
+
+    rep = run_parity(wl, prompt_hook=prompt_hook, decode_hook=decode_hook)
+    assert_report(rep, wl.dtype)
+
+
+def test_more_sinks_than_budget_is_rejected(cuda_device):
+    from parity import make_ctx
+    wl = small(prompt_len=128, decode_steps=2, n_sink=40, min_budget=8)
+    with pytest.raises(B.D2OError) as e:
+        make_ctx(wl)
+    assert e.value.status == 1            # min_budget must leave room for the sinks and one more token
+
+
 def test_budget_never_reached_equals_full_attention():
     """With S_l >= prompt + steps nothing is evicted and the output is plain softmax attention."""
     wl = small(prompt_len=200, decode_steps=7, rho=1.035)
