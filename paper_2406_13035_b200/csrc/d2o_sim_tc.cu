@@ -21,6 +21,7 @@
 // (ordered max_j k_i.k_j/|k_j|, 0x7fffffff - slot).  neighbour_reduce_kernel takes the maximum over
 // the chunks at the evicted positions and multiplies by 1/|k_i|.
 #include <cuda.h>
+#include <limits.h>
 #include <math.h>
 
 #include "d2o_common.cuh"
@@ -53,34 +54,31 @@ __host__ __device__ __forceinline__ int chunk_columns(int S) {
 
 // One block of 32 accumulator columns of one row: times 1/|k_c| per column, maximum and its column (the lowest
 // on ties), merged into the row's running (best, best_col).  cl0 = chunk-local column of the block.
+//
+// The maximum is tracked on the bit patterns as signed integers: for values >= +0 that is the order of the floats,
+// and every negative value (and -0) sorts below +0, in the wrong order among themselves.  A row whose true maximum is
+// negative therefore ends with a negative pattern; it is reported as "nothing found" and neighbour_reduce_kernel
+// redoes that row with plain fp32 arithmetic.  In exchange the compare and the value select are one integer
+// max-with-predicate instruction, which is what the scan is bound by.
 __device__ __forceinline__ void scan_block(const uint32_t (&r)[32], const float* s_rn, int cl0, int n_cols, int c0,
-                                           float& best, int& best_col) {
-  // four interleaved running maxima (columns i mod 4) keep the compare chains short
-  float tb[4]; int ti[4];
+                                           int& best, int& best_col) {
+  // four interleaved running maxima (columns i mod 4) keep the dependent chains short
+  int tb[4], ti[4];
 #pragma unroll
-  for (int w = 0; w < 4; ++w) { tb[w] = -INFINITY; ti[w] = w; }
+  for (int w = 0; w < 4; ++w) { tb[w] = INT_MIN; ti[w] = w; }
   const float4* rn4 = reinterpret_cast<const float4*>(s_rn + cl0);
-  if (cl0 + 32 <= n_cols) {
+  const bool whole = cl0 + 32 <= n_cols;                          // else: columns past the chunk hold other slices' rows
 #pragma unroll
-    for (int i4 = 0; i4 < 8; ++i4) {
-      const float4 q = rn4[i4];
-      const float rv[4] = {q.x, q.y, q.z, q.w};
+  for (int i4 = 0; i4 < 8; ++i4) {
+    const float4 q = rn4[i4];
+    const float rv[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const float x = __uint_as_float(r[i4 * 4 + w]) * rv[w];
-        if (x > tb[w]) { tb[w] = x; ti[w] = i4 * 4 + w; }
-      }
-    }
-  } else {                                                        // columns past the chunk hold other slices' rows
-#pragma unroll
-    for (int i4 = 0; i4 < 8; ++i4) {
-      const float4 q = rn4[i4];
-      const float rv[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const float x = __uint_as_float(r[i4 * 4 + w]) * rv[w];
-        if (cl0 + i4 * 4 + w < n_cols && x > tb[w]) { tb[w] = x; ti[w] = i4 * 4 + w; }
-      }
+    for (int w = 0; w < 4; ++w) {
+      int x = __float_as_int(__uint_as_float(r[i4 * 4 + w]) * rv[w]);
+      if (!whole && cl0 + i4 * 4 + w >= n_cols) x = INT_MIN;
+      bool keep;
+      tb[w] = __vibmax_s32(tb[w], x, &keep);                      // keep = (tb >= x): the earlier column stays on ties
+      ti[w] = keep ? ti[w] : i4 * 4 + w;
     }
   }
   // larger value wins, equal values go to the lower column
@@ -218,7 +216,7 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
       tc::fence_after_sync();
       if (n_blk > 0) tc::tmem_ld32_issue(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(blk0 * 32), ra);
     }
-    float best = -INFINITY; int best_col = 0x7fffffff;
+    int best = INT_MIN, best_col = 0x7fffffff;               // bit pattern of the best value so far (see scan_block)
 #pragma unroll 1
     for (int job = 0; job < n_jobs; ++job) {
       const int t = t0 + job / n_nt, j = job % n_nt;
@@ -246,10 +244,10 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
       }
       if (n_blk > 1) scan_block(rb, s_rn, col0 + 32, n_cols, c0, best, best_col);
       if (j == n_nt - 1) {
-        // (ordered value, inverted slot): larger is better, ties go to the lower slot; -0 counts as +0
-        if (best == 0.f) best = 0.f;
-        const unsigned long long key = best > -INFINITY
-            ? (((unsigned long long)float_ord(best) << 32) | (uint32_t)(0x7fffffff - best_col)) : 0ull;
+        // (ordered value, inverted slot): larger is better, ties go to the lower slot.  A non-negative float's
+        // ordered form is its pattern with the top bit set; a negative pattern means "nothing found" (key 0)
+        const unsigned long long key = best >= 0
+            ? (((unsigned long long)(0x80000000u | (uint32_t)best) << 32) | (uint32_t)(0x7fffffff - best_col)) : 0ull;
         if (part > 0) s_pair[(part - 1) * kTileM + row] = key;
         asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
         if (part == 0) {
@@ -260,7 +258,7 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
           if (pos < a.P) out_keys[pos] = k;
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
-        best = -INFINITY; best_col = 0x7fffffff;
+        best = INT_MIN; best_col = 0x7fffffff;
       }
     }
   }
@@ -275,45 +273,65 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
 
 // mx_i = 1/|k_i| * max over the chunks of the partial maxima, nn_i = its slot, for the evicted positions.
 struct NnReduceArgs {
-  const int32_t* budgets;
+  const int32_t* budgets; const int64_t* row_off;
   const int32_t* evict_idx;
   const unsigned long long* part_key;
+  const float* rnorm;                       // pool-wide 1/|k_c|
   float* evict_mx; int32_t* evict_nn;
   int L, layer, Hkv, P, n_chunks_max;
 };
 
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
-neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K) {
+neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K, const T* __restrict__ kpool) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;
   const int slice = blockIdx.y;
-  const int b = slice / a.Hkv;
+  const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int S = a.budgets[b * a.L + a.layer];
   const int Le = a.P - S;
   const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
   const int i = blockIdx.x * (blockDim.x / LPR) + grp;
   if (i >= Le) return;
+  const unsigned gmask = group_mask<LPR>();
   const int pos = a.evict_idx[(size_t)slice * a.P + i];
   float f[EPV];
   Elem<T>::unpack(ld_global_v4(K + ((size_t)slice * a.P + pos) * D + lig * EPV), f);
   float ss = 0.f;
 #pragma unroll
   for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
-  ss = group_sum<LPR>(ss, group_mask<LPR>());
-  if (lig == 0) {
-    const int n_chunks = (S + kChunkN - 1) / kChunkN;
-    unsigned long long key = 0ull;
-    for (int c = 0; c < n_chunks; ++c) {
-      const unsigned long long k2 = a.part_key[((size_t)slice * a.n_chunks_max + c) * a.P + pos];
-      key = k2 > key ? k2 : key;
+  ss = group_sum<LPR>(ss, gmask);
+  const float rn = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+  const int n_chunks = (S + kChunkN - 1) / kChunkN;
+  unsigned long long key = 0ull;
+  for (int c = 0; c < n_chunks; ++c) {
+    const unsigned long long k2 = a.part_key[((size_t)slice * a.n_chunks_max + c) * a.P + pos];
+    key = k2 > key ? k2 : key;
+  }
+  int slot = 0x7fffffff - (int)(uint32_t)(key & 0xffffffffu);
+  float mx = ord_float((uint32_t)(key >> 32)) * rn;
+  bool found = key != 0ull && (unsigned)slot < (unsigned)S;
+  if (!found) {
+    // No chunk reported a non-negative maximum: every similarity of this row is negative (or not finite).  The row
+    // is redone here in fp32, all retained rows in slot order (the first maximum stays).  A row without any finite
+    // similarity gets maximum -inf and neighbour 0 and is never merged.
+    const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
+    float best = -INFINITY; int bj = 0;
+    for (int j = 0; j < S; ++j) {
+      float g[EPV];
+      Elem<T>::unpack(ld_global_v4(kpool + (row0 + j) * D + lig * EPV), g);
+      float dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPV; ++e) dot = fmaf(f[e], g[e], dot);
+      dot = group_sum<LPR>(dot, gmask);
+      const float u = __fadd_rn(dot * rn * a.rnorm[row0 + j], 0.f);
+      if (u > best) { best = u; bj = j; }
     }
-    const float rn = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
-    // a row whose partial maxima are all empty (non-finite keys) gets maximum -inf, neighbour 0 and is never merged
-    const int slot = 0x7fffffff - (int)(uint32_t)(key & 0xffffffffu);
-    const bool found = key != 0ull && (unsigned)slot < (unsigned)S;
-    a.evict_mx[(size_t)slice * a.P + i] = found ? ord_float((uint32_t)(key >> 32)) * rn : -INFINITY;
-    a.evict_nn[(size_t)slice * a.P + i] = found ? slot : 0;
+    mx = best; slot = bj;
+  }
+  if (lig == 0) {
+    a.evict_mx[(size_t)slice * a.P + i] = mx;
+    a.evict_nn[(size_t)slice * a.P + i] = slot;
   }
 }
 
@@ -403,7 +421,8 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   if (e != cudaSuccess) return e;
 
   NnReduceArgs r;
-  r.budgets = a.budgets; r.evict_idx = (const int32_t*)(X + c->slay.evict_idx); r.part_key = a.part_key;
+  r.budgets = a.budgets; r.row_off = a.row_off; r.rnorm = a.rnorm;
+  r.evict_idx = (const int32_t*)(X + c->slay.evict_idx); r.part_key = a.part_key;
   r.evict_mx = (float*)(X + c->slay.evict_mx); r.evict_nn = (int32_t*)(X + c->slay.evict_nn);
   r.L = g.n_layers; r.layer = layer; r.Hkv = Hkv; r.P = P; r.n_chunks_max = n_chunks_max;
   int minS = P;
@@ -413,11 +432,11 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   const int lpr = D * 2 / 16;
   dim3 rgrid((maxLe + 256 / lpr - 1) / (256 / lpr), n_slices);
   if (g.dtype == D2O_F16) {
-    if (D == 128) neighbour_reduce_kernel<__half, 128><<<rgrid, 256, 0, st>>>(r, (const __half*)K);
-    else neighbour_reduce_kernel<__half, 64><<<rgrid, 256, 0, st>>>(r, (const __half*)K);
+    if (D == 128) neighbour_reduce_kernel<__half, 128><<<rgrid, 256, 0, st>>>(r, (const __half*)K, (const __half*)(S + c->lay.kpool));
+    else neighbour_reduce_kernel<__half, 64><<<rgrid, 256, 0, st>>>(r, (const __half*)K, (const __half*)(S + c->lay.kpool));
   } else {
-    if (D == 128) neighbour_reduce_kernel<__nv_bfloat16, 128><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K);
-    else neighbour_reduce_kernel<__nv_bfloat16, 64><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K);
+    if (D == 128) neighbour_reduce_kernel<__nv_bfloat16, 128><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K, (const __nv_bfloat16*)(S + c->lay.kpool));
+    else neighbour_reduce_kernel<__nv_bfloat16, 64><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K, (const __nv_bfloat16*)(S + c->lay.kpool));
   }
   return cudaGetLastError();
 }

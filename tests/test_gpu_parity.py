@@ -168,6 +168,24 @@ def test_zero_norm_keys(name):
     assert_report(rep, wl.dtype)
 
 
+@pytest.mark.parametrize("name", ["cfg1", "cfg2"])
+def test_rows_with_only_negative_similarities(name):
+    # every key in the positive orthant except one in the negative orthant: all its cosines are negative, which the
+    # tensor-core similarity kernel hands to the fp32 redo path of the reduce kernel
+    wl = dataclasses.replace(W.twin(name), n_layers=2, decode_steps=4)
+    seen = {"n": 0}
+
+    def prompt_hook(l, Q, K, V):
+        K = K.abs()
+        K[:, :, 7] = -K[:, :, 7]
+        seen["n"] += 1
+        return Q, K, V
+
+    rep = run_parity(wl, prompt_hook=prompt_hook)
+    assert_report(rep, wl.dtype)
+    assert seen["n"] == 2
+
+
 def test_more_sinks_than_budget_is_rejected(cuda_device):
     from parity import make_ctx
     wl = small(prompt_len=128, decode_steps=2, n_sink=40, min_budget=8)
