@@ -108,6 +108,8 @@ typedef struct {
   uint32_t error_word;       /* 0 = none; else first device-side anomaly (d2o_status)         */
   uint32_t error_detail;
   uint64_t decode_launches;  /* decode kernels launched so far (a step over all layers may take two)  */
+  uint64_t guess_misses;     /* evictions whose victim was not among the rows guessed before the step (the keys
+                              * of that slice were then read a second time)                                   */
 } d2o_stats;
 
 const char* d2o_status_string(d2o_status s);

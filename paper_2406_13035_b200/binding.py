@@ -50,7 +50,8 @@ class D2OView(C.Structure):
 class D2OStats(C.Structure):
     _fields_ = [("decode_steps", C.c_uint64), ("evictions", C.c_uint64), ("merges", C.c_uint64),
                 ("discards", C.c_uint64), ("prefill_evicted", C.c_uint64), ("prefill_merged", C.c_uint64),
-                ("error_word", C.c_uint32), ("error_detail", C.c_uint32), ("decode_launches", C.c_uint64)]
+                ("error_word", C.c_uint32), ("error_detail", C.c_uint32), ("decode_launches", C.c_uint64),
+                ("guess_misses", C.c_uint64)]
 
 
 class D2OError(RuntimeError):

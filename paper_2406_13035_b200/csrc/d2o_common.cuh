@@ -129,7 +129,7 @@ __device__ __forceinline__ void report_error(uint32_t* status_word, uint32_t cod
 
 // ----------------------------------------------------------------------------- counters
 enum Counter { kCntDecodeSteps = 0, kCntEvictions, kCntMerges, kCntDiscards, kCntPrefillEvicted,
-               kCntPrefillMerged, kNumCounters = 8 };
+               kCntPrefillMerged, kCntGuessMisses, kNumCounters = 8 };
 
 // ----------------------------------------------------------------------------- context
 struct Layout {            // byte offsets into `state`

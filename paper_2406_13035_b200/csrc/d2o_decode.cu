@@ -2,24 +2,29 @@
 //
 // One CTA handles one slice = (layer, sequence, KV head) with its G query heads, and streams the
 // slice's cache rows through a ring of shared-memory stages filled by bulk asynchronous copies
-// (cp.async.bulk, completion on mbarriers).  A producer warp runs ahead of eight consumer warps by
-// the depth of the ring, across the boundaries of the passes, so the reductions between two passes
+// (cp.async.bulk, completion on mbarriers).  A producer warp runs ahead of the consumer warps by
+// the depth of the ring, across the boundary of the two passes, so the reductions between them
 // do not drain the memory pipeline:
 //
-//   pass K   keys once from HBM: logits of the G heads (plus the new token's row from the inputs)
+//   guess    before the keys arrive: the rows with the lowest accumulated scores among those that may
+//            be evicted in this step (Eq. 7-8) are the likely victims; their keys join the queries
+//   pass K   keys once from HBM: logits of the G heads and the dot products with the guessed victims
+//            (Eq. 9), the new token's row from the inputs
 //            -> softmax normaliser -> AttnScore += probabilities (Eq. 6 case 2)
 //            -> victim = lowest score outside the T sinks and the M most recent positions (Eq. 7-8)
-//   pass K'  keys again, now served by L2 (the first pass asks L2 to keep them, the later passes
-//            ask it to drop what they touch): cosine of the victim with every other row (Eq. 9)
+//            -> if it was guessed (it nearly always is), its cosines are already there; if not, the
+//               keys are read once more, directly from L2, for this one slice
 //            -> nearest neighbour, tau_t (Eq. 10), merge decision, merged key row (Eq. 11-12)
 //   pass V   values once from HBM: outputs (Eq. 3); the value rows of the victim and of the
 //            neighbour are picked out of the stream for the merge (Eq. 11)
 //   then     merged value row, the new token takes the victim's row.
-// Pass K' is skipped while the cache is not full.  Everything that needs the whole slice is a
-// block-wide reduction inside one CTA; there is no inter-CTA communication.
+// The guess changes no result: the victim is always the exact arg-min of the updated scores, and the
+// cosines of a guessed row are the same dot products a second pass would compute.
+// Everything that needs the whole slice is a block-wide reduction inside one CTA; there is no
+// inter-CTA communication.
 //
 // Arithmetic: fp32 FMAs on unpacked rows (one query head per KV head, or fp32 caches), or, for 16-bit caches with
-// grouped queries, mma.sync for all three passes on stages that arrive through tiled tensor maps with the 128-byte
+// grouped queries, mma.sync for both passes on stages that arrive through tiled tensor maps with the 128-byte
 // swizzle.  A decode step over all layers runs the slices largest first and, where a few slices are much longer
 // than the rest, those in a launch of their own with sixteen consumer warps (see launch_decode).
 #include <math.h>
@@ -93,6 +98,23 @@ __device__ __forceinline__ void stage_wait(unsigned long long* bar, uint32_t par
 // Similarity as an ordered key: -0 (a zero-norm row times a negative dot product) must count as +0, or equal
 // similarities would not tie.
 __device__ __forceinline__ uint32_t sim_ord(float u) { return float_ord(__fadd_rn(u, 0.f)); }
+// d = a * b + c on two fp32 lanes at once (one issue slot instead of two)
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<const unsigned long long*>(&a)), "l"(*reinterpret_cast<const unsigned long long*>(&b)),
+        "l"(*reinterpret_cast<const unsigned long long*>(&c)));
+  return *reinterpret_cast<float2*>(&d);
+}
+// dot product of two pieces of N floats each, accumulated in two interleaved fp32 chains
+template <int N>
+__device__ __forceinline__ float dot_pairs(const float (&a)[N], const float (&b)[N]) {
+  float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int i = 0; i < N; i += 2) acc = ffma2(make_float2(a[i], a[i + 1]), make_float2(b[i], b[i + 1]), acc);
+  return acc.x + acc.y;
+}
 // next slot of the ring; the parity flips on wrap-around
 __device__ __forceinline__ void ring_next(int& slot, uint32_t& ph, int stages) {
   if (++slot == stages) { slot = 0; ph ^= 1u; }
@@ -347,14 +369,14 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
       }
-      const int n_pass = evict ? 3 : 2;
       int slot = 0, q = 0;
       uint32_t ph = 1;                                               // parity of the previous use of a slot
-      for (int p = 0; p < n_pass; ++p) {
-        const bool is_v = (p == n_pass - 1);
+      for (int p = 0; p < 2; ++p) {
+        const bool is_v = (p == 1);
         const T* pool = is_v ? vpool : kpool;
         const T* fresh = is_v ? v_new : k_new;
         const bool hint = a.l2_hints != 0;
+        // keys may be read once more (a victim that was not guessed): they leave L2 after the values
         const unsigned long long pol = (p == 0 && evict) ? keep : drop;
         for (int s = 0; s < n_st; ++s, ++q, ring_next(slot, ph, NS)) {
           if (q >= NS) stage_wait(&s_empty[slot], ph, &s_timeout);
@@ -362,9 +384,9 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
           const int np = max(0, min(a1, n_old) - a0);                // cache rows of the stage
           const bool nw = n_old >= a0 && n_old < a1;                 // the new token's row falls into the stage
           uint4* dst = ring + (size_t)slot * SR * LPR;
-          // pass K' also needs 1/|k| and the position of its rows (16-byte granules: up to 3 entries past n_old
-          // come from the slice's padding and are never used)
-          const bool with_meta = evict && p == 1 && np > 0;
+          // the cosines of pass K also need 1/|k| and the position of the rows (16-byte granules: up to 3 entries past
+          // n_old come from the slice's padding and are never used)
+          const bool with_meta = evict && p == 0 && np > 0;
           const int np4 = (np + 3) & ~3;
           if (kTensor) {
             // swizzled [d half][SR rows][128 B]; the box always has SR rows (what lies past the cache rows is never
@@ -399,8 +421,10 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     }
     // A grid launched with programmatic stream serialisation may run beside its predecessor, but it must not be
     // complete before it: whatever the stream runs next (the next step, a copy of the outputs) is ordered behind
-    // this grid only.  Returns at once in an ordinarily launched grid.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // this grid only.  One CTA that stays until the predecessor has finished is enough for that, and keeps the other
+    // CTAs' places free for the rest of this grid: the last one, which holds the shortest slice.  The instruction
+    // returns at once in an ordinarily launched grid.
+    if (blockIdx.x == gridDim.x - 1) asm volatile("griddepcontrol.wait;" ::: "memory");
     return;
   }
 
@@ -438,7 +462,103 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   uint4 knew = make_uint4(0, 0, 0, 0), vnew = make_uint4(0, 0, 0, 0);
   if (grp == 0) { knew = ld_global_v4(k_new + lig * EPV); vnew = ld_global_v4(v_new + lig * EPV); }
 
-  // ---- pass K: logits
+  // ---- guess of the victim: the NC rows with the lowest accumulated score (ties: the later position) among the rows
+  // that may be evicted in this step, taken from the scores as they stand before the step (Eq. 7-8 on the old scores).
+  // This step's probabilities are small against the differences between accumulated scores, so the victim that is
+  // chosen after the softmax is nearly always one of them.  Their keys are multiplied with every row during pass K.
+  constexpr int NC = kTensor ? 2 : 1;
+  constexpr int kCandTig = G < 8 ? G / 2 : 0;                          // tensor path: the lanes whose columns hold the candidates
+  int cand_li[NC];                                                     // row of candidate c in the slice, -1: none
+  float cand_rn[NC];                                                   // its 1/|k|
+  unsigned long long cbest[NC];                                        // this thread's best (cosine, earliest position) per candidate
+  int cbest_li[NC];
+  float ck[kTensor ? 1 : NC][EPV];                                     // FMA path: this lane's piece of the candidates' keys
+  uint4 cb[D / 32];                                                    // tensor path, G = 8: fragments of candidate `gid`
+#pragma unroll
+  for (int c = 0; c < NC; ++c) { cand_li[c] = -1; cand_rn[c] = 0.f; cbest[c] = 0ull; cbest_li[c] = -1; }
+#pragma unroll
+  for (int j = 0; j < D / 32; ++j) cb[j] = make_uint4(0, 0, 0, 0);
+  if (evict) {
+    if (warp == 0) {
+      // the new token's inverse norm, from the row as stored
+      float f[EPV];
+      Elem<T>::unpack(knew, f);
+      float ss = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
+      ss = warp_sum(ss);                                               // lanes >= LPR hold zeros
+      if (lane == 0) s_new_rn = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+    }
+    unsigned long long my[NC];
+    int my_li[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) { my[c] = ~0ull; my_li[c] = -1; }
+    auto offer = [&](float sc, int pz, int li) {
+      if (pz >= Tn && pz <= a.t - M) {
+        unsigned long long key = ((unsigned long long)float_ord(sc) << 32) | (uint32_t)(0x7fffffff - pz);
+        int kl = li;
+#pragma unroll
+        for (int c = 0; c < NC; ++c)
+          if (key < my[c]) { const unsigned long long tk = my[c]; const int tl = my_li[c]; my[c] = key; my_li[c] = kl; key = tk; kl = tl; }
+      }
+    };
+    const int n_vec4 = (n_old / 4) * 4;
+    for (int li = tid * 4; li < n_vec4; li += kConsThreads * 4) {
+      const float4 sc = *reinterpret_cast<const float4*>(a.score + row0 + li);
+      const int4 pz = *reinterpret_cast<const int4*>(a.pos + row0 + li);
+      offer(sc.x, pz.x, li); offer(sc.y, pz.y, li + 1); offer(sc.z, pz.z, li + 2); offer(sc.w, pz.w, li + 3);
+    }
+    for (int li = n_vec4 + tid; li < n_old; li += kConsThreads) offer(a.score[row0 + li], a.pos[row0 + li], li);
+    int taken = 0;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      unsigned long long k = ~0ull; int kl = -1;
+#pragma unroll
+      for (int j = 0; j < NC; ++j) if (taken == j) { k = my[j]; kl = my_li[j]; }
+      block_arg_extreme<true, CW>(k, kl, s_key, s_li, &s_best_key, &s_best_li);
+      consumer_sync<CW>();
+      const unsigned long long bk = s_best_key;
+      cand_li[c] = bk == ~0ull ? -1 : s_best_li;
+      if (bk != ~0ull && bk == k) ++taken;                             // this thread's row was taken
+    }
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      if (cand_li[c] < 0) continue;
+      const T* row = kpool + (row0 + cand_li[c]) * D;
+      cand_rn[c] = a.rnorm[row0 + cand_li[c]];
+      if constexpr (!kTensor) {
+        Elem<T>::unpack(ld_global_v4(row + lig * EPV), ck[c]);
+      } else if constexpr (G < 8) {
+        // the candidates take the columns after the query heads of the same tensor-core steps
+        if (gid == G + c) {
+#pragma unroll
+          for (int j = 0; j < D / 32; ++j) qb[j] = ld_global_v4(row + ((j >> 1) * 8 + 2 * tig + (j & 1)) * 8);
+        }
+      } else {
+        if (gid == c) {
+#pragma unroll
+          for (int j = 0; j < D / 32; ++j) cb[j] = ld_global_v4(row + ((j >> 1) * 8 + 2 * tig + (j & 1)) * 8);
+        }
+      }
+    }
+    if constexpr (!kTensor) {
+#pragma unroll
+      for (int c = 0; c < NC; ++c)
+        if (cand_li[c] < 0) {
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) ck[c][e] = 0.f;
+        }
+    }
+  }
+  // cosine of row li (inverse norm rn, position pz) with candidate c, from their dot product: keeps this thread's best
+  auto cand_update = [&](int c, float dot, float rn, int pz, int li) {
+    if (li != cand_li[c]) {
+      const unsigned long long key = ((unsigned long long)sim_ord(dot * cand_rn[c] * rn) << 32) | (uint32_t)(0x7fffffff - pz);
+      if (key > cbest[c]) { cbest[c] = key; cbest_li[c] = li; }
+    }
+  };
+
+  // ---- pass K: logits, and the candidates' dot products
   float mloc[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) mloc[g] = -INFINITY;
@@ -462,8 +582,26 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       const int lt = s * SR + tile * 16;                             // first row of the tile
       const bool mine = tile >= 0 && lt < n_old;
       if (mine) tile_dots<T, D, SR>(st, tile, qb, acc);
+      float acc2[4] = {0.f, 0.f, 0.f, 0.f};
+      if constexpr (G == 8) {
+        if (mine && evict) tile_dots<T, D, SR>(st, tile, cb, acc2);  // eight heads leave no column free: a second set of steps
+      }
+      // the candidates' columns belong to the lanes with tig = kCandTig: rows gid, gid + 8 of the tile; their 1/|k| and
+      // positions leave the stage before it is released
+      const bool cand_lane = evict && mine && tig == kCandTig;
+      const int lr0 = tile * 16 + gid;
+      float rn0 = 0.f, rn1 = 0.f; int ps0 = 0, ps1 = 0;
+      if (cand_lane) {
+        rn0 = meta_rn[(size_t)slot * SR + lr0]; ps0 = meta_ps[(size_t)slot * SR + lr0];
+        rn1 = meta_rn[(size_t)slot * SR + lr0 + 8]; ps1 = meta_ps[(size_t)slot * SR + lr0 + 8];
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_empty[slot]);
+      if (cand_lane) {
+        const float* ca = G < 8 ? acc : acc2;
+        if (lt + gid < n_old) { cand_update(0, ca[0], rn0, ps0, lt + gid); cand_update(1, ca[1], rn0, ps0, lt + gid); }
+        if (lt + gid + 8 < n_old) { cand_update(0, ca[2], rn1, ps1, lt + gid + 8); cand_update(1, ca[3], rn1, ps1, lt + gid + 8); }
+      }
       if (mine && 2 * tig < G) {
         const int li0 = lt + gid, li1 = li0 + 8;
         const float x00 = acc[0] * qscale, x01 = acc[1] * qscale, x10 = acc[2] * qscale, x11 = acc[3] * qscale;
@@ -510,6 +648,20 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         if (lane == 0) pl_put(g, n_old, x);
         mloc[g] = fmaxf(mloc[g], x);
       }
+      if (evict) {
+        // the new token is not in the stream: its cosines with the candidates come from the inputs
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          if (cand_li[c] < 0) continue;
+          float cf[EPV];
+          Elem<T>::unpack(lane < LPR ? ld_global_v4(kpool + (row0 + cand_li[c]) * D + lane * EPV) : make_uint4(0, 0, 0, 0), cf);
+          float x = 0.f;
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) x = fmaf(cf[e], kf[e], x);
+          x = warp_sum(x);
+          if (lane == 0) cand_update(c, x, s_new_rn, a.t, n_old);
+        }
+      }
     }
   } else {
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
@@ -525,22 +677,36 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         for (int u = 0; u < 4; ++u)
           raw[u] = s * SR + u * NGRP + grp < n ? st[(size_t)u * NGRP * LPR] : make_uint4(0, 0, 0, 0);
       }
-      float dot[G][4];
+      float dot[G][4], cdot[NC][4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         float f[EPV];
         Elem<T>::unpack(raw[u], f);
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-          float x = 0.f;
+          dot[g][u] = dot_pairs<EPV>(qf[g], f);
+        }
+        if (evict) {
 #pragma unroll
-          for (int e = 0; e < EPV; ++e) x = fmaf(qf[g][e], f[e], x);
-          dot[g][u] = x;
+          for (int c = 0; c < NC; ++c) {
+            cdot[c][u] = dot_pairs<EPV>(ck[c], f);
+          }
         }
       }
+      const int li = s * SR + (lig / QL) * NGRP + grp;               // the row whose total this lane receives
+      // its 1/|k| and position leave the stage before the stage is released
+      const bool cand_lane = evict && li < n && lig % QL == 0;
+      float rn_li = s_new_rn; int ps_li = a.t;
+      if (cand_lane && li < n_old) { rn_li = meta_rn[(size_t)slot * SR + (li - s * SR)]; ps_li = meta_ps[(size_t)slot * SR + (li - s * SR)]; }
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_empty[slot]);
-      const int li = s * SR + (lig / QL) * NGRP + grp;               // the row whose total this lane receives
+      if (evict) {
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          const float r = reduce4<LPR>(cdot[c][0], cdot[c][1], cdot[c][2], cdot[c][3], lig);
+          if (cand_lane) cand_update(c, r, rn_li, ps_li, li);
+        }
+      }
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         const float r = reduce4<LPR>(dot[g][0], dot[g][1], dot[g][2], dot[g][3], lig);
@@ -555,8 +721,8 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     }
   }
   // ---- softmax normaliser, probabilities, accumulated attention (Eq. 6 case 2), victim candidate
-  if (warp == 0) {
-    // the new token's metadata; its inverse norm from the row as stored
+  if (warp == 0 && !evict) {
+    // the new token's inverse norm from the row as stored (when a row is evicted it was needed before pass K)
     float f[EPV];
     Elem<T>::unpack(knew, f);
     float ss = 0.f;
@@ -653,7 +819,8 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     if (evict) block_arg_extreme<true, CW>(my_min, my_min_li, s_key, s_li, &s_best_key, &s_best_li);
     consumer_sync<CW>();
   }
-  // ---- victim (Eq. 7-8), pass K': cosine with every other row (Eq. 9), tau_t (Eq. 10), merged key (Eq. 11-12)
+  // ---- victim (Eq. 7-8); its cosine with every other row (Eq. 9): from the guess, or from a second look at the keys;
+  // tau_t (Eq. 10), merged key (Eq. 11-12)
   int vic_li = -1, nn_li = -1;
   bool merge = false, nn_is_new = false;
   float w_e = 0.f, w_c = 1.f, rn_slot = 0.f;
@@ -662,9 +829,9 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     vic_li = s_best_li;
     if (s_best_key == ~0ull) {
       // nothing may be evicted (S_l < T + M): report, drop the new token, keep the cache as it is.  The producer
-      // still delivers two passes; they are drained without being used.
+      // still delivers the value pass; it is drained without being used.
       if (tid == 0) report_error(a.status, D2O_ERR_STATE, 0xDEC00000u | (uint32_t)(sl & 0xfffff));
-      for (int s = 0; s < 2 * n_st; ++s, ring_next(slot, ph, NS)) {
+      for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
         stage_wait(&s_full[slot], ph, &s_timeout);
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_empty[slot]);
@@ -675,88 +842,38 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     float kvic[EPV];
     Elem<T>::unpack(ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) + lig * EPV), kvic);
     unsigned long long best = 0ull; int best_li = -1;
-    if constexpr (kTensor) {
-      // the victim's key as the only vector of the B operand: lanes with tig = 0 receive the dot products
-      uint4 vb[D / 32];
+    int hit = -1;
 #pragma unroll
-      for (int j = 0; j < D / 32; ++j)
-        vb[j] = gid == 0 ? ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) +
-                                        ((j >> 1) * 8 + 2 * tig + (j & 1)) * 8)
-                         : make_uint4(0, 0, 0, 0);
-      for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
-        stage_wait(&s_full[slot], ph, &s_timeout);
-        const unsigned char* st = reinterpret_cast<const unsigned char*>(ring) + (size_t)slot * kStageBytes;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        const int tile = kHalfTiles ? warp - (s & 1) * kTiles : warp;
-        const bool active = tile >= 0 && tile < kTiles && s * SR + tile * 16 < n_old;
-        if (active) tile_dots<T, D, SR>(st, tile, vb, acc);
-        // 1/|k| and position of this thread's two rows leave the stage before the stage is released
-        const int lr0 = tile * 16 + gid, li0 = s * SR + lr0, li1 = li0 + 8;
-        const bool m0 = active && tig == 0 && li0 < n_old && li0 != vic_li, m1 = active && tig == 0 && li1 < n_old && li1 != vic_li;
-        float rn0 = 0.f, rn1 = 0.f; int ps0 = 0, ps1 = 0;
-        if (m0) { rn0 = meta_rn[(size_t)slot * SR + lr0]; ps0 = meta_ps[(size_t)slot * SR + lr0]; }
-        if (m1) { rn1 = meta_rn[(size_t)slot * SR + lr0 + 8]; ps1 = meta_ps[(size_t)slot * SR + lr0 + 8]; }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s_empty[slot]);
-        if (m0) {                                                    // max similarity, ties -> earliest position
-          const unsigned long long key = ((unsigned long long)sim_ord(acc[0] * vic_rn * rn0) << 32) | (uint32_t)(0x7fffffff - ps0);
-          if (key > best) { best = key; best_li = li0; }
-        }
-        if (m1) {
-          const unsigned long long key = ((unsigned long long)sim_ord(acc[2] * vic_rn * rn1) << 32) | (uint32_t)(0x7fffffff - ps1);
-          if (key > best) { best = key; best_li = li1; }
-        }
-      }
-      if (warp == 0 && vic_li != n_old) {
-        // the new token as a merge target: its key row is held by the first LPR lanes
-        float kf[EPV];
-        Elem<T>::unpack(knew, kf);
-        float x = 0.f;
-        if (lane < LPR) {
+    for (int c = 0; c < NC; ++c) if (cand_li[c] == vic_li) hit = c;
+    if (hit >= 0) {
 #pragma unroll
-          for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], kf[e], x);
-        }
-        x = warp_sum(x);
-        const unsigned long long key = ((unsigned long long)sim_ord(x * vic_rn * s_new_rn) << 32) | (uint32_t)(0x7fffffff - a.t);
-        if (lane == 0 && key > best) { best = key; best_li = n_old; }
-      }
+      for (int c = 0; c < NC; ++c) if (hit == c) { best = cbest[c]; best_li = cbest_li[c]; }
     } else {
-    for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
-        stage_wait(&s_full[slot], ph, &s_timeout);
-        const uint4* st = ring + (size_t)slot * SR * LPR + (size_t)grp * LPR + lig;
-        const bool full = (s + 1) * SR <= n;
-        uint4 raw[4];
-        if (full) {
+      // The victim was not among the guessed rows (or is the new token itself): the keys once more, straight from
+      // global memory, where L2 still holds most of them.  One row per group of LPR lanes.
+      if (tid == 0) atomicAdd(&a.counters[kCntGuessMisses], 1ull);
+      for (int li = grp; li < n_old; li += NGRP) {
+        float f[EPV];
+        Elem<T>::unpack(ld_global_v4(kpool + (row0 + li) * D + lig * EPV), f);
+        float x = 0.f;
 #pragma unroll
-          for (int u = 0; u < 4; ++u) raw[u] = st[(size_t)u * NGRP * LPR];
-        } else {
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-            raw[u] = s * SR + u * NGRP + grp < n ? st[(size_t)u * NGRP * LPR] : make_uint4(0, 0, 0, 0);
-        }
-        float dot[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          float f[EPV];
-          Elem<T>::unpack(raw[u], f);
-          float x = 0.f;
-#pragma unroll
-          for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], f[e], x);
-          dot[u] = x;
-        }
-        // the row whose total this lane receives; its 1/|k| and position leave the stage before the stage is released
-        const int li = s * SR + (lig / QL) * NGRP + grp;
-        const bool mine = li < n && lig % QL == 0 && li != vic_li;
-        float rn_li = s_new_rn; int ps_li = a.t;
-        if (mine && li < n_old) { rn_li = meta_rn[(size_t)slot * SR + (li - s * SR)]; ps_li = meta_ps[(size_t)slot * SR + (li - s * SR)]; }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s_empty[slot]);
-        const float r = reduce4<LPR>(dot[0], dot[1], dot[2], dot[3], lig);
-        if (mine) {                                                    // max similarity, ties -> earliest position
-          const float u = r * vic_rn * rn_li;
-          const unsigned long long key = ((unsigned long long)sim_ord(u) << 32) | (uint32_t)(0x7fffffff - ps_li);
+        for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], f[e], x);
+        x = group_sum<LPR>(x, gmask);
+        if (lig == 0 && li != vic_li) {                              // max similarity, ties -> earliest position
+          const unsigned long long key = ((unsigned long long)sim_ord(x * vic_rn * a.rnorm[row0 + li]) << 32) |
+                                         (uint32_t)(0x7fffffff - a.pos[row0 + li]);
           if (key > best) { best = key; best_li = li; }
         }
+      }
+      if (grp == 0 && vic_li != n_old) {                             // the new token as a merge target
+        float f[EPV];
+        Elem<T>::unpack(knew, f);
+        float x = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], f[e], x);
+        x = group_sum<LPR>(x, gmask);
+        const unsigned long long key = ((unsigned long long)sim_ord(x * vic_rn * s_new_rn) << 32) | (uint32_t)(0x7fffffff - a.t);
+        if (lig == 0 && key > best) { best = key; best_li = n_old; }
       }
     }
     block_arg_extreme<false, CW>(best, best_li, s_key, s_li, &s_best_key, &s_best_li);
@@ -930,7 +1047,10 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
           for (int g = 0; g < G; ++g) {
             const float p = pl[(size_t)g * a.row_cap + lbase + u * NGRP];
 #pragma unroll
-            for (int e = 0; e < EPV; ++e) acc[g][e] = fmaf(p, f[e], acc[g][e]);
+            for (int e = 0; e < EPV; e += 2) {
+              const float2 r = ffma2(make_float2(p, p), make_float2(f[e], f[e + 1]), make_float2(acc[g][e], acc[g][e + 1]));
+              acc[g][e] = r.x; acc[g][e + 1] = r.y;
+            }
           }
         }
       } else {
@@ -947,7 +1067,10 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
             for (int g = 0; g < G; ++g) {
               const float p = pl_get(g, li);
 #pragma unroll
-              for (int e = 0; e < EPV; ++e) acc[g][e] = fmaf(p, f[e], acc[g][e]);
+              for (int e = 0; e < EPV; e += 2) {
+                const float2 r = ffma2(make_float2(p, p), make_float2(f[e], f[e + 1]), make_float2(acc[g][e], acc[g][e + 1]));
+                acc[g][e] = r.x; acc[g][e + 1] = r.y;
+              }
             }
           }
         }

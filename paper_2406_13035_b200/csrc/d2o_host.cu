@@ -376,6 +376,7 @@ extern "C" d2o_status d2o_get_stats(d2o_ctx* c, d2o_stats* out, void* stream) {
   out->error_word = word[0];
   out->error_detail = word[1];
   out->decode_launches = c->decode_launches;
+  out->guess_misses = cnt[kCntGuessMisses];
   return D2O_OK;
 }
 

@@ -149,7 +149,7 @@ def test_zero_norm_keys(name):
     # a zero key has similarity 0 to everything: as an evicted prompt token, as a retained one (window), as the
     # key of a generated token, and as the victim of a later step
     base = W.CONFIGS["cfg0"] if name == "cfg0" else W.twin(name)
-    wl = dataclasses.replace(base, prompt_len=256, decode_steps=10, n_layers=min(base.n_layers, 2))
+    wl = dataclasses.replace(base, prompt_len=256, decode_steps=10, n_layers=min(base.n_layers, 2), max_budget=0)
 
     def prompt_hook(l, Q, K, V):
         K = K.clone()
