@@ -137,10 +137,10 @@ def workload_string(wl: W.Workload, nd: int) -> str:
 
 def algorithmic_decode_bytes(wl: W.Workload, rows_held: float) -> float:
     """Bytes one decode step over all layers must move: K_c and V_c rows once, per-row score/pos/norm read (12 B)
-    and score write (4 B), q/k/v in and out once.  `rows_held` = cache rows per KV head summed over (sequence,
-    layer)."""
+    and score write (4 B), q/k/v in and out once.  `rows_held` = cache rows summed over (sequence, layer, KV
+    head)."""
     e = 4 if wl.dtype == "f32" else 2
-    rows = float(rows_held) * wl.n_kv_heads
+    rows = float(rows_held)
     per_row = 2 * wl.d_head * e + 16
     io = wl.n_layers * wl.batch * (2 * wl.n_q_heads + 2 * wl.n_kv_heads) * wl.d_head * e
     return rows * per_row + io
@@ -184,10 +184,11 @@ def kernels_per_pass(wl: W.Workload) -> int:
 
 
 def roofline_of_decode(wl, budgets, nd, decode_ms, launches_per_step, peaks):
+    """`budgets`: host int tensor [B, L, Hkv]."""
     P = wl.prompt_len
     rows = 0.0
     for s in range(nd):
-        rows += float(torch.clamp(budgets.double(), max=P + s).sum())          # rows held before step s
+        rows += float(torch.clamp(budgets.double(), max=P + s).sum())          # cache rows held before step s
     bytes_per_step = algorithmic_decode_bytes(wl, rows / nd)
     step_ms = decode_ms / nd
     peak = float(peaks.get("hbm_gbs", 6650.0))
@@ -376,8 +377,8 @@ def tensor_phase_rates(wl, budgets, stats_ms, compress_ms, peaks):
         return None
     P, L = wl.prompt_len, wl.n_layers
     tpeak = float(peaks.get("bf16_tflops_sustained", 1400.0))
-    Le = P - budgets.double()                                     # evicted rows per (sequence, layer)
-    sim_flops = float((2.0 * Le * budgets.double() * wl.d_head).sum()) * wl.n_kv_heads
+    Le = P - budgets.double()                                     # evicted rows per (sequence, layer, KV head)
+    sim_flops = float((2.0 * Le * budgets.double() * wl.d_head).sum())
     attn_flops = 2.0 * wl.batch * wl.n_q_heads * L * float(P) * P * wl.d_head      # two causal sweeps of P^2 d
     return [
         {"phase": "d2o_layer_stats (attn_tc_kernel x 2 sweeps + density)", "bound": "tensor",

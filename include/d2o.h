@@ -71,20 +71,31 @@ typedef struct {
   int32_t head_reduce;     /* layer weight w_l from the per-head densities: 0: sum_h exp(-F_lh/gamma)
                             * (Appendix A.5); 1: exp(-mean_h F_lh/gamma); reciprocal-of-variance allocation of
                             * the ablation (Section 5.4, setting 2): 2: sum_h 1/F_lh; 3: 1/mean_h F_lh          */
+  int32_t budget_rule;     /* 0: one size per layer, Eq. 5 with the weights of head_reduce;
+                            * 1: one size per (layer, KV head), S_l^h = alpha_l^h * S_total of Appendix A.5, the
+                            *    weight of a KV head being the sum of exp(-F/gamma) over its query heads and
+                            *    S_total = round(rho * L * Hkv * L_prompt) (head_reduce is ignored);
+                            * 2: "exponential decay allocation" of the ablation (Section 5.4, setting 3):
+                            *    S_l = round(mean_h exp(-F_lh/gamma) * L_prompt), clamped; the total is not fixed,
+                            *    rho is ignored and the cache pool is sized for n_layers * max_budget rows    */
+  int32_t sim_feature;     /* rows the similarity of Eq. 9 is computed on: 0: keys (the method); 1: values (the
+                            * ablation's "Feature choice" row V)                                                  */
+  int32_t merge_policy;    /* 0: similarity-weighted merge (Eq. 11-12); 1: average merge (ablation "Merge policy"):
+                            * a kept token and the tokens merged into it weigh the same                           */
 } d2o_config;
 
 typedef struct d2o_ctx d2o_ctx;
 
 /* Device pointers into `state` for inspection / checkpointing.  Per-layer fields refer to the
  * layer passed to d2o_get_view().  The cache rows of slice (b, layer, h) are
- * [row_off[b, layer] + h * stride, ... + len), stride = S_l rounded up to a multiple of 8.
- * All DEVICE. */
+ * [row_off[b, layer, h], ... + len).  With the per-layer budget rules all KV heads of a layer have the
+ * same size.  All DEVICE. */
 typedef struct {
   const float*   colsum;     /* [B, Hq, P]   column sums of the prompt attention (Eq. 4)      */
   const double*  density;    /* [B, L, Hq]   F_v per sequence, layer, query head (all layers) */
-  const int32_t* budgets;    /* [B, L]       S_l (all layers)                                  */
-  const int32_t* windows;    /* [B, L]       M_l (all layers)                                  */
-  const int64_t* row_off;    /* [B, L]       first cache row of (b, layer); slice (b,h) starts at row_off + h*roundup8(S_l) */
+  const int32_t* budgets;    /* [B, L, Hkv]  cache size of every slice (all layers)            */
+  const int32_t* windows;    /* [B, L, Hkv]  recent window M of every slice (all layers)       */
+  const int64_t* row_off;    /* [B, L, Hkv]  first cache row of every slice, a multiple of 8   */
   void*          k_cache;    /* base of the K pool, rows of d_head elements (all layers)      */
   void*          v_cache;    /* base of the V pool                                             */
   int32_t*       pos;        /* [rows]       original position of each cache row (pool-wide)  */
@@ -132,19 +143,19 @@ void d2o_destroy(d2o_ctx* ctx);
 d2o_status d2o_layer_stats(d2o_ctx* ctx, int32_t layer, const void* Q, const void* K,
                            const float* lse, void* stream);
 
-/* (1') Eq. 5 / Appendix A.2 once every layer has been fed: S_l for all layers and sequences.
- * Writes budgets_host (HOST int32 [B, L], may be NULL).  Synchronises `stream`: the host
- * needs S_l to lay out the cache.  */
+/* (1') Eq. 5 / Appendix A.2 once every layer has been fed: the cache size of every slice.
+ * Writes budgets_host (HOST int32 [B, L, Hkv], may be NULL).  Synchronises `stream`: the host
+ * needs the sizes to lay out the cache and to plan the decode launches.  */
 d2o_status d2o_layer_budgets(d2o_ctx* ctx, int32_t* budgets_host, void* stream);
 
-/* Eq. 5 as a pure function: density DEVICE double [B, L, H] -> budgets DEVICE int32 [B, L]
- * (and, if not NULL, windows DEVICE int32 [B, L], row offsets DEVICE int64 [B, L]).
- * No context; asynchronous. */
+/* Eq. 5 as a pure function: density DEVICE double [B, L, H] -> budgets DEVICE int32 [B, L, Hkv]
+ * (and, if not NULL, windows DEVICE int32 [B, L, Hkv], row offsets DEVICE int64 [B, L, Hkv]).
+ * budget_rule and head_reduce as in d2o_config.  No context; asynchronous. */
 d2o_status d2o_budgets_from_density(const double* density, int32_t batch, int32_t n_layers,
                                     int32_t n_heads, int32_t n_kv_heads, int32_t prompt_len,
                                     float rho, int32_t min_budget, int32_t max_budget,
-                                    float density_temp, int32_t head_reduce, int32_t n_sink,
-                                    int32_t window, float nm_ratio, int32_t* budgets,
+                                    float density_temp, int32_t head_reduce, int32_t budget_rule,
+                                    int32_t n_sink, int32_t window, float nm_ratio, int32_t* budgets,
                                     int32_t* windows, int64_t* row_off, int32_t* status_word,
                                     void* stream);
 

@@ -203,9 +203,12 @@ def head_budgets(F: np.ndarray, P: int, rho: float, group: int = 1, min_budget: 
     L, H = F.shape
     assert H % group == 0
     Hkv = H // group
-    wq = np.exp(-(F - F.min()) / gamma)                            # [L, H]
-    w = wq.reshape(L, Hkv, group).sum(axis=2).reshape(-1)          # [L * Hkv]
-    S_tot = int(math.floor(rho * L * Hkv * P + 0.5))
+    wq = np.exp(-(F - F.min()) / gamma).reshape(L, Hkv, group)     # [L, Hkv, G]
+    w = np.zeros((L, Hkv))
+    for g in range(group):                                         # query heads of a KV head, in order
+        w = w + wq[:, :, g]
+    w = w.reshape(-1)                                              # [L * Hkv]
+    S_tot = int(math.floor(rho * (L * Hkv) * P + 0.5))
     cap = max_budget if max_budget > 0 else P
     return allocate_budgets(w, S_tot, min_budget, cap).reshape(L, Hkv)
 
@@ -221,7 +224,11 @@ def exp_decay_budgets(F: np.ndarray, P: int, min_budget: int = 1, gamma: float =
     F = np.asarray(F, dtype=np.float64)
     if F.ndim == 1:
         F = F[:, None]
-    alpha = np.exp(-F / gamma).sum(axis=1) / F.shape[1]
+    e = np.exp(-F / gamma)
+    alpha = np.zeros(F.shape[0])
+    for h in range(F.shape[1]):                                    # query heads in order
+        alpha = alpha + e[:, h]
+    alpha = alpha / F.shape[1]
     cap = max_budget if max_budget > 0 else P
     S = np.floor(alpha * P + 0.5).astype(np.int64)
     return np.clip(S, min_budget, cap)

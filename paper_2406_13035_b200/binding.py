@@ -36,7 +36,8 @@ class D2OConfig(C.Structure):
                 ("prompt_len", C.c_int32), ("max_new_tokens", C.c_int32), ("rho", C.c_float),
                 ("n_sink", C.c_int32), ("window", C.c_int32), ("nm_ratio", C.c_float), ("beta", C.c_float),
                 ("tau_override", C.c_float), ("density_temp", C.c_float), ("min_budget", C.c_int32),
-                ("max_budget", C.c_int32), ("head_reduce", C.c_int32)]
+                ("max_budget", C.c_int32), ("head_reduce", C.c_int32), ("budget_rule", C.c_int32),
+                ("sim_feature", C.c_int32), ("merge_policy", C.c_int32)]
 
 
 class D2OView(C.Structure):
@@ -82,7 +83,7 @@ def load_library() -> C.CDLL:
     lib.d2o_destroy.restype = None
     lib.d2o_layer_stats.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.d2o_layer_budgets.argtypes = [vp, vp, vp]
-    lib.d2o_budgets_from_density.argtypes = [vp, i32, i32, i32, i32, i32, f32, i32, i32, f32, i32, i32, i32, f32,
+    lib.d2o_budgets_from_density.argtypes = [vp, i32, i32, i32, i32, i32, f32, i32, i32, f32, i32, i32, i32, i32, f32,
                                              vp, vp, vp, vp, vp]
     lib.d2o_prefill_compress.argtypes = [vp, i32, vp, vp, vp]
     lib.d2o_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
@@ -126,10 +127,10 @@ def f32(x: float) -> float:
 
 def make_config(*, n_layers, batch, n_q_heads, n_kv_heads, d_head, dtype, prompt_len, max_new_tokens, rho,
                 n_sink=1, window=0, nm_ratio=3.0, beta=0.7, tau_override=float("nan"), density_temp=1.0,
-                min_budget=8, max_budget=0, head_reduce=0) -> D2OConfig:
+                min_budget=8, max_budget=0, head_reduce=0, budget_rule=0, sim_feature=0, merge_policy=0) -> D2OConfig:
     return D2OConfig(n_layers, batch, n_q_heads, n_kv_heads, d_head, DTYPE_CODE[dtype], prompt_len, max_new_tokens,
                      rho, n_sink, window, nm_ratio, beta, tau_override, density_temp, min_budget, max_budget,
-                     head_reduce)
+                     head_reduce, budget_rule, sim_feature, merge_policy)
 
 
 def d2o_workspace_size(cfg: D2OConfig):
@@ -175,7 +176,7 @@ class D2OContext:
         _check(self.lib.d2o_layer_stats(self.handle, layer, _ptr(Q), _ptr(K), _ptr(lse), _stream()), "d2o_layer_stats")
 
     def d2o_layer_budgets(self) -> torch.Tensor:
-        out = torch.empty(self.cfg.batch, self.cfg.n_layers, dtype=torch.int32)
+        out = torch.empty(self.cfg.batch, self.cfg.n_layers, self.cfg.n_kv_heads, dtype=torch.int32)
         _check(self.lib.d2o_layer_budgets(self.handle, out.data_ptr(), _stream()), "d2o_layer_budgets")
         self.budgets_host = out
         return out
@@ -232,13 +233,14 @@ class D2OContext:
                           (c.batch, c.n_layers, c.n_q_heads))
 
     def tables(self):
-        """(budgets [B,L], windows [B,L], row_off [B,L]) as host tensors."""
+        """(budgets, windows, row_off), each [B, L, Hkv], as host tensors."""
         c = self.cfg
         v = self._view(0)
-        n = c.batch * c.n_layers
-        b = self._wrap(v.budgets, n * 4, torch.int32, (c.batch, c.n_layers)).cpu()
-        w = self._wrap(v.windows, n * 4, torch.int32, (c.batch, c.n_layers)).cpu()
-        o = self._wrap(v.row_off, n * 8, torch.int64, (c.batch, c.n_layers)).cpu()
+        shape = (c.batch, c.n_layers, c.n_kv_heads)
+        n = c.batch * c.n_layers * c.n_kv_heads
+        b = self._wrap(v.budgets, n * 4, torch.int32, shape).cpu()
+        w = self._wrap(v.windows, n * 4, torch.int32, shape).cpu()
+        o = self._wrap(v.row_off, n * 8, torch.int64, shape).cpu()
         return b, w, o
 
     def slice_state(self, layer: int, b: int, h: int, tables=None):
@@ -246,8 +248,8 @@ class D2OContext:
         c = self.cfg
         v = self._view(layer)
         bud, win, off = tables if tables is not None else self.tables()
-        S = int(bud[b, layer])
-        r0 = int(off[b, layer]) + h * ((S + 7) // 8 * 8)      # slices start at multiples of 8 rows
+        S = int(bud[b, layer, h])
+        r0 = int(off[b, layer, h])
         esz = 4 if c.dtype == D2O_F32 else 2
         rows = v.pool_rows
         sidx = (layer * c.batch + b) * c.n_kv_heads + h
@@ -259,7 +261,7 @@ class D2OContext:
         rnorm = self._wrap(v.rnorm, rows * 4, torch.float32, (rows,))[r0:r0 + ln].cpu()
         K = self._wrap(v.k_cache, rows * c.d_head * esz, self.tdtype, (rows, c.d_head))[r0:r0 + ln].cpu()
         V = self._wrap(v.v_cache, rows * c.d_head * esz, self.tdtype, (rows, c.d_head))[r0:r0 + ln].cpu()
-        return dict(pos=pos, score=score, rnorm=rnorm, K=K, V=V, len=ln, tau=tau, S=S, M=int(win[b, layer]))
+        return dict(pos=pos, score=score, rnorm=rnorm, K=K, V=V, len=ln, tau=tau, S=S, M=int(win[b, layer, h]))
 
     def evict_lists(self, b: int, h: int, Le: int):
         """Scratch of the layer compressed last: evicted positions, Max(U[i,:]) and Argmax slot."""
@@ -275,17 +277,17 @@ class D2OContext:
 
 def d2o_budgets_from_density(density: torch.Tensor, *, n_kv_heads: int, prompt_len: int, rho: float,
                              min_budget: int, max_budget: int = 0, density_temp: float = 1.0, head_reduce: int = 0,
-                             n_sink: int = 1, window: int = 0, nm_ratio: float = 3.0):
-    """density: CUDA float64 [B, L, H] -> (budgets, windows, row_off) CUDA tensors [B, L]."""
+                             budget_rule: int = 0, n_sink: int = 1, window: int = 0, nm_ratio: float = 3.0):
+    """density: CUDA float64 [B, L, H] -> (budgets, windows, row_off) CUDA tensors [B, L, Hkv]."""
     lib = load_library()
     B, L, H = density.shape
     dev = density.device
-    budgets = torch.zeros(B, L, dtype=torch.int32, device=dev)
-    windows = torch.zeros(B, L, dtype=torch.int32, device=dev)
-    row_off = torch.zeros(B, L, dtype=torch.int64, device=dev)
+    budgets = torch.zeros(B, L, n_kv_heads, dtype=torch.int32, device=dev)
+    windows = torch.zeros(B, L, n_kv_heads, dtype=torch.int32, device=dev)
+    row_off = torch.zeros(B, L, n_kv_heads, dtype=torch.int64, device=dev)
     status = torch.zeros(4, dtype=torch.int32, device=dev)
     _check(lib.d2o_budgets_from_density(_ptr(density), B, L, H, n_kv_heads, prompt_len, rho, min_budget, max_budget,
-                                        density_temp, head_reduce, n_sink, window, nm_ratio, _ptr(budgets),
+                                        density_temp, head_reduce, budget_rule, n_sink, window, nm_ratio, _ptr(budgets),
                                         _ptr(windows), _ptr(row_off), _ptr(status), _stream()),
            "d2o_budgets_from_density")
     return budgets, windows, row_off, status

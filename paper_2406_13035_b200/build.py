@@ -29,7 +29,10 @@ def _stale(out: str, deps) -> bool:
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compiles every .cu file to an object (in _build/) and links libd2o.so next to this file."""
+    """Compiles every .cu file to an object (in _build/) and links libd2o.so next to this file.
+    With D2O_SKIP_BUILD=1 in the environment an existing libd2o.so is used as it is."""
+    if os.environ.get("D2O_SKIP_BUILD") == "1" and os.path.exists(LIB) and not force:
+        return LIB
     nvcc = _nvcc()
     bdir = os.path.join(HERE, "_build")
     os.makedirs(bdir, exist_ok=True)

@@ -122,6 +122,9 @@ __device__ __forceinline__ float ord_float(uint32_t o) {
 // per-row arrays (pos, score, rnorm) of a slice start on a 32-byte boundary (bulk copies need 16).
 __host__ __device__ __forceinline__ int slice_stride(int S) { return (S + 7) & ~7; }
 
+// index of slice (sequence b, layer, KV head h) in the [B, L, Hkv] tables (budgets, windows, row offsets)
+__host__ __device__ __forceinline__ int slice_entry(int b, int layer, int h, int L, int Hkv) { return (b * L + layer) * Hkv + h; }
+
 // device-side anomaly report: first writer wins
 __device__ __forceinline__ void report_error(uint32_t* status_word, uint32_t code, uint32_t detail) {
   if (atomicCAS(status_word, 0u, code) == 0u) status_word[1] = detail;
@@ -156,9 +159,11 @@ struct d2o_ctx {
   size_t state_bytes, scratch_bytes;
   // host mirrors, valid after d2o_layer_budgets
   bool have_budgets;
-  int32_t* h_budgets;          // [B, L]
-  int32_t* h_windows;          // [B, L]
-  int64_t* h_row_off;          // [B, L]
+  int32_t* h_budgets;          // [B, L, Hkv]
+  int32_t* h_windows;          // [B, L, Hkv]
+  int64_t* h_row_off;          // [B, L, Hkv]
+  int32_t* h_pair_max;         // [B, L] largest cache size over the KV heads of the pair
+  int64_t* h_pair_sum;         // [B, L] cache sizes summed over the KV heads of the pair
   uint8_t* layer_fed;          // [L] stats seen
   uint8_t* layer_compressed;   // [L]
   int32_t* layer_steps;        // [L] decode steps taken
@@ -179,8 +184,8 @@ namespace d2o {
 cudaError_t launch_layer_stats(const d2o_ctx* c, int layer, const void* Q, const void* K, const float* lse,
                                cudaStream_t st);
 cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, int P, float rho, int min_budget,
-                           int max_budget, float gamma, int head_reduce, int n_sink, int window, float nm_ratio,
-                           int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
+                           int max_budget, float gamma, int head_reduce, int budget_rule, int n_sink, int window,
+                           float nm_ratio, int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
                            cudaStream_t st);
 cudaError_t launch_prefill_compress(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st);
 cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const void* k, const void* v, void* out,

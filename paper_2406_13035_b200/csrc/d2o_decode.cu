@@ -59,6 +59,7 @@ struct DecodeArgs {
   int l2_hints;                     // 1: pass K asks L2 to keep its lines, later passes to drop theirs
   const int32_t* order;             // NULL: CTAs take (layer, b, h) in index order; else (layer * B + b) per group of Hkv CTAs
   int pair_base;                    // first entry of `order` this launch works on
+  int average;                      // 1: average merge (both rows weigh 1/2) instead of the weights of Eq. 12
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -313,9 +314,9 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   const T* v_new = v_in + (size_t)sl * D;
 
   // ---- slice parameters
-  const int S = a.budgets[b * a.L + layer];
-  const int M = a.windows[b * a.L + layer];
-  const int64_t row0 = a.row_off[b * a.L + layer] + (int64_t)h * slice_stride(S);
+  const int S = a.budgets[slice_entry(b, layer, h, a.L, a.Hkv)];
+  const int M = a.windows[slice_entry(b, layer, h, a.L, a.Hkv)];
+  const int64_t row0 = a.row_off[slice_entry(b, layer, h, a.L, a.Hkv)];
   const int sidx = (layer * a.B + b) * a.Hkv + h;
   const int n_old = a.len[sidx];
   const float tau_old = a.tau[sidx];
@@ -885,7 +886,8 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     merge = mx >= thr;
     nn_is_new = (nn_li == n_old);
     const float ew = expf(mx);
-    w_e = ew / (ew + kEuler); w_c = kEuler / (ew + kEuler);
+    w_e = a.average ? 0.5f : ew / (ew + kEuler);
+    w_c = a.average ? 0.5f : kEuler / (ew + kEuler);
     if (tid == 0) {
       a.tau[sidx] = tau_new;
       atomicAdd(&a.counters[kCntDecodeSteps], 1ull);
@@ -1240,28 +1242,29 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   a.counters = (unsigned long long*)(S + c->lay.counters); a.status = (uint32_t*)(S + c->lay.status);
   a.L = L; a.l0 = l0; a.B = B; a.Hkv = g.n_kv_heads; a.T = g.n_sink;
   a.t = g.prompt_len + c->layer_steps[l0];
-  a.beta = g.beta; a.tau_override = g.tau_override;
+  a.beta = g.beta; a.tau_override = g.tau_override; a.average = g.merge_policy;
   a.l2_hints = c->decode_l2_hints;
   const int G = c->group, Hkv = g.n_kv_heads;
   const int row_bytes = g.d_head * c->elem_size;
   void* kpool = S + c->lay.kpool; void* vpool = S + c->lay.vpool;
+  // rows of the longest slice of a pair, and the mean over all slices (a cache cannot hold more than was generated)
+  const int t_now = g.prompt_len + c->layer_steps[l0];
   int max_rows = 0;
-  long long sum_rows = 0;
+  double sum_rows = 0.0;
   for (int l = l0; l < l1; ++l)
     for (int b = 0; b < B; ++b) {
-      const int r = min(c->h_budgets[b * L + l], g.prompt_len + c->layer_steps[l0]) + 1;
-      max_rows = max(max_rows, r);
-      sum_rows += r;
+      max_rows = max(max_rows, min(c->h_pair_max[b * L + l], t_now) + 1);
+      sum_rows += (double)min((long long)c->h_pair_sum[b * L + l], (long long)t_now * g.n_kv_heads) / g.n_kv_heads + 1.0;
     }
   // all layers in one call: CTAs take the slices largest cache first, so the long ones do not end up in the tail
   const bool ordered = (l0 == 0 && l1 == L);
   a.order = ordered ? (const int32_t*)(S + c->lay.order) : nullptr;
   a.spill = (float*)(c->scratch + c->slay.pl_spill);
   const int n_pairs = (l1 - l0) * B;
-  const double mean_rows = (double)sum_rows / n_pairs;
-  auto rows_of_pair = [&](int i) {                                    // i-th pair in launch order
+  const double mean_rows = sum_rows / n_pairs;
+  auto rows_of_pair = [&](int i) {                                    // i-th pair in launch order: its longest slice
     const int pr = ordered ? c->h_order[i] : (l0 * B + i);
-    return min(c->h_budgets[(pr % B) * L + pr / B], g.prompt_len + c->layer_steps[l0]) + 1;
+    return min(c->h_pair_max[(pr % B) * L + pr / B], t_now) + 1;
   };
 
   // A step takes at least as long as its longest slice takes in one CTA.  Where that is more than the whole step

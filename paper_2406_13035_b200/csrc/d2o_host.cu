@@ -60,11 +60,28 @@ static d2o_status validate(const d2o_config* c, int64_t* total_budget, int* max_
   if (!(c->beta >= 0.0f && c->beta <= 1.0f)) return D2O_ERR_INVALID_ARG;
   if (!(c->density_temp > 0.0f) || !isfinite(c->density_temp)) return D2O_ERR_INVALID_ARG;
   if (c->head_reduce < 0 || c->head_reduce > 3) return D2O_ERR_UNSUPPORTED;
+  if (c->budget_rule < 0 || c->budget_rule > 2) return D2O_ERR_UNSUPPORTED;
+  if (c->sim_feature < 0 || c->sim_feature > 1 || c->merge_policy < 0 || c->merge_policy > 1) return D2O_ERR_UNSUPPORTED;
+  // the value-feature ablation is built for the prompt stage; the decode kernel computes its cosines on the keys
+  if (c->sim_feature == 1 && c->max_new_tokens > 0) return D2O_ERR_UNSUPPORTED;
   int maxb = c->max_budget > 0 ? c->max_budget : c->prompt_len;
   if (maxb > c->prompt_len + c->max_new_tokens) return D2O_ERR_INVALID_ARG;
   if (c->min_budget < 1 || c->min_budget < c->n_sink + 1 || c->min_budget > maxb) return D2O_ERR_INVALID_ARG;
+  // cache rows per KV head and sequence, summed over the layers: fixed by rho (rules 0 and 1), or bounded by the
+  // upper clamp (rule 2, whose total depends on the densities)
   double tot = floor((double)c->rho * (double)c->n_layers * (double)c->prompt_len + 0.5);
-  if (tot < (double)c->n_layers * c->min_budget || tot > (double)c->n_layers * maxb) return D2O_ERR_INVALID_ARG;
+  if (c->budget_rule == 1) {
+    // per-head sizes add up to round(rho * L * Hkv * P) per sequence; per KV head that is at most this many rows more
+    // than the mean, so the pool is sized by the total over heads (see layouts)
+    tot = floor((double)c->rho * ((double)c->n_layers * c->n_kv_heads) * (double)c->prompt_len + 0.5);
+    if (tot < (double)c->n_layers * c->n_kv_heads * c->min_budget || tot > (double)c->n_layers * c->n_kv_heads * maxb)
+      return D2O_ERR_INVALID_ARG;
+    if ((size_t)c->n_layers * c->n_kv_heads > 4096) return D2O_ERR_UNSUPPORTED;   // work arrays of the budget kernel
+  } else if (c->budget_rule == 2) {
+    tot = (double)c->n_layers * maxb;
+  } else if (tot < (double)c->n_layers * c->min_budget || tot > (double)c->n_layers * maxb) {
+    return D2O_ERR_INVALID_ARG;
+  }
   // the prompt-stage segment kernel keeps one counter per retained row of a slice in shared memory
   if (maxb + 1 > kMaxSliceRows) return D2O_ERR_UNSUPPORTED;
   *total_budget = (int64_t)tot;
@@ -75,15 +92,18 @@ static d2o_status validate(const d2o_config* c, int64_t* total_budget, int* max_
 static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, Layout* l, ScratchLayout* s) {
   const size_t B = c->batch, L = c->n_layers, Hq = c->n_q_heads, Hkv = c->n_kv_heads, P = c->prompt_len;
   const size_t d = c->d_head, e = elem_size_of(c->dtype);
-  const size_t rows = B * Hkv * ((size_t)total_budget + 7 * L);     // every slice starts at a multiple of 8 rows
+  // every slice starts at a multiple of 8 rows; total_budget counts rows per KV head (per-layer rules) or over all KV
+  // heads (per-head rule) of one sequence
+  const size_t rows = c->budget_rule == 1 ? B * ((size_t)total_budget + 7 * L * Hkv)
+                                          : B * Hkv * ((size_t)total_budget + 7 * L);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
   l->status = take(16);
   l->counters = take(kNumCounters * 8);
   l->density = take(B * L * Hq * 8);
-  l->budgets = take(B * L * 4);
-  l->windows = take(B * L * 4);
-  l->row_off = take(B * L * 8);
+  l->budgets = take(B * L * Hkv * 4);
+  l->windows = take(B * L * Hkv * 4);
+  l->row_off = take(B * L * Hkv * 8);
   l->order = take(B * L * 4);
   l->len = take(L * B * Hkv * 4);
   l->tau = take(L * B * Hkv * 4);
@@ -140,7 +160,9 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
   c->elem_size = elem_size_of(cfg->dtype);
   c->max_budget = maxb;
   c->total_budget = tot;
-  c->pool_rows = (int64_t)cfg->batch * cfg->n_kv_heads * (tot + 7 * (int64_t)cfg->n_layers);
+  c->pool_rows = cfg->budget_rule == 1
+      ? (int64_t)cfg->batch * (tot + 7 * (int64_t)cfg->n_layers * cfg->n_kv_heads)
+      : (int64_t)cfg->batch * cfg->n_kv_heads * (tot + 7 * (int64_t)cfg->n_layers);
   c->lay = l; c->slay = s;
   c->decode_l2_hints = 1;
   {
@@ -156,9 +178,12 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
   c->state = (char*)state; c->scratch = (char*)scratch;
   c->state_bytes = state_bytes; c->scratch_bytes = scratch_bytes;
   const size_t BL = (size_t)cfg->batch * cfg->n_layers;
-  c->h_budgets = (int32_t*)calloc(BL, 4);
-  c->h_windows = (int32_t*)calloc(BL, 4);
-  c->h_row_off = (int64_t*)calloc(BL, 8);
+  const size_t BLH = BL * cfg->n_kv_heads;
+  c->h_budgets = (int32_t*)calloc(BLH, 4);
+  c->h_windows = (int32_t*)calloc(BLH, 4);
+  c->h_row_off = (int64_t*)calloc(BLH, 8);
+  c->h_pair_max = (int32_t*)calloc(BL, 4);
+  c->h_pair_sum = (int64_t*)calloc(BL, 8);
   c->layer_fed = (uint8_t*)calloc(cfg->n_layers, 1);
   c->layer_compressed = (uint8_t*)calloc(cfg->n_layers, 1);
   c->layer_steps = (int32_t*)calloc(cfg->n_layers, 4);
@@ -172,7 +197,7 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
 
 extern "C" void d2o_destroy(d2o_ctx* c) {
   if (!c) return;
-  free(c->h_budgets); free(c->h_windows); free(c->h_row_off);
+  free(c->h_budgets); free(c->h_windows); free(c->h_row_off); free(c->h_pair_max); free(c->h_pair_sum);
   free(c->layer_fed); free(c->layer_compressed); free(c->layer_steps); free(c->h_order);
   free(c);
 }
@@ -191,19 +216,22 @@ extern "C" d2o_status d2o_layer_stats(d2o_ctx* c, int32_t layer, const void* Q, 
 extern "C" d2o_status d2o_budgets_from_density(const double* density, int32_t batch, int32_t n_layers,
                                                int32_t n_heads, int32_t n_kv_heads, int32_t prompt_len, float rho,
                                                int32_t min_budget, int32_t max_budget, float density_temp,
-                                               int32_t head_reduce, int32_t n_sink, int32_t window, float nm_ratio,
-                                               int32_t* budgets, int32_t* windows, int64_t* row_off,
-                                               int32_t* status_word, void* stream) {
+                                               int32_t head_reduce, int32_t budget_rule, int32_t n_sink,
+                                               int32_t window, float nm_ratio, int32_t* budgets, int32_t* windows,
+                                               int64_t* row_off, int32_t* status_word, void* stream) {
   if (!density || !budgets || batch < 1 || n_layers < 1 || n_layers > 1024 || n_heads < 1 || n_kv_heads < 1 ||
-      prompt_len < 1)
+      prompt_len < 1 || n_heads % n_kv_heads != 0)
     return D2O_ERR_INVALID_ARG;
   if (!(rho > 0.0f) || !(density_temp > 0.0f) || head_reduce < 0 || head_reduce > 3) return D2O_ERR_INVALID_ARG;
+  if (budget_rule < 0 || budget_rule > 2) return D2O_ERR_INVALID_ARG;
   if (max_budget <= 0) max_budget = prompt_len;
   if (min_budget < 1 || min_budget > max_budget) return D2O_ERR_INVALID_ARG;
-  double tot = floor((double)rho * n_layers * prompt_len + 0.5);
-  if (tot < (double)n_layers * min_budget || tot > (double)n_layers * max_budget) return D2O_ERR_INVALID_ARG;
+  const double units = budget_rule == 1 ? (double)n_layers * n_kv_heads : (double)n_layers;
+  if (units > 4096) return D2O_ERR_UNSUPPORTED;
+  double tot = floor((double)rho * units * prompt_len + 0.5);
+  if (budget_rule != 2 && (tot < units * min_budget || tot > units * max_budget)) return D2O_ERR_INVALID_ARG;
   CUDA_TRY(launch_budgets(density, batch, n_layers, n_heads, n_kv_heads, prompt_len, rho, min_budget, max_budget,
-                          density_temp, head_reduce, n_sink, window, nm_ratio, budgets, windows, row_off,
+                          density_temp, head_reduce, budget_rule, n_sink, window, nm_ratio, budgets, windows, row_off,
                           (uint32_t*)status_word, (cudaStream_t)stream));
   return D2O_OK;
 }
@@ -219,24 +247,31 @@ extern "C" d2o_status d2o_layer_budgets(d2o_ctx* c, int32_t* budgets_host, void*
   int64_t* d_o = (int64_t*)(c->state + c->lay.row_off);
   CUDA_TRY(launch_budgets((const double*)(c->state + c->lay.density), g.batch, g.n_layers, g.n_q_heads,
                           g.n_kv_heads, g.prompt_len, g.rho, g.min_budget, c->max_budget, g.density_temp,
-                          g.head_reduce, g.n_sink, g.window, g.nm_ratio, d_b, d_w, d_o,
+                          g.head_reduce, g.budget_rule, g.n_sink, g.window, g.nm_ratio, d_b, d_w, d_o,
                           (uint32_t*)(c->state + c->lay.status), st));
   const size_t BL = (size_t)g.batch * g.n_layers;
-  CUDA_TRY(cudaMemcpyAsync(c->h_budgets, d_b, BL * 4, cudaMemcpyDeviceToHost, st));
-  CUDA_TRY(cudaMemcpyAsync(c->h_windows, d_w, BL * 4, cudaMemcpyDeviceToHost, st));
-  CUDA_TRY(cudaMemcpyAsync(c->h_row_off, d_o, BL * 8, cudaMemcpyDeviceToHost, st));
+  const size_t Hkv = g.n_kv_heads, BLH = BL * Hkv;
+  CUDA_TRY(cudaMemcpyAsync(c->h_budgets, d_b, BLH * 4, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaMemcpyAsync(c->h_windows, d_w, BLH * 4, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaMemcpyAsync(c->h_row_off, d_o, BLH * 8, cudaMemcpyDeviceToHost, st));
   CUDA_TRY(cudaStreamSynchronize(st));
   // the device computed offsets for the pool; make sure they fit what the caller gave us
-  for (size_t i = 0; i < BL; ++i) {
-    int64_t end = c->h_row_off[i] + (int64_t)g.n_kv_heads * slice_stride(c->h_budgets[i]);
+  for (size_t i = 0; i < BLH; ++i) {
+    int64_t end = c->h_row_off[i] + (int64_t)slice_stride(c->h_budgets[i]);
     if (c->h_budgets[i] < 1 || c->h_budgets[i] > c->max_budget || c->h_row_off[i] < 0 || end > c->pool_rows)
       return D2O_ERR_STATE;
+  }
+  // largest and summed cache size over the KV heads of every (sequence, layer) pair
+  for (size_t i = 0; i < BL; ++i) {
+    int32_t mx = 0; int64_t sm = 0;
+    for (size_t h = 0; h < Hkv; ++h) { mx = std::max(mx, c->h_budgets[i * Hkv + h]); sm += c->h_budgets[i * Hkv + h]; }
+    c->h_pair_max[i] = mx; c->h_pair_sum[i] = sm;
   }
   // (layer, sequence) pairs by cache size, largest first: the decode kernel takes its slices in this order
   for (size_t i = 0; i < BL; ++i) c->h_order[i] = (int32_t)i;                  // i = layer * B + b
   {
     const int Bn = g.batch, Ln = g.n_layers;
-    const int32_t* hb = c->h_budgets;
+    const int32_t* hb = c->h_pair_max;                                           // [B, L]
     std::stable_sort(c->h_order, c->h_order + BL, [=](int32_t x, int32_t y) {
       return hb[(x % Bn) * Ln + x / Bn] > hb[(y % Bn) * Ln + y / Bn];
     });
@@ -244,7 +279,7 @@ extern "C" d2o_status d2o_layer_budgets(d2o_ctx* c, int32_t* budgets_host, void*
   CUDA_TRY(cudaMemcpyAsync(c->state + c->lay.order, c->h_order, BL * 4, cudaMemcpyHostToDevice, st));
   CUDA_TRY(cudaStreamSynchronize(st));
   c->have_budgets = true;
-  if (budgets_host) memcpy(budgets_host, c->h_budgets, BL * 4);
+  if (budgets_host) memcpy(budgets_host, c->h_budgets, BLH * 4);
   return D2O_OK;
 }
 

@@ -33,6 +33,7 @@ struct SelectArgs {
   uint32_t* status;
   int L, layer, B, Hq, Hkv, G, P, T;
   int keys_in_smem;
+  int value_feature;       // 1: the similarity of Eq. 9 is taken on the value rows (ablation), so the norms are theirs
 };
 
 __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* total) {
@@ -69,10 +70,10 @@ select_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
   const int slice = blockIdx.x;                 // b * Hkv + h
   const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int P = a.P;
-  const int S = a.budgets[b * a.L + a.layer];
+  const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int Tn = a.T < S ? a.T : S;
-  const int M = a.windows[b * a.L + a.layer];
-  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
+  const int M = a.windows[slice_entry(b, a.layer, h, a.L, a.Hkv)];
+  const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int sidx = (a.layer * a.B + b) * a.Hkv + h;
   float* keys = a.keys_in_smem ? reinterpret_cast<float*>(sel_smem) : a.keys_spill + (size_t)slice * P;
   // group score: sum over the G query heads of this KV head, fixed order (Eq. 6 case 1)
@@ -159,9 +160,9 @@ gather_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
   const int slice = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int P = a.P;
-  const int S = a.budgets[b * a.L + a.layer];
+  const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int n_keep = S >= P ? P : S;
-  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
+  const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
   const T* Ks = K + (size_t)slice * P * D;
   const T* Vs = V + (size_t)slice * P * D;
@@ -172,7 +173,7 @@ gather_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
     const uint4 vv = ld_global_v4(Vs + (size_t)j * D + lig * EPV);
     *reinterpret_cast<uint4*>(kpool + (row0 + r) * D + lig * EPV) = kv;
     *reinterpret_cast<uint4*>(vpool + (row0 + r) * D + lig * EPV) = vv;
-    float f[EPV]; Elem<T>::unpack(kv, f);
+    float f[EPV]; Elem<T>::unpack(a.value_feature ? vv : kv, f);
     float ss = 0.f;
 #pragma unroll
     for (int i = 0; i < EPV; ++i) ss = fmaf(f[i], f[i], ss);
@@ -202,11 +203,11 @@ similarity_kernel(SimArgs a, const T* __restrict__ K, const T* __restrict__ kpoo
   float* crn = ern + kSimTile;              // [64] inverse norms of the retained rows
   const int slice = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
-  const int S = a.budgets[b * a.L + a.layer];
+  const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int Le = a.P - S;
   const int i0 = blockIdx.x * kSimTile;
   if (Le <= 0 || i0 >= Le) return;
-  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
+  const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const T* Ks = K + (size_t)slice * a.P * D;
   const int32_t* ev = a.evict_idx + (size_t)slice * a.P;
   constexpr int EPV = Elem<T>::kPerVec;
@@ -328,7 +329,7 @@ segment_kernel(SegArgs a) {
   __shared__ int s_total;
   const int slice = blockIdx.x;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
-  const int S = a.budgets[b * a.L + a.layer];
+  const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int Le = a.P - S;
   const int sidx = (a.layer * a.B + b) * a.Hkv + h;
   const float* mx = a.evict_mx + (size_t)slice * a.P;
@@ -453,6 +454,8 @@ struct MergeArgs {
   const int32_t* seg_start; const int32_t* seg_items;
   float* rnorm;
   int L, layer, Hkv, P, seg_stride;
+  int average;             // 1: average merge (every token of a merge weighs the same) instead of Eq. 12
+  int value_feature;       // 1: the cached inverse norms belong to the value rows
 };
 
 template <typename T, int D>
@@ -463,7 +466,7 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   constexpr int LPR = D / EPV;
   const int slice = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
-  const int S = a.budgets[b * a.L + a.layer];
+  const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   if (a.P - S <= 0) return;
   const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
   const int j = blockIdx.x * (blockDim.x / LPR) + grp;
@@ -471,7 +474,7 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   const int32_t* start = a.seg_start + (size_t)slice * a.seg_stride;
   const int s0 = start[j], s1 = start[j + 1];
   if (s1 == s0) return;                              // nothing merged: the row stays bit-identical
-  const int64_t row = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S) + j;
+  const int64_t row = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)] + j;
   const int32_t* items = a.seg_items + (size_t)slice * a.P;
   const int32_t* ev = a.evict_idx + (size_t)slice * a.P;
   const float* mx = a.evict_mx + (size_t)slice * a.P;
@@ -479,15 +482,16 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   const T* Vs = V + (size_t)slice * a.P * D;
   float ka[EPV], va[EPV], f[EPV];
   Elem<T>::unpack(ld_global_v4(kpool + row * D + lig * EPV), f);
+  const float own = a.average ? 1.0f : kEuler;       // weight of the retained token itself: e^{self-similarity}, or 1
 #pragma unroll
-  for (int i = 0; i < EPV; ++i) ka[i] = kEuler * f[i];
+  for (int i = 0; i < EPV; ++i) ka[i] = own * f[i];
   Elem<T>::unpack(ld_global_v4(vpool + row * D + lig * EPV), f);
 #pragma unroll
-  for (int i = 0; i < EPV; ++i) va[i] = kEuler * f[i];
-  float den = kEuler;
+  for (int i = 0; i < EPV; ++i) va[i] = own * f[i];
+  float den = own;
   for (int s = s0; s < s1; ++s) {
     const int i = items[s];
-    const float w = expf(mx[i]);
+    const float w = a.average ? 1.0f : expf(mx[i]);
     const int pj = ev[i];
     den += w;
     Elem<T>::unpack(ld_global_v4(Ks + (size_t)pj * D + lig * EPV), f);
@@ -500,10 +504,10 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   const float inv = 1.0f / den;
 #pragma unroll
   for (int e = 0; e < EPV; ++e) { ka[e] = ka[e] * inv; va[e] = va[e] * inv; }
-  const uint4 kv = Elem<T>::pack(ka);
+  const uint4 kv = Elem<T>::pack(ka), vv = Elem<T>::pack(va);
   *reinterpret_cast<uint4*>(kpool + row * D + lig * EPV) = kv;
-  *reinterpret_cast<uint4*>(vpool + row * D + lig * EPV) = Elem<T>::pack(va);
-  Elem<T>::unpack(kv, f);                            // the norm of what is actually stored
+  *reinterpret_cast<uint4*>(vpool + row * D + lig * EPV) = vv;
+  Elem<T>::unpack(a.value_feature ? vv : kv, f);     // the norm of what is actually stored
   float ss = 0.f;
 #pragma unroll
   for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
@@ -521,7 +525,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   T* kpool = (T*)(S + c->lay.kpool);
   T* vpool = (T*)(S + c->lay.vpool);
   int maxS = 0;
-  for (int b = 0; b < B; ++b) maxS = max(maxS, c->h_budgets[b * L + layer]);
+  for (int b = 0; b < B; ++b) maxS = max(maxS, c->h_pair_max[b * L + layer]);
   const int seg_stride = c->max_budget + 2;
 
   SelectArgs sa;
@@ -538,6 +542,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   sa.L = L; sa.layer = layer; sa.B = B; sa.Hq = g.n_q_heads; sa.Hkv = Hkv; sa.G = c->group; sa.P = P; sa.T = g.n_sink;
   const size_t key_bytes = (size_t)P * sizeof(float);
   sa.keys_in_smem = key_bytes <= 200 * 1024;
+  sa.value_feature = g.sim_feature;
   const size_t sel_sm = sa.keys_in_smem ? key_bytes : 0;
   cudaError_t e = cudaFuncSetAttribute(select_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)(sel_sm > 48 * 1024 ? sel_sm : 48 * 1024));
@@ -550,7 +555,8 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   }
 
   int minS = P;
-  for (int b = 0; b < B; ++b) minS = min(minS, c->h_budgets[b * L + layer]);
+  for (int b = 0; b < B; ++b)
+    for (int h = 0; h < Hkv; ++h) minS = min(minS, c->h_budgets[(b * L + layer) * Hkv + h]);
   const int maxLe = P - minS;
   if (maxLe <= 0) return cudaGetLastError();
 
@@ -561,12 +567,15 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   const size_t sim_sm = ((size_t)2 * D * kSimTile + 2 * kSimTile) * sizeof(float);
   e = cudaFuncSetAttribute(similarity_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sim_sm);
   if (e != cudaSuccess) return e;
+  // rows the similarity is computed on: the keys (Eq. 9), or the values (ablation "Feature choice")
+  const void* feat = g.sim_feature ? V : K;
+  const T* feat_pool = g.sim_feature ? vpool : kpool;
   if (sizeof(T) == 2 && c->similarity_path == 0) {
-    e = launch_similarity_tc(c, layer, K, maxS, st);
+    e = launch_similarity_tc(c, layer, feat, maxS, st);
     if (e != cudaSuccess) return e;
   } else {
     dim3 sgrid((maxLe + kSimTile - 1) / kSimTile, n_slices);
-    similarity_kernel<T, D><<<sgrid, kSimThreads, sim_sm, st>>>(ma, (const T*)K, kpool);
+    similarity_kernel<T, D><<<sgrid, kSimThreads, sim_sm, st>>>(ma, (const T*)feat, feat_pool);
   }
 
   SegArgs ga;
@@ -586,7 +595,8 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   MergeArgs mg;
   mg.budgets = sa.budgets; mg.row_off = sa.row_off; mg.evict_idx = sa.evict_idx; mg.evict_mx = ma.evict_mx;
   mg.seg_start = ga.seg_start; mg.seg_items = ga.seg_items; mg.rnorm = sa.rnorm;
-  mg.L = L; mg.layer = layer; mg.Hkv = Hkv; mg.P = P; mg.seg_stride = seg_stride;
+  mg.L = L; mg.layer = layer; mg.Hkv = Hkv; mg.P = P; mg.seg_stride = seg_stride; mg.average = g.merge_policy;
+  mg.value_feature = g.sim_feature;
   constexpr int LPR = D / Elem<T>::kPerVec;
   const int rows_per_cta = 256 / LPR;
   dim3 mgrid((maxS + rows_per_cta - 1) / rows_per_cta, n_slices);

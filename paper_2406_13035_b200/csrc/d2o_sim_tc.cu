@@ -109,7 +109,7 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
   const int slice = blockIdx.z;
   const int nc = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
-  const int S = a.budgets[b * a.L + a.layer];
+  const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int chunk_cols = chunk_columns(S);                   // the retained rows are split evenly over the chunks
   const int c0 = nc * chunk_cols;                            // first retained slot of the chunk
   if (c0 >= S || a.P - S <= 0) return;                       // uniform for the CTA: nothing to do
@@ -120,7 +120,7 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
   const int t0 = blockIdx.x * a.tiles_per_cta;
   const int t1 = min(n_tiles_all, t0 + a.tiles_per_cta);
   if (t0 >= t1) return;
-  const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
+  const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   if ((tc::smem_u32(tc_smem) & 1023u) != 0u) {               // swizzled tiles need 1024-byte aligned shared memory
     if (tid == 0) report_error(a.status, D2O_ERR_STATE, 0x51C10000u);
     return;
@@ -288,7 +288,7 @@ neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K, const T* __rest
   constexpr int LPR = D / EPV;
   const int slice = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
-  const int S = a.budgets[b * a.L + a.layer];
+  const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int Le = a.P - S;
   const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
   const int i = blockIdx.x * (blockDim.x / LPR) + grp;
@@ -315,7 +315,7 @@ neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K, const T* __rest
     // No chunk reported a non-negative maximum: every similarity of this row is negative (or not finite).  The row
     // is redone here in fp32, all retained rows in slot order (the first maximum stays).  A row without any finite
     // similarity gets maximum -inf and neighbour 0 and is never merged.
-    const int64_t row0 = a.row_off[b * a.L + a.layer] + (int64_t)h * slice_stride(S);
+    const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
     float best = -INFINITY; int bj = 0;
     for (int j = 0; j < S; ++j) {
       float g[EPV];
@@ -379,7 +379,9 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   char* S = c->state; char* X = c->scratch;
   CUtensorMap map_k, map_pool;
   if (!encode_rows_2d(&map_k, g.dtype, K, (uint64_t)n_slices * P, D, kTileM)) return cudaErrorNotSupported;
-  if (!encode_rows_2d(&map_pool, g.dtype, S + c->lay.kpool, (uint64_t)c->pool_rows, D, kBBoxRows)) return cudaErrorNotSupported;
+  // the retained rows of the same kind: K_c, or V_c when the similarity is taken on the values
+  char* pool = S + (g.sim_feature ? c->lay.vpool : c->lay.kpool);
+  if (!encode_rows_2d(&map_pool, g.dtype, pool, (uint64_t)c->pool_rows, D, kBBoxRows)) return cudaErrorNotSupported;
   const int n_chunks_max = (c->max_budget + kChunkN - 1) / kChunkN;
   const int n_chunks = (max_S + kChunkN - 1) / kChunkN;
   const int n_tiles = (P + kTileM - 1) / kTileM;
@@ -426,17 +428,18 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   r.evict_mx = (float*)(X + c->slay.evict_mx); r.evict_nn = (int32_t*)(X + c->slay.evict_nn);
   r.L = g.n_layers; r.layer = layer; r.Hkv = Hkv; r.P = P; r.n_chunks_max = n_chunks_max;
   int minS = P;
-  for (int bb = 0; bb < B; ++bb) minS = min(minS, c->h_budgets[bb * g.n_layers + layer]);
+  for (int bb = 0; bb < B; ++bb)
+    for (int hh = 0; hh < Hkv; ++hh) minS = min(minS, c->h_budgets[(bb * g.n_layers + layer) * Hkv + hh]);
   const int maxLe = P - minS;
   if (maxLe <= 0) return cudaSuccess;
   const int lpr = D * 2 / 16;
   dim3 rgrid((maxLe + 256 / lpr - 1) / (256 / lpr), n_slices);
   if (g.dtype == D2O_F16) {
-    if (D == 128) neighbour_reduce_kernel<__half, 128><<<rgrid, 256, 0, st>>>(r, (const __half*)K, (const __half*)(S + c->lay.kpool));
-    else neighbour_reduce_kernel<__half, 64><<<rgrid, 256, 0, st>>>(r, (const __half*)K, (const __half*)(S + c->lay.kpool));
+    if (D == 128) neighbour_reduce_kernel<__half, 128><<<rgrid, 256, 0, st>>>(r, (const __half*)K, (const __half*)pool);
+    else neighbour_reduce_kernel<__half, 64><<<rgrid, 256, 0, st>>>(r, (const __half*)K, (const __half*)pool);
   } else {
-    if (D == 128) neighbour_reduce_kernel<__nv_bfloat16, 128><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K, (const __nv_bfloat16*)(S + c->lay.kpool));
-    else neighbour_reduce_kernel<__nv_bfloat16, 64><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K, (const __nv_bfloat16*)(S + c->lay.kpool));
+    if (D == 128) neighbour_reduce_kernel<__nv_bfloat16, 128><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K, (const __nv_bfloat16*)pool);
+    else neighbour_reduce_kernel<__nv_bfloat16, 64><<<rgrid, 256, 0, st>>>(r, (const __nv_bfloat16*)K, (const __nv_bfloat16*)pool);
   }
   return cudaGetLastError();
 }

@@ -214,121 +214,159 @@ density_kernel(const float* __restrict__ colsum, double* __restrict__ density, i
   }
 }
 
-// Eq. 5 with S_l = clip(lambda * w_l, S_min, S_max), sum_l S_l = S_tot, then floor + largest remainder.
-// One thread per sequence; per-thread work arrays (w, kinks, x) live in dynamic shared memory.
+// Cache sizes from the densities.  budget_rule 0 (Eq. 5): S_l = clip(lambda * w_l, S_min, S_max) with
+// sum_l S_l = S_tot, then floor + largest remainder; rule 1 (per-head sizes of Appendix A.5): the same over the
+// (layer, KV head) units; rule 2 (exponential-decay allocation of the ablation): S_l = round(mean_h exp(-F/gamma) P),
+// clamped, no fixed total.  One thread per sequence; its work arrays (w, kinks, x) live in dynamic shared memory.
+// Output tables are [B, L, Hkv]; the per-layer rules give every KV head of a layer the same size.
 __device__ inline double clipd(double v, double lo, double hi) { return v < lo ? lo : (v > hi ? hi : v); }
 
 __global__ void budget_kernel(const double* __restrict__ density, int B, int L, int H, int Hkv, int P, double rho,
-                              int min_budget, int max_budget, double gamma, int head_reduce, int n_sink, int window,
-                              double nm_ratio, int32_t* __restrict__ budgets, int32_t* __restrict__ windows,
-                              int64_t* __restrict__ row_off, uint32_t* status_word) {
+                              int min_budget, int max_budget, double gamma, int head_reduce, int budget_rule,
+                              int n_sink, int window, double nm_ratio, int32_t* __restrict__ budgets,
+                              int32_t* __restrict__ windows, int64_t* __restrict__ row_off, uint32_t* status_word) {
   extern __shared__ __align__(16) double dsm[];
-  double* w = dsm + (size_t)threadIdx.x * 4 * L;
-  double* kinks = w + L;        // [2L]
-  double* x = kinks + 2 * L;    // [L]
+  const int n = budget_rule == 1 ? L * Hkv : L;                       // allocation units
+  const int G = H / Hkv;
+  double* w = dsm + (size_t)threadIdx.x * 4 * n;
+  double* kinks = w + n;        // [2n]
+  double* x = kinks + 2 * n;    // [n]
   const double lo = (double)min_budget, hi = (double)max_budget;
-  const long long S_tot = (long long)floor(rho * (double)L * (double)P + 0.5);
+  const long long S_tot = (long long)floor(rho * (double)n * (double)P + 0.5);
   for (int b = threadIdx.x; b < B; b += blockDim.x) {
     const double* F = density + (size_t)b * L * H;
-    if (head_reduce == 0) {
-      double fmin = F[0];
-      for (int i = 1; i < L * H; ++i) fmin = fmin < F[i] ? fmin : F[i];
+    int32_t* bud = budgets + (size_t)b * L * Hkv;
+    // unit u -> its (first) entry of the [L, Hkv] table
+    auto slot_of = [&](int u) { return budget_rule == 1 ? u : u * Hkv; };
+    if (budget_rule == 2) {
       for (int l = 0; l < L; ++l) {
         double a = 0.0;
-        for (int h = 0; h < H; ++h) a = __dadd_rn(a, exp(-__ddiv_rn(__dadd_rn(F[l * H + h], -fmin), gamma)));
-        w[l] = a;
-      }
-    } else if (head_reduce == 2) {
-      // reciprocal of the variance, per head (a zero variance counts as the smallest positive one)
-      for (int l = 0; l < L; ++l) {
-        double a = 0.0;
-        for (int h = 0; h < H; ++h) {
-          const double f = F[l * H + h];
-          a = __dadd_rn(a, __ddiv_rn(1.0, f > 1e-300 ? f : 1e-300));
-        }
-        w[l] = a;
+        for (int h = 0; h < H; ++h) a = __dadd_rn(a, exp(-__ddiv_rn(F[l * H + h], gamma)));
+        const double s = floor(__dadd_rn(__dmul_rn(__ddiv_rn(a, (double)H), (double)P), 0.5));
+        bud[l * Hkv] = (int32_t)clipd(s, lo, hi);
       }
     } else {
-      double fmin = INFINITY;
-      for (int l = 0; l < L; ++l) {
-        double a = 0.0;
-        for (int h = 0; h < H; ++h) a = __dadd_rn(a, F[l * H + h]);
-        x[l] = __ddiv_rn(a, (double)H);
-        fmin = fmin < x[l] ? fmin : x[l];
-      }
-      if (head_reduce == 1) {
-        for (int l = 0; l < L; ++l) w[l] = exp(-__ddiv_rn(__dadd_rn(x[l], -fmin), gamma));
+      if (budget_rule == 1) {
+        double fmin = F[0];
+        for (int i = 1; i < L * H; ++i) fmin = fmin < F[i] ? fmin : F[i];
+        for (int u = 0; u < n; ++u) {
+          double a = 0.0;
+          for (int g = 0; g < G; ++g) a = __dadd_rn(a, exp(-__ddiv_rn(__dadd_rn(F[u * G + g], -fmin), gamma)));
+          w[u] = a;
+        }
+      } else if (head_reduce == 0) {
+        double fmin = F[0];
+        for (int i = 1; i < L * H; ++i) fmin = fmin < F[i] ? fmin : F[i];
+        for (int l = 0; l < L; ++l) {
+          double a = 0.0;
+          for (int h = 0; h < H; ++h) a = __dadd_rn(a, exp(-__ddiv_rn(__dadd_rn(F[l * H + h], -fmin), gamma)));
+          w[l] = a;
+        }
+      } else if (head_reduce == 2) {
+        // reciprocal of the variance, per head (a zero variance counts as the smallest positive one)
+        for (int l = 0; l < L; ++l) {
+          double a = 0.0;
+          for (int h = 0; h < H; ++h) {
+            const double f = F[l * H + h];
+            a = __dadd_rn(a, __ddiv_rn(1.0, f > 1e-300 ? f : 1e-300));
+          }
+          w[l] = a;
+        }
       } else {
-        for (int l = 0; l < L; ++l) w[l] = __ddiv_rn(1.0, x[l] > 1e-300 ? x[l] : 1e-300);
+        double fmin = INFINITY;
+        for (int l = 0; l < L; ++l) {
+          double a = 0.0;
+          for (int h = 0; h < H; ++h) a = __dadd_rn(a, F[l * H + h]);
+          x[l] = __ddiv_rn(a, (double)H);
+          fmin = fmin < x[l] ? fmin : x[l];
+        }
+        if (head_reduce == 1) {
+          for (int l = 0; l < L; ++l) w[l] = exp(-__ddiv_rn(__dadd_rn(x[l], -fmin), gamma));
+        } else {
+          for (int l = 0; l < L; ++l) w[l] = __ddiv_rn(1.0, x[l] > 1e-300 ? x[l] : 1e-300);
+        }
+      }
+      for (int u = 0; u < n; ++u) w[u] = w[u] > 1e-300 ? (w[u] < 1e300 ? w[u] : 1e300) : 1e-300;
+      // kinks of the piecewise-linear total(lambda), ascending (insertion sort)
+      int nk = 0;
+      for (int u = 0; u < n; ++u) {
+        const double cand[2] = {__ddiv_rn(lo, w[u]), __ddiv_rn(hi, w[u])};
+        for (int c = 0; c < 2; ++c) {
+          int i = nk++;
+          while (i > 0 && kinks[i - 1] > cand[c]) { kinks[i] = kinks[i - 1]; --i; }
+          kinks[i] = cand[c];
+        }
+      }
+      auto total = [&](double lam) {
+        double t = 0.0;
+        for (int u = 0; u < n; ++u) t = __dadd_rn(t, clipd(__dmul_rn(lam, w[u]), lo, hi));
+        return t;
+      };
+      // total() is non-decreasing: the first kink that reaches S_tot, by bisection
+      int k = 0, k_hi = nk;
+      while (k < k_hi) {
+        const int mid = (k + k_hi) >> 1;
+        if (total(kinks[mid]) < (double)S_tot) k = mid + 1; else k_hi = mid;
+      }
+      double lam;
+      if (k == 0) lam = kinks[0];
+      else if (k == nk) lam = kinks[nk - 1];
+      else {
+        const double a = kinks[k - 1], bb = kinks[k];
+        const double mid = __dmul_rn(0.5, __dadd_rn(a, bb));
+        double fixed = 0.0, wf = 0.0;
+        for (int u = 0; u < n; ++u) {
+          const double v = __dmul_rn(mid, w[u]);
+          if (v > lo && v < hi) wf = __dadd_rn(wf, w[u]);
+          else fixed = __dadd_rn(fixed, clipd(v, lo, hi));
+        }
+        lam = wf > 0.0 ? __ddiv_rn(__dadd_rn((double)S_tot, -fixed), wf) : bb;
+        lam = lam < a ? a : (lam > bb ? bb : lam);
+      }
+      long long sum = 0;
+      for (int u = 0; u < n; ++u) {
+        x[u] = clipd(__dmul_rn(lam, w[u]), lo, hi);
+        const double fl = floor(x[u]);
+        bud[slot_of(u)] = (int32_t)fl;
+        x[u] = x[u] - fl;                                   // remainder
+        sum += (long long)fl;
+      }
+      long long left = S_tot - sum;
+      if (left < 0 || left > n) { report_error(status_word, D2O_ERR_STATE, 0xB0000000u | (uint32_t)b); left = 0; }
+      while (left > 0) {                                     // largest remainder first, ties -> lower unit
+        int best = -1;
+        for (int u = 0; u < n; ++u)
+          if (x[u] >= 0.0 && bud[slot_of(u)] < max_budget && (best < 0 || x[u] > x[best])) best = u;
+        if (best < 0) { report_error(status_word, D2O_ERR_STATE, 0xB1000000u | (uint32_t)b); break; }
+        bud[slot_of(best)] += 1;
+        x[best] = -1.0;                                      // taken
+        --left;
       }
     }
-    for (int l = 0; l < L; ++l) w[l] = w[l] > 1e-300 ? (w[l] < 1e300 ? w[l] : 1e300) : 1e-300;
-    // kinks of the piecewise-linear total(lambda), ascending (insertion sort)
-    int nk = 0;
-    for (int l = 0; l < L; ++l) {
-      const double cand[2] = {__ddiv_rn(lo, w[l]), __ddiv_rn(hi, w[l])};
-      for (int c = 0; c < 2; ++c) {
-        int i = nk++;
-        while (i > 0 && kinks[i - 1] > cand[c]) { kinks[i] = kinks[i - 1]; --i; }
-        kinks[i] = cand[c];
-      }
-    }
-    auto total = [&](double lam) {
-      double t = 0.0;
-      for (int l = 0; l < L; ++l) t = __dadd_rn(t, clipd(__dmul_rn(lam, w[l]), lo, hi));
-      return t;
-    };
-    int k = 0;
-    while (k < nk && total(kinks[k]) < (double)S_tot) ++k;
-    double lam;
-    if (k == 0) lam = kinks[0];
-    else if (k == nk) lam = kinks[nk - 1];
-    else {
-      const double a = kinks[k - 1], bb = kinks[k];
-      const double mid = __dmul_rn(0.5, __dadd_rn(a, bb));
-      double fixed = 0.0, wf = 0.0;
-      for (int l = 0; l < L; ++l) {
-        const double v = __dmul_rn(mid, w[l]);
-        if (v > lo && v < hi) wf = __dadd_rn(wf, w[l]);
-        else fixed = __dadd_rn(fixed, clipd(v, lo, hi));
-      }
-      lam = wf > 0.0 ? __ddiv_rn(__dadd_rn((double)S_tot, -fixed), wf) : bb;
-      lam = lam < a ? a : (lam > bb ? bb : lam);
-    }
-    long long sum = 0;
-    for (int l = 0; l < L; ++l) {
-      x[l] = clipd(__dmul_rn(lam, w[l]), lo, hi);
-      const double fl = floor(x[l]);
-      budgets[b * L + l] = (int32_t)fl;
-      x[l] = x[l] - fl;                                   // remainder
-      sum += (long long)fl;
-    }
-    long long left = S_tot - sum;
-    if (left < 0 || left > L) { report_error(status_word, D2O_ERR_STATE, 0xB0000000u | (uint32_t)b); left = 0; }
-    while (left > 0) {                                     // largest remainder first, ties -> lower layer
-      int best = -1;
+    if (budget_rule != 1) {                                  // one size per layer: every KV head gets it
       for (int l = 0; l < L; ++l)
-        if (x[l] >= 0.0 && budgets[b * L + l] < max_budget && (best < 0 || x[l] > x[best])) best = l;
-      if (best < 0) { report_error(status_word, D2O_ERR_STATE, 0xB1000000u | (uint32_t)b); break; }
-      budgets[b * L + best] += 1;
-      x[best] = -1.0;                                      // taken
-      --left;
+        for (int h = 1; h < Hkv; ++h) bud[l * Hkv + h] = bud[l * Hkv];
     }
     if (windows) {
-      for (int l = 0; l < L; ++l) {
-        const int S = budgets[b * L + l];
+      for (int i = 0; i < L * Hkv; ++i) {
+        const int S = bud[i];
         const int T = n_sink < S ? n_sink : S;
         int M = window > 0 ? window : (int)floor((double)(S - T) / (1.0 + nm_ratio) + 0.5);
         M = M < 0 ? 0 : (M > S - T ? S - T : M);
-        windows[b * L + l] = M;
+        windows[(size_t)b * L * Hkv + i] = M;
       }
     }
   }
   __syncthreads();
-  if (threadIdx.x == 0 && row_off) {                       // cache rows laid out layer-major, then sequence
+  if (threadIdx.x == 0 && row_off) {                       // cache rows laid out layer-major, then sequence, then head
     long long o = 0;
     for (int l = 0; l < L; ++l)
-      for (int b = 0; b < B; ++b) { row_off[b * L + l] = o; o += (long long)Hkv * slice_stride(budgets[b * L + l]); }
+      for (int b = 0; b < B; ++b)
+        for (int h = 0; h < Hkv; ++h) {
+          const size_t i = ((size_t)b * L + l) * Hkv + h;
+          row_off[i] = o;
+          o += (long long)slice_stride(budgets[i]);
+        }
   }
 }
 
@@ -376,18 +414,20 @@ cudaError_t launch_layer_stats(const d2o_ctx* c, int layer, const void* Q, const
 }
 
 cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, int P, float rho, int min_budget,
-                           int max_budget, float gamma, int head_reduce, int n_sink, int window, float nm_ratio,
-                           int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
+                           int max_budget, float gamma, int head_reduce, int budget_rule, int n_sink, int window,
+                           float nm_ratio, int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
                            cudaStream_t st) {
-  const size_t per_thread = (size_t)4 * L * sizeof(double);
+  const size_t n_units = budget_rule == 1 ? (size_t)L * Hkv : (size_t)L;
+  const size_t per_thread = 4 * n_units * sizeof(double);
   int threads = B < 32 ? B : 32;
   while (threads > 1 && per_thread * threads > 160 * 1024) threads /= 2;
   const size_t sm = per_thread * threads;
+  if (sm > 200 * 1024) return cudaErrorInvalidValue;          // more allocation units than the work arrays hold
   cudaError_t e = cudaFuncSetAttribute(budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
   if (e != cudaSuccess) return e;
   budget_kernel<<<1, threads, sm, st>>>(density, B, L, H, Hkv, P, (double)rho, min_budget, max_budget, (double)gamma,
-                                        head_reduce, n_sink, window, (double)nm_ratio, budgets, windows, row_off,
-                                        status_word);
+                                        head_reduce, budget_rule, n_sink, window, (double)nm_ratio, budgets, windows,
+                                        row_off, status_word);
   return cudaGetLastError();
 }
 

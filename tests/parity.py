@@ -91,7 +91,9 @@ def make_oracle(wl: W.Workload, cfg: B.D2OConfig) -> O.OracleStack:
                          rho=float(cfg.rho), n_sink=cfg.n_sink, window=cfg.window, nm_ratio=float(cfg.nm_ratio),
                          beta=float(cfg.beta), density_temp=float(cfg.density_temp), min_budget=cfg.min_budget,
                          head_reduce=cfg.head_reduce, tau_override=float(cfg.tau_override),
-                         max_budget=cfg.max_budget)
+                         max_budget=cfg.max_budget, feature=("k", "v")[cfg.sim_feature],
+                         policy=("weighted", "average")[cfg.merge_policy],
+                         budget_rule=("layer", "head", "exp_decay")[cfg.budget_rule])
 
 
 def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int, int, int]]] = None,
@@ -151,8 +153,9 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
     tabs = ctx.tables()
     for b in range(Bn):
         for l in range(L):
-            S, T, M = orc.slice_params(b, l)
-            assert int(tabs[1][b, l]) == M, f"window mismatch at b={b} l={l}: {int(tabs[1][b, l])} vs {M}"
+            for h in range(Hkv):
+                S, T, M = orc.slice_params(b, l, h)
+                assert int(tabs[1][b, l, h]) == M, f"window mismatch at b={b} l={l} h={h}: {int(tabs[1][b, l, h])} vs {M}"
     # ---------------- (2) prompt-stage compression
     for l in range(L):
         K, V = KV[l]

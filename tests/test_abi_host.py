@@ -50,7 +50,7 @@ def test_workspace_size_and_validation(lib):
     bad = [dict(n_q_heads=7), dict(d_head=96), dict(dtype="f32", d_head=32), dict(rho=0.0), dict(rho=float("nan")),
            dict(beta=1.5), dict(n_layers=0), dict(prompt_len=0), dict(min_budget=0), dict(min_budget=1, n_sink=4),
            dict(rho=2.0), dict(density_temp=0.0), dict(head_reduce=7), dict(n_q_heads=24, n_kv_heads=8),
-           dict(max_budget=4096)]
+           dict(max_budget=4096), dict(budget_rule=3), dict(sim_feature=2), dict(merge_policy=-1)]
     for kw in bad:
         with pytest.raises(B.D2OError) as ei:
             B.d2o_workspace_size(good(**kw))
@@ -73,7 +73,7 @@ def test_null_and_misaligned_arguments(lib):
     assert lib.d2o_full_decode_step(1, 96, 1, 1, 16, 0, 16, 16, 16, 16, 16, 16, None) == 2
     assert lib.d2o_full_decode_step(1, 128, 1, 1, 16, 16, 16, 16, 16, 16, 16, 16, None) == 1     # len >= capacity
     assert lib.d2o_full_decode_step(1, 128, 1, 1, 16, 0, 8, 16, 16, 16, 16, 16, None) == 1       # misaligned cache
-    assert lib.d2o_budgets_from_density(None, 1, 1, 1, 1, 16, 0.5, 1, 0, 1.0, 0, 1, 0, 3.0, None, None, None,
+    assert lib.d2o_budgets_from_density(None, 1, 1, 1, 1, 16, 0.5, 1, 0, 1.0, 0, 0, 1, 0, 3.0, None, None, None,
                                         None, None) == 1
     assert lib.d2o_status_string(0) == b"ok" and b"order" in lib.d2o_status_string(4)
     lib.d2o_destroy(None)

@@ -186,6 +186,50 @@ def test_rows_with_only_negative_similarities(name):
     assert seen["n"] == 2
 
 
+@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfg2"])
+def test_average_merge_policy(name):
+    # the ablation's average merging: a kept token and everything merged into it weigh the same
+    wl = small(prompt_len=320, decode_steps=8) if name == "cfg0" else dataclasses.replace(W.twin(name), n_layers=2,
+                                                                                            decode_steps=8)
+    rep = run_parity(wl, ctx_over=dict(merge_policy=1))
+    assert_report(rep, wl.dtype)
+    assert rep.merges > 0
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg0"])
+def test_per_head_budgets(name):
+    # S_l^h = alpha_l^h * S_total: every (layer, KV head) has its own cache size, window and threshold
+    wl = dataclasses.replace(W.CONFIGS["cfg0"], n_layers=3, prompt_len=384, decode_steps=8, density_temp=40.0,
+                             min_budget=24) if name == "cfg0" else dataclasses.replace(W.twin(name), decode_steps=8)
+    rep = run_parity(wl, ctx_over=dict(budget_rule=1))
+    assert_report(rep, wl.dtype)
+    assert rep.merges + rep.discards > 0
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2"])
+def test_exponential_decay_budgets(name):
+    # S_l = exp(-F_l / gamma) * P, not normalised: gamma of the order of the densities keeps the sizes between the clamps
+    wl = dataclasses.replace(W.twin(name), decode_steps=6)
+    rep = run_parity(wl, ctx_over=dict(budget_rule=2, density_temp=float(wl.prompt_len) / 1.5,
+                                       max_budget=wl.prompt_len // 2))
+    assert_report(rep, wl.dtype)
+    assert rep.merges + rep.discards > 0
+
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfg2"])
+def test_value_feature_prompt_stage(name):
+    # the ablation's "Feature choice" V: nearest neighbours, tau_0 and merge weights from the cosine of the values
+    wl = small(prompt_len=320, decode_steps=0) if name == "cfg0" else dataclasses.replace(W.twin(name), n_layers=2,
+                                                                                            decode_steps=0)
+    rep = run_parity(wl, ctx_over=dict(sim_feature=1))
+    assert_report(rep, wl.dtype)
+    assert rep.steps == 0 and rep.gpu_stats.prefill_merged > 0
+    from parity import make_ctx
+    with pytest.raises(B.D2OError) as e:                  # generation with this switch is not built
+        make_ctx(dataclasses.replace(wl, decode_steps=4), sim_feature=1)
+    assert e.value.status == 2
+
+
 def test_more_sinks_than_budget_is_rejected(cuda_device):
     from parity import make_ctx
     wl = small(prompt_len=128, decode_steps=2, n_sink=40, min_budget=8)
@@ -215,34 +259,82 @@ def test_budgets_large_temperature_gives_uniform_allocation(cuda_device):
 
 def test_budgets_pure_function_matches_oracle(cuda_device):
     r = np.random.default_rng(5)
-    for trial in range(40):
-        Bn, L, H = int(r.integers(1, 4)), int(r.integers(1, 40)), int(r.integers(1, 9))
+    done = 0
+    for trial in range(60):
+        Bn, L, H = int(r.integers(1, 4)), int(r.integers(1, 40)), 2 * int(r.integers(1, 5))
         P = int(r.integers(64, 9000))
         rho = B.f32(float(r.uniform(0.05, 1.0)))
         gamma = B.f32(float(r.choice([1.0, 10.0, 1000.0])))
         smin = int(r.integers(1, 12))
         F = r.gamma(1.0, size=(Bn, L, H)) * float(r.choice([0.01, 1.0, 30.0, 3000.0]))
-        if L * smin > math.floor(rho * L * P + 0.5):
+        tot = math.floor(rho * L * P + 0.5)
+        # every other trial with an upper clamp between the mean and four times the mean
+        cap = 0 if trial % 2 == 0 else int(min(P, max(smin, math.ceil(tot / L * float(r.uniform(1.0, 4.0))))))
+        if L * smin > tot or (cap and L * cap < tot):
             continue
         hr = int(trial % 4)                                          # both softmax rules and both reciprocal rules
         nm = B.f32(3.0)
         bud, win, off, status = B.d2o_budgets_from_density(torch.tensor(F, device=cuda_device), n_kv_heads=2,
-                                                           prompt_len=P, rho=rho, min_budget=smin,
+                                                           prompt_len=P, rho=rho, min_budget=smin, max_budget=cap,
                                                            density_temp=gamma, head_reduce=hr, n_sink=1, window=0,
                                                            nm_ratio=nm)
         bud = bud.cpu().numpy()
         assert int(status[0]) == 0
         for b in range(Bn):
-            ref = O.layer_budgets(F[b], P, rho, smin, gamma, hr)
-            np.testing.assert_array_equal(bud[b], ref)
+            ref = O.layer_budgets(F[b], P, rho, smin, gamma, hr, cap)
+            np.testing.assert_array_equal(bud[b, :, 0], ref)
+            np.testing.assert_array_equal(bud[b, :, 1], ref)          # every KV head of a layer gets the layer's size
             for l in range(L):
-                assert int(win[b, l]) == O.window_size(int(ref[l]), min(1, int(ref[l])), 0, nm)
+                assert int(win[b, l, 0]) == O.window_size(int(ref[l]), min(1, int(ref[l])), 0, nm)
         o = off.cpu().numpy()
-        flat = [(l, b) for l in range(L) for b in range(Bn)]
         run = 0
-        for l, b in flat:
-            assert o[b, l] == run
-            run += 2 * ((bud[b, l] + 7) // 8 * 8)          # slices start at multiples of 8 rows
+        for l in range(L):
+            for b in range(Bn):
+                for h in range(2):
+                    assert o[b, l, h] == run
+                    run += (bud[b, l, h] + 7) // 8 * 8      # slices start at multiples of 8 rows
+        done += 1
+    assert done > 30
+
+
+def test_per_head_and_exponential_decay_budgets_match_oracle(cuda_device):
+    r = np.random.default_rng(15)
+    done = 0
+    for trial in range(40):
+        Bn, L, Hkv, G = int(r.integers(1, 3)), int(r.integers(1, 33)), int(r.choice([1, 2, 8, 32])), int(r.choice([1, 2, 4, 8]))
+        H = Hkv * G
+        P = int(r.integers(64, 9000))
+        rho = B.f32(float(r.uniform(0.05, 1.0)))
+        gamma = B.f32(float(r.choice([1.0, 10.0, 1000.0])))
+        smin = int(r.integers(1, 12))
+        F = r.gamma(1.0, size=(Bn, L, H)) * float(r.choice([0.01, 1.0, 30.0, 3000.0]))
+        tot = math.floor(rho * (L * Hkv) * P + 0.5)
+        cap = 0 if trial % 2 == 0 else int(min(P, max(smin, math.ceil(tot / (L * Hkv) * float(r.uniform(1.0, 4.0))))))
+        if L * Hkv * smin > tot or (cap and L * Hkv * cap < tot):
+            continue
+        kw = dict(n_kv_heads=Hkv, prompt_len=P, rho=rho, min_budget=smin, max_budget=cap, density_temp=gamma,
+                  n_sink=1, window=0, nm_ratio=B.f32(3.0))
+        bud, _, off, status = B.d2o_budgets_from_density(torch.tensor(F, device=cuda_device), budget_rule=1, **kw)
+        assert int(status[0]) == 0
+        bud = bud.cpu().numpy()
+        for b in range(Bn):
+            np.testing.assert_array_equal(bud[b], O.head_budgets(F[b], P, rho, G, smin, gamma, cap))
+        o = off.cpu().numpy()
+        run = 0
+        for l in range(L):
+            for b in range(Bn):
+                for h in range(Hkv):
+                    assert o[b, l, h] == run
+                    run += (bud[b, l, h] + 7) // 8 * 8
+        bud2, _, _, status = B.d2o_budgets_from_density(torch.tensor(F, device=cuda_device), budget_rule=2, **kw)
+        assert int(status[0]) == 0
+        bud2 = bud2.cpu().numpy()
+        for b in range(Bn):
+            ref = O.exp_decay_budgets(F[b], P, smin, gamma, cap)
+            for h in range(Hkv):
+                np.testing.assert_array_equal(bud2[b, :, h], ref)
+        done += 1
+    assert done > 20
 
 
 @pytest.mark.parametrize("dtype,d,G,n_slices,cap,length", [("f16", 128, 1, 6, 700, 513), ("bf16", 128, 4, 3, 4100, 4099),
