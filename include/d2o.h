@@ -246,6 +246,15 @@ d2o_status d2o_set_tuning(d2o_ctx* ctx, int32_t decode_stages, int32_t decode_l2
                           int32_t similarity_path, int32_t stats_path, int32_t decode_warps,
                           int32_t decode_smem_rows, int32_t decode_long_pairs);
 
+/* For failure-detection tests (Section 4.2's decode step has no counterpart; this exercises the library's own
+ * promise that no device-side wait is unbounded).  wait_limit_us: how long the decode kernel waits for a stage
+ * of cache rows before it gives up (0 = the default of one second).  producer_stop_stage: the kernel's copy
+ * engine issues no copy from this stage of a slice on (-1 = never), so that the wait for it runs out.  A wait
+ * that runs out sets the error word to D2O_ERR_TIMEOUT (see d2o_get_stats); the kernel returns, the slices
+ * whose wait ran out during the key pass are left untouched, and every later decode step on this context does
+ * nothing.  Nothing traps and the CUDA context stays usable. */
+d2o_status d2o_set_fault_injection(d2o_ctx* ctx, int32_t wait_limit_us, int32_t producer_stop_stage);
+
 #ifdef __cplusplus
 }
 #endif

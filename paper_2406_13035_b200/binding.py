@@ -25,7 +25,7 @@ EXPORTS = [
     "d2o_status_string", "d2o_last_cuda_error", "d2o_workspace_size", "d2o_create", "d2o_destroy",
     "d2o_layer_stats", "d2o_layer_budgets", "d2o_budgets_from_density", "d2o_prefill_compress",
     "d2o_decode_step", "d2o_decode_step_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
-    "d2o_set_tuning", "d2o_layer_stats_static",
+    "d2o_set_tuning", "d2o_layer_stats_static", "d2o_set_fault_injection",
 ]
 STATIC_LSE_FLOATS = 1 << 20      # D2O_STATIC_LSE_FLOATS of include/d2o.h
 
@@ -93,6 +93,7 @@ def load_library() -> C.CDLL:
     lib.d2o_get_stats.argtypes = [vp, C.POINTER(D2OStats), vp]
     lib.d2o_set_tuning.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32]
     lib.d2o_layer_stats_static.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.d2o_set_fault_injection.argtypes = [vp, i32, i32]
     for name in EXPORTS:
         if name not in ("d2o_status_string", "d2o_last_cuda_error", "d2o_destroy"):
             getattr(lib, name).restype = C.c_int
@@ -199,6 +200,10 @@ class D2OContext:
                        decode_long_pairs: int = 0):
         _check(self.lib.d2o_set_tuning(self.handle, decode_stages, decode_l2_hints, similarity_path, stats_path,
                                        decode_warps, decode_smem_rows, decode_long_pairs), "d2o_set_tuning")
+
+    def d2o_set_fault_injection(self, wait_limit_us: int = 0, producer_stop_stage: int = -1):
+        _check(self.lib.d2o_set_fault_injection(self.handle, wait_limit_us, producer_stop_stage),
+               "d2o_set_fault_injection")
 
     def d2o_get_stats(self) -> D2OStats:
         s = D2OStats()

@@ -176,6 +176,8 @@ struct d2o_ctx {
   int decode_l2_hints;         // tuning: 1 = the decode kernel's copies carry L2 eviction hints
   int similarity_path;         // tuning: 0 = tensor cores for 16-bit keys, 1 = FFMA kernel for every dtype
   int stats_path;              // tuning: 0 = tensor cores for the column sums of 16-bit Q/K, 1 = FFMA kernels
+  int wait_limit_us;           // failure-detection tests: limit of a device-side wait in microseconds (0 = one second)
+  int producer_stop_stage;     // failure-detection tests: the decode producer issues no copy from this stage on (-1 = never)
 };
 
 namespace d2o {

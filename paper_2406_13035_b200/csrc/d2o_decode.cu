@@ -60,6 +60,8 @@ struct DecodeArgs {
   const int32_t* order;             // NULL: CTAs take (layer, b, h) in index order; else (layer * B + b) per group of Hkv CTAs
   int pair_base;                    // first entry of `order` this launch works on
   int average;                      // 1: average merge (both rows weigh 1/2) instead of the weights of Eq. 12
+  unsigned long long wait_ns;       // a wait for a stage gives up after this long
+  int stop_stage;                   // failure-detection tests: the producer issues no copy from this stage on (-1: never)
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -88,13 +90,23 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
 }
 // Wait for a stage in the kernel's loops: one probe when the phase is already complete (the common case); otherwise
 // poll until it completes, another thread has recorded a timeout, or this one does.
-__device__ __forceinline__ void stage_wait(unsigned long long* bar, uint32_t parity, volatile int* timeout) {
+__device__ __forceinline__ void stage_wait(unsigned long long* bar, uint32_t parity, volatile int* timeout,
+                                           unsigned long long limit_ns) {
   if (mbar_try_wait(bar, parity)) return;
   const unsigned long long t0 = global_ns();
   while (*timeout == 0) {
     if (mbar_try_wait(bar, parity)) return;
-    if (global_ns() - t0 > kWaitNs) { *timeout = 2; return; }
+    if (global_ns() - t0 > limit_ns) { *timeout = 2; return; }
   }
+}
+// The same without giving up early when another thread has recorded a timeout: used by the producer to see its own
+// copies land before it leaves.  false = the limit ran out.
+__device__ __forceinline__ bool landed_wait(unsigned long long* bar, uint32_t parity, unsigned long long limit_ns) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (!mbar_try_wait(bar, parity))
+    if (global_ns() - t0 > limit_ns) return false;
+  return true;
 }
 // Similarity as an ordered key: -0 (a zero-norm row times a negative dot product) must count as +0, or equal
 // similarities would not tie.
@@ -351,16 +363,19 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   __shared__ float s_red[2][kConsWarps][G];
   __shared__ unsigned long long s_key[kConsWarps], s_best_key;
   __shared__ int s_li[kConsWarps], s_best_li;
-  __shared__ volatile int s_timeout;
+  __shared__ volatile int s_timeout;                                 // 1: an earlier launch recorded an anomaly; 2: a wait of this CTA ran out
+  __shared__ int s_bail;
 
   if (tid == 0) {
-    // once an anomaly has been recorded (by this or an earlier launch) no wait is attempted any more
     s_timeout = *reinterpret_cast<volatile uint32_t*>(a.status) != 0u;
     for (int s = 0; s < NS; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kConsWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  // once an anomaly has been recorded the state is no longer trusted: later steps do nothing (the error word stays
+  // set and the caller finds it with d2o_get_stats)
+  if (s_timeout != 0) return;
 
   // =========================================================================== producer warp
   if (warp == kConsWarps) {
@@ -372,7 +387,8 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       }
       int slot = 0, q = 0;
       uint32_t ph = 1;                                               // parity of the previous use of a slot
-      for (int p = 0; p < 2; ++p) {
+      bool stopped = false;
+      for (int p = 0; p < 2 && !stopped; ++p) {
         const bool is_v = (p == 1);
         const T* pool = is_v ? vpool : kpool;
         const T* fresh = is_v ? v_new : k_new;
@@ -380,7 +396,10 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         // keys may be read once more (a victim that was not guessed): they leave L2 after the values
         const unsigned long long pol = (p == 0 && evict) ? keep : drop;
         for (int s = 0; s < n_st; ++s, ++q, ring_next(slot, ph, NS)) {
-          if (q >= NS) stage_wait(&s_empty[slot], ph, &s_timeout);
+          if (q >= NS) stage_wait(&s_empty[slot], ph, &s_timeout, a.wait_ns);
+          // a wait ran out somewhere in this CTA, or the failure-detection tests asked for a stage that never
+          // arrives: nothing more is issued
+          if (s_timeout != 0 || (a.stop_stage >= 0 && q >= a.stop_stage)) { stopped = true; break; }
           const int a0 = s * SR, a1 = min(n, a0 + SR);
           const int np = max(0, min(a1, n_old) - a0);                // cache rows of the stage
           const bool nw = n_old >= a0 && n_old < a1;                 // the new token's row falls into the stage
@@ -417,6 +436,16 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
             else bulk_g2s(dst, pool + (row0 + a0) * D, (uint32_t)(np * ROWB), &s_full[slot]);
           }
           if (nw) bulk_g2s(dst + (size_t)(n_old - a0) * LPR, fresh, (uint32_t)ROWB, &s_full[slot]);
+        }
+      }
+      if (stopped) {
+        // The consumers will run into a wait that gives up and may leave early.  The CTA must not end while copies
+        // are on their way into its shared memory: see the last (up to NS) issued stages land, each wait bounded.
+        const int n_back = q < NS ? q : NS;
+        int sl_i = slot; uint32_t ph_i = ph;                         // `slot` is the stage that was not issued
+        for (int i = 0; i < n_back; ++i) {
+          if (sl_i == 0) { sl_i = NS - 1; ph_i ^= 1u; } else --sl_i;
+          if (!landed_wait(&s_full[sl_i], ph_i ^ 1u, a.wait_ns)) break;
         }
       }
     }
@@ -576,7 +605,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     const int tile_odd = kHalfTiles ? (warp >= kTiles ? warp - kTiles : -1) : warp;
     float* const pl_mine = pl + (size_t)(2 * tig) * a.row_cap + gid;
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
-      stage_wait(&s_full[slot], ph, &s_timeout);
+      stage_wait(&s_full[slot], ph, &s_timeout, a.wait_ns);
       const unsigned char* st = reinterpret_cast<const unsigned char*>(ring) + (size_t)slot * kStageBytes;
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
       const int tile = (s & 1) ? tile_odd : tile_even;
@@ -666,7 +695,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     }
   } else {
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
-      stage_wait(&s_full[slot], ph, &s_timeout);
+      stage_wait(&s_full[slot], ph, &s_timeout, a.wait_ns);
       const uint4* st = ring + (size_t)slot * SR * LPR + (size_t)grp * LPR + lig;   // this thread's piece of row grp
       const bool full = (s + 1) * SR <= n_plain_fma;                 // every row of the stage is a plain row
       uint4 raw[4];
@@ -736,7 +765,13 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   {
 #pragma unroll
     for (int g = 0; g < G; ++g) { const float w = warp_max(mloc[g]); if (lane == 0) s_red[0][warp][g] = w; }
+    if (tid == 0) s_bail = s_timeout;
     consumer_sync<CW>();                                                 // logits, maxima and the new token's metadata
+    if (s_bail != 0) {
+      // a wait of the key pass ran out: the logits are not to be trusted, so nothing of the slice's state is touched
+      if (tid == 0) report_error(a.status, D2O_ERR_TIMEOUT, 0xDEC10000u | (uint32_t)(sl & 0xffff));
+      return;
+    }
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       float t = s_red[0][0][g];
@@ -833,7 +868,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       // still delivers the value pass; it is drained without being used.
       if (tid == 0) report_error(a.status, D2O_ERR_STATE, 0xDEC00000u | (uint32_t)(sl & 0xfffff));
       for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
-        stage_wait(&s_full[slot], ph, &s_timeout);
+        stage_wait(&s_full[slot], ph, &s_timeout, a.wait_ns);
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_empty[slot]);
       }
@@ -883,7 +918,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     const float mx = ord_float((uint32_t)(s_best_key >> 32));
     const float tau_new = a.beta * mx + (1.0f - a.beta) * tau_old;
     const float thr = isnan(a.tau_override) ? tau_new : a.tau_override;
-    merge = mx >= thr;
+    merge = mx >= thr && nn_li >= 0;
     nn_is_new = (nn_li == n_old);
     const float ew = expf(mx);
     w_e = a.average ? 0.5f : ew / (ew + kEuler);
@@ -954,7 +989,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     const int vic_row = vic_li < n_old ? vic_li : -64, nn_row = nn_li < n_old ? nn_li : -64;
     int li0 = rt * 16;                                               // first row of this warp's tile
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS), li0 += SR, wrow += SR) {
-      stage_wait(&s_full[slot], ph, &s_timeout);
+      stage_wait(&s_full[slot], ph, &s_timeout, a.wait_ns);
       const uint32_t stage_u32 = ring_u32 + (uint32_t)slot * (uint32_t)kStageBytes;
       if (li0 < n_old) {
         uint32_t bh0, bl0, bh1, bl1;
@@ -1031,7 +1066,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
 #pragma unroll
       for (int e = 0; e < EPV; ++e) acc[g][e] = 0.f;
     for (int s = 0; s < n_st; ++s, ring_next(slot, ph, NS)) {
-      stage_wait(&s_full[slot], ph, &s_timeout);
+      stage_wait(&s_full[slot], ph, &s_timeout, a.wait_ns);
       const uint4* st = ring + (size_t)slot * SR * LPR + (size_t)grp * LPR + lig;
       const int lbase = s * SR + grp;                                // this thread's rows: lbase + u * NGRP
       // a plain stage: all rows are cache rows with their weights in shared memory, neither victim nor neighbour
@@ -1243,6 +1278,8 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   a.L = L; a.l0 = l0; a.B = B; a.Hkv = g.n_kv_heads; a.T = g.n_sink;
   a.t = g.prompt_len + c->layer_steps[l0];
   a.beta = g.beta; a.tau_override = g.tau_override; a.average = g.merge_policy;
+  a.wait_ns = c->wait_limit_us > 0 ? (unsigned long long)c->wait_limit_us * 1000ull : kWaitNs;
+  a.stop_stage = c->producer_stop_stage;
   a.l2_hints = c->decode_l2_hints;
   const int G = c->group, Hkv = g.n_kv_heads;
   const int row_bytes = g.d_head * c->elem_size;

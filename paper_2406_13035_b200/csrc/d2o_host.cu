@@ -165,6 +165,7 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
       : (int64_t)cfg->batch * cfg->n_kv_heads * (tot + 7 * (int64_t)cfg->n_layers);
   c->lay = l; c->slay = s;
   c->decode_l2_hints = 1;
+  c->producer_stop_stage = -1;
   {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -431,5 +432,12 @@ extern "C" d2o_status d2o_set_tuning(d2o_ctx* c, int32_t decode_stages, int32_t 
   c->decode_warps = decode_warps;
   c->decode_smem_rows = decode_smem_rows;
   c->decode_long_pairs = decode_long_pairs;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_set_fault_injection(d2o_ctx* c, int32_t wait_limit_us, int32_t producer_stop_stage) {
+  if (!c || wait_limit_us < 0 || producer_stop_stage < -1) return D2O_ERR_INVALID_ARG;
+  c->wait_limit_us = wait_limit_us;
+  c->producer_stop_stage = producer_stop_stage;
   return D2O_OK;
 }
