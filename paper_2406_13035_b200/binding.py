@@ -64,6 +64,12 @@ class D2OError(RuntimeError):
 _lib = None
 
 
+def use_library(path: str):
+    """Selects the shared object the binding loads next (libd2o.so, or the checked build libd2o_checked.so)."""
+    global _lib, LIB_PATH
+    _lib, LIB_PATH = None, path
+
+
 def load_library() -> C.CDLL:
     """Loads libd2o.so (built by paper_2406_13035_b200.build).  Raises if it is missing."""
     global _lib

@@ -10,6 +10,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libd2o.so")
+LIB_CHECKED = os.path.join(HERE, "libd2o_checked.so")      # the same sources with -DD2O_CHECKED (index checks)
 SOURCES = ["d2o_host.cu", "d2o_stats.cu", "d2o_prefill.cu", "d2o_decode.cu", "d2o_full_decode.cu", "d2o_sim_tc.cu", "d2o_colsum_tc.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
@@ -28,13 +29,15 @@ def _stale(out: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compiles every .cu file to an object (in _build/) and links libd2o.so next to this file.
-    With D2O_SKIP_BUILD=1 in the environment an existing libd2o.so is used as it is."""
+def build_library(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compiles every .cu file to an object (in _build/) and links libd2o.so next to this file; `checked` builds
+    libd2o_checked.so (objects in _build_checked/), whose kernels verify every data-derived index before using it.
+    With D2O_SKIP_BUILD=1 in the environment an existing library is used as it is."""
+    LIB = LIB_CHECKED if checked else globals()["LIB"]
     if os.environ.get("D2O_SKIP_BUILD") == "1" and os.path.exists(LIB) and not force:
         return LIB
     nvcc = _nvcc()
-    bdir = os.path.join(HERE, "_build")
+    bdir = os.path.join(HERE, "_build_checked" if checked else "_build")
     os.makedirs(bdir, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     headers.append(os.path.join(os.path.dirname(HERE), "include", "d2o.h"))
@@ -48,7 +51,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         objs.append(obj)
         if force or _stale(obj, [src] + headers):
             cmd = [nvcc, *ARCH, "-O3", "-lineinfo", "-std=c++17", "-Xcompiler", "-fPIC", "-Xptxas", "-v",
-                   "-c", src, "-o", obj]
+                   *(["-DD2O_CHECKED"] if checked else []), "-c", src, "-o", obj]
             procs.append((s, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     failed = False
     for s, p in procs:
@@ -69,4 +72,4 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

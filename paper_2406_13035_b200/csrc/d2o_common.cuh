@@ -130,6 +130,16 @@ __device__ __forceinline__ void report_error(uint32_t* status_word, uint32_t cod
   if (atomicCAS(status_word, 0u, code) == 0u) status_word[1] = detail;
 }
 
+// Checked build (-DD2O_CHECKED, libd2o_checked.so): every index that a kernel derives from data (a position read
+// from a list, a victim or neighbour row, a cache row computed from the tables) is compared with its range before it
+// is used.  A violation records D2O_ERR_STATE with a code naming the check and the access is skipped; nothing traps.
+// In the ordinary build the guard is the constant `true`.
+#ifdef D2O_CHECKED
+#define D2O_GUARD(cond, status_word, code) ((cond) ? true : (d2o::report_error((status_word), D2O_ERR_STATE, (code)), false))
+#else
+#define D2O_GUARD(cond, status_word, code) true
+#endif
+
 // ----------------------------------------------------------------------------- counters
 enum Counter { kCntDecodeSteps = 0, kCntEvictions, kCntMerges, kCntDiscards, kCntPrefillEvicted,
                kCntPrefillMerged, kCntGuessMisses, kNumCounters = 8 };

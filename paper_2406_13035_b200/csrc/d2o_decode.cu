@@ -62,6 +62,7 @@ struct DecodeArgs {
   int average;                      // 1: average merge (both rows weigh 1/2) instead of the weights of Eq. 12
   unsigned long long wait_ns;       // a wait for a stage gives up after this long
   int stop_stage;                   // failure-detection tests: the producer issues no copy from this stage on (-1: never)
+  long long pool_rows;              // rows of the cache pool (bounds of the checked build)
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -332,6 +333,9 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   const int sidx = (layer * a.B + b) * a.Hkv + h;
   const int n_old = a.len[sidx];
   const float tau_old = a.tau[sidx];
+  if (!D2O_GUARD(S >= 1 && n_old >= 0 && n_old <= S && row0 >= 0 && row0 + slice_stride(S) <= a.pool_rows, a.status,
+                 0xC4EC0010u))
+    return;                                                          // uniform for the CTA, before any barrier or copy
   const int n = n_old + 1;                                         // rows attended: cache + the new token
   const int Tn = a.T < S ? a.T : S;
   const bool evict = n > S;
@@ -874,6 +878,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       }
       return;
     }
+    if (!D2O_GUARD(vic_li >= 0 && vic_li <= n_old, a.status, 0xC4EC0011u)) vic_li = n_old;
     const float vic_rn = vic_li < n_old ? a.rnorm[row0 + vic_li] : s_new_rn;
     float kvic[EPV];
     Elem<T>::unpack(ld_global_v4((vic_li < n_old ? kpool + (row0 + vic_li) * D : k_new) + lig * EPV), kvic);
@@ -919,6 +924,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     const float tau_new = a.beta * mx + (1.0f - a.beta) * tau_old;
     const float thr = isnan(a.tau_override) ? tau_new : a.tau_override;
     merge = mx >= thr && nn_li >= 0;
+    if (!D2O_GUARD(nn_li >= 0 && nn_li <= n_old && nn_li != vic_li, a.status, 0xC4EC0012u)) merge = false;
     nn_is_new = (nn_li == n_old);
     const float ew = expf(mx);
     w_e = a.average ? 0.5f : ew / (ew + kEuler);
@@ -1280,6 +1286,7 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   a.beta = g.beta; a.tau_override = g.tau_override; a.average = g.merge_policy;
   a.wait_ns = c->wait_limit_us > 0 ? (unsigned long long)c->wait_limit_us * 1000ull : kWaitNs;
   a.stop_stage = c->producer_stop_stage;
+  a.pool_rows = c->pool_rows;
   a.l2_hints = c->decode_l2_hints;
   const int G = c->group, Hkv = g.n_kv_heads;
   const int row_bytes = g.d_head * c->elem_size;

@@ -33,6 +33,7 @@ struct SelectArgs {
   uint32_t* status;
   int L, layer, B, Hq, Hkv, G, P, T;
   int keys_in_smem;
+  long long pool_rows;     // rows of the cache pool (bounds of the checked build)
   int value_feature;       // 1: the similarity of Eq. 9 is taken on the value rows (ablation), so the norms are theirs
 };
 
@@ -130,10 +131,13 @@ select_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
     if (j < P) {
       if (keep) {
         const int slot = n_ret + kr;
-        a.pos[row0 + slot] = j;
-        a.score[row0 + slot] = keys[j];
+        if (D2O_GUARD(slot < (keep_all ? P : S) && row0 + slot < a.pool_rows, a.status, 0xC4EC0001u)) {
+          a.pos[row0 + slot] = j;
+          a.score[row0 + slot] = keys[j];
+        }
       } else {
-        a.evict_idx[(size_t)slice * P + n_ev + (threadIdx.x - kr)] = j;
+        const int at = n_ev + (threadIdx.x - kr);
+        if (D2O_GUARD(at >= 0 && at < P, a.status, 0xC4EC0002u)) a.evict_idx[(size_t)slice * P + at] = j;
       }
     }
     const int valid = min((int)blockDim.x, P - base);
@@ -169,6 +173,7 @@ gather_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
   const int r1 = min(n_keep, ((int)blockIdx.x + 1) * 64);
   for (int r = blockIdx.x * 64 + grp; r < r1; r += blockDim.x / LPR) {
     const int j = a.pos[row0 + r];
+    if (!D2O_GUARD(j >= 0 && j < P && row0 + r < a.pool_rows, a.status, 0xC4EC0003u)) continue;
     const uint4 kv = ld_global_v4(Ks + (size_t)j * D + lig * EPV);
     const uint4 vv = ld_global_v4(Vs + (size_t)j * D + lig * EPV);
     *reinterpret_cast<uint4*>(kpool + (row0 + r) * D + lig * EPV) = kv;
@@ -190,6 +195,7 @@ struct SimArgs {
   const int32_t* budgets; const int64_t* row_off;
   const int32_t* evict_idx; float* evict_mx; int32_t* evict_nn;
   const float* rnorm; const int32_t* pos;
+  uint32_t* status;
   int L, layer, Hkv, P;
 };
 
@@ -215,8 +221,9 @@ similarity_kernel(SimArgs a, const T* __restrict__ K, const T* __restrict__ kpoo
   const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
   {  // evicted tile: gather rows by index, transposed, plus inverse norms
     const int r = threadIdx.x % kSimTile;
-    const bool ok = i0 + r < Le;
+    bool ok = i0 + r < Le;
     const int j = ok ? ev[i0 + r] : 0;
+    if (ok && !D2O_GUARD(j >= 0 && j < a.P, a.status, 0xC4EC0004u)) ok = false;
     float ss = 0.f;
     for (int vi = threadIdx.x / kSimTile; vi < VPR; vi += kSimThreads / kSimTile) {
       float f[EPV];
@@ -454,6 +461,7 @@ struct MergeArgs {
   const int32_t* seg_start; const int32_t* seg_items;
   float* rnorm;
   int L, layer, Hkv, P, seg_stride;
+  uint32_t* status;
   int average;             // 1: average merge (every token of a merge weighs the same) instead of Eq. 12
   int value_feature;       // 1: the cached inverse norms belong to the value rows
 };
@@ -474,6 +482,7 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   const int32_t* start = a.seg_start + (size_t)slice * a.seg_stride;
   const int s0 = start[j], s1 = start[j + 1];
   if (s1 == s0) return;                              // nothing merged: the row stays bit-identical
+  if (!D2O_GUARD(s0 >= 0 && s0 < s1 && s1 <= a.P - S, a.status, 0xC4EC0007u)) return;
   const int64_t row = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)] + j;
   const int32_t* items = a.seg_items + (size_t)slice * a.P;
   const int32_t* ev = a.evict_idx + (size_t)slice * a.P;
@@ -491,8 +500,10 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   float den = own;
   for (int s = s0; s < s1; ++s) {
     const int i = items[s];
+    if (!D2O_GUARD(i >= 0 && i < a.P - S, a.status, 0xC4EC0005u)) continue;
     const float w = a.average ? 1.0f : expf(mx[i]);
     const int pj = ev[i];
+    if (!D2O_GUARD(pj >= 0 && pj < a.P, a.status, 0xC4EC0006u)) continue;
     den += w;
     Elem<T>::unpack(ld_global_v4(Ks + (size_t)pj * D + lig * EPV), f);
 #pragma unroll
@@ -542,6 +553,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   sa.L = L; sa.layer = layer; sa.B = B; sa.Hq = g.n_q_heads; sa.Hkv = Hkv; sa.G = c->group; sa.P = P; sa.T = g.n_sink;
   const size_t key_bytes = (size_t)P * sizeof(float);
   sa.keys_in_smem = key_bytes <= 200 * 1024;
+  sa.pool_rows = c->pool_rows;
   sa.value_feature = g.sim_feature;
   const size_t sel_sm = sa.keys_in_smem ? key_bytes : 0;
   cudaError_t e = cudaFuncSetAttribute(select_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -563,7 +575,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   SimArgs ma;
   ma.budgets = sa.budgets; ma.row_off = sa.row_off;
   ma.evict_idx = sa.evict_idx; ma.evict_mx = (float*)(X + c->slay.evict_mx); ma.evict_nn = (int32_t*)(X + c->slay.evict_nn);
-  ma.rnorm = sa.rnorm; ma.pos = sa.pos; ma.L = L; ma.layer = layer; ma.Hkv = Hkv; ma.P = P;
+  ma.rnorm = sa.rnorm; ma.pos = sa.pos; ma.status = sa.status; ma.L = L; ma.layer = layer; ma.Hkv = Hkv; ma.P = P;
   const size_t sim_sm = ((size_t)2 * D * kSimTile + 2 * kSimTile) * sizeof(float);
   e = cudaFuncSetAttribute(similarity_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sim_sm);
   if (e != cudaSuccess) return e;
@@ -596,7 +608,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   mg.budgets = sa.budgets; mg.row_off = sa.row_off; mg.evict_idx = sa.evict_idx; mg.evict_mx = ma.evict_mx;
   mg.seg_start = ga.seg_start; mg.seg_items = ga.seg_items; mg.rnorm = sa.rnorm;
   mg.L = L; mg.layer = layer; mg.Hkv = Hkv; mg.P = P; mg.seg_stride = seg_stride; mg.average = g.merge_policy;
-  mg.value_feature = g.sim_feature;
+  mg.value_feature = g.sim_feature; mg.status = sa.status;
   constexpr int LPR = D / Elem<T>::kPerVec;
   const int rows_per_cta = 256 / LPR;
   dim3 mgrid((maxS + rows_per_cta - 1) / rows_per_cta, n_slices);

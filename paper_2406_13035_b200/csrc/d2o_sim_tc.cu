@@ -278,6 +278,7 @@ struct NnReduceArgs {
   const unsigned long long* part_key;
   const float* rnorm;                       // pool-wide 1/|k_c|
   float* evict_mx; int32_t* evict_nn;
+  uint32_t* status;
   int L, layer, Hkv, P, n_chunks_max;
 };
 
@@ -295,6 +296,7 @@ neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K, const T* __rest
   if (i >= Le) return;
   const unsigned gmask = group_mask<LPR>();
   const int pos = a.evict_idx[(size_t)slice * a.P + i];
+  if (!D2O_GUARD(pos >= 0 && pos < a.P, a.status, 0xC4EC0008u)) return;      // uniform for the row's lanes
   float f[EPV];
   Elem<T>::unpack(ld_global_v4(K + ((size_t)slice * a.P + pos) * D + lig * EPV), f);
   float ss = 0.f;
@@ -423,7 +425,7 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   if (e != cudaSuccess) return e;
 
   NnReduceArgs r;
-  r.budgets = a.budgets; r.row_off = a.row_off; r.rnorm = a.rnorm;
+  r.budgets = a.budgets; r.row_off = a.row_off; r.rnorm = a.rnorm; r.status = a.status;
   r.evict_idx = (const int32_t*)(X + c->slay.evict_idx); r.part_key = a.part_key;
   r.evict_mx = (float*)(X + c->slay.evict_mx); r.evict_nn = (int32_t*)(X + c->slay.evict_nn);
   r.L = g.n_layers; r.layer = layer; r.Hkv = Hkv; r.P = P; r.n_chunks_max = n_chunks_max;
