@@ -107,6 +107,7 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   l->order = take(B * L * 4);
   l->len = take(L * B * Hkv * 4);
   l->tau = take(L * B * Hkv * 4);
+  l->guess = take(L * B * Hkv * 2 * 4);
   l->colsum = take(L * B * Hq * P * 4);
   l->pos = take(rows * 4);
   l->score = take(rows * 4);

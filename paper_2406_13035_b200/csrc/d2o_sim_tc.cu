@@ -54,31 +54,34 @@ __host__ __device__ __forceinline__ int chunk_columns(int S) {
 
 // One block of 32 accumulator columns of one row: times 1/|k_c| per column, maximum and its column (the lowest
 // on ties), merged into the row's running (best, best_col).  cl0 = chunk-local column of the block.
-//
-// The maximum is tracked on the bit patterns as signed integers: for values >= +0 that is the order of the floats,
-// and every negative value (and -0) sorts below +0, in the wrong order among themselves.  A row whose true maximum is
-// negative therefore ends with a negative pattern; it is reported as "nothing found" and neighbour_reduce_kernel
-// redoes that row with plain fp32 arithmetic.  In exchange the compare and the value select are one integer
-// max-with-predicate instruction, which is what the scan is bound by.
 __device__ __forceinline__ void scan_block(const uint32_t (&r)[32], const float* s_rn, int cl0, int n_cols, int c0,
-                                           int& best, int& best_col) {
-  // four interleaved running maxima (columns i mod 4) keep the dependent chains short
-  int tb[4], ti[4];
+                                           float& best, int& best_col) {
+  // four interleaved running maxima (columns i mod 4) keep the compare chains short
+  float tb[4]; int ti[4];
 #pragma unroll
-  for (int w = 0; w < 4; ++w) { tb[w] = INT_MIN; ti[w] = w; }
+  for (int w = 0; w < 4; ++w) { tb[w] = -INFINITY; ti[w] = w; }
   const float4* rn4 = reinterpret_cast<const float4*>(s_rn + cl0);
-  const bool whole = cl0 + 32 <= n_cols;                          // else: columns past the chunk hold other slices' rows
+  if (cl0 + 32 <= n_cols) {
 #pragma unroll
-  for (int i4 = 0; i4 < 8; ++i4) {
-    const float4 q = rn4[i4];
-    const float rv[4] = {q.x, q.y, q.z, q.w};
+    for (int i4 = 0; i4 < 8; ++i4) {
+      const float4 q = rn4[i4];
+      const float rv[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      int x = __float_as_int(__uint_as_float(r[i4 * 4 + w]) * rv[w]);
-      if (!whole && cl0 + i4 * 4 + w >= n_cols) x = INT_MIN;
-      bool keep;
-      tb[w] = __vibmax_s32(tb[w], x, &keep);                      // keep = (tb >= x): the earlier column stays on ties
-      ti[w] = keep ? ti[w] : i4 * 4 + w;
+      for (int w = 0; w < 4; ++w) {
+        const float x = __uint_as_float(r[i4 * 4 + w]) * rv[w];
+        if (x > tb[w]) { tb[w] = x; ti[w] = i4 * 4 + w; }
+      }
+    }
+  } else {                                                        // columns past the chunk hold other slices' rows
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4) {
+      const float4 q = rn4[i4];
+      const float rv[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float x = __uint_as_float(r[i4 * 4 + w]) * rv[w];
+        if (cl0 + i4 * 4 + w < n_cols && x > tb[w]) { tb[w] = x; ti[w] = i4 * 4 + w; }
+      }
     }
   }
   // larger value wins, equal values go to the lower column
@@ -216,7 +219,7 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
       tc::fence_after_sync();
       if (n_blk > 0) tc::tmem_ld32_issue(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(blk0 * 32), ra);
     }
-    int best = INT_MIN, best_col = 0x7fffffff;               // bit pattern of the best value so far (see scan_block)
+    float best = -INFINITY; int best_col = 0x7fffffff;
 #pragma unroll 1
     for (int job = 0; job < n_jobs; ++job) {
       const int t = t0 + job / n_nt, j = job % n_nt;
@@ -244,10 +247,10 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
       }
       if (n_blk > 1) scan_block(rb, s_rn, col0 + 32, n_cols, c0, best, best_col);
       if (j == n_nt - 1) {
-        // (ordered value, inverted slot): larger is better, ties go to the lower slot.  A non-negative float's
-        // ordered form is its pattern with the top bit set; a negative pattern means "nothing found" (key 0)
-        const unsigned long long key = best >= 0
-            ? (((unsigned long long)(0x80000000u | (uint32_t)best) << 32) | (uint32_t)(0x7fffffff - best_col)) : 0ull;
+        // (ordered value, inverted slot): larger is better, ties go to the lower slot; -0 counts as +0
+        if (best == 0.f) best = 0.f;
+        const unsigned long long key = best > -INFINITY
+            ? (((unsigned long long)float_ord(best) << 32) | (uint32_t)(0x7fffffff - best_col)) : 0ull;
         if (part > 0) s_pair[(part - 1) * kTileM + row] = key;
         asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
         if (part == 0) {
@@ -258,7 +261,7 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
           if (pos < a.P) out_keys[pos] = k;
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
-        best = INT_MIN; best_col = 0x7fffffff;
+        best = -INFINITY; best_col = 0x7fffffff;
       }
     }
   }
@@ -314,9 +317,9 @@ neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K, const T* __rest
   float mx = ord_float((uint32_t)(key >> 32)) * rn;
   bool found = key != 0ull && (unsigned)slot < (unsigned)S;
   if (!found) {
-    // No chunk reported a non-negative maximum: every similarity of this row is negative (or not finite).  The row
-    // is redone here in fp32, all retained rows in slot order (the first maximum stays).  A row without any finite
-    // similarity gets maximum -inf and neighbour 0 and is never merged.
+    // No chunk reported a maximum (no finite similarity in the row: non-finite keys).  The row is redone here in
+    // fp32, all retained rows in slot order (the first maximum stays); without any finite similarity it gets maximum
+    // -inf and neighbour 0 and is never merged.
     const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
     float best = -INFINITY; int bj = 0;
     for (int j = 0; j < S; ++j) {
