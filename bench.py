@@ -518,6 +518,8 @@ def run_ours(args, wl, rank, world, device):
             todo.append((f"cfg4_B{bsz}", c, True))
         todo.append(("cfg4_B8_unclamped", dataclasses.replace(W.CONFIGS["cfg4"], max_budget=0, name="cfg4[B=8,unclamped]"),
                      False))
+        # the multi-turn (streaming) shape of the paper's appendix: fixed budget 2048 = 48 important + 2000 recent tokens
+        todo.append(("streaming_session", W.CONFIGS["session"], False))
         for key, c, fc in todo:
             try:
                 per[key] = per_config_entry(B, c, device, args, peaks, full_cache=fc)

@@ -136,6 +136,14 @@ d2o_status d2o_create(const d2o_config* cfg, void* state, size_t state_bytes,
                       void* scratch, size_t scratch_bytes, void* stream, d2o_ctx** out);
 void d2o_destroy(d2o_ctx* ctx);
 
+/* Ragged batches: lens HOST int32 [B], the prompt length of every sequence (1 .. prompt_len).  The prompt
+ * tensors keep their layout for prompt_len positions per sequence; the positions beyond a sequence's length are
+ * padding and are never used.  Every sequence gets Eq. 4-5 over its own prompt (its own S_l with
+ * sum_l S_l = round(rho * L * its length)), and its generated tokens continue at its own length.  Call before
+ * the first d2o_layer_stats of a prompt; returns D2O_ERR_STATE afterwards, D2O_ERR_INVALID_ARG if a length
+ * does not satisfy the conditions d2o_create checks for prompt_len.  Synchronises `stream`. */
+d2o_status d2o_set_prompt_lens(d2o_ctx* ctx, const int32_t* lens, void* stream);
+
 /* (1) Eq. 4 for one layer.  Q DEVICE [B, Hq, P, d], K DEVICE [B, Hkv, P, d].
  * Computes s = column sums of the causal prompt attention Softmax(Q K^T / sqrt(d)) per query
  * head and F_v = Var(s).  `lse` (DEVICE float [B, Hq, P], natural-log row normalisers of that

@@ -25,7 +25,7 @@ EXPORTS = [
     "d2o_status_string", "d2o_last_cuda_error", "d2o_workspace_size", "d2o_create", "d2o_destroy",
     "d2o_layer_stats", "d2o_layer_budgets", "d2o_budgets_from_density", "d2o_prefill_compress",
     "d2o_decode_step", "d2o_decode_step_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
-    "d2o_set_tuning", "d2o_layer_stats_static", "d2o_set_fault_injection",
+    "d2o_set_tuning", "d2o_layer_stats_static", "d2o_set_fault_injection", "d2o_set_prompt_lens",
 ]
 STATIC_LSE_FLOATS = 1 << 20      # D2O_STATIC_LSE_FLOATS of include/d2o.h
 
@@ -100,6 +100,7 @@ def load_library() -> C.CDLL:
     lib.d2o_set_tuning.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32]
     lib.d2o_layer_stats_static.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.d2o_set_fault_injection.argtypes = [vp, i32, i32]
+    lib.d2o_set_prompt_lens.argtypes = [vp, vp, vp]
     for name in EXPORTS:
         if name not in ("d2o_status_string", "d2o_last_cuda_error", "d2o_destroy"):
             getattr(lib, name).restype = C.c_int
@@ -179,6 +180,11 @@ class D2OContext:
             pass
 
     # ---- the path
+    def d2o_set_prompt_lens(self, lens):
+        t = torch.as_tensor(lens, dtype=torch.int32).contiguous()
+        assert t.numel() == self.cfg.batch and t.device.type == "cpu"
+        _check(self.lib.d2o_set_prompt_lens(self.handle, t.data_ptr(), _stream()), "d2o_set_prompt_lens")
+
     def d2o_layer_stats(self, layer: int, Q: torch.Tensor, K: torch.Tensor, lse: Optional[torch.Tensor] = None):
         _check(self.lib.d2o_layer_stats(self.handle, layer, _ptr(Q), _ptr(K), _ptr(lse), _stream()), "d2o_layer_stats")
 

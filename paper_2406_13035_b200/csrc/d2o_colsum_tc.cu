@@ -34,7 +34,8 @@ struct ColsumTcArgs {
   float* lse2;                               // [B, Hq, P] log2-domain row normalisers (written by sweep 1, read by sweep 2)
   float* colsum;                             // [B, Hq, P] (sweep 2)
   uint32_t* status;
-  int P, Hq, group;
+  const int32_t* plen;                       // [B] prompt length of every sequence (<= P)
+  int P, Hq, group;                          // P: the length the tensors are laid out for
 };
 
 namespace tc {
@@ -70,16 +71,17 @@ attn_tc_kernel(ColsumTcArgs a, const __grid_constant__ CUtensorMap map_q, const 
   __shared__ int s_fail;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int P = a.P;
+  const int bh = blockIdx.x;                                 // b * Hq + hq (fastest index: all heads of the heaviest pair first)
+  const int b = bh / a.Hq, hq = bh % a.Hq;
+  const int P = a.plen[b];                                   // this sequence's prompt; rows beyond it are padding
   const int n_pairs = (P + 2 * kCsTile - 1) / (2 * kCsTile);
   const int n_tiles = (P + kCsTile - 1) / kCsTile;
-  const int bh = blockIdx.y;                                 // b * Hq + hq
-  const int b = bh / a.Hq, hq = bh % a.Hq;
+  if ((int)blockIdx.y >= n_pairs) return;                    // the grid is sized for the longest prompt
   const int Hkv = a.Hq / a.group;
-  const int q_base = bh * P;                                 // first row of this head in the [B*Hq*P, d] view of Q
-  const int k_base = (b * Hkv + hq / a.group) * P;
+  const int q_base = bh * a.P;                               // first row of this head in the [B*Hq*P, d] view of Q
+  const int k_base = (b * Hkv + hq / a.group) * a.P;
   // heaviest CTAs first: sweep 1 -> the last rows see the most keys; sweep 2 -> the first keys see the most rows
-  const int pair = SWEEP == kSweepRows ? n_pairs - 1 - (int)blockIdx.x : (int)blockIdx.x;
+  const int pair = SWEEP == kSweepRows ? n_pairs - 1 - (int)blockIdx.y : (int)blockIdx.y;
   const int a0 = pair * 2 * kCsTile;                         // first A row (query position or key position)
   // streamed tiles: sweep 1 keys [0, a0 + 256), sweep 2 queries [a0, P)
   const int bt0 = SWEEP == kSweepRows ? 0 : a0 / kCsTile;
@@ -123,12 +125,13 @@ attn_tc_kernel(ColsumTcArgs a, const __grid_constant__ CUtensorMap map_q, const 
         if (job >= kCsStages && !s_fail && !tc::mbar_wait(&b_empty[s], (uint32_t)(((job / kCsStages) - 1) & 1))) s_fail = 1;
         const int r0 = (bt0 + job) * kCsTile;                // first B row of the tile
         uint32_t bytes = (uint32_t)TILE;
-        const int n_lse = SWEEP == kSweepCols ? min(kCsTile, P - r0) : 0;      // P is a multiple of 4: 16-byte granules
+        // 16-byte granules: up to three entries past the prompt come from the row's padding and are masked
+        const int n_lse = SWEEP == kSweepCols ? min(kCsTile, ((P + 3) & ~3) - r0) : 0;
         bytes += (uint32_t)(n_lse * 4);
         tc::mbar_expect_tx(&b_full[s], bytes);
         for (int kb = 0; kb < KB; ++kb)
           tc::tma_load_2d(sB + s * TILE + kb * BLOCK, map_b, kb * 64, b_base + r0, &b_full[s]);
-        if (n_lse > 0) tc::bulk_g2s(s_lse + s * kCsTile, a.lse2 + (size_t)bh * P + r0, (uint32_t)(n_lse * 4), &b_full[s]);
+        if (n_lse > 0) tc::bulk_g2s(s_lse + s * kCsTile, a.lse2 + (size_t)bh * a.P + r0, (uint32_t)(n_lse * 4), &b_full[s]);
       }
     }
   } else if (warp == 1) {
@@ -250,13 +253,13 @@ attn_tc_kernel(ColsumTcArgs a, const __grid_constant__ CUtensorMap map_q, const 
         const float mm = fmaxf(m_run, m2);
         const float ll = (m_run > -INFINITY ? l_run * exp2f((m_run - mm) * c) : 0.f) +
                          (m2 > -INFINITY ? l2 * exp2f((m2 - mm) * c) : 0.f);
-        a.lse2[(size_t)bh * P + arow] = fmaf(mm, c, log2f(ll));
+        a.lse2[(size_t)bh * a.P + arow] = fmaf(mm, c, log2f(ll));
       }
     } else {
       double* dcomb = reinterpret_cast<double*>(s_comb);
       if (bhalf == 1) dcomb[at * kCsTile + r] = col_acc;
       asm volatile("bar.sync 1, %0;" ::"n"(kCsEpiWarps * 32) : "memory");
-      if (bhalf == 0 && arow < P) a.colsum[(size_t)bh * P + arow] = (float)(col_acc + dcomb[at * kCsTile + r]);
+      if (bhalf == 0 && arow < P) a.colsum[(size_t)bh * a.P + arow] = (float)(col_acc + dcomb[at * kCsTile + r]);
     }
   }
   tc::fence_before_sync();
@@ -265,7 +268,7 @@ attn_tc_kernel(ColsumTcArgs a, const __grid_constant__ CUtensorMap map_q, const 
     tc::fence_after_sync();
     tc::tmem_dealloc(tmem_base, 512);
   }
-  if (tid == 0 && s_fail) report_error(a.status, D2O_ERR_TIMEOUT, 0xC5C00000u | (uint32_t)(blockIdx.y & 0xfffff));
+  if (tid == 0 && s_fail) report_error(a.status, D2O_ERR_TIMEOUT, 0xC5C00000u | (uint32_t)(bh & 0xfffff));
 }
 
 // natural-log row normalisers supplied by the caller -> log2 domain
@@ -291,10 +294,12 @@ cudaError_t launch_colsum_tc(const d2o_ctx* c, const void* Q, const void* K, con
   a.colsum = colsum;
   a.status = (uint32_t*)(c->state + c->lay.status);
   a.P = P; a.Hq = Hq; a.group = c->group;
+  a.plen = (const int32_t*)(c->state + c->lay.plen);
   const int KB = D / 64;
   const size_t smem = (size_t)(2 + kCsStages) * KB * kCsTile * 128 + (size_t)kCsStages * kCsTile * 4 + 4 * kCsTile * 4;
   const int n_pairs = (P + 2 * kCsTile - 1) / (2 * kCsTile);
-  dim3 grid(n_pairs, B * Hq);
+  // heaviest CTAs first over the whole launch: the pair index is the slow grid dimension
+  dim3 grid(B * Hq, n_pairs);
   const int fmt = g.dtype == D2O_F16 ? 0 : 1;
   cudaError_t e;
 #define D2O_LAUNCH_CS(DD, FF, SW)                                                                                  \

@@ -146,7 +146,7 @@ enum Counter { kCntDecodeSteps = 0, kCntEvictions, kCntMerges, kCntDiscards, kCn
 
 // ----------------------------------------------------------------------------- context
 struct Layout {            // byte offsets into `state`
-  size_t status, counters, density, budgets, windows, row_off, order, len, tau, guess, colsum, pos, score, rnorm, kpool, vpool, end;
+  size_t status, counters, density, budgets, windows, row_off, order, plen, len, tau, guess, sim_items, colsum, pos, score, rnorm, kpool, vpool, end;
 };
 struct ScratchLayout {     // byte offsets into `scratch`
   size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, seg_tmp, part_key, pl_spill, stage_q, stage_k, stage_v, stage_out, end;
@@ -177,6 +177,9 @@ struct d2o_ctx {
   uint8_t* layer_fed;          // [L] stats seen
   uint8_t* layer_compressed;   // [L]
   int32_t* layer_steps;        // [L] decode steps taken
+  int32_t* h_plen;             // [B] prompt length of every sequence (prompt_len unless d2o_set_prompt_lens was called)
+  int32_t* h_sim_count;        // [L] work items of the tensor-core similarity kernel per layer
+  int4* h_sim_items;           // host copy of the work lists (device copy in `state`)
   int32_t* h_order;            // [L * B] (layer * B + b) sorted by cache size, largest first (device copy in `state`)
   int decode_stages;           // tuning: stages of the decode kernel's ring, 0 = auto
   int decode_warps;            // tuning: consumer warps per decode CTA (4, 8, 16), 0 = auto
@@ -198,7 +201,7 @@ cudaError_t launch_layer_stats(const d2o_ctx* c, int layer, const void* Q, const
 cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, int P, float rho, int min_budget,
                            int max_budget, float gamma, int head_reduce, int budget_rule, int n_sink, int window,
                            float nm_ratio, int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
-                           cudaStream_t st);
+                           const int32_t* plen, cudaStream_t st);
 cudaError_t launch_prefill_compress(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st);
 cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const void* k, const void* v, void* out,
                           cudaStream_t st, d2o_status* why);
@@ -209,6 +212,8 @@ cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int ca
 // tensor-core similarity + nearest neighbour for 16-bit keys (d2o_sim_tc.cu); fills evict_mx / evict_nn
 cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int max_S, cudaStream_t st);
 size_t sim_tc_part_key_bytes(const d2o_config* cfg, int max_budget);
+size_t sim_tc_max_items(const d2o_config* cfg, int max_budget);
+void sim_tc_build_items(const d2o_ctx* c, int n_sms, int4* items, int32_t* count);
 // tensor-core column sums of the prompt attention for 16-bit Q/K (d2o_colsum_tc.cu)
 bool colsum_tc_supported(const d2o_config* cfg);
 cudaError_t launch_colsum_tc(const d2o_ctx* c, const void* Q, const void* K, const float* lse_in, float* colsum,

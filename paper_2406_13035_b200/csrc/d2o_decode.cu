@@ -52,7 +52,8 @@ struct DecodeArgs {
   int32_t* len; float* tau;                                                  // [L, B, Hkv]
   int32_t* guess;                                                            // [L, B, Hkv][2] rows guessed for the next step's victim (-2: none yet)
   unsigned long long* counters; uint32_t* status;
-  int L, l0, B, Hkv, T, t;          // t = position of the token generated in this step
+  const int32_t* plen;              // [B] prompt length of every sequence
+  int L, l0, B, Hkv, T, step;       // step = number of tokens generated before this one: its position is plen[b] + step
   float beta, tau_override;
   int row_cap;                      // rows of a slice whose logits / probabilities live in shared memory (multiple of 8)
   float* spill;                     // the same for rows >= row_cap: [(row0 + 8 slice) G + g (stride(S) + 8) + row], stays in L2
@@ -328,6 +329,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   const T* v_new = v_in + (size_t)sl * D;
 
   // ---- slice parameters
+  const int t_pos = a.plen[b] + a.step;                                // position of the token generated in this step
   const int S = a.budgets[slice_entry(b, layer, h, a.L, a.Hkv)];
   const int M = a.windows[slice_entry(b, layer, h, a.L, a.Hkv)];
   const int64_t row0 = a.row_off[slice_entry(b, layer, h, a.L, a.Hkv)];
@@ -540,7 +542,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
 #pragma unroll
     for (int c = 0; c < NC; ++c) { my[c] = ~0ull; my_li[c] = -1; }
     auto offer = [&](float sc, int pz, int li) {
-      if (pz >= Tn && pz <= a.t - M) {
+      if (pz >= Tn && pz <= t_pos - M) {
         unsigned long long key = ((unsigned long long)float_ord(sc) << 32) | (uint32_t)(0x7fffffff - pz);
         int kl = li;
 #pragma unroll
@@ -707,7 +709,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
 #pragma unroll
           for (int e = 0; e < EPV; ++e) x = fmaf(cf[e], kf[e], x);
           x = warp_sum(x);
-          if (lane == 0) cand_update(c, x, s_new_rn, a.t, n_old);
+          if (lane == 0) cand_update(c, x, s_new_rn, t_pos, n_old);
         }
       }
     }
@@ -744,7 +746,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       const int li = s * SR + (lig / QL) * NGRP + grp;               // the row whose total this lane receives
       // its 1/|k| and position leave the stage before the stage is released
       const bool cand_lane = evict && li < n && lig % QL == 0;
-      float rn_li = s_new_rn; int ps_li = a.t;
+      float rn_li = s_new_rn; int ps_li = t_pos;
       if (cand_lane && li < n_old) { rn_li = meta_rn[(size_t)slot * SR + (li - s * SR)]; ps_li = meta_ps[(size_t)slot * SR + (li - s * SR)]; }
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_empty[slot]);
@@ -839,7 +841,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
 #pragma unroll
     for (int c = 0; c < NG; ++c) { nx[c] = ~0ull; nx_li[c] = -1; }
     auto offer_next = [&](float sc, int pz, int li) {
-      if (pz >= Tn && pz <= a.t + 1 - M) {
+      if (pz >= Tn && pz <= t_pos + 1 - M) {
         unsigned long long key = ((unsigned long long)float_ord(sc) << 32) | (uint32_t)(0x7fffffff - pz);
         int kl = li;
 #pragma unroll
@@ -865,7 +867,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         const int pv[4] = {pz.x, pz.y, pz.z, pz.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          if (pv[j] >= Tn && pv[j] <= a.t - M) {
+          if (pv[j] >= Tn && pv[j] <= t_pos - M) {
             const unsigned long long key = ((unsigned long long)float_ord(sv[j]) << 32) | (uint32_t)(0x7fffffff - pv[j]);
             if (key < my_min) { my_min = key; my_min_li = li + j; }
           }
@@ -880,8 +882,8 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       const float s_new = (li < n_old ? a.score[row0 + li] : 0.f) + p;
       if (li < n_old || !evict) a.score[row0 + li] = s_new;          // the new token's score is placed with its row
       else s_new_score = s_new;
-      const int pz = li < n_old ? a.pos[row0 + li] : a.t;
-      if (evict && pz >= Tn && pz <= a.t - M) {                      // lowest score, ties -> latest position
+      const int pz = li < n_old ? a.pos[row0 + li] : t_pos;
+      if (evict && pz >= Tn && pz <= t_pos - M) {                      // lowest score, ties -> latest position
         const unsigned long long key = ((unsigned long long)float_ord(s_new) << 32) | (uint32_t)(0x7fffffff - pz);
         if (key < my_min) { my_min = key; my_min_li = li; }
       }
@@ -976,7 +978,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
 #pragma unroll
         for (int e = 0; e < EPV; ++e) x = fmaf(kvic[e], f[e], x);
         x = group_sum<LPR>(x, gmask);
-        const unsigned long long key = ((unsigned long long)sim_ord(x * vic_rn * s_new_rn) << 32) | (uint32_t)(0x7fffffff - a.t);
+        const unsigned long long key = ((unsigned long long)sim_ord(x * vic_rn * s_new_rn) << 32) | (uint32_t)(0x7fffffff - t_pos);
         if (lig == 0 && key > best) { best = key; best_li = n_old; }
       }
     }
@@ -1022,7 +1024,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       if (vic_li != n_old) {
         *reinterpret_cast<uint4*>(kpool + (row0 + vic_li) * D + lane * EPV) = kslot;
         if (lane == 0) {
-          a.pos[row0 + vic_li] = a.t;
+          a.pos[row0 + vic_li] = t_pos;
           a.score[row0 + vic_li] = s_new_score;
           a.rnorm[row0 + vic_li] = rn_slot;
         }
@@ -1213,7 +1215,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     if (grp == 0) {
       *reinterpret_cast<uint4*>(kpool + (row0 + n_old) * D + lig * EPV) = knew;
       *reinterpret_cast<uint4*>(vpool + (row0 + n_old) * D + lig * EPV) = vnew;
-      if (lig == 0) { a.pos[row0 + n_old] = a.t; a.rnorm[row0 + n_old] = s_new_rn; }
+      if (lig == 0) { a.pos[row0 + n_old] = t_pos; a.rnorm[row0 + n_old] = s_new_rn; }
     }
     if (tid == 0) {
       a.len[sidx] = n;
@@ -1346,7 +1348,8 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   a.guess = (int32_t*)(S + c->lay.guess);
   a.counters = (unsigned long long*)(S + c->lay.counters); a.status = (uint32_t*)(S + c->lay.status);
   a.L = L; a.l0 = l0; a.B = B; a.Hkv = g.n_kv_heads; a.T = g.n_sink;
-  a.t = g.prompt_len + c->layer_steps[l0];
+  a.step = c->layer_steps[l0];
+  a.plen = (const int32_t*)(S + c->lay.plen);
   a.beta = g.beta; a.tau_override = g.tau_override; a.average = g.merge_policy;
   a.wait_ns = c->wait_limit_us > 0 ? (unsigned long long)c->wait_limit_us * 1000ull : kWaitNs;
   a.stop_stage = c->producer_stop_stage;

@@ -105,9 +105,11 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   l->windows = take(B * L * Hkv * 4);
   l->row_off = take(B * L * Hkv * 8);
   l->order = take(B * L * 4);
+  l->plen = take(B * 4);
   l->len = take(L * B * Hkv * 4);
   l->tau = take(L * B * Hkv * 4);
   l->guess = take(L * B * Hkv * 2 * 4);
+  l->sim_items = take(c->dtype == D2O_F32 ? 0 : L * sim_tc_max_items(c, max_budget) * 16);
   l->colsum = take(L * B * Hq * P * 4);
   l->pos = take(rows * 4);
   l->score = take(rows * 4);
@@ -190,8 +192,15 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
   c->layer_compressed = (uint8_t*)calloc(cfg->n_layers, 1);
   c->layer_steps = (int32_t*)calloc(cfg->n_layers, 4);
   c->h_order = (int32_t*)calloc(BL, 4);
+  c->h_plen = (int32_t*)calloc(cfg->batch, 4);
+  c->h_sim_count = (int32_t*)calloc(cfg->n_layers, 4);
+  c->h_sim_items = cfg->dtype == D2O_F32 ? nullptr
+      : (int4*)malloc((size_t)cfg->n_layers * sim_tc_max_items(cfg, maxb) * sizeof(int4));
+  for (int b = 0; b < cfg->batch; ++b) c->h_plen[b] = cfg->prompt_len;
   // bookkeeping (status, counters, density, budgets ... tau) starts at zero
   cudaError_t e = cudaMemsetAsync(c->state, 0, l.colsum, (cudaStream_t)stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(c->state + l.plen, c->h_plen, (size_t)cfg->batch * 4, cudaMemcpyHostToDevice, (cudaStream_t)stream);
   if (e != cudaSuccess) { d2o_destroy(c); return cuda_fail(e, "cudaMemsetAsync(state)"); }
   *out = c;
   return D2O_OK;
@@ -200,7 +209,7 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
 extern "C" void d2o_destroy(d2o_ctx* c) {
   if (!c) return;
   free(c->h_budgets); free(c->h_windows); free(c->h_row_off); free(c->h_pair_max); free(c->h_pair_sum);
-  free(c->layer_fed); free(c->layer_compressed); free(c->layer_steps); free(c->h_order);
+  free(c->layer_fed); free(c->layer_compressed); free(c->layer_steps); free(c->h_order); free(c->h_plen); free(c->h_sim_count); free(c->h_sim_items);
   free(c);
 }
 
@@ -234,7 +243,7 @@ extern "C" d2o_status d2o_budgets_from_density(const double* density, int32_t ba
   if (budget_rule != 2 && (tot < units * min_budget || tot > units * max_budget)) return D2O_ERR_INVALID_ARG;
   CUDA_TRY(launch_budgets(density, batch, n_layers, n_heads, n_kv_heads, prompt_len, rho, min_budget, max_budget,
                           density_temp, head_reduce, budget_rule, n_sink, window, nm_ratio, budgets, windows, row_off,
-                          (uint32_t*)status_word, (cudaStream_t)stream));
+                          (uint32_t*)status_word, nullptr, (cudaStream_t)stream));
   return D2O_OK;
 }
 
@@ -248,9 +257,9 @@ extern "C" d2o_status d2o_layer_budgets(d2o_ctx* c, int32_t* budgets_host, void*
   int32_t* d_w = (int32_t*)(c->state + c->lay.windows);
   int64_t* d_o = (int64_t*)(c->state + c->lay.row_off);
   CUDA_TRY(launch_budgets((const double*)(c->state + c->lay.density), g.batch, g.n_layers, g.n_q_heads,
-                          g.n_kv_heads, g.prompt_len, g.rho, g.min_budget, c->max_budget, g.density_temp,
+                          g.n_kv_heads, g.prompt_len, g.rho, g.min_budget, g.max_budget, g.density_temp,
                           g.head_reduce, g.budget_rule, g.n_sink, g.window, g.nm_ratio, d_b, d_w, d_o,
-                          (uint32_t*)(c->state + c->lay.status), st));
+                          (uint32_t*)(c->state + c->lay.status), (const int32_t*)(c->state + c->lay.plen), st));
   const size_t BL = (size_t)g.batch * g.n_layers;
   const size_t Hkv = g.n_kv_heads, BLH = BL * Hkv;
   CUDA_TRY(cudaMemcpyAsync(c->h_budgets, d_b, BLH * 4, cudaMemcpyDeviceToHost, st));
@@ -279,6 +288,13 @@ extern "C" d2o_status d2o_layer_budgets(d2o_ctx* c, int32_t* budgets_host, void*
     });
   }
   CUDA_TRY(cudaMemcpyAsync(c->state + c->lay.order, c->h_order, BL * 4, cudaMemcpyHostToDevice, st));
+  if (c->h_sim_items) {
+    // work lists of the tensor-core similarity kernel for every layer (the budgets are all it needs)
+    sim_tc_build_items(c, c->n_sms, c->h_sim_items, c->h_sim_count);
+    CUDA_TRY(cudaMemcpyAsync(c->state + c->lay.sim_items, c->h_sim_items,
+                             (size_t)g.n_layers * sim_tc_max_items(&g, c->max_budget) * sizeof(int4),
+                             cudaMemcpyHostToDevice, st));
+  }
   CUDA_TRY(cudaStreamSynchronize(st));
   c->have_budgets = true;
   if (budgets_host) memcpy(budgets_host, c->h_budgets, BLH * 4);
@@ -440,5 +456,27 @@ extern "C" d2o_status d2o_set_fault_injection(d2o_ctx* c, int32_t wait_limit_us,
   if (!c || wait_limit_us < 0 || producer_stop_stage < -1) return D2O_ERR_INVALID_ARG;
   c->wait_limit_us = wait_limit_us;
   c->producer_stop_stage = producer_stop_stage;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_set_prompt_lens(d2o_ctx* c, const int32_t* lens_host, void* stream) {
+  if (!c || !lens_host) return D2O_ERR_INVALID_ARG;
+  const d2o_config& g = c->cfg;
+  for (int l = 0; l < g.n_layers; ++l)
+    if (c->layer_fed[l]) return D2O_ERR_STATE;                 // the lengths belong to the prompt that is about to be fed
+  for (int b = 0; b < g.batch; ++b) {
+    const int P = lens_host[b];
+    if (P < 1 || P > g.prompt_len) return D2O_ERR_INVALID_ARG;
+    // the same conditions d2o_create checks for prompt_len, for this sequence
+    const int maxb = g.max_budget > 0 ? g.max_budget : P;
+    if (maxb > P + g.max_new_tokens || g.min_budget > maxb) return D2O_ERR_INVALID_ARG;
+    const double units = g.budget_rule == 1 ? (double)g.n_layers * g.n_kv_heads : (double)g.n_layers;
+    const double tot = floor((double)g.rho * units * (double)P + 0.5);
+    if (g.budget_rule != 2 && (tot < units * g.min_budget || tot > units * maxb)) return D2O_ERR_INVALID_ARG;
+  }
+  memcpy(c->h_plen, lens_host, (size_t)g.batch * 4);
+  CUDA_TRY(cudaMemcpyAsync(c->state + c->lay.plen, c->h_plen, (size_t)g.batch * 4, cudaMemcpyHostToDevice,
+                           (cudaStream_t)stream));
+  CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));      // h_plen may change again before the copy would run
   return D2O_OK;
 }

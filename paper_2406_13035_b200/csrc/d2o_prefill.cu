@@ -32,6 +32,7 @@ struct SelectArgs {
   float* keys_spill;       // [B, Hkv, P] group scores when P does not fit in shared memory (may alias evict_mx)
   unsigned long long* counters;
   uint32_t* status;
+  const int32_t* plen;     // [B] prompt length of every sequence; P below is the length the tensors are laid out for
   int L, layer, B, Hq, Hkv, G, P, T;
   int keys_in_smem;
   long long pool_rows;     // rows of the cache pool (bounds of the checked build)
@@ -71,18 +72,19 @@ select_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
   __shared__ int s_need;
   const int slice = blockIdx.x;                 // b * Hkv + h
   const int b = slice / a.Hkv, h = slice % a.Hkv;
-  const int P = a.P;
+  const int Pmax = a.P;                         // row stride of the per-position arrays
+  const int P = a.plen[b];                      // this sequence's prompt length
   const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int Tn = a.T < S ? a.T : S;
   const int M = a.windows[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int sidx = (a.layer * a.B + b) * a.Hkv + h;
-  float* keys = a.keys_in_smem ? reinterpret_cast<float*>(sel_smem) : a.keys_spill + (size_t)slice * P;
+  float* keys = a.keys_in_smem ? reinterpret_cast<float*>(sel_smem) : a.keys_spill + (size_t)slice * Pmax;
   // group score: sum over the G query heads of this KV head, fixed order (Eq. 6 case 1)
-  const float* cs = a.colsum + ((size_t)b * a.Hq + (size_t)h * a.G) * P;
+  const float* cs = a.colsum + ((size_t)b * a.Hq + (size_t)h * a.G) * Pmax;
   for (int j = threadIdx.x; j < P; j += blockDim.x) {
     float t = cs[j];
-    for (int g = 1; g < a.G; ++g) t += cs[(size_t)g * P + j];
+    for (int g = 1; g < a.G; ++g) t += cs[(size_t)g * Pmax + j];
     keys[j] = t;
   }
   __syncthreads();
@@ -138,7 +140,7 @@ select_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
         }
       } else {
         const int at = n_ev + (threadIdx.x - kr);
-        if (D2O_GUARD(at >= 0 && at < P, a.status, 0xC4EC0002u)) a.evict_idx[(size_t)slice * P + at] = j;
+        if (D2O_GUARD(at >= 0 && at < P, a.status, 0xC4EC0002u)) a.evict_idx[(size_t)slice * Pmax + at] = j;
       }
     }
     const int valid = min((int)blockDim.x, P - base);
@@ -165,13 +167,13 @@ gather_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
   constexpr int LPR = D / EPV;                   // lanes per row
   const int slice = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
-  const int P = a.P;
+  const int P = a.plen[b];
   const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int n_keep = S >= P ? P : S;
   const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
-  const T* Ks = K + (size_t)slice * P * D;
-  const T* Vs = V + (size_t)slice * P * D;
+  const T* Ks = K + (size_t)slice * a.P * D;
+  const T* Vs = V + (size_t)slice * a.P * D;
   const int r1 = min(n_keep, ((int)blockIdx.x + 1) * 64);
   for (int r = blockIdx.x * 64 + grp; r < r1; r += blockDim.x / LPR) {
     const int j = a.pos[row0 + r];
@@ -198,6 +200,7 @@ struct SimArgs {
   const int32_t* evict_idx; float* evict_mx; int32_t* evict_nn;
   const float* rnorm; const int32_t* pos;
   uint32_t* status;
+  const int32_t* plen;
   int L, layer, Hkv, P;
 };
 
@@ -212,7 +215,7 @@ similarity_kernel(SimArgs a, const T* __restrict__ K, const T* __restrict__ kpoo
   const int slice = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
-  const int Le = a.P - S;
+  const int Le = a.plen[b] - S;
   const int i0 = blockIdx.x * kSimTile;
   if (Le <= 0 || i0 >= Le) return;
   const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
@@ -225,7 +228,7 @@ similarity_kernel(SimArgs a, const T* __restrict__ K, const T* __restrict__ kpoo
     const int r = threadIdx.x % kSimTile;
     bool ok = i0 + r < Le;
     const int j = ok ? ev[i0 + r] : 0;
-    if (ok && !D2O_GUARD(j >= 0 && j < a.P, a.status, 0xC4EC0004u)) ok = false;
+    if (ok && !D2O_GUARD(j >= 0 && j < a.plen[b], a.status, 0xC4EC0004u)) ok = false;
     float ss = 0.f;
     for (int vi = threadIdx.x / kSimTile; vi < VPR; vi += kSimThreads / kSimTile) {
       float f[EPV];
@@ -325,6 +328,7 @@ struct SegArgs {
   int32_t* seg_start; int32_t* seg_items; int32_t* seg_tmp; float* tau;
   unsigned long long* counters;
   uint32_t* status;
+  const int32_t* plen;
   int L, layer, B, Hkv, P, seg_stride;
   float tau_override;
 };
@@ -339,7 +343,7 @@ segment_kernel(SegArgs a) {
   const int slice = blockIdx.x;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
-  const int Le = a.P - S;
+  const int Le = a.plen[b] - S;
   const int sidx = (a.layer * a.B + b) * a.Hkv + h;
   const float* mx = a.evict_mx + (size_t)slice * a.P;
   const int32_t* nn = a.evict_nn + (size_t)slice * a.P;
@@ -462,6 +466,7 @@ struct MergeArgs {
   const int32_t* evict_idx; const float* evict_mx;
   const int32_t* seg_start; const int32_t* seg_items;
   float* rnorm;
+  const int32_t* plen;
   int L, layer, Hkv, P, seg_stride;
   uint32_t* status;
   int average;             // 1: average merge (every token of a merge weighs the same) instead of Eq. 12
@@ -477,14 +482,15 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   const int slice = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
-  if (a.P - S <= 0) return;
+  const int Le = a.plen[b] - S;
+  if (Le <= 0) return;
   const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
   const int j = blockIdx.x * (blockDim.x / LPR) + grp;
   if (j >= S) return;
   const int32_t* start = a.seg_start + (size_t)slice * a.seg_stride;
   const int s0 = start[j], s1 = start[j + 1];
   if (s1 == s0) return;                              // nothing merged: the row stays bit-identical
-  if (!D2O_GUARD(s0 >= 0 && s0 < s1 && s1 <= a.P - S, a.status, 0xC4EC0007u)) return;
+  if (!D2O_GUARD(s0 >= 0 && s0 < s1 && s1 <= Le, a.status, 0xC4EC0007u)) return;
   const int64_t row = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)] + j;
   const int32_t* items = a.seg_items + (size_t)slice * a.P;
   const int32_t* ev = a.evict_idx + (size_t)slice * a.P;
@@ -502,10 +508,10 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   float den = own;
   for (int s = s0; s < s1; ++s) {
     const int i = items[s];
-    if (!D2O_GUARD(i >= 0 && i < a.P - S, a.status, 0xC4EC0005u)) continue;
+    if (!D2O_GUARD(i >= 0 && i < Le, a.status, 0xC4EC0005u)) continue;
     const float w = a.average ? 1.0f : expf(mx[i]);
     const int pj = ev[i];
-    if (!D2O_GUARD(pj >= 0 && pj < a.P, a.status, 0xC4EC0006u)) continue;
+    if (!D2O_GUARD(pj >= 0 && pj < a.plen[b], a.status, 0xC4EC0006u)) continue;
     den += w;
     Elem<T>::unpack(ld_global_v4(Ks + (size_t)pj * D + lig * EPV), f);
 #pragma unroll
@@ -553,6 +559,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   sa.keys_spill = (float*)(X + c->slay.evict_mx);
   sa.counters = (unsigned long long*)(S + c->lay.counters);
   sa.status = (uint32_t*)(S + c->lay.status);
+  sa.plen = (const int32_t*)(S + c->lay.plen);
   sa.L = L; sa.layer = layer; sa.B = B; sa.Hq = g.n_q_heads; sa.Hkv = Hkv; sa.G = c->group; sa.P = P; sa.T = g.n_sink;
   const size_t key_bytes = (size_t)P * sizeof(float);
   sa.keys_in_smem = key_bytes <= 200 * 1024;
@@ -569,16 +576,15 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
     gather_kernel<T, D><<<ggrid, 256, 0, st>>>(sa, (const T*)K, (const T*)V, kpool, vpool);
   }
 
-  int minS = P;
+  int maxLe = 0;                                 // most evicted rows of any slice of this layer
   for (int b = 0; b < B; ++b)
-    for (int h = 0; h < Hkv; ++h) minS = min(minS, c->h_budgets[(b * L + layer) * Hkv + h]);
-  const int maxLe = P - minS;
+    for (int h = 0; h < Hkv; ++h) maxLe = max(maxLe, c->h_plen[b] - c->h_budgets[(b * L + layer) * Hkv + h]);
   if (maxLe <= 0) return cudaGetLastError();
 
   SimArgs ma;
   ma.budgets = sa.budgets; ma.row_off = sa.row_off;
   ma.evict_idx = sa.evict_idx; ma.evict_mx = (float*)(X + c->slay.evict_mx); ma.evict_nn = (int32_t*)(X + c->slay.evict_nn);
-  ma.rnorm = sa.rnorm; ma.pos = sa.pos; ma.status = sa.status; ma.L = L; ma.layer = layer; ma.Hkv = Hkv; ma.P = P;
+  ma.rnorm = sa.rnorm; ma.pos = sa.pos; ma.status = sa.status; ma.plen = sa.plen; ma.L = L; ma.layer = layer; ma.Hkv = Hkv; ma.P = P;
   const size_t sim_sm = ((size_t)2 * D * kSimTile + 2 * kSimTile) * sizeof(float);
   e = cudaFuncSetAttribute(similarity_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sim_sm);
   if (e != cudaSuccess) return e;
@@ -598,6 +604,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   ga.seg_start = (int32_t*)(X + c->slay.seg_start); ga.seg_items = (int32_t*)(X + c->slay.seg_items);
   ga.seg_tmp = (int32_t*)(X + c->slay.seg_tmp);
   ga.tau = sa.tau; ga.counters = sa.counters; ga.status = sa.status;
+  ga.plen = sa.plen;
   ga.L = L; ga.layer = layer; ga.B = B; ga.Hkv = Hkv; ga.P = P; ga.seg_stride = seg_stride;
   ga.tau_override = g.tau_override;
   // counts / cursors per retained slot, later the radix histograms (32 warps x 64 digits)
@@ -610,6 +617,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   MergeArgs mg;
   mg.budgets = sa.budgets; mg.row_off = sa.row_off; mg.evict_idx = sa.evict_idx; mg.evict_mx = ma.evict_mx;
   mg.seg_start = ga.seg_start; mg.seg_items = ga.seg_items; mg.rnorm = sa.rnorm;
+  mg.plen = sa.plen;
   mg.L = L; mg.layer = layer; mg.Hkv = Hkv; mg.P = P; mg.seg_stride = seg_stride; mg.average = g.merge_policy;
   mg.value_feature = g.sim_feature; mg.status = sa.status;
   constexpr int LPR = D / Elem<T>::kPerVec;

@@ -23,6 +23,11 @@
 #include <cuda.h>
 #include <limits.h>
 #include <math.h>
+#include <stdlib.h>
+
+#include <algorithm>
+#include <utility>
+#include <vector>
 
 #include "d2o_common.cuh"
 #include "d2o_tc.cuh"
@@ -42,7 +47,9 @@ struct SimTcArgs {
   const float* rnorm;                       // pool-wide 1/|k_c|
   unsigned long long* part_key;             // [slices][n_chunks_max][P]
   uint32_t* status;
-  int L, layer, Hkv, P, n_chunks_max, tiles_per_cta;
+  const int32_t* plen;                      // [B] prompt length of every sequence; P is the row stride per slice
+  const int4* items;                        // work list of this layer: (slice, chunk, first tile, end tile) per CTA
+  int L, layer, Hkv, P, n_chunks_max;
 };
 
 // Retained rows per chunk for a slice of S rows: ceil(S / kChunkN) chunks of equal size, rounded up to the MMA's
@@ -109,19 +116,21 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
   __shared__ int s_fail;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int slice = blockIdx.z;
-  const int nc = blockIdx.y;
+  const int4 item = a.items[blockIdx.x];
+  const int slice = item.x;
+  const int nc = item.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   const int chunk_cols = chunk_columns(S);                   // the retained rows are split evenly over the chunks
   const int c0 = nc * chunk_cols;                            // first retained slot of the chunk
-  if (c0 >= S || a.P - S <= 0) return;                       // uniform for the CTA: nothing to do
+  const int Pb = a.plen[b];                                  // this sequence's prompt length
+  if (c0 >= S || Pb - S <= 0) return;                        // uniform for the CTA: nothing to do
   const int n_cols = min(chunk_cols, S - c0);
   const int n_nt = (n_cols + kTileN - 1) / kTileN;           // MMA column tiles in this chunk (1 or 2)
   const int n_last = (n_cols - (n_nt - 1) * kTileN + 15) & ~15;   // columns of the last tile's MMA (multiple of 16)
-  const int n_tiles_all = (a.P + kTileM - 1) / kTileM;
-  const int t0 = blockIdx.x * a.tiles_per_cta;
-  const int t1 = min(n_tiles_all, t0 + a.tiles_per_cta);
+  const int n_tiles_all = (Pb + kTileM - 1) / kTileM;
+  const int t0 = item.z;
+  const int t1 = min(n_tiles_all, item.w);
   if (t0 >= t1) return;
   const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   if ((tc::smem_u32(tc_smem) & 1023u) != 0u) {               // swizzled tiles need 1024-byte aligned shared memory
@@ -258,7 +267,7 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
 #pragma unroll
           for (int o = 0; o < 3; ++o) { const unsigned long long other = s_pair[o * kTileM + row]; k = other > k ? other : k; }
           const int pos = t * kTileM + row;
-          if (pos < a.P) out_keys[pos] = k;
+          if (pos < Pb) out_keys[pos] = k;
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
         best = -INFINITY; best_col = 0x7fffffff;
@@ -271,7 +280,7 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
     tc::fence_after_sync();
     tc::tmem_dealloc(tmem_base, 512);
   }
-  if (tid == 0 && s_fail) report_error(a.status, D2O_ERR_TIMEOUT, 0x51C00000u | (uint32_t)(blockIdx.z & 0xfffff));
+  if (tid == 0 && s_fail) report_error(a.status, D2O_ERR_TIMEOUT, 0x51C00000u | (uint32_t)(slice & 0xfffff));
 }
 
 // mx_i = 1/|k_i| * max over the chunks of the partial maxima, nn_i = its slot, for the evicted positions.
@@ -282,6 +291,7 @@ struct NnReduceArgs {
   const float* rnorm;                       // pool-wide 1/|k_c|
   float* evict_mx; int32_t* evict_nn;
   uint32_t* status;
+  const int32_t* plen;
   int L, layer, Hkv, P, n_chunks_max;
 };
 
@@ -293,13 +303,13 @@ neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K, const T* __rest
   const int slice = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
-  const int Le = a.P - S;
+  const int Le = a.plen[b] - S;
   const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
   const int i = blockIdx.x * (blockDim.x / LPR) + grp;
   if (i >= Le) return;
   const unsigned gmask = group_mask<LPR>();
   const int pos = a.evict_idx[(size_t)slice * a.P + i];
-  if (!D2O_GUARD(pos >= 0 && pos < a.P, a.status, 0xC4EC0008u)) return;      // uniform for the row's lanes
+  if (!D2O_GUARD(pos >= 0 && pos < a.plen[b], a.status, 0xC4EC0008u)) return;      // uniform for the row's lanes
   float f[EPV];
   Elem<T>::unpack(ld_global_v4(K + ((size_t)slice * a.P + pos) * D + lig * EPV), f);
   float ss = 0.f;
@@ -371,6 +381,66 @@ bool encode_rows_2d(CUtensorMap* map, int dtype, const void* base, uint64_t rows
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Upper bound of the work items of one layer: one per (slice, chunk) plus the splits into tile ranges.
+size_t sim_tc_max_items(const d2o_config* cfg, int max_budget) {
+  const size_t chunks = ((size_t)max_budget + kChunkN - 1) / kChunkN;
+  return (size_t)cfg->batch * cfg->n_kv_heads * chunks + 2048;
+}
+
+// The work lists of all layers, built on the host once the budgets are known: every (slice, chunk of retained rows)
+// is cut into ranges of prompt tiles of about equal work (tiles x columns), so that one launch is several full waves
+// of CTAs of the same length whatever the spread of the budgets; longest first.  `items` has room for
+// n_layers * sim_tc_max_items() entries, `count[layer]` receives the entries of each layer.
+void sim_tc_build_items(const d2o_ctx* c, int n_sms, int4* items, int32_t* count) {
+  const d2o_config& g = c->cfg;
+  const int B = g.batch, Hkv = g.n_kv_heads, L = g.n_layers;
+  const size_t cap = sim_tc_max_items(&g, c->max_budget);
+  struct Piece { int slice, chunk, tiles, cols; };
+  Piece* pieces = (Piece*)malloc(sizeof(Piece) * (size_t)B * Hkv * ((c->max_budget + kChunkN - 1) / kChunkN + 1));
+  for (int layer = 0; layer < L; ++layer) {
+    int4* out = items + (size_t)layer * cap;
+    size_t n_pieces = 0;
+    double total = 0.0;
+    for (int b = 0; b < B; ++b)
+      for (int h = 0; h < Hkv; ++h) {
+        const int S = c->h_budgets[((size_t)b * L + layer) * Hkv + h];
+        const int P = c->h_plen[b];
+        if (P - S <= 0) continue;
+        const int n_chunks = (S + kChunkN - 1) / kChunkN, cc = chunk_columns(S);
+        const int tiles = (P + kTileM - 1) / kTileM;
+        for (int nc = 0; nc < n_chunks; ++nc) {
+          const int cols = min(cc, S - nc * cc);
+          if (cols <= 0) continue;
+          pieces[n_pieces++] = {b * Hkv + h, nc, tiles, cols};
+          total += (double)tiles * (cols + 64);                // + a per-tile cost that does not depend on the columns
+        }
+      }
+    size_t n = 0;
+    if (n_pieces > 0) {
+      // aim at five waves of equal items, at least four tiles each (a CTA first loads its chunk of retained rows)
+      const double target = total / ((double)n_sms * 5.0);
+      std::vector<std::pair<double, int4>> list;
+      for (size_t i = 0; i < n_pieces; ++i) {
+        const Piece& p = pieces[i];
+        const double work = (double)p.tiles * (p.cols + 64);
+        int k = (int)(work / target + 0.5);
+        k = max(1, min(k, max(1, p.tiles / 4)));
+        if (list.size() + k + (n_pieces - i) > cap) k = 1;     // never more entries than the list holds
+        for (int j = 0; j < k; ++j) {
+          const int t0 = (int)((long long)p.tiles * j / k), t1 = (int)((long long)p.tiles * (j + 1) / k);
+          if (t1 > t0) list.push_back({(double)(t1 - t0) * (p.cols + 64), make_int4(p.slice, p.chunk, t0, t1)});
+        }
+      }
+      // longest first; ties keep the slice order
+      std::stable_sort(list.begin(), list.end(),
+                       [](const std::pair<double, int4>& x, const std::pair<double, int4>& y) { return x.first > y.first; });
+      for (const auto& e : list) out[n++] = e.second;
+    }
+    count[layer] = (int32_t)n;
+  }
+  free(pieces);
+}
+
 size_t sim_tc_part_key_bytes(const d2o_config* cfg, int max_budget) {
   const size_t chunks = ((size_t)max_budget + kChunkN - 1) / kChunkN;
   return (size_t)cfg->batch * cfg->n_kv_heads * chunks * cfg->prompt_len * 8;
@@ -388,31 +458,21 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   char* pool = S + (g.sim_feature ? c->lay.vpool : c->lay.kpool);
   if (!encode_rows_2d(&map_pool, g.dtype, pool, (uint64_t)c->pool_rows, D, kBBoxRows)) return cudaErrorNotSupported;
   const int n_chunks_max = (c->max_budget + kChunkN - 1) / kChunkN;
-  const int n_chunks = (max_S + kChunkN - 1) / kChunkN;
-  const int n_tiles = (P + kTileM - 1) / kTileM;
-  // One CTA per SM at a time.  Split the prompt tiles so that the waves are full: cost of a split count =
-  // waves x (start-up of a CTA + its tiles), in units of one tile's work.
-  int sms = 148;
-  { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
-  int splits = 1; double best_cost = 1e30;
-  for (int sp = 1; sp <= n_tiles; ++sp) {
-    const int tpc = (n_tiles + sp - 1) / sp;
-    const int ctas = ((n_tiles + tpc - 1) / tpc) * n_chunks * n_slices;
-    const double cost = (double)((ctas + sms - 1) / sms) * (3.0 + tpc);
-    if (cost < best_cost - 1e-9) { best_cost = cost; splits = sp; }
-  }
-  const int tiles_per_cta = (n_tiles + splits - 1) / splits;
-  splits = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
+  (void)max_S;
+  const int n_items = c->h_sim_count[layer];
+  if (n_items == 0) return cudaSuccess;                      // nothing was evicted in this layer
 
   SimTcArgs a;
   a.budgets = (const int32_t*)(S + c->lay.budgets); a.row_off = (const int64_t*)(S + c->lay.row_off);
   a.rnorm = (const float*)(S + c->lay.rnorm);
   a.part_key = (unsigned long long*)(X + c->slay.part_key);
   a.status = (uint32_t*)(S + c->lay.status);
-  a.L = g.n_layers; a.layer = layer; a.Hkv = Hkv; a.P = P; a.n_chunks_max = n_chunks_max; a.tiles_per_cta = tiles_per_cta;
+  a.plen = (const int32_t*)(S + c->lay.plen);
+  a.L = g.n_layers; a.layer = layer; a.Hkv = Hkv; a.P = P; a.n_chunks_max = n_chunks_max;
+  a.items = (const int4*)(S + c->lay.sim_items) + (size_t)layer * sim_tc_max_items(&g, c->max_budget);
   const int KB = D / 64;
   const size_t smem = (size_t)KB * kChunkN * 128 + (size_t)kAStages * KB * kTileM * 128 + kChunkN * 4 + 3 * kTileM * 8;
-  dim3 grid(splits, n_chunks, n_slices);
+  dim3 grid((unsigned)n_items);
   const int fmt = g.dtype == D2O_F16 ? 0 : 1;
   cudaError_t e;
 #define D2O_LAUNCH_TC(DD, FF)                                                                                     \
@@ -428,14 +488,13 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   if (e != cudaSuccess) return e;
 
   NnReduceArgs r;
-  r.budgets = a.budgets; r.row_off = a.row_off; r.rnorm = a.rnorm; r.status = a.status;
+  r.budgets = a.budgets; r.row_off = a.row_off; r.rnorm = a.rnorm; r.status = a.status; r.plen = a.plen;
   r.evict_idx = (const int32_t*)(X + c->slay.evict_idx); r.part_key = a.part_key;
   r.evict_mx = (float*)(X + c->slay.evict_mx); r.evict_nn = (int32_t*)(X + c->slay.evict_nn);
   r.L = g.n_layers; r.layer = layer; r.Hkv = Hkv; r.P = P; r.n_chunks_max = n_chunks_max;
-  int minS = P;
+  int maxLe = 0;
   for (int bb = 0; bb < B; ++bb)
-    for (int hh = 0; hh < Hkv; ++hh) minS = min(minS, c->h_budgets[(bb * g.n_layers + layer) * Hkv + hh]);
-  const int maxLe = P - minS;
+    for (int hh = 0; hh < Hkv; ++hh) maxLe = max(maxLe, c->h_plen[bb] - c->h_budgets[(bb * g.n_layers + layer) * Hkv + hh]);
   if (maxLe <= 0) return cudaSuccess;
   const int lpr = D * 2 / 16;
   dim3 rgrid((maxLe + 256 / lpr - 1) / (256 / lpr), n_slices);

@@ -63,16 +63,19 @@ __device__ __forceinline__ void tile_dot(const float* qt, const float* kt, int t
 // lse2[b,hq,i] = log2 sum_{j<=i} 2^{(q_i.k_j) * scale * log2e}, stored as natural log.
 template <typename T, int D>
 __global__ void __launch_bounds__(kStatThreads)
-lse_kernel(const T* __restrict__ Q, const T* __restrict__ K, float* __restrict__ lse, int P, int Hq, int group) {
+lse_kernel(const T* __restrict__ Q, const T* __restrict__ K, float* __restrict__ lse, int Pmax, int Hq, int group,
+           const int32_t* __restrict__ plen) {
   extern __shared__ __align__(16) float smem[];
   float* qt = smem;
   float* kt = smem + D * kTile;
   const int it = gridDim.x - 1 - blockIdx.x;          // heaviest row tiles first
   const int bh = blockIdx.y;
   const int b = bh / Hq, hq = bh % Hq;
+  const int P = plen ? plen[b] : Pmax;                 // this sequence's prompt length; tensors are laid out for Pmax
+  if (it * kTile >= P) return;
   const int Hkv = Hq / group;
-  const T* q = Q + ((size_t)b * Hq + hq) * (size_t)P * D;
-  const T* k = K + ((size_t)b * Hkv + hq / group) * (size_t)P * D;
+  const T* q = Q + ((size_t)b * Hq + hq) * (size_t)Pmax * D;
+  const T* k = K + ((size_t)b * Hkv + hq / group) * (size_t)Pmax * D;
   const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
   const float mul = (D == 64 ? 0.125f : 0.08838834764831845f) * kLog2e;
   load_tile_transposed<T, D>(qt, q, it * kTile, P, mul);
@@ -118,27 +121,29 @@ lse_kernel(const T* __restrict__ Q, const T* __restrict__ K, float* __restrict__
       m[r] = mn;
     }
     const int row = it * kTile + ty * 4 + r;
-    if (tx == 0 && row < P) lse[((size_t)b * Hq + hq) * P + row] = (m[r] + log2f(l[r])) * 0.6931471805599453f;
+    if (tx == 0 && row < P) lse[((size_t)b * Hq + hq) * Pmax + row] = (m[r] + log2f(l[r])) * 0.6931471805599453f;
   }
 }
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kStatThreads)
 colsum_kernel(const T* __restrict__ Q, const T* __restrict__ K, const float* __restrict__ lse,
-              float* __restrict__ colsum, int P, int Hq, int group) {
+              float* __restrict__ colsum, int Pmax, int Hq, int group, const int32_t* __restrict__ plen) {
   extern __shared__ __align__(16) float smem[];
   float* qt = smem;
   float* kt = smem + D * kTile;
   float* lse2 = kt + D * kTile;                        // [64]
   double* red = reinterpret_cast<double*>(lse2 + kTile);  // [16][64]
   const int jt = blockIdx.x;                          // column tile 0 has the most rows: first
-  const int nT = gridDim.x;
   const int bh = blockIdx.y;
   const int b = bh / Hq, hq = bh % Hq;
+  const int P = plen ? plen[b] : Pmax;
+  const int nT = (P + kTile - 1) / kTile;
+  if (jt >= nT) return;
   const int Hkv = Hq / group;
-  const T* q = Q + ((size_t)b * Hq + hq) * (size_t)P * D;
-  const T* k = K + ((size_t)b * Hkv + hq / group) * (size_t)P * D;
-  const float* ls = lse + ((size_t)b * Hq + hq) * P;
+  const T* q = Q + ((size_t)b * Hq + hq) * (size_t)Pmax * D;
+  const T* k = K + ((size_t)b * Hkv + hq / group) * (size_t)Pmax * D;
+  const float* ls = lse + ((size_t)b * Hq + hq) * Pmax;
   const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
   const float mul = (D == 64 ? 0.125f : 0.08838834764831845f) * kLog2e;
   load_tile_transposed<T, D>(kt, k, jt * kTile, P, 1.0f);
@@ -176,18 +181,20 @@ colsum_kernel(const T* __restrict__ Q, const T* __restrict__ K, const float* __r
 #pragma unroll
     for (int y = 0; y < 16; ++y) t += red[y * kTile + threadIdx.x];
     const int col = jt * kTile + threadIdx.x;
-    if (col < P) colsum[((size_t)b * Hq + hq) * P + col] = (float)t;
+    if (col < P) colsum[((size_t)b * Hq + hq) * Pmax + col] = (float)t;
   }
 }
 
 // F[b, layer, hq] = (1/P) sum_j (s_j - mean)^2, mean = (1/P) sum_j s_j   (Eq. 4; population variance)
 __global__ void __launch_bounds__(256)
-density_kernel(const float* __restrict__ colsum, double* __restrict__ density, int P, int Hq, int L, int layer) {
+density_kernel(const float* __restrict__ colsum, double* __restrict__ density, int Pmax, int Hq, int L, int layer,
+               const int32_t* __restrict__ plen) {
   __shared__ double part[8];
   __shared__ double mean_s;
   const int bh = blockIdx.x;
   const int b = bh / Hq, hq = bh % Hq;
-  const float* s = colsum + (size_t)bh * P;
+  const int P = plen ? plen[b] : Pmax;
+  const float* s = colsum + (size_t)bh * Pmax;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   double t = 0.0;
   for (int j = threadIdx.x; j < P; j += blockDim.x) t += (double)s[j];
@@ -221,19 +228,23 @@ density_kernel(const float* __restrict__ colsum, double* __restrict__ density, i
 // Output tables are [B, L, Hkv]; the per-layer rules give every KV head of a layer the same size.
 __device__ inline double clipd(double v, double lo, double hi) { return v < lo ? lo : (v > hi ? hi : v); }
 
-__global__ void budget_kernel(const double* __restrict__ density, int B, int L, int H, int Hkv, int P, double rho,
-                              int min_budget, int max_budget, double gamma, int head_reduce, int budget_rule,
+__global__ void budget_kernel(const double* __restrict__ density, int B, int L, int H, int Hkv, int Pmax, double rho,
+                              int min_budget, int max_budget_cfg, double gamma, int head_reduce, int budget_rule,
                               int n_sink, int window, double nm_ratio, int32_t* __restrict__ budgets,
-                              int32_t* __restrict__ windows, int64_t* __restrict__ row_off, uint32_t* status_word) {
+                              int32_t* __restrict__ windows, int64_t* __restrict__ row_off, uint32_t* status_word,
+                              const int32_t* __restrict__ plen) {
   extern __shared__ __align__(16) double dsm[];
   const int n = budget_rule == 1 ? L * Hkv : L;                       // allocation units
   const int G = H / Hkv;
   double* w = dsm + (size_t)threadIdx.x * 4 * n;
   double* kinks = w + n;        // [2n]
   double* x = kinks + 2 * n;    // [n]
-  const double lo = (double)min_budget, hi = (double)max_budget;
-  const long long S_tot = (long long)floor(rho * (double)n * (double)P + 0.5);
+  const double lo = (double)min_budget;
   for (int b = threadIdx.x; b < B; b += blockDim.x) {
+    const int P = plen ? plen[b] : Pmax;                              // this sequence's prompt length
+    const int max_budget = max_budget_cfg > 0 ? max_budget_cfg : P;   // no clamp given: a layer cannot hold more than the prompt
+    const double hi = (double)max_budget;
+    const long long S_tot = (long long)floor(rho * (double)n * (double)P + 0.5);
     const double* F = density + (size_t)b * L * H;
     int32_t* bud = budgets + (size_t)b * L * Hkv;
     // unit u -> its (first) entry of the [L, Hkv] table
@@ -378,10 +389,11 @@ static cudaError_t run_stats(const d2o_ctx* c, int layer, const void* Q, const v
   const int nT = (P + kTile - 1) / kTile;
   float* colsum = (float*)(c->state + c->lay.colsum) + (size_t)layer * B * Hq * P;
   double* density = (double*)(c->state + c->lay.density);
+  const int32_t* plen = (const int32_t*)(c->state + c->lay.plen);
   if (c->stats_path == 0 && colsum_tc_supported(&g)) {
     cudaError_t e = launch_colsum_tc(c, Q, K, lse_in, colsum, st);
     if (e != cudaSuccess) return e;
-    density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, g.n_layers, layer);
+    density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, g.n_layers, layer, plen);
     return cudaGetLastError();
   }
   const float* lse = lse_in;
@@ -391,14 +403,14 @@ static cudaError_t run_stats(const d2o_ctx* c, int layer, const void* Q, const v
     const size_t sm = (size_t)2 * D * kTile * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(lse_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
-    lse_kernel<T, D><<<grid, kStatThreads, sm, st>>>((const T*)Q, (const T*)K, lse_buf, P, Hq, c->group);
+    lse_kernel<T, D><<<grid, kStatThreads, sm, st>>>((const T*)Q, (const T*)K, lse_buf, P, Hq, c->group, plen);
     lse = lse_buf;
   }
   const size_t sm2 = (size_t)2 * D * kTile * sizeof(float) + kTile * sizeof(float) + 16 * kTile * sizeof(double);
   cudaError_t e = cudaFuncSetAttribute(colsum_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
   if (e != cudaSuccess) return e;
-  colsum_kernel<T, D><<<grid, kStatThreads, sm2, st>>>((const T*)Q, (const T*)K, lse, colsum, P, Hq, c->group);
-  density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, g.n_layers, layer);
+  colsum_kernel<T, D><<<grid, kStatThreads, sm2, st>>>((const T*)Q, (const T*)K, lse, colsum, P, Hq, c->group, plen);
+  density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, g.n_layers, layer, plen);
   return cudaGetLastError();
 }
 
@@ -416,7 +428,7 @@ cudaError_t launch_layer_stats(const d2o_ctx* c, int layer, const void* Q, const
 cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, int P, float rho, int min_budget,
                            int max_budget, float gamma, int head_reduce, int budget_rule, int n_sink, int window,
                            float nm_ratio, int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
-                           cudaStream_t st) {
+                           const int32_t* plen, cudaStream_t st) {
   const size_t n_units = budget_rule == 1 ? (size_t)L * Hkv : (size_t)L;
   const size_t per_thread = 4 * n_units * sizeof(double);
   int threads = B < 32 ? B : 32;
@@ -427,7 +439,7 @@ cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, 
   if (e != cudaSuccess) return e;
   budget_kernel<<<1, threads, sm, st>>>(density, B, L, H, Hkv, P, (double)rho, min_budget, max_budget, (double)gamma,
                                         head_reduce, budget_rule, n_sink, window, (double)nm_ratio, budgets, windows,
-                                        row_off, status_word);
+                                        row_off, status_word, plen);
   return cudaGetLastError();
 }
 
@@ -445,12 +457,12 @@ static cudaError_t run_stats_static(const void* Q, const void* K, float* lse_buf
   const size_t sm = (size_t)2 * D * kTile * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(lse_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
   if (e != cudaSuccess) return e;
-  lse_kernel<T, D><<<grid, kStatThreads, sm, st>>>((const T*)Q, (const T*)K, lse_buf, P, Hq, group);
+  lse_kernel<T, D><<<grid, kStatThreads, sm, st>>>((const T*)Q, (const T*)K, lse_buf, P, Hq, group, nullptr);
   const size_t sm2 = sm + kTile * sizeof(float) + 16 * kTile * sizeof(double);
   e = cudaFuncSetAttribute(colsum_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
   if (e != cudaSuccess) return e;
-  colsum_kernel<T, D><<<grid, kStatThreads, sm2, st>>>((const T*)Q, (const T*)K, lse_buf, colsum, P, Hq, group);
-  density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, 1, 0);
+  colsum_kernel<T, D><<<grid, kStatThreads, sm2, st>>>((const T*)Q, (const T*)K, lse_buf, colsum, P, Hq, group, nullptr);
+  density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, 1, 0, nullptr);
   return cudaGetLastError();
 }
 

@@ -116,6 +116,17 @@ CONFIGS: Dict[str, Workload] = {
 }
 
 
+# Not one of the five benchmark configurations: the steady state of the paper's multi-turn (streaming) setting,
+# appendix "Generated Samples of Multi-turn Conversations": every layer holds a fixed budget of 2048 tokens, of which
+# N = 48 are important tokens and M = 2000 the recent window (no sinks: 48 + 2000 = 2048).  The "prompt" is the 2048
+# tokens the conversation has accumulated, so nothing is evicted at the prompt stage and every generated token
+# evicts one.  Llama-2-7B-shaped heads, four sessions.
+CONFIGS["session"] = Workload("session", batch=4, n_layers=32, n_q_heads=32, n_kv_heads=32, d_head=128,
+                              dtype="f16", prompt_len=2048, decode_steps=256, rho=1.0, n_sink=0, window=2000,
+                              beta=0.7, rank=8, heavy_frac=0.05, temp_first=1.0, temp_last=0.25,
+                              density_temp=1e30, min_budget=2048, max_budget=2048, seed=2406135)
+
+
 def twin(name: str) -> Workload:
     """Scaled twin used by the whole-pipeline parity tests (4 layers, P/8, B<=2)."""
     return CONFIGS[name].scaled(n_layers=4, prompt_div=8, batch=2, steps=16)

@@ -84,7 +84,7 @@ def make_ctx(wl: W.Workload, device="cuda:0", **over) -> B.D2OContext:
     return B.D2OContext(B.make_config(**kw), device)
 
 
-def make_oracle(wl: W.Workload, cfg: B.D2OConfig) -> O.OracleStack:
+def make_oracle(wl: W.Workload, cfg: B.D2OConfig, prompt_lens=None) -> O.OracleStack:
     # float parameters take the values the C floats hold
     return O.OracleStack(n_layers=cfg.n_layers, batch=cfg.batch, n_q_heads=cfg.n_q_heads,
                          n_kv_heads=cfg.n_kv_heads, d_head=cfg.d_head, dtype=wl.dtype, prompt_len=cfg.prompt_len,
@@ -93,7 +93,7 @@ def make_oracle(wl: W.Workload, cfg: B.D2OConfig) -> O.OracleStack:
                          head_reduce=cfg.head_reduce, tau_override=float(cfg.tau_override),
                          max_budget=cfg.max_budget, feature=("k", "v")[cfg.sim_feature],
                          policy=("weighted", "average")[cfg.merge_policy],
-                         budget_rule=("layer", "head", "exp_decay")[cfg.budget_rule])
+                         budget_rule=("layer", "head", "exp_decay")[cfg.budget_rule], prompt_lens=prompt_lens)
 
 
 def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int, int, int]]] = None,
@@ -102,7 +102,7 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
                similarity_path: int = 0, stats_path: int = 0, decode_warps: int = 0,
                decode_smem_rows: int = 0, decode_long_pairs: int = 0,
                check_stats_all: Optional[bool] = None, prompt_hook=None, decode_hook=None,
-               max_ties: Optional[int] = None) -> Report:
+               max_ties: Optional[int] = None, prompt_lens=None) -> Report:
     """`slices`: (layer, b, kv_head) triples checked against the oracle (None = all).
     The GPU always runs the whole workload.  `prompt_hook(layer, Q, K, V)` and `decode_hook(step, q, k, v)` may
     return edited input tensors (both sides then see the edited ones)."""
@@ -113,7 +113,9 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
             or decode_long_pairs):
         ctx.d2o_set_tuning(decode_stages, decode_l2_hints, similarity_path, stats_path, decode_warps,
                            decode_smem_rows, decode_long_pairs)
-    orc = make_oracle(wl, cfg)
+    orc = make_oracle(wl, cfg, prompt_lens)
+    if prompt_lens is not None:                        # ragged batch: the tensors stay padded to wl.prompt_len
+        ctx.d2o_set_prompt_lens(prompt_lens)
     L, Bn, Hq, Hkv, G, P = wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.group, wl.prompt_len
     all_slices = [(l, b, h) for l in range(L) for b in range(Bn) for h in range(Hkv)]
     chk = all_slices if slices is None else slices
@@ -136,8 +138,8 @@ def run_parity(wl: W.Workload, device="cuda:0", slices: Optional[List[Tuple[int,
             orc.layer_stats(l, _lazy64(Qc), _lazy64(Kc), heads)
             cs = ctx.colsum(l).cpu().double().numpy()
             for b, hq in heads:
-                ref = orc.colsum[l, b, hq]
-                rep.err("colsum_rel", np.max(np.abs(cs[b, hq] - ref) / np.maximum(np.abs(ref), 1e-6)))
+                ref = orc.colsum[l, b, hq, :orc.Pb[b]]
+                rep.err("colsum_rel", np.max(np.abs(cs[b, hq, :orc.Pb[b]] - ref) / np.maximum(np.abs(ref), 1e-6)))
         del Q
     budgets = ctx.d2o_layer_budgets().numpy().astype(np.int64)
     F_gpu = ctx.density().cpu().numpy()

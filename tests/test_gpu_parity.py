@@ -230,6 +230,53 @@ def test_value_feature_prompt_stage(name):
     assert e.value.status == 2
 
 
+@pytest.mark.parametrize("name", ["cfg0", "cfg2"])
+def test_streaming_session_shape(name):
+    # The multi-turn setting of the paper's appendix (fixed budget 2048 with N = 48 important and M = 2000 recent
+    # tokens, no sinks), scaled by 1/16: the prompt is shorter than the budget, so the cache first grows by appending,
+    # then every new token evicts one; the cache is almost all window.
+    base = W.CONFIGS["cfg0"] if name == "cfg0" else W.twin("cfg2")
+    wl = dataclasses.replace(base, n_layers=2, batch=1, prompt_len=64, decode_steps=100, rho=2.0, n_sink=0,
+                             window=125, min_budget=128, max_budget=128, density_temp=1e30)
+    rep = run_parity(wl)
+    assert_report(rep, wl.dtype)
+    assert rep.merges + rep.discards == rep.checked_slices * (100 - 64)      # evictions start once 128 rows are held
+
+
+@pytest.mark.parametrize("name,lens", [("cfg0", [384, 131]), ("cfg1", [512, 77]), ("cfg2", [1024, 389]),
+                                       ("cfg2", [300, 1024])])
+def test_ragged_batch(name, lens):
+    # per-sequence prompt lengths in one padded batch: own column sums, budgets, eviction and token positions
+    base = dataclasses.replace(W.CONFIGS["cfg0"], n_layers=2, batch=2, prompt_len=384, density_temp=40.0,
+                               min_budget=16) if name == "cfg0" else W.twin(name)
+    wl = dataclasses.replace(base, batch=2, decode_steps=6, max_budget=0, min_budget=min(base.min_budget, 16))
+    assert wl.prompt_len == max(lens)
+    rep = run_parity(wl, prompt_lens=lens)
+    # a 77-token prompt has many nearly equal small scores at its end: one Top-N boundary of the 256 slices of the
+    # fp16 case is a tie below 1e-6 relative between float32 and float64 (counted, followed)
+    assert_report(rep, wl.dtype, max_ties=1 if name == "cfg1" else 0)
+    print("ragged", name, lens, rep.ties)
+    assert rep.merges + rep.discards == rep.checked_slices * 6
+
+
+def test_ragged_lengths_are_validated(cuda_device):
+    from parity import make_ctx
+    wl = small(prompt_len=256, decode_steps=2, batch=2)
+    ctx = make_ctx(wl)
+    for bad in ([256, 0], [257, 10], [256, 20]):         # 20 positions cannot hold L * min_budget = 8 rows at rho 0.25
+        with pytest.raises(B.D2OError) as e:
+            ctx.d2o_set_prompt_lens(bad)
+        assert e.value.status == 1
+    ctx.d2o_set_prompt_lens([256, 100])
+    s = W.LayerStream(wl, 0, "cuda:0")
+    Q, K, V = s.prompt()
+    ctx.d2o_layer_stats(0, Q, K)
+    with pytest.raises(B.D2OError) as e:                  # too late: the prompt is being fed
+        ctx.d2o_set_prompt_lens([256, 100])
+    assert e.value.status == 4
+    ctx.close()
+
+
 def test_more_sinks_than_budget_is_rejected(cuda_device):
     from parity import make_ctx
     wl = small(prompt_len=128, decode_steps=2, n_sink=40, min_budget=8)

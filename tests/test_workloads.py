@@ -6,7 +6,9 @@ from paper_2406_13035_b200 import workloads as W
 
 
 def test_configs_cover_the_five_benchmark_shapes():
-    assert set(W.CONFIGS) == {"cfg0", "cfg1", "cfg2", "cfg3", "cfg4"}
+    assert set(W.CONFIGS) == {"cfg0", "cfg1", "cfg2", "cfg3", "cfg4", "session"}
+    ses = W.CONFIGS["session"]                          # the multi-turn shape: 2048 = 48 important + 2000 recent tokens
+    assert ses.max_budget == ses.min_budget == 2048 and ses.window == 2000 and ses.n_sink == 0
     c1 = W.CONFIGS["cfg1"]
     assert (c1.n_layers, c1.n_q_heads, c1.n_kv_heads, c1.d_head, c1.dtype, c1.prompt_len) == (32, 32, 32, 128, "f16", 4096)
     assert W.CONFIGS["cfg2"].group == 4 and W.CONFIGS["cfg3"].prompt_len == 32768
