@@ -146,7 +146,7 @@ enum Counter { kCntDecodeSteps = 0, kCntEvictions, kCntMerges, kCntDiscards, kCn
 
 // ----------------------------------------------------------------------------- context
 struct Layout {            // byte offsets into `state`
-  size_t status, counters, density, budgets, windows, row_off, order, plen, len, tau, guess, sim_items, colsum, pos, score, rnorm, kpool, vpool, end;
+  size_t status, counters, density, budgets, windows, row_off, order, plen, len, tau, sim_items, colsum, pos, score, rnorm, kpool, vpool, end;
 };
 struct ScratchLayout {     // byte offsets into `scratch`
   size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, seg_tmp, part_key, pl_spill, stage_q, stage_k, stage_v, stage_out, end;

@@ -50,7 +50,6 @@ struct DecodeArgs {
   const int32_t* budgets; const int32_t* windows; const int64_t* row_off;   // [B, L]
   int32_t* pos; float* score; float* rnorm;                                  // pool-wide
   int32_t* len; float* tau;                                                  // [L, B, Hkv]
-  int32_t* guess;                                                            // [L, B, Hkv][2] rows guessed for the next step's victim (-2: none yet)
   unsigned long long* counters; uint32_t* status;
   const int32_t* plen;              // [B] prompt length of every sequence
   int L, l0, B, Hkv, T, step;       // step = number of tokens generated before this one: its position is plen[b] + step
@@ -372,8 +371,6 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   __shared__ int s_li[kConsWarps], s_best_li;
   __shared__ volatile int s_timeout;                                 // 1: an earlier launch recorded an anomaly; 2: a wait of this CTA ran out
   __shared__ int s_bail;
-  __shared__ unsigned long long s_gk[kConsWarps][3];                 // per warp: lowest keys among the rows evictable next step
-  __shared__ int s_gl[kConsWarps][3];
 
   if (tid == 0) {
     s_timeout = *reinterpret_cast<volatile uint32_t*>(a.status) != 0u;
@@ -517,9 +514,6 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   for (int c = 0; c < NC; ++c) { cand_li[c] = -1; cand_rn[c] = 0.f; cbest[c] = 0ull; cbest_li[c] = -1; }
 #pragma unroll
   for (int j = 0; j < D / 32; ++j) cb[j] = make_uint4(0, 0, 0, 0);
-  // The previous step left its guess behind (see below, after the victim search); only the first evicting step of a
-  // slice has to look through the scores itself.
-  const int stored0 = evict ? a.guess[2 * sidx] : -2, stored1 = evict ? a.guess[2 * sidx + 1] : -2;
   if (evict) {
     if (warp == 0) {
       // the new token's inverse norm, from the row as stored
@@ -531,12 +525,6 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       ss = warp_sum(ss);                                               // lanes >= LPR hold zeros
       if (lane == 0) s_new_rn = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
     }
-    consumer_sync<CW>();                                                 // s_new_rn is read during pass K
-  }
-  if (evict && stored0 != -2) {
-    cand_li[0] = (unsigned)stored0 < (unsigned)n_old ? stored0 : -1;
-    if (NC > 1) cand_li[NC - 1] = (unsigned)stored1 < (unsigned)n_old && stored1 != stored0 ? stored1 : -1;
-  } else if (evict) {
     unsigned long long my[NC];
     int my_li[NC];
 #pragma unroll
@@ -834,21 +822,6 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       inv_l[g] = 1.0f / t;
     }
     unsigned long long my_min = ~0ull; int my_min_li = -1;
-    // the same search over the rows that may be evicted at the NEXT step (one more position leaves the window): the
-    // lowest NC + 1 of them, of which the victim will be struck, are the next step's guess
-    constexpr int NG = NC + 1;
-    unsigned long long nx[NG]; int nx_li[NG];
-#pragma unroll
-    for (int c = 0; c < NG; ++c) { nx[c] = ~0ull; nx_li[c] = -1; }
-    auto offer_next = [&](float sc, int pz, int li) {
-      if (pz >= Tn && pz <= t_pos + 1 - M) {
-        unsigned long long key = ((unsigned long long)float_ord(sc) << 32) | (uint32_t)(0x7fffffff - pz);
-        int kl = li;
-#pragma unroll
-        for (int c = 0; c < NG; ++c)
-          if (key < nx[c]) { const unsigned long long tk = nx[c]; const int tl = nx_li[c]; nx[c] = key; nx_li[c] = kl; key = tk; kl = tl; }
-      }
-    };
     for (int li = tid * 4; li < n_vec; li += kConsThreads * 4) {
       float4 p = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -871,7 +844,6 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
             const unsigned long long key = ((unsigned long long)float_ord(sv[j]) << 32) | (uint32_t)(0x7fffffff - pv[j]);
             if (key < my_min) { my_min = key; my_min_li = li + j; }
           }
-          offer_next(sv[j], pv[j], li + j);
         }
       }
     }
@@ -887,42 +859,9 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         const unsigned long long key = ((unsigned long long)float_ord(s_new) << 32) | (uint32_t)(0x7fffffff - pz);
         if (key < my_min) { my_min = key; my_min_li = li; }
       }
-      if (evict && li < n_old) offer_next(s_new, pz, li);
     }
-    if (evict) {
-      // per warp: its lowest NG keys, by NG rounds of a warp-wide minimum (the owner of a minimum moves on to its next)
-      int head = 0;
-#pragma unroll
-      for (int r = 0; r < NG; ++r) {
-        unsigned long long k = ~0ull; int kl = -1;
-#pragma unroll
-        for (int j = 0; j < NG; ++j) if (head == j) { k = nx[j]; kl = nx_li[j]; }
-        const unsigned long long w = warp_min_u64(k);
-        const unsigned vote = __ballot_sync(0xffffffffu, k == w);
-        const int src = __ffs(vote) - 1;
-        const int wl = __shfl_sync(0xffffffffu, kl, src);
-        if (lane == src && w != ~0ull) ++head;
-        if (lane == 0) { s_gk[warp][r] = w; s_gl[warp][r] = w == ~0ull ? -1 : wl; }
-      }
-      block_arg_extreme<true, CW>(my_min, my_min_li, s_key, s_li, &s_best_key, &s_best_li);
-    }
+    if (evict) block_arg_extreme<true, CW>(my_min, my_min_li, s_key, s_li, &s_best_key, &s_best_li);
     consumer_sync<CW>();
-    if (evict && tid == 32) {
-      // next step's guess: the lowest keys over the warps' lists, without the row that is evicted now
-      const int vic = s_best_li;
-      int g0 = -1, g1 = -1;
-      unsigned long long k0 = ~0ull, k1 = ~0ull;
-      for (int w = 0; w < kConsWarps; ++w)
-        for (int r = 0; r < NG; ++r) {
-          const unsigned long long k = s_gk[w][r];
-          const int l = s_gl[w][r];
-          if (l < 0 || l == vic) continue;
-          if (k < k0) { k1 = k0; g1 = g0; k0 = k; g0 = l; }
-          else if (k < k1) { k1 = k; g1 = l; }
-        }
-      a.guess[2 * sidx] = g0;
-      a.guess[2 * sidx + 1] = g1;
-    }
   }
   // ---- victim (Eq. 7-8); its cosine with every other row (Eq. 9): from the guess, or from a second look at the keys;
   // tau_t (Eq. 10), merged key (Eq. 11-12)
@@ -1345,7 +1284,6 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   a.row_off = (const int64_t*)(S + c->lay.row_off);
   a.pos = (int32_t*)(S + c->lay.pos); a.score = (float*)(S + c->lay.score); a.rnorm = (float*)(S + c->lay.rnorm);
   a.len = (int32_t*)(S + c->lay.len); a.tau = (float*)(S + c->lay.tau);
-  a.guess = (int32_t*)(S + c->lay.guess);
   a.counters = (unsigned long long*)(S + c->lay.counters); a.status = (uint32_t*)(S + c->lay.status);
   a.L = L; a.l0 = l0; a.B = B; a.Hkv = g.n_kv_heads; a.T = g.n_sink;
   a.step = c->layer_steps[l0];

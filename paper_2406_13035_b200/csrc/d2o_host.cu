@@ -108,7 +108,6 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   l->plen = take(B * 4);
   l->len = take(L * B * Hkv * 4);
   l->tau = take(L * B * Hkv * 4);
-  l->guess = take(L * B * Hkv * 2 * 4);
   l->sim_items = take(c->dtype == D2O_F32 ? 0 : L * sim_tc_max_items(c, max_budget) * 16);
   l->colsum = take(L * B * Hq * P * 4);
   l->pos = take(rows * 4);

@@ -27,7 +27,6 @@ struct SelectArgs {
   const int64_t* row_off;  // [B, L]
   int32_t* pos; float* score; float* rnorm;   // pool-wide
   int32_t* len; float* tau;                   // [L, B, Hkv]
-  int32_t* guess;          // [L, B, Hkv][2] the decode kernel's victim guesses: none yet (-2)
   int32_t* evict_idx;      // [B, Hkv, P]
   float* keys_spill;       // [B, Hkv, P] group scores when P does not fit in shared memory (may alias evict_mx)
   unsigned long long* counters;
@@ -151,7 +150,6 @@ select_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
   if (threadIdx.x == 0) {
     a.len[sidx] = n_keep;
     a.tau[sidx] = 0.f;
-    a.guess[2 * sidx] = -2; a.guess[2 * sidx + 1] = -2;
     if (n_ret != n_keep) report_error(a.status, D2O_ERR_STATE, 0x5E000000u | (uint32_t)slice);
     atomicAdd(&a.counters[kCntPrefillEvicted], (unsigned long long)(P - n_keep));
   }
@@ -554,7 +552,6 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   sa.row_off = (const int64_t*)(S + c->lay.row_off);
   sa.pos = (int32_t*)(S + c->lay.pos); sa.score = (float*)(S + c->lay.score); sa.rnorm = (float*)(S + c->lay.rnorm);
   sa.len = (int32_t*)(S + c->lay.len); sa.tau = (float*)(S + c->lay.tau);
-  sa.guess = (int32_t*)(S + c->lay.guess);
   sa.evict_idx = (int32_t*)(X + c->slay.evict_idx);
   sa.keys_spill = (float*)(X + c->slay.evict_mx);
   sa.counters = (unsigned long long*)(S + c->lay.counters);

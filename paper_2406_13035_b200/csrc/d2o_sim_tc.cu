@@ -8,15 +8,17 @@
 // tiled TMA load of 128 consecutive prompt rows, and the few retained rows among them cost
 // S/P extra work.
 //
-// One CTA = (slice, chunk of up to 448 retained rows, range of 128-row prompt tiles).
-//   warp 0      TMA producer: the retained chunk once (B operand, stays in shared memory), then the
-//               prompt tiles through a 3-stage ring (A operand); 128-byte swizzled K-major tiles
-//   warp 1      allocates tensor memory, issues tcgen05.mma: 128 x 256 x 16 per instruction, d/16 per job,
-//               accumulators double-buffered in 2 x 256 tensor-memory columns
-//   warps 2-17  epilogue: tcgen05.ld of the accumulators, times 1/|k_c| per column, running max and
-//               arg-max per row (ties -> lowest slot); four warps share a row (quarters of the column blocks);
-//               the scan is bound by instruction issue (about five per accumulator element), which is
-//               why it gets sixteen warps
+// One CTA = one work item = (slice, chunk of up to 384 retained rows, range of 128-row prompt tiles); the host
+// cuts every (slice, chunk) into ranges of about equal work once the budgets are known (sim_tc_build_items).
+//   warp 0      TMA producer: the retained chunk once (B operand, stays in shared memory), then the prompt tiles
+//               (A operand) into four slots, one per part; 128-byte swizzled K-major tiles
+//   warp 1      allocates tensor memory, issues tcgen05.mma: one job = 128 x 128 x d (d/16 instructions) into the
+//               part's own 128-column accumulator, the parts in turn
+//   warps 2-17  epilogue: four parts of four warps.  A part owns every fourth prompt tile; each of its threads owns
+//               one row (tensor-memory lane) of that tile and scans all retained columns of it, job after job:
+//               tcgen05.ld of the accumulator, times 1/|k_c| per column, running max and arg-max (ties -> lowest
+//               slot) in registers.  No exchange between warps and no barrier per tile; while one part drains its
+//               accumulator the tensor cores work for the other three.
 // Output: for every prompt position of the tile range and this chunk, the packed key
 // (ordered max_j k_i.k_j/|k_j|, 0x7fffffff - slot).  neighbour_reduce_kernel takes the maximum over
 // the chunks at the evicted positions and multiplies by 1/|k_i|.
@@ -37,10 +39,10 @@ namespace d2o {
 constexpr int kTcEpiWarps = 16;             // four per quarter of the tensor-memory lanes
 constexpr int kTcThreads = (2 + kTcEpiWarps) * 32;
 constexpr int kTileM = 128;                 // prompt rows per A tile
-constexpr int kTileN = 256;                 // retained rows per MMA
-constexpr int kChunkN = 448;                // retained rows resident per CTA (112 KB for d = 128)
+constexpr int kJobN = 128;                  // retained rows per MMA job (one 128 x 128 fp32 accumulator)
+constexpr int kChunkN = 384;                // retained rows resident per CTA (96 KB for d = 128)
 constexpr int kBBoxRows = 64;               // rows per TMA box of the B operand
-constexpr int kAStages = 3;                 // 3 x 32 KB of prompt tiles in flight
+constexpr int kParts = 4;                   // prompt tiles in flight: each with its own accumulator and four epilogue warps
 
 struct SimTcArgs {
   const int32_t* budgets; const int64_t* row_off;
@@ -103,15 +105,14 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_pool) {
   constexpr int KB = D / 64;                                 // 64-element (128-byte) blocks along d
   constexpr int A_BLOCK = kTileM * 128;                      // bytes of one A k-block
-  constexpr int A_STAGE = KB * A_BLOCK;
+  constexpr int A_TILE = KB * A_BLOCK;
   constexpr int B_BLOCK = kChunkN * 128;                     // bytes of one B k-block (all chunk rows)
 
   extern __shared__ __align__(1024) unsigned char tc_smem[];
   unsigned char* sB = tc_smem;                               // [KB][kChunkN rows][128 B]
-  unsigned char* sA = tc_smem + KB * B_BLOCK;                // [kAStages][KB][128 rows][128 B]
-  float* s_rn = reinterpret_cast<float*>(sA + kAStages * A_STAGE);                 // [kChunkN] 1/|k_c| of the chunk
-  unsigned long long* s_pair = reinterpret_cast<unsigned long long*>(s_rn + kChunkN);   // [3][128] keys of the other column quarters
-  __shared__ unsigned long long b_full, a_full[kAStages], a_empty[kAStages], tm_full[2], tm_empty[2];
+  unsigned char* sA = tc_smem + KB * B_BLOCK;                // [kParts][KB][128 rows][128 B]: the prompt tile of each part
+  float* s_rn = reinterpret_cast<float*>(sA + kParts * A_TILE);                    // [kChunkN] 1/|k_c| of the chunk
+  __shared__ unsigned long long b_full, a_full[kParts], a_empty[kParts], tm_full[kParts], tm_empty[kParts];
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
 
@@ -126,12 +127,13 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
   const int Pb = a.plen[b];                                  // this sequence's prompt length
   if (c0 >= S || Pb - S <= 0) return;                        // uniform for the CTA: nothing to do
   const int n_cols = min(chunk_cols, S - c0);
-  const int n_nt = (n_cols + kTileN - 1) / kTileN;           // MMA column tiles in this chunk (1 or 2)
-  const int n_last = (n_cols - (n_nt - 1) * kTileN + 15) & ~15;   // columns of the last tile's MMA (multiple of 16)
+  const int n_j = (n_cols + kJobN - 1) / kJobN;              // MMA column tiles (jobs) per prompt tile: 1 .. 3
+  const int n_last = (n_cols - (n_j - 1) * kJobN + 15) & ~15;    // columns of the last job's MMA (multiple of 16)
   const int n_tiles_all = (Pb + kTileM - 1) / kTileM;
   const int t0 = item.z;
   const int t1 = min(n_tiles_all, item.w);
   if (t0 >= t1) return;
+  const int T = t1 - t0;                                     // prompt tiles of this CTA; part p takes tiles p, p + 4, ...
   const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
   if ((tc::smem_u32(tc_smem) & 1023u) != 0u) {               // swizzled tiles need 1024-byte aligned shared memory
     if (tid == 0) report_error(a.status, D2O_ERR_STATE, 0x51C10000u);
@@ -141,12 +143,14 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
   if (tid == 0) {
     s_fail = 0;
     tc::mbar_init(&b_full, 1);
-    for (int s = 0; s < kAStages; ++s) { tc::mbar_init(&a_full[s], 1); tc::mbar_init(&a_empty[s], 1); }
-    for (int i = 0; i < 2; ++i) { tc::mbar_init(&tm_full[i], 1); tc::mbar_init(&tm_empty[i], kTcEpiWarps); }
+    for (int p = 0; p < kParts; ++p) {
+      tc::mbar_init(&a_full[p], 1); tc::mbar_init(&a_empty[p], 1);
+      tc::mbar_init(&tm_full[p], 1); tc::mbar_init(&tm_empty[p], kTcEpiWarps / kParts);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {                                           // 512 columns: two 128 x 256 fp32 accumulators
+  if (warp == 1) {                                           // 512 columns: one 128 x 128 fp32 accumulator per part
     tc::tmem_alloc(&s_tmem, 512);
     tc::tmem_relinquish();
   }
@@ -163,115 +167,103 @@ sim_tc_kernel(SimTcArgs a, const __grid_constant__ CUtensorMap map_k, const __gr
       for (int kb = 0; kb < KB; ++kb)
         for (int j = 0; j < n_box; ++j)
           tc::tma_load_2d(sB + kb * B_BLOCK + j * kBBoxRows * 128, &map_pool, kb * 64, (int)(row0 + c0 + j * kBBoxRows), &b_full);
-      int it = 0;
-      for (int t = t0; t < t1; ++t, ++it) {
-        const int s = it % kAStages;
-        if (it >= kAStages && !s_fail && !tc::mbar_wait(&a_empty[s], (uint32_t)(((it / kAStages) - 1) & 1))) s_fail = 1;
-        tc::mbar_expect_tx(&a_full[s], (uint32_t)A_STAGE);
+      for (int i = 0; i < T; ++i) {                            // tile i goes to part i % 4, its k-th tile with k = i / 4
+        const int p = i % kParts, k = i / kParts;
+        if (k >= 1 && !s_fail && !tc::mbar_wait(&a_empty[p], (uint32_t)((k - 1) & 1))) s_fail = 1;
+        tc::mbar_expect_tx(&a_full[p], (uint32_t)A_TILE);
         for (int kb = 0; kb < KB; ++kb)
-          tc::tma_load_2d(sA + s * A_STAGE + kb * A_BLOCK, &map_k, kb * 64, slice * a.P + t * kTileM, &a_full[s]);
+          tc::tma_load_2d(sA + p * A_TILE + kb * A_BLOCK, &map_k, kb * 64, slice * a.P + (t0 + i) * kTileM, &a_full[p]);
       }
     }
   } else if (warp == 1) {
     // ======================================================================= MMA issuer
+    // Jobs are issued part by part in turn, so that while one part's epilogue drains its accumulator the tensor
+    // cores work for the other three.
     if (lane == 0) {
       if (!tc::mbar_wait(&b_full, 0)) s_fail = 1;
-      int it = 0, job = 0;
-      for (int t = t0; t < t1; ++t, ++it) {
-        const int s = it % kAStages;
-        if (!s_fail && !tc::mbar_wait(&a_full[s], (uint32_t)((it / kAStages) & 1))) s_fail = 1;
-        for (int j = 0; j < n_nt; ++j, ++job) {
-          const int buf = job & 1;
-          // the epilogue must have drained this accumulator (the first use of each buffer passes at once)
-          if (!s_fail && !tc::mbar_wait(&tm_empty[buf], (uint32_t)(((job >> 1) & 1) ^ 1))) s_fail = 1;
-          tc::fence_after_sync();
-          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kTileN);
-          const uint32_t idesc = make_idesc(FMT, kTileM, j == n_nt - 1 ? (uint32_t)n_last : (uint32_t)kTileN);
+      const int rounds = (T + kParts - 1) / kParts;
+      for (int k = 0; k < rounds; ++k)
+        for (int j = 0; j < n_j; ++j)
+          for (int p = 0; p < kParts; ++p) {
+            if (k * kParts + p >= T) continue;
+            if (j == 0 && !s_fail && !tc::mbar_wait(&a_full[p], (uint32_t)(k & 1))) s_fail = 1;
+            const int cnt = k * n_j + j;                         // jobs issued to this part before this one
+            // the part's epilogue must have drained its accumulator (the first use passes at once)
+            if (!s_fail && !tc::mbar_wait(&tm_empty[p], (uint32_t)((cnt & 1) ^ 1))) s_fail = 1;
+            tc::fence_after_sync();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(p * kJobN);
+            const uint32_t idesc = make_idesc(FMT, kTileM, j == n_j - 1 ? (uint32_t)n_last : (uint32_t)kJobN);
 #pragma unroll
-          for (int kb = 0; kb < KB; ++kb) {
-            const uint64_t adesc = tc::smem_desc_sw128(tc::smem_u32(sA + s * A_STAGE + kb * A_BLOCK));
-            const uint64_t bdesc = tc::smem_desc_sw128(tc::smem_u32(sB + kb * B_BLOCK + j * kTileN * 128));
+            for (int kb = 0; kb < KB; ++kb) {
+              const uint64_t adesc = tc::smem_desc_sw128(tc::smem_u32(sA + p * A_TILE + kb * A_BLOCK));
+              const uint64_t bdesc = tc::smem_desc_sw128(tc::smem_u32(sB + kb * B_BLOCK + j * kJobN * 128));
 #pragma unroll
-            for (int k = 0; k < 4; ++k)                      // 16 elements = 32 bytes along K per instruction
-              tc::mma_f16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+              for (int kk = 0; kk < 4; ++kk)                     // 16 elements = 32 bytes along K per instruction
+                tc::mma_f16(d_tmem, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), idesc, (kb | kk) != 0 ? 1u : 0u);
+            }
+            tc::mma_commit(&tm_full[p]);
+            if (j == n_j - 1) tc::mma_commit(&a_empty[p]);       // the tile's slot is free once its MMAs have read it
           }
-          tc::mma_commit(&tm_full[buf]);
-        }
-        tc::mma_commit(&a_empty[s]);                         // the stage is free once its MMAs have read it
-      }
     }
   } else {
     // ======================================================================= epilogue warps
+    // Four warps per part, one per quarter of the tensor-memory lanes: a thread owns one row of its part's prompt
+    // tile and scans all retained columns of it, job after job, so that the row's maximum never leaves its registers
+    // (no exchange between warps, no barrier per tile).
     const int e = warp - 2;
     const int quarter = warp & 3;                            // tensor-memory lanes this warp may read: 32*quarter ..
-    const int part = e >> 2;                                 // which quarter of a tile's column blocks this warp scans
-    const int row = quarter * 32 + lane;                     // row of the A tile owned by this thread
+    const int p = e >> 2;                                    // part
+    const int row = quarter * 32 + lane;                     // row of the prompt tile owned by this thread
     for (int i = tid - 64; i < kChunkN; i += kTcEpiWarps * 32)
       s_rn[i] = i < n_cols ? a.rnorm[row0 + c0 + i] : 0.f;
     asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
     unsigned long long* out_keys = a.part_key + ((size_t)slice * a.n_chunks_max + nc) * a.P;
-    // The (at most eight) 32-column blocks of a job that hold retained rows are dealt to the four warps of a row,
-    // at most two each (slots 0 and 1).  Loads run one block ahead of the scan, across job boundaries: the first
-    // block of the next job is requested before the second block of this job is scanned.
-    auto blocks_of = [&](int j, int& blk0, int& n_blk) {
-      const int n_blk_all = (min(kTileN, n_cols - j * kTileN) + 31) / 32;
-      const int per = (n_blk_all + 3) / 4;
-      blk0 = part * per;
-      n_blk = max(0, min(per, n_blk_all - blk0));
-    };
-    const int n_jobs = (t1 - t0) * n_nt;
+    const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(p * kJobN);
     uint32_t ra[32], rb[32];
-    {
-      int blk0, n_blk;
-      blocks_of(0, blk0, n_blk);
-      if (!s_fail && !tc::mbar_wait(&tm_full[0], 0u)) s_fail = 1;
-      tc::fence_after_sync();
-      if (n_blk > 0) tc::tmem_ld32_issue(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(blk0 * 32), ra);
-    }
-    float best = -INFINITY; int best_col = 0x7fffffff;
-#pragma unroll 1
-    for (int job = 0; job < n_jobs; ++job) {
-      const int t = t0 + job / n_nt, j = job % n_nt;
-      const int buf = job & 1;
-      int blk0, n_blk;
-      blocks_of(j, blk0, n_blk);
-      const int col0 = j * kTileN + blk0 * 32;                // chunk-local column of this warp's first block
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kTileN + blk0 * 32);
-      if (n_blk > 0) tc::tmem_ld_wait(ra);
-      if (n_blk > 1) tc::tmem_ld32_issue(taddr + 32u, rb);
-      if (n_blk > 0) scan_block(ra, s_rn, col0, n_cols, c0, best, best_col);
-      if (n_blk > 1) tc::tmem_ld_wait(rb);
-      // every load of this job has landed in registers: hand the accumulator back to the MMA warp
+    const int n_tp = p < T ? (T - p + kParts - 1) / kParts : 0;   // tiles of this part
+    // every load of a job has landed in registers: hand the accumulator back to the MMA warp
+    auto release = [&]() {
       tc::fence_before_sync();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&tm_empty[buf]);
-      if (job + 1 < n_jobs) {
-        const int nj = (job + 1) % n_nt;
-        int nblk0, nn_blk;
-        blocks_of(nj, nblk0, nn_blk);
-        if (!s_fail && !tc::mbar_wait(&tm_full[buf ^ 1], (uint32_t)(((job + 1) >> 1) & 1))) s_fail = 1;
+      if (lane == 0) tc::mbar_arrive(&tm_empty[p]);
+    };
+#pragma unroll 1
+    for (int k = 0; k < n_tp; ++k) {
+      float best = -INFINITY; int best_col = 0x7fffffff;
+#pragma unroll 1
+      for (int j = 0; j < n_j; ++j) {
+        const int cnt = k * n_j + j;
+        if (!s_fail && !tc::mbar_wait(&tm_full[p], (uint32_t)(cnt & 1))) s_fail = 1;
         tc::fence_after_sync();
-        if (nn_blk > 0)
-          tc::tmem_ld32_issue(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf ^ 1) * kTileN + nblk0 * 32), ra);
-      }
-      if (n_blk > 1) scan_block(rb, s_rn, col0 + 32, n_cols, c0, best, best_col);
-      if (j == n_nt - 1) {
-        // (ordered value, inverted slot): larger is better, ties go to the lower slot; -0 counts as +0
-        if (best == 0.f) best = 0.f;
-        const unsigned long long key = best > -INFINITY
-            ? (((unsigned long long)float_ord(best) << 32) | (uint32_t)(0x7fffffff - best_col)) : 0ull;
-        if (part > 0) s_pair[(part - 1) * kTileM + row] = key;
-        asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
-        if (part == 0) {
-          unsigned long long k = key;
-#pragma unroll
-          for (int o = 0; o < 3; ++o) { const unsigned long long other = s_pair[o * kTileM + row]; k = other > k ? other : k; }
-          const int pos = t * kTileM + row;
-          if (pos < Pb) out_keys[pos] = k;
+        const int cl = j * kJobN;                              // chunk-local column of the job's first block
+        const int nb = (min(kJobN, n_cols - cl) + 31) / 32;    // 32-column blocks with retained rows: 1 .. 4
+        // loads run one block ahead of the scan
+        tc::tmem_ld32_issue(lane_base, ra);
+        tc::tmem_ld_wait(ra);
+        if (nb > 1) tc::tmem_ld32_issue(lane_base + 32u, rb); else release();
+        scan_block(ra, s_rn, cl, n_cols, c0, best, best_col);
+        if (nb > 1) {
+          tc::tmem_ld_wait(rb);
+          if (nb > 2) tc::tmem_ld32_issue(lane_base + 64u, ra); else release();
+          scan_block(rb, s_rn, cl + 32, n_cols, c0, best, best_col);
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kTcEpiWarps * 32) : "memory");
-        best = -INFINITY; best_col = 0x7fffffff;
+        if (nb > 2) {
+          tc::tmem_ld_wait(ra);
+          if (nb > 3) tc::tmem_ld32_issue(lane_base + 96u, rb); else release();
+          scan_block(ra, s_rn, cl + 64, n_cols, c0, best, best_col);
+        }
+        if (nb > 3) {
+          tc::tmem_ld_wait(rb);
+          release();
+          scan_block(rb, s_rn, cl + 96, n_cols, c0, best, best_col);
+        }
       }
+      // (ordered value, inverted slot): larger is better, ties go to the lower slot; -0 counts as +0
+      if (best == 0.f) best = 0.f;
+      const unsigned long long key = best > -INFINITY
+          ? (((unsigned long long)float_ord(best) << 32) | (uint32_t)(0x7fffffff - best_col)) : 0ull;
+      const int pos = (t0 + k * kParts + p) * kTileM + row;
+      if (pos < Pb) out_keys[pos] = key;
     }
   }
   tc::fence_before_sync();
@@ -417,14 +409,14 @@ void sim_tc_build_items(const d2o_ctx* c, int n_sms, int4* items, int32_t* count
       }
     size_t n = 0;
     if (n_pieces > 0) {
-      // aim at five waves of equal items, at least four tiles each (a CTA first loads its chunk of retained rows)
+      // aim at five waves of equal items, at least eight tiles each (a CTA first loads its chunk of retained rows and keeps four tiles in flight)
       const double target = total / ((double)n_sms * 5.0);
       std::vector<std::pair<double, int4>> list;
       for (size_t i = 0; i < n_pieces; ++i) {
         const Piece& p = pieces[i];
         const double work = (double)p.tiles * (p.cols + 64);
         int k = (int)(work / target + 0.5);
-        k = max(1, min(k, max(1, p.tiles / 4)));
+        k = max(1, min(k, max(1, p.tiles / 8)));
         if (list.size() + k + (n_pieces - i) > cap) k = 1;     // never more entries than the list holds
         for (int j = 0; j < k; ++j) {
           const int t0 = (int)((long long)p.tiles * j / k), t1 = (int)((long long)p.tiles * (j + 1) / k);
@@ -471,7 +463,7 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
   a.L = g.n_layers; a.layer = layer; a.Hkv = Hkv; a.P = P; a.n_chunks_max = n_chunks_max;
   a.items = (const int4*)(S + c->lay.sim_items) + (size_t)layer * sim_tc_max_items(&g, c->max_budget);
   const int KB = D / 64;
-  const size_t smem = (size_t)KB * kChunkN * 128 + (size_t)kAStages * KB * kTileM * 128 + kChunkN * 4 + 3 * kTileM * 8;
+  const size_t smem = (size_t)KB * kChunkN * 128 + (size_t)kParts * KB * kTileM * 128 + kChunkN * 4;
   dim3 grid((unsigned)n_items);
   const int fmt = g.dtype == D2O_F16 ? 0 : 1;
   cudaError_t e;
