@@ -47,7 +47,7 @@ constexpr int kTensorMinG = 2;                          // query heads per KV he
 constexpr uint32_t kSuspendNs = 4000u;                  // a waiting thread may stay suspended this long before it looks again
 
 struct DecodeArgs {
-  const int32_t* budgets; const int32_t* windows; const int64_t* row_off;   // [B, L]
+  const int32_t* budgets; const int32_t* windows; const int64_t* row_off;   // [B, L, Hkv]
   int32_t* pos; float* score; float* rnorm;                                  // pool-wide
   int32_t* len; float* tau;                                                  // [L, B, Hkv]
   unsigned long long* counters; uint32_t* status;

@@ -22,9 +22,9 @@ constexpr int kSelThreads = 1024;
 
 struct SelectArgs {
   const float* colsum;     // [B, Hq, P] of this layer
-  const int32_t* budgets;  // [B, L]
-  const int32_t* windows;  // [B, L]
-  const int64_t* row_off;  // [B, L]
+  const int32_t* budgets;  // [B, L, Hkv]
+  const int32_t* windows;  // [B, L, Hkv]
+  const int64_t* row_off;  // [B, L, Hkv]
   int32_t* pos; float* score; float* rnorm;   // pool-wide
   int32_t* len; float* tau;                   // [L, B, Hkv]
   int32_t* evict_idx;      // [B, Hkv, P]
@@ -504,19 +504,42 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
 #pragma unroll
   for (int i = 0; i < EPV; ++i) va[i] = own * f[i];
   float den = own;
-  for (int s = s0; s < s1; ++s) {
-    const int i = items[s];
-    if (!D2O_GUARD(i >= 0 && i < Le, a.status, 0xC4EC0005u)) continue;
-    const float w = a.average ? 1.0f : expf(mx[i]);
-    const int pj = ev[i];
-    if (!D2O_GUARD(pj >= 0 && pj < a.plen[b], a.status, 0xC4EC0006u)) continue;
-    den += w;
-    Elem<T>::unpack(ld_global_v4(Ks + (size_t)pj * D + lig * EPV), f);
+  // The lanes of the row first fetch the list entries of up to LPR merged tokens side by side (entry -> similarity and
+  // prompt position), then the rows are added in list order, two tokens' key and value rows in flight at a time: the
+  // chain entry -> position -> row is three dependent loads per token otherwise.
+  const unsigned gm = group_mask<LPR>();
+  for (int s = s0; s < s1; s += LPR) {
+    const int cnt = min(LPR, s1 - s);
+    float my_w = 0.f; int my_pj = 0;
+    if (lig < cnt) {
+      const int i = items[s + lig];
+      if (D2O_GUARD(i >= 0 && i < Le, a.status, 0xC4EC0005u)) {
+        const int pj = ev[i];
+        if (D2O_GUARD(pj >= 0 && pj < a.plen[b], a.status, 0xC4EC0006u)) { my_pj = pj; my_w = a.average ? 1.0f : expf(mx[i]); }
+      }
+    }
+    for (int t = 0; t < cnt; t += 2) {
+      const float w0 = __shfl_sync(gm, my_w, t, LPR), w1 = t + 1 < cnt ? __shfl_sync(gm, my_w, t + 1, LPR) : 0.f;
+      const int p0 = __shfl_sync(gm, my_pj, t, LPR), p1 = t + 1 < cnt ? __shfl_sync(gm, my_pj, t + 1, LPR) : p0;
+      const uint4 k0 = ld_global_v4(Ks + (size_t)p0 * D + lig * EPV), v0 = ld_global_v4(Vs + (size_t)p0 * D + lig * EPV);
+      const uint4 k1 = ld_global_v4(Ks + (size_t)p1 * D + lig * EPV), v1 = ld_global_v4(Vs + (size_t)p1 * D + lig * EPV);
+      den += w0;
+      Elem<T>::unpack(k0, f);
 #pragma unroll
-    for (int e = 0; e < EPV; ++e) ka[e] = fmaf(w, f[e], ka[e]);
-    Elem<T>::unpack(ld_global_v4(Vs + (size_t)pj * D + lig * EPV), f);
+      for (int e = 0; e < EPV; ++e) ka[e] = fmaf(w0, f[e], ka[e]);
+      Elem<T>::unpack(v0, f);
 #pragma unroll
-    for (int e = 0; e < EPV; ++e) va[e] = fmaf(w, f[e], va[e]);
+      for (int e = 0; e < EPV; ++e) va[e] = fmaf(w0, f[e], va[e]);
+      if (t + 1 < cnt) {                                   // a token whose check failed has weight 0: its terms are +0
+        den += w1;
+        Elem<T>::unpack(k1, f);
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) ka[e] = fmaf(w1, f[e], ka[e]);
+        Elem<T>::unpack(v1, f);
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) va[e] = fmaf(w1, f[e], va[e]);
+      }
+    }
   }
   const float inv = 1.0f / den;
 #pragma unroll
