@@ -61,27 +61,60 @@ __host__ __device__ __forceinline__ int chunk_columns(int S) {
   return (((S + n_chunks - 1) / n_chunks) + 15) & ~15;
 }
 
+// (x0, x1) = (a0 * b0, a1 * b1), each product rounded to nearest as a single multiply would.
+__device__ __forceinline__ void mul_pair(float a0, float a1, float b0, float b1, float& x0, float& x1) {
+  unsigned long long a, b, d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "f"(a0), "f"(a1));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(b) : "f"(b0), "f"(b1));
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(d));
+}
+
+// Maximum of three; a NaN operand is ignored.
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 // One block of 32 accumulator columns of one row: times 1/|k_c| per column, maximum and its column (the lowest
 // on ties), merged into the row's running (best, best_col).  cl0 = chunk-local column of the block.
 __device__ __forceinline__ void scan_block(const uint32_t (&r)[32], const float* s_rn, int cl0, int n_cols, int c0,
                                            float& best, int& best_col) {
-  // four interleaved running maxima (columns i mod 4) keep the compare chains short
-  float tb[4]; int ti[4];
-#pragma unroll
-  for (int w = 0; w < 4; ++w) { tb[w] = -INFINITY; ti[w] = w; }
   const float4* rn4 = reinterpret_cast<const float4*>(s_rn + cl0);
   if (cl0 + 32 <= n_cols) {
+    // Columns go in pairs (2i, 2i + 1): one packed multiply, one three-input maximum against the running value,
+    // one compare and two selects per pair.  The chain remembers the winning pair and that pair's first value,
+    // from which the column inside the pair follows at the end.  Two chains (pairs i mod 2) keep them short.
+    // max.f32 drops a NaN operand, as the compare of the scalar form does.
+    float pb[2] = {-INFINITY, -INFINITY}, plo[2] = {-INFINITY, -INFINITY};
+    int pi[2] = {0, 1};
 #pragma unroll
     for (int i4 = 0; i4 < 8; ++i4) {
       const float4 q = rn4[i4];
       const float rv[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const float x = __uint_as_float(r[i4 * 4 + w]) * rv[w];
-        if (x > tb[w]) { tb[w] = x; ti[w] = i4 * 4 + w; }
+      for (int w = 0; w < 2; ++w) {
+        float x0, x1;
+        mul_pair(__uint_as_float(r[i4 * 4 + 2 * w]), __uint_as_float(r[i4 * 4 + 2 * w + 1]), rv[2 * w], rv[2 * w + 1], x0, x1);
+        const float m = max3(pb[w], x0, x1);
+        const bool up = m > pb[w];
+        pi[w] = up ? i4 * 2 + w : pi[w];
+        plo[w] = up ? x0 : plo[w];
+        pb[w] = m;
       }
     }
-  } else {                                                        // columns past the chunk hold other slices' rows
+    // the later chain wins only with a larger value or an equal one from an earlier pair
+    if (pb[1] > pb[0] || (pb[1] == pb[0] && pi[1] < pi[0])) { pb[0] = pb[1]; pi[0] = pi[1]; plo[0] = plo[1]; }
+    const int col = 2 * pi[0] + (plo[0] == pb[0] ? 0 : 1);        // equal values inside the pair: the lower column
+    if (pb[0] > best) { best = pb[0]; best_col = c0 + cl0 + col; }
+    return;
+  }
+  // four interleaved running maxima (columns i mod 4) keep the compare chains short
+  float tb[4]; int ti[4];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) { tb[w] = -INFINITY; ti[w] = w; }
+  {                                                               // columns past the chunk hold other slices' rows
 #pragma unroll
     for (int i4 = 0; i4 < 8; ++i4) {
       const float4 q = rn4[i4];
