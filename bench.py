@@ -41,6 +41,7 @@ NOMINAL_HBM_GBS = 8000.0          # the figure the metric quotes; the measured c
 # dram__bytes_read.sum + dram__bytes_write.sum of the decode_kernel launches of one step under ncu, divided by the
 # algorithmic bytes of that step, per workload the counters were taken on (None: not captured for this kernel build)
 DECODE_TRAFFIC_RATIO = {"cfg1": None, "cfg2": None}
+NO_CHAIN = False                  # --single-step-calls: one d2o_decode_step call per token in the timed passes too
 
 
 def parse():
@@ -66,6 +67,8 @@ def parse():
     ap.add_argument("--no-per-config", action="store_true", help="skip the shorter measurements of the other configs")
     ap.add_argument("--unclamped", action="store_true", help="run the main config without the upper budget clamp")
     ap.add_argument("--layers-per-call", type=int, default=0)
+    ap.add_argument("--single-step-calls", action="store_true",
+                    help="decode with one d2o_decode_step call per token instead of d2o_decode_steps")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling captures)")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences (the serving sweep of config 4)")
     return ap.parse_args()
@@ -201,7 +204,10 @@ def measure_resident(ctx, wl, prompts, dq, dk, dv, nd, lpc, warmup, steps, world
     """`steps` timed passes of the whole path with every input resident; returns per-phase milliseconds (mean over
     the passes), the budgets, the launch count, and the decode-step percentiles of one extra pass."""
     L = wl.n_layers
-    dout = torch.empty_like(dq[0])
+    # all layers per call: the decode steps of a pass go through the multi-step entry point (their inputs are all
+    # resident, which is what it asks for); the extra pass below steps call by call
+    chain = (lpc == L) and not NO_CHAIN
+    dout = torch.empty_like(dq) if chain else torch.empty_like(dq[0])
     launches = {"n": 0, "decode_seen": ctx.d2o_get_stats().decode_launches}
 
     def one_pass(timed: bool, step_events=None):
@@ -215,12 +221,16 @@ def measure_resident(ctx, wl, prompts, dq, dk, dv, nd, lpc, warmup, steps, world
         for l in range(L):
             ctx.d2o_prefill_compress(l, prompts[l][1], prompts[l][2])
         e[3].record()
-        for s in range(nd):
-            for l0 in range(0, L, lpc):
-                l1 = min(L, l0 + lpc)
-                ctx.d2o_decode_step(l0, l1, dq[s, l0:l1], dk[s, l0:l1], dv[s, l0:l1], dout[l0:l1])
-            if step_events is not None:
-                step_events[s + 1].record()
+        if chain and step_events is None:
+            ctx.d2o_decode_steps(0, L, nd, dq, dk, dv, dout)
+        else:
+            o = dout[0] if chain else dout
+            for s in range(nd):
+                for l0 in range(0, L, lpc):
+                    l1 = min(L, l0 + lpc)
+                    ctx.d2o_decode_step(l0, l1, dq[s, l0:l1], dk[s, l0:l1], dv[s, l0:l1], o[l0:l1])
+                if step_events is not None:
+                    step_events[s + 1].record()
         e[4].record()
         dl = ctx.d2o_get_stats().decode_launches      # the library counts its decode launches (a step may take two)
         if timed:
@@ -255,13 +265,15 @@ def measure_resident(ctx, wl, prompts, dq, dk, dv, nd, lpc, warmup, steps, world
         torch.cuda.synchronize()
         step_us = sorted(step_ev[i].elapsed_time(step_ev[i + 1]) * 1e3 for i in range(nd))
         step_pct = {"p50": round(step_us[nd // 2], 2), "p99": round(step_us[min(nd - 1, (nd * 99) // 100)], 2),
-                    "max": round(step_us[-1], 2)}
+                    "max": round(step_us[-1], 2), "mean": round(step_ev[0].elapsed_time(step_ev[nd]) * 1e3 / nd, 2),
+                    "entry_point": "d2o_decode_step, one call per token (an event after every call)"}
     seg = [[p[0][i].elapsed_time(p[0][i + 1]) for i in range(4)] for p in passes]          # ms
     means = [statistics.mean(s[i] for s in seg) for i in range(4)]
     means.append(sum(means))
     stats_ms, budget_ms, compress_ms, decode_ms, pass_ms = max_over_ranks(means, world, device)
     return dict(stats_ms=stats_ms, budget_ms=budget_ms, compress_ms=compress_ms, decode_ms=decode_ms, pass_ms=pass_ms,
-                budgets=passes[-1][1], launches=launches["n"], clocks=clocks, wall_s=t_wall, step_pct=step_pct)
+                budgets=passes[-1][1], launches=launches["n"], clocks=clocks, wall_s=t_wall, step_pct=step_pct,
+                chained=chain)
 
 
 def measure_streamed(B, wl, nd, warmup, steps, device, args, with_lse=False):
@@ -269,8 +281,10 @@ def measure_streamed(B, wl, nd, warmup, steps, device, args, with_lse=False):
     the compression stage), so that batches whose prompts do not fit all at once can be measured.  Only the library
     calls are inside the event pairs.  Returns the same per-phase means as measure_resident."""
     L = wl.n_layers
-    ctx = make_context(B, wl, nd, device, args)
+    chain = not NO_CHAIN
+    ctx = make_context(B, wl, 2 * nd if chain else nd, device, args)
     acc = []
+    single_ms = []
     lse_ms = None
     for it in range(warmup + steps):
         t_stats = t_comp = 0.0
@@ -294,14 +308,26 @@ def measure_streamed(B, wl, nd, warmup, steps, device, args, with_lse=False):
             del K, V
             streams.append(s)
         dq, dk, dv = decode_inputs(streams, nd)
-        dout = torch.empty_like(dq[0])
+        dout = torch.empty_like(dq) if chain else torch.empty_like(dq[0])
         a, b = ev(), ev()
         a.record()
-        for s in range(nd):
-            ctx.d2o_decode_step(0, L, dq[s], dk[s], dv[s], dout)
+        if chain:
+            ctx.d2o_decode_steps(0, L, nd, dq, dk, dv, dout)
+        else:
+            for s in range(nd):
+                ctx.d2o_decode_step(0, L, dq[s], dk[s], dv[s], dout)
         b.record()
         pend.append((3, a, b))
+        if chain:
+            # the same number of further tokens, one call per token (same inputs again: the sizes are what matters)
+            a2, b2 = ev(), ev()
+            a2.record()
+            for s in range(nd):
+                ctx.d2o_decode_step(0, L, dq[s], dk[s], dv[s], dout[0])
+            b2.record()
         torch.cuda.synchronize()
+        if chain and it >= warmup:
+            single_ms.append(a2.elapsed_time(b2))
         tot = [0.0, 0.0, 0.0, 0.0]
         for k, a, b in pend:
             tot[k] += a.elapsed_time(b)
@@ -330,7 +356,8 @@ def measure_streamed(B, wl, nd, warmup, steps, device, args, with_lse=False):
     torch.cuda.empty_cache()
     m = [statistics.mean(x[i] for x in acc) for i in range(4)]
     return dict(stats_ms=m[0], budget_ms=m[1], compress_ms=m[2], decode_ms=m[3], pass_ms=sum(m), budgets=budgets,
-                stats_with_lse_ms=lse_ms, merges_discards=[int(st.merges), int(st.discards)])
+                stats_with_lse_ms=lse_ms, merges_discards=[int(st.merges), int(st.discards)],
+                decode_single_calls_ms=statistics.mean(single_ms) if single_ms else None)
 
 
 def full_cache_decode(B, wl, nd, device, peak, world=1):
@@ -395,6 +422,9 @@ def per_config_entry(B, wl, device, args, peaks, full_cache=False):
     m = measure_streamed(B, wl, nd, 1, 2, device, args, with_lse=(wl.dtype != "f32"))
     bytes_per_step, achieved, peak = roofline_of_decode(wl, m["budgets"], nd, m["decode_ms"], 1, peaks)
     out = {"workload": workload_string(wl, nd), "decode_us_per_step": round(m["decode_ms"] * 1e3 / nd, 2),
+           "decode_entry_point": "d2o_decode_step" if NO_CHAIN else "d2o_decode_steps",
+           "decode_us_per_step_single_calls": (None if m["decode_single_calls_ms"] is None
+                                               else round(m["decode_single_calls_ms"] * 1e3 / nd, 2)),
            "tokens_per_s": round(wl.batch * nd / (m["decode_ms"] * 1e-3), 1),
            "frac_of_measured_hbm": round(achieved / peak, 4), "frac_of_nominal_hbm": round(achieved / NOMINAL_HBM_GBS, 4),
            "achieved_GBps": round(achieved, 1), "stats_ms": round(m["stats_ms"], 3),
@@ -497,7 +527,9 @@ def run_ours(args, wl, rank, world, device):
                    "layers_per_decode_call": lpc, "decode_ring_stages": args.stages or "auto",
                    "sequences_per_gpu": wl.batch, "parallelism": "replicas (independent sequences per GPU)"},
         "decode_steps_per_s_per_gpu": round(steps_per_s, 2), "decode_us_per_step": round(decode_ms * 1e3 / nd, 2),
-        "decode_step_us_percentiles": m["step_pct"],
+        "decode_entry_point": ("d2o_decode_steps (all decode steps of a pass in one call, inputs resident)"
+                               if m["chained"] else "d2o_decode_step (one call per token)"),
+        "decode_step_us_single_calls": m["step_pct"],
         "stats_ms": round(m["stats_ms"], 3), "budgets_ms": round(m["budget_ms"], 3),
         "prefill_compress_ms": round(m["compress_ms"], 3), "decode_ms": round(decode_ms, 3),
         "wall_s": round(m["wall_s"], 3), "budgets_min_max": [int(budgets.min()), int(budgets.max())],
@@ -619,7 +651,9 @@ def spawn_ranks(n: int) -> int:
 
 
 def main():
+    global NO_CHAIN
     args = parse()
+    NO_CHAIN = args.single_step_calls
     wl = W.CONFIGS[args.config] if args.config in W.CONFIGS else W.twin(args.config.replace("_twin", ""))
     if args.batch:
         wl = dataclasses.replace(wl, batch=args.batch, name=f"{wl.name}[B={args.batch}]")

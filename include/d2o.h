@@ -181,6 +181,22 @@ d2o_status d2o_prefill_compress(d2o_ctx* ctx, int32_t layer, const void* K, cons
 d2o_status d2o_decode_step(d2o_ctx* ctx, int32_t l0, int32_t l1, const void* q, const void* k,
                            const void* v, void* out, void* stream);
 
+/* n_steps consecutive generated tokens for layers [l0, l1) whose inputs are all resident
+ * (Section 4.2, one eviction per generated token; Eq. 2-3, 6-12 per step as in
+ * d2o_decode_step).  DEVICE tensors: q [n_steps, l1-l0, B, Hq, d], k and v
+ * [n_steps, l1-l0, B, Hkv, d], out [n_steps, l1-l0, B, Hq, d]; every entry must be complete
+ * (stream-ordered) before the call, so a step's inputs cannot depend on an earlier step's
+ * output.  The results are those of n_steps calls of d2o_decode_step, bit for bit.  What
+ * differs is the launch: from the second step on a step's grids are launched with
+ * programmatic stream serialisation and start while the previous step's last CTAs still
+ * run; every CTA then waits (with the limit of every other wait in the kernel) for a
+ * per-slice step counter that the slice's previous CTA publishes as its last act, not for
+ * the whole previous grid.  Whatever follows on `stream` is ordered behind all n_steps.
+ * Errors: as d2o_decode_step; D2O_ERR_STATE if fewer than n_steps tokens remain of
+ * max_new_tokens (nothing is launched then). */
+d2o_status d2o_decode_steps(d2o_ctx* ctx, int32_t l0, int32_t l1, int32_t n_steps, const void* q,
+                            const void* k, const void* v, void* out, void* stream);
+
 /* Same with HOST buffers (pinned memory recommended): copies q, k, v to the device, runs the
  * step, copies `out` back and synchronises `stream`.  If q, k and v lie back to back in host
  * memory in this order they travel in one transfer. */

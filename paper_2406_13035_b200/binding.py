@@ -24,7 +24,7 @@ TORCH_DTYPE = {D2O_F32: torch.float32, D2O_F16: torch.float16, D2O_BF16: torch.b
 EXPORTS = [
     "d2o_status_string", "d2o_last_cuda_error", "d2o_workspace_size", "d2o_create", "d2o_destroy",
     "d2o_layer_stats", "d2o_layer_budgets", "d2o_budgets_from_density", "d2o_prefill_compress",
-    "d2o_decode_step", "d2o_decode_step_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
+    "d2o_decode_step", "d2o_decode_steps", "d2o_decode_step_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
     "d2o_set_tuning", "d2o_layer_stats_static", "d2o_set_fault_injection", "d2o_set_prompt_lens",
 ]
 STATIC_LSE_FLOATS = 1 << 20      # D2O_STATIC_LSE_FLOATS of include/d2o.h
@@ -94,6 +94,7 @@ def load_library() -> C.CDLL:
     lib.d2o_prefill_compress.argtypes = [vp, i32, vp, vp, vp]
     lib.d2o_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.d2o_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.d2o_decode_steps.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.d2o_full_decode_step.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.d2o_get_view.argtypes = [vp, i32, C.POINTER(D2OView)]
     lib.d2o_get_stats.argtypes = [vp, C.POINTER(D2OStats), vp]
@@ -200,6 +201,10 @@ class D2OContext:
     def d2o_decode_step(self, l0: int, l1: int, q, k, v, out):
         _check(self.lib.d2o_decode_step(self.handle, l0, l1, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream()),
                "d2o_decode_step")
+
+    def d2o_decode_steps(self, l0: int, l1: int, n_steps: int, q, k, v, out):
+        _check(self.lib.d2o_decode_steps(self.handle, l0, l1, n_steps, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream()),
+               "d2o_decode_steps")
 
     def d2o_decode_step_host(self, l0: int, l1: int, q, k, v, out):
         for t in (q, k, v, out):

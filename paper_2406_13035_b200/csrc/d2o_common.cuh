@@ -146,7 +146,7 @@ enum Counter { kCntDecodeSteps = 0, kCntEvictions, kCntMerges, kCntDiscards, kCn
 
 // ----------------------------------------------------------------------------- context
 struct Layout {            // byte offsets into `state`
-  size_t status, counters, density, budgets, windows, row_off, order, plen, len, tau, sim_items, colsum, pos, score, rnorm, kpool, vpool, end;
+  size_t status, counters, density, budgets, windows, row_off, order, plen, len, tau, steps_done, sim_items, colsum, pos, score, rnorm, kpool, vpool, end;
 };
 struct ScratchLayout {     // byte offsets into `scratch`
   size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, seg_tmp, part_key, pl_spill, stage_q, stage_k, stage_v, stage_out, end;
@@ -204,7 +204,7 @@ cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, 
                            const int32_t* plen, cudaStream_t st);
 cudaError_t launch_prefill_compress(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st);
 cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const void* k, const void* v, void* out,
-                          cudaStream_t st, d2o_status* why);
+                          cudaStream_t st, d2o_status* why, bool chained = false, bool publish = false);
 cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int capacity, int len, void* kc, void* vc,
                                const void* q, const void* k, const void* v, void* out, cudaStream_t st,
                                d2o_status* why);

@@ -64,6 +64,9 @@ struct DecodeArgs {
   unsigned long long wait_ns;       // a wait for a stage gives up after this long
   int stop_stage;                   // failure-detection tests: the producer issues no copy from this stage on (-1: never)
   long long pool_rows;              // rows of the cache pool (bounds of the checked build)
+  int32_t* steps_done;              // [L, B, Hkv] decode steps completed on the slice: written as a CTA's last act
+  int chained;                      // 1: the previous step's grids may still be running (see slice_ready)
+  int publish;                      // 1: a chained step follows: the CTA publishes the slice's step counter at its end
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -109,6 +112,20 @@ __device__ __forceinline__ bool landed_wait(unsigned long long* bar, uint32_t pa
   while (!mbar_try_wait(bar, parity))
     if (global_ns() - t0 > limit_ns) return false;
   return true;
+}
+// Waits, with a limit, until the slice's step counter has reached `want`: the CTA that ran the slice's previous
+// decode step has finished and its stores are visible.  0: ready; 1: an anomaly was recorded meanwhile (the state is
+// no longer trusted); 2: the wait ran out.
+__device__ __forceinline__ int slice_ready(const int32_t* flag, int want, const uint32_t* status, unsigned long long limit_ns) {
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v >= want) return 0;
+    if (*reinterpret_cast<const volatile uint32_t*>(status) != 0u) return 1;
+    if (global_ns() - t0 > limit_ns) return 2;
+    __nanosleep(200);
+  }
 }
 // Similarity as an ordered key: -0 (a zero-norm row times a negative dot product) must count as +0, or equal
 // similarities would not tie.
@@ -333,6 +350,17 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   const int M = a.windows[slice_entry(b, layer, h, a.L, a.Hkv)];
   const int64_t row0 = a.row_off[slice_entry(b, layer, h, a.L, a.Hkv)];
   const int sidx = (layer * a.B + b) * a.Hkv + h;
+  // a chained step runs beside the grids of the step before it: the slice is this CTA's once that step's CTA has
+  // published it
+  __shared__ int s_chain;
+  if (a.chained) {
+    if (tid == 0) s_chain = slice_ready(a.steps_done + sidx, a.step, a.status, a.wait_ns);
+    __syncthreads();
+    if (s_chain != 0) {                                              // uniform for the CTA, before any barrier or copy
+      if (tid == 0 && s_chain == 2) report_error(a.status, D2O_ERR_TIMEOUT, 0xDEC20000u | (uint32_t)(sl & 0xffff));
+      return;
+    }
+  }
   const int n_old = a.len[sidx];
   const float tau_old = a.tau[sidx];
   if (!D2O_GUARD(S >= 1 && n_old >= 0 && n_old <= S && row0 >= 0 && row0 + slice_stride(S) <= a.pool_rows, a.status,
@@ -371,10 +399,12 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   __shared__ int s_li[kConsWarps], s_best_li;
   __shared__ volatile int s_timeout;                                 // 1: an earlier launch recorded an anomaly; 2: a wait of this CTA ran out
   __shared__ int s_bail;
+  __shared__ unsigned long long s_done;                              // arrivals of the consumer warps at the kernel's end
 
   if (tid == 0) {
     s_timeout = *reinterpret_cast<volatile uint32_t*>(a.status) != 0u;
     for (int s = 0; s < NS; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kConsWarps); }
+    mbar_init(&s_done, kConsWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -386,6 +416,8 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
   // =========================================================================== producer warp
   if (warp == kConsWarps) {
     if (lane == 0) {
+      // rows that the previous step's CTA wrote with ordinary stores are read here by bulk copies
+      if (a.chained) asm volatile("fence.proxy.async.global;" ::: "memory");
       unsigned long long keep = 0, drop = 0;
       if (a.l2_hints) {
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
@@ -453,6 +485,14 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
           if (sl_i == 0) { sl_i = NS - 1; ph_i ^= 1u; } else --sl_i;
           if (!landed_wait(&s_full[sl_i], ph_i ^ 1u, a.wait_ns)) break;
         }
+      }
+      // a chained step follows: once every consumer warp has arrived (the slice's state is complete and ordered
+      // before this thread by the arrivals), publish the slice's step counter.  Not after a wait ran out: the step
+      // after this one then finds the error word, or runs into its own limit.
+      if (a.publish && !stopped) {
+        stage_wait(&s_done, 0u, &s_timeout, a.wait_ns);
+        if (s_timeout == 0)
+          asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(a.steps_done + sidx), "r"(a.step + 1) : "memory");
       }
     }
     // A grid launched with programmatic stream serialisation may run beside its predecessor, but it must not be
@@ -1149,6 +1189,16 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     }
   }
   if (tid == 0 && s_timeout == 2) report_error(a.status, D2O_ERR_TIMEOUT, 0xDEC10000u | (uint32_t)(sl & 0xffff));
+  // This warp's part of the slice's state is complete.  When a chained step follows, the producer warp waits for
+  // every consumer warp's arrival and publishes the slice's step counter.  The next step's CTA reads the rows,
+  // positions and norms that warp 0 writes last with bulk copies, hence the proxy fence in that warp.
+  auto consumer_done = [&]() {
+    if (a.publish) {
+      if (warp == 0) asm volatile("fence.proxy.async.global;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_done);
+    }
+  };
   if (!evict) {
     // the cache is not full yet: append the new token's row
     if (grp == 0) {
@@ -1160,6 +1210,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       a.len[sidx] = n;
       atomicAdd(&a.counters[kCntDecodeSteps], 1ull);
     }
+    consumer_done();
     return;
   }
   // ---- merged value row (Eq. 11); the new token's value takes the victim's row
@@ -1177,6 +1228,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     }
     if (vic_li != n_old) *reinterpret_cast<uint4*>(vpool + (row0 + vic_li) * D + lane * EPV) = vslot;
   }
+  consumer_done();
 }
 
 // ------------------------------------------------------------------------------------ launch
@@ -1273,8 +1325,13 @@ static int smem_rows_for(int max_rows, double mean_rows, int G) {
   return min(max_rows, max(free_rows, (int)(2.0 * mean_rows)));
 }
 
+// `chained`: this step follows another decode step of the same layers on the same stream, and its inputs were
+// complete before that one was launched.  Its grids are then launched with programmatic stream serialisation and
+// may start while the previous step's last CTAs are still running; every CTA waits for its own slice's step counter
+// instead of the whole previous grid.  `publish`: a chained step follows this one, so every CTA writes its slice's
+// step counter when the slice's state is complete.
 cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const void* k, const void* v, void* out,
-                          cudaStream_t st, d2o_status* why) {
+                          cudaStream_t st, d2o_status* why, bool chained, bool publish) {
   const d2o_config& g = c->cfg;
   const int B = g.batch, L = g.n_layers;
   DecodeArgs a = {};
@@ -1292,6 +1349,9 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   a.wait_ns = c->wait_limit_us > 0 ? (unsigned long long)c->wait_limit_us * 1000ull : kWaitNs;
   a.stop_stage = c->producer_stop_stage;
   a.pool_rows = c->pool_rows;
+  a.steps_done = (int32_t*)(S + c->lay.steps_done);
+  a.chained = chained ? 1 : 0;
+  a.publish = publish ? 1 : 0;
   a.l2_hints = c->decode_l2_hints;
   const int G = c->group, Hkv = g.n_kv_heads;
   const int row_bytes = g.d_head * c->elem_size;
@@ -1387,7 +1447,7 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
   };
 
   if (n_long > 0) {
-    cudaError_t e = launch_class(0, n_long, 16, false);
+    cudaError_t e = launch_class(0, n_long, 16, chained);
     if (e != cudaSuccess || *why != D2O_OK) return e;
     const int rest = (n_pairs - n_long) * Hkv;
     int rest_max = rows_of_pair(n_long);
@@ -1406,7 +1466,7 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     if (G <= 2 && n_slices >= 8 * c->n_sms * 4 && max_rows <= 1536) cw = 4;
     if (G >= 4 && n_slices <= c->n_sms * 8 && max_rows > 2.0 * mean_rows) cw = 16;
   }
-  return launch_class(0, n_pairs, cw, false);
+  return launch_class(0, n_pairs, cw, chained);
 }
 
 }  // namespace d2o

@@ -108,6 +108,7 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   l->plen = take(B * 4);
   l->len = take(L * B * Hkv * 4);
   l->tau = take(L * B * Hkv * 4);
+  l->steps_done = take(L * B * Hkv * 4);
   l->sim_items = take(c->dtype == D2O_F32 ? 0 : L * sim_tc_max_items(c, max_budget) * 16);
   l->colsum = take(L * B * Hq * P * 4);
   l->pos = take(rows * 4);
@@ -330,6 +331,29 @@ extern "C" d2o_status d2o_decode_step(d2o_ctx* c, int32_t l0, int32_t l1, const 
   if (why != D2O_OK) return why;
   if (e != cudaSuccess) return cuda_fail(e, "launch_decode");
   for (int l = l0; l < l1; ++l) c->layer_steps[l] += 1;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_decode_steps(d2o_ctx* c, int32_t l0, int32_t l1, int32_t n_steps, const void* q,
+                                       const void* k, const void* v, void* out, void* stream) {
+  d2o_status st = check_decode_range(c, l0, l1);
+  if (st != D2O_OK) return st;
+  if (n_steps < 1) return D2O_ERR_INVALID_ARG;
+  if (c->layer_steps[l0] + n_steps > c->cfg.max_new_tokens) return D2O_ERR_STATE;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return D2O_ERR_INVALID_ARG;
+  const d2o_config& g = c->cfg;
+  const size_t nl = (size_t)(l1 - l0);
+  const size_t qb = nl * g.batch * g.n_q_heads * g.d_head * c->elem_size;     // bytes of one step's q and out
+  const size_t kb = nl * g.batch * g.n_kv_heads * g.d_head * c->elem_size;    // of its k and v
+  for (int s = 0; s < n_steps; ++s) {
+    d2o_status why = D2O_OK;
+    // the first step is ordered behind whatever the stream ran before; the later ones are chained to their predecessor
+    cudaError_t e = launch_decode(c, l0, l1, (const char*)q + s * qb, (const char*)k + s * kb, (const char*)v + s * kb,
+                                  (char*)out + s * qb, (cudaStream_t)stream, &why, s > 0, s + 1 < n_steps);
+    if (why != D2O_OK) return why;
+    if (e != cudaSuccess) return cuda_fail(e, "launch_decode");
+    for (int l = l0; l < l1; ++l) c->layer_steps[l] += 1;
+  }
   return D2O_OK;
 }
 

@@ -27,6 +27,7 @@ struct SelectArgs {
   const int64_t* row_off;  // [B, L, Hkv]
   int32_t* pos; float* score; float* rnorm;   // pool-wide
   int32_t* len; float* tau;                   // [L, B, Hkv]
+  int32_t* steps_done;                        // [L, B, Hkv] decode steps completed on the slice
   int32_t* evict_idx;      // [B, Hkv, P]
   float* keys_spill;       // [B, Hkv, P] group scores when P does not fit in shared memory (may alias evict_mx)
   unsigned long long* counters;
@@ -149,6 +150,7 @@ select_kernel(SelectArgs a, const T* __restrict__ K, const T* __restrict__ V, T*
   const int n_keep = keep_all ? P : S;
   if (threadIdx.x == 0) {
     a.len[sidx] = n_keep;
+    a.steps_done[sidx] = 0;
     a.tau[sidx] = 0.f;
     if (n_ret != n_keep) report_error(a.status, D2O_ERR_STATE, 0x5E000000u | (uint32_t)slice);
     atomicAdd(&a.counters[kCntPrefillEvicted], (unsigned long long)(P - n_keep));
@@ -575,6 +577,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   sa.row_off = (const int64_t*)(S + c->lay.row_off);
   sa.pos = (int32_t*)(S + c->lay.pos); sa.score = (float*)(S + c->lay.score); sa.rnorm = (float*)(S + c->lay.rnorm);
   sa.len = (int32_t*)(S + c->lay.len); sa.tau = (float*)(S + c->lay.tau);
+  sa.steps_done = (int32_t*)(S + c->lay.steps_done);
   sa.evict_idx = (int32_t*)(X + c->slay.evict_idx);
   sa.keys_spill = (float*)(X + c->slay.evict_mx);
   sa.counters = (unsigned long long*)(S + c->lay.counters);
