@@ -218,8 +218,11 @@ def measure_resident(ctx, wl, prompts, dq, dk, dv, nd, lpc, warmup, steps, world
         e[1].record()
         budgets = ctx.d2o_layer_budgets()
         e[2].record()
-        for l in range(L):
-            ctx.d2o_prefill_compress(l, prompts[l][1], prompts[l][2])
+        if NO_CHAIN:
+            for l in range(L):
+                ctx.d2o_prefill_compress(l, prompts[l][1], prompts[l][2])
+        else:                                             # every layer's K and V are resident: one call
+            ctx.d2o_prefill_compress_layers(0, L, [p[1] for p in prompts], [p[2] for p in prompts])
         e[3].record()
         if chain and step_events is None:
             ctx.d2o_decode_steps(0, L, nd, dq, dk, dv, dout)
@@ -299,14 +302,24 @@ def measure_streamed(B, wl, nd, warmup, steps, device, args, with_lse=False):
         a.record(); budgets = ctx.d2o_layer_budgets(); b.record()
         pend.append((1, a, b))
         streams = []
-        for l in range(L):
-            s = W.LayerStream(wl, l, device)
-            _, K, V = s.prompt()
+        group = 1 if NO_CHAIN else 4                      # layers whose K and V are on the device together
+        for l0 in range(0, L, group):
+            l1 = min(L, l0 + group)
+            Ks, Vs = [], []
+            for l in range(l0, l1):
+                s = W.LayerStream(wl, l, device)
+                _, K, V = s.prompt()
+                Ks.append(K); Vs.append(V)
+                streams.append(s)
             a, b = ev(), ev()
-            a.record(); ctx.d2o_prefill_compress(l, K, V); b.record()
+            a.record()
+            if group == 1:
+                ctx.d2o_prefill_compress(l0, Ks[0], Vs[0])
+            else:
+                ctx.d2o_prefill_compress_layers(l0, l1, Ks, Vs)
+            b.record()
             pend.append((2, a, b))
-            del K, V
-            streams.append(s)
+            del Ks, Vs, K, V
         dq, dk, dv = decode_inputs(streams, nd)
         dout = torch.empty_like(dq) if chain else torch.empty_like(dq[0])
         a, b = ev(), ev()

@@ -174,6 +174,19 @@ d2o_status d2o_budgets_from_density(const double* density, int32_t batch, int32_
 d2o_status d2o_prefill_compress(d2o_ctx* ctx, int32_t layer, const void* K, const void* V,
                                 void* stream);
 
+/* The same for layers [l0, l1) in one call (Eq. 5 needs every layer's density before any layer
+ * can be compressed, so at this point the caller holds all layers' K and V anyway).
+ * K, V: HOST arrays of l1-l0 DEVICE pointers, each [B, Hkv, P, d].  The layers are independent
+ * (Eq. 6-12 act per layer and head); the library works on up to four of them side by side, each
+ * on a stream of its own with its own part of `scratch`, so that the per-layer kernels of a small
+ * batch (B * Hkv CTAs each) fill the GPU together.  The internal streams start behind everything
+ * `stream` holds at the call, and `stream` continues behind all of them; the first call creates
+ * them (streams and events only, no device memory).  Results are those of l1-l0 calls of
+ * d2o_prefill_compress, bit for bit; the inspection arrays of d2o_get_view (evicted positions,
+ * Max(U), Argmax) then show one of the layers, not necessarily the last. */
+d2o_status d2o_prefill_compress_layers(d2o_ctx* ctx, int32_t l0, int32_t l1, const void* const* K,
+                                       const void* const* V, void* stream);
+
 /* (3) One generated token for layers [l0, l1).  DEVICE tensors:
  * q [l1-l0, B, Hq, d], k and v [l1-l0, B, Hkv, d], out [l1-l0, B, Hq, d].
  * Every call advances the token position of those layers by one; all layers must be

@@ -24,7 +24,7 @@ TORCH_DTYPE = {D2O_F32: torch.float32, D2O_F16: torch.float16, D2O_BF16: torch.b
 EXPORTS = [
     "d2o_status_string", "d2o_last_cuda_error", "d2o_workspace_size", "d2o_create", "d2o_destroy",
     "d2o_layer_stats", "d2o_layer_budgets", "d2o_budgets_from_density", "d2o_prefill_compress",
-    "d2o_decode_step", "d2o_decode_steps", "d2o_decode_step_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
+    "d2o_prefill_compress_layers", "d2o_decode_step", "d2o_decode_steps", "d2o_decode_step_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
     "d2o_set_tuning", "d2o_layer_stats_static", "d2o_set_fault_injection", "d2o_set_prompt_lens",
 ]
 STATIC_LSE_FLOATS = 1 << 20      # D2O_STATIC_LSE_FLOATS of include/d2o.h
@@ -92,6 +92,7 @@ def load_library() -> C.CDLL:
     lib.d2o_budgets_from_density.argtypes = [vp, i32, i32, i32, i32, i32, f32, i32, i32, f32, i32, i32, i32, i32, f32,
                                              vp, vp, vp, vp, vp]
     lib.d2o_prefill_compress.argtypes = [vp, i32, vp, vp, vp]
+    lib.d2o_prefill_compress_layers.argtypes = [vp, i32, i32, C.POINTER(vp), C.POINTER(vp), vp]
     lib.d2o_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.d2o_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.d2o_decode_steps.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
@@ -197,6 +198,15 @@ class D2OContext:
 
     def d2o_prefill_compress(self, layer: int, K: torch.Tensor, V: torch.Tensor):
         _check(self.lib.d2o_prefill_compress(self.handle, layer, _ptr(K), _ptr(V), _stream()), "d2o_prefill_compress")
+
+    def d2o_prefill_compress_layers(self, l0: int, l1: int, Ks, Vs):
+        """`Ks`, `Vs`: one device tensor per layer of [l0, l1)."""
+        n = l1 - l0
+        assert len(Ks) == n and len(Vs) == n
+        ka = (C.c_void_p * n)(*[_ptr(t) for t in Ks])
+        va = (C.c_void_p * n)(*[_ptr(t) for t in Vs])
+        _check(self.lib.d2o_prefill_compress_layers(self.handle, l0, l1, ka, va, _stream()),
+               "d2o_prefill_compress_layers")
 
     def d2o_decode_step(self, l0: int, l1: int, q, k, v, out):
         _check(self.lib.d2o_decode_step(self.handle, l0, l1, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream()),

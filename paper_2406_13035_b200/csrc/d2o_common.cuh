@@ -150,7 +150,9 @@ struct Layout {            // byte offsets into `state`
 };
 struct ScratchLayout {     // byte offsets into `scratch`
   size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, seg_tmp, part_key, pl_spill, stage_q, stage_k, stage_v, stage_out, end;
+  size_t lane_stride;      // evict_idx .. part_key are the working set of one layer's compression: kCompressLanes copies, this far apart
 };
+constexpr int kCompressLanes = 4;   // layers that d2o_prefill_compress_layers works on side by side
 
 }  // namespace d2o
 
@@ -191,6 +193,11 @@ struct d2o_ctx {
   int stats_path;              // tuning: 0 = tensor cores for the column sums of 16-bit Q/K, 1 = FFMA kernels
   int wait_limit_us;           // failure-detection tests: limit of a device-side wait in microseconds (0 = one second)
   int producer_stop_stage;     // failure-detection tests: the decode producer issues no copy from this stage on (-1 = never)
+  // d2o_prefill_compress_layers: one stream per lane, created with the first call (no device memory involved)
+  cudaStream_t lane_stream[d2o::kCompressLanes];
+  cudaEvent_t lane_done[d2o::kCompressLanes];
+  cudaEvent_t lane_fork;
+  bool lanes_ready;
 };
 
 namespace d2o {
@@ -202,7 +209,7 @@ cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, 
                            int max_budget, float gamma, int head_reduce, int budget_rule, int n_sink, int window,
                            float nm_ratio, int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
                            const int32_t* plen, cudaStream_t st);
-cudaError_t launch_prefill_compress(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st);
+cudaError_t launch_prefill_compress(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st, int lane = 0);
 cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const void* k, const void* v, void* out,
                           cudaStream_t st, d2o_status* why, bool chained = false, bool publish = false);
 cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int capacity, int len, void* kc, void* vc,
@@ -210,7 +217,7 @@ cudaError_t launch_full_decode(int dtype, int d, int n_slices, int group, int ca
                                d2o_status* why);
 
 // tensor-core similarity + nearest neighbour for 16-bit keys (d2o_sim_tc.cu); fills evict_mx / evict_nn
-cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int max_S, cudaStream_t st);
+cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int max_S, cudaStream_t st, int lane = 0);
 size_t sim_tc_part_key_bytes(const d2o_config* cfg, int max_budget);
 size_t sim_tc_max_items(const d2o_config* cfg, int max_budget);
 void sim_tc_build_items(const d2o_ctx* c, int n_sms, int4* items, int32_t* count);

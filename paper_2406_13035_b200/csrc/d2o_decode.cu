@@ -1376,19 +1376,22 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     return min(c->h_pair_max[(pr % B) * L + pr / B], t_now) + 1;
   };
 
-  // A step takes at least as long as its longest slice takes in one CTA.  Where that is more than the whole step
-  // would otherwise need (few sequences, a few layers with several times the mean budget), the longest slices go
-  // into a launch of their own with sixteen consumer warps per CTA, and the rest follows in a second launch that
-  // is allowed to start while the first is still running (the two share no slice).  Estimate with rough per-row
-  // costs of an eight-warp CTA; exactness does not matter, the split only has to catch the outliers.
+  // A step takes at least as long as its longest slice takes in one CTA, and in a chain of steps a slice's CTAs
+  // follow one another.  On the tensor path, where a few layers hold several times the mean budget and an
+  // eight-warp CTA streams about 15 GB/s, the longest slices go into a launch of their own with sixteen consumer
+  // warps per CTA, and the rest follows in a second launch that is allowed to start while the first is still running
+  // (the two share no slice).  Estimate with rough per-row costs of an eight-warp CTA; exactness does not matter,
+  // the split only has to catch the outliers.  On the FMA path an eight-warp CTA streams a 2048-row slice in well
+  // under a step and the split only costs (measured with and without on the 7B-shaped configs, single and chained
+  // steps): one launch.
   int n_long = 0;
-  if (ordered && c->decode_warps == 0 && c->decode_long_pairs == 0 && n_pairs > 1) {
-    const double fixed_us = 8.0, row_us = tensor_path(c->elem_size, G) ? 0.025 : 0.05;
+  if (ordered && c->decode_warps == 0 && c->decode_long_pairs == 0 && n_pairs > 1 && tensor_path(c->elem_size, G)) {
+    const double fixed_us = 8.0, row_us = 0.025;
     const double slots = (double)c->n_sms * ctas_per_sm(8, G, c->elem_size);
     double work = 0.0;
     for (int i = 0; i < n_pairs; ++i) work += Hkv * (fixed_us + row_us * rows_of_pair(i));
-    // measured optimum: four pairs on the 7B-shaped config (FMA path), twelve on the long-context one (tensor path)
-    const double limit = (tensor_path(c->elem_size, G) ? 0.55 : 0.65) * work / slots;
+    // measured optimum on the long-context config: twelve pairs
+    const double limit = 0.55 * work / slots;
     while (n_long < n_pairs && (n_long + 1) * Hkv <= 2 * c->n_sms && fixed_us + row_us * rows_of_pair(n_long) > limit) ++n_long;
     if (n_long == n_pairs) n_long = 0;
   } else if (ordered && c->decode_long_pairs > 0) {

@@ -126,6 +126,8 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   s->seg_items = take(B * Hkv * P * 4);
   s->seg_tmp = take(B * Hkv * P * 4);
   s->part_key = take(c->dtype == D2O_F32 ? 0 : sim_tc_part_key_bytes(c, max_budget));
+  s->lane_stride = o - s->evict_idx;                       // the arrays above, once more per further lane
+  o += (size_t)(kCompressLanes - 1) * s->lane_stride;
   s->pl_spill = take((rows + 8 * L * B * Hkv) * (Hq / Hkv) * 4);
   s->stage_q = take(L * B * Hq * d * e);
   s->stage_k = take(L * B * Hkv * d * e);
@@ -208,6 +210,10 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
 
 extern "C" void d2o_destroy(d2o_ctx* c) {
   if (!c) return;
+  if (c->lanes_ready) {
+    for (int i = 0; i < kCompressLanes; ++i) { cudaStreamDestroy(c->lane_stream[i]); cudaEventDestroy(c->lane_done[i]); }
+    cudaEventDestroy(c->lane_fork);
+  }
   free(c->h_budgets); free(c->h_windows); free(c->h_row_off); free(c->h_pair_max); free(c->h_pair_sum);
   free(c->layer_fed); free(c->layer_compressed); free(c->layer_steps); free(c->h_order); free(c->h_plen); free(c->h_sim_count); free(c->h_sim_items);
   free(c);
@@ -308,6 +314,42 @@ extern "C" d2o_status d2o_prefill_compress(d2o_ctx* c, int32_t layer, const void
   CUDA_TRY(launch_prefill_compress(c, layer, K, V, (cudaStream_t)stream));
   c->layer_compressed[layer] = 1;
   c->layer_steps[layer] = 0;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_prefill_compress_layers(d2o_ctx* c, int32_t l0, int32_t l1, const void* const* K,
+                                                  const void* const* V, void* stream) {
+  if (!c || !K || !V || l0 < 0 || l1 > c->cfg.n_layers || l0 >= l1) return D2O_ERR_INVALID_ARG;
+  for (int l = l0; l < l1; ++l)
+    if (!aligned16(K[l - l0]) || !aligned16(V[l - l0])) return D2O_ERR_INVALID_ARG;
+  if (!c->have_budgets) return D2O_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (l1 - l0 == 1) {
+    CUDA_TRY(launch_prefill_compress(c, l0, K[0], V[0], st));
+  } else {
+    if (!c->lanes_ready) {
+      // streams and events only: no device memory
+      for (int i = 0; i < kCompressLanes; ++i) {
+        CUDA_TRY(cudaStreamCreateWithFlags(&c->lane_stream[i], cudaStreamNonBlocking));
+        CUDA_TRY(cudaEventCreateWithFlags(&c->lane_done[i], cudaEventDisableTiming));
+      }
+      CUDA_TRY(cudaEventCreateWithFlags(&c->lane_fork, cudaEventDisableTiming));
+      c->lanes_ready = true;
+    }
+    // the lanes start behind everything the caller's stream holds, the caller's stream goes on behind every lane
+    const int lanes = min(kCompressLanes, l1 - l0);
+    CUDA_TRY(cudaEventRecord(c->lane_fork, st));
+    for (int i = 0; i < lanes; ++i) CUDA_TRY(cudaStreamWaitEvent(c->lane_stream[i], c->lane_fork, 0));
+    for (int l = l0; l < l1; ++l) {
+      const int lane = (l - l0) % lanes;                     // a lane's layers follow one another on its stream
+      CUDA_TRY(launch_prefill_compress(c, l, K[l - l0], V[l - l0], c->lane_stream[lane], lane));
+    }
+    for (int i = 0; i < lanes; ++i) {
+      CUDA_TRY(cudaEventRecord(c->lane_done[i], c->lane_stream[i]));
+      CUDA_TRY(cudaStreamWaitEvent(st, c->lane_done[i], 0));
+    }
+  }
+  for (int l = l0; l < l1; ++l) { c->layer_compressed[l] = 1; c->layer_steps[l] = 0; }
   return D2O_OK;
 }
 

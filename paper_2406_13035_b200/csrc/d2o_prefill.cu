@@ -559,11 +559,11 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
 
 // ------------------------------------------------------------------------------------ launcher
 template <typename T, int D>
-static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st) {
+static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st, int lane) {
   const d2o_config& g = c->cfg;
   const int B = g.batch, Hkv = g.n_kv_heads, P = g.prompt_len, L = g.n_layers;
   const int n_slices = B * Hkv;
-  char* S = c->state; char* X = c->scratch;
+  char* S = c->state; char* X = c->scratch + (size_t)lane * c->slay.lane_stride;   // only the lane's arrays are used below
   T* kpool = (T*)(S + c->lay.kpool);
   T* vpool = (T*)(S + c->lay.vpool);
   int maxS = 0;
@@ -615,7 +615,7 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   const void* feat = g.sim_feature ? V : K;
   const T* feat_pool = g.sim_feature ? vpool : kpool;
   if (sizeof(T) == 2 && c->similarity_path == 0) {
-    e = launch_similarity_tc(c, layer, feat, maxS, st);
+    e = launch_similarity_tc(c, layer, feat, maxS, st, lane);
     if (e != cudaSuccess) return e;
   } else {
     dim3 sgrid((maxLe + kSimTile - 1) / kSimTile, n_slices);
@@ -650,13 +650,13 @@ static cudaError_t run_prefill(const d2o_ctx* c, int layer, const void* K, const
   return cudaGetLastError();
 }
 
-cudaError_t launch_prefill_compress(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st) {
+cudaError_t launch_prefill_compress(const d2o_ctx* c, int layer, const void* K, const void* V, cudaStream_t st, int lane) {
   const int d = c->cfg.d_head;
   switch (c->cfg.dtype) {
-    case D2O_F32: return d == 64 ? run_prefill<float, 64>(c, layer, K, V, st) : run_prefill<float, 128>(c, layer, K, V, st);
-    case D2O_F16: return d == 64 ? run_prefill<__half, 64>(c, layer, K, V, st) : run_prefill<__half, 128>(c, layer, K, V, st);
-    default: return d == 64 ? run_prefill<__nv_bfloat16, 64>(c, layer, K, V, st)
-                            : run_prefill<__nv_bfloat16, 128>(c, layer, K, V, st);
+    case D2O_F32: return d == 64 ? run_prefill<float, 64>(c, layer, K, V, st, lane) : run_prefill<float, 128>(c, layer, K, V, st, lane);
+    case D2O_F16: return d == 64 ? run_prefill<__half, 64>(c, layer, K, V, st, lane) : run_prefill<__half, 128>(c, layer, K, V, st, lane);
+    default: return d == 64 ? run_prefill<__nv_bfloat16, 64>(c, layer, K, V, st, lane)
+                            : run_prefill<__nv_bfloat16, 128>(c, layer, K, V, st, lane);
   }
 }
 

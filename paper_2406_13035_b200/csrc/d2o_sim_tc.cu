@@ -472,11 +472,11 @@ size_t sim_tc_part_key_bytes(const d2o_config* cfg, int max_budget) {
 }
 
 // Returns cudaErrorNotSupported if the tensor maps cannot be built.
-cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int max_S, cudaStream_t st) {
+cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int max_S, cudaStream_t st, int lane) {
   const d2o_config& g = c->cfg;
   const int B = g.batch, Hkv = g.n_kv_heads, P = g.prompt_len, D = g.d_head;
   const int n_slices = B * Hkv;
-  char* S = c->state; char* X = c->scratch;
+  char* S = c->state; char* X = c->scratch + (size_t)lane * c->slay.lane_stride;   // only the lane's arrays are used below
   CUtensorMap map_k, map_pool;
   if (!encode_rows_2d(&map_k, g.dtype, K, (uint64_t)n_slices * P, D, kTileM)) return cudaErrorNotSupported;
   // the retained rows of the same kind: K_c, or V_c when the similarity is taken on the values

@@ -137,7 +137,7 @@ def test_chained_steps_argument_checks():
 
 @pytest.mark.slow
 def test_chained_steps_full_size_config_1():
-    """All 32 layers of the 7B-shaped config (1024 slices, two launch classes per step), 48 tokens in one call."""
+    """All 32 layers of the 7B-shaped config (1024 slices), 48 tokens in one call."""
     wl = dataclasses.replace(W.CONFIGS["cfg1"], decode_steps=48)
     r = np.random.default_rng(5)
     picks = sorted({(int(r.integers(wl.n_layers)), 0, int(r.integers(wl.n_kv_heads))) for _ in range(48)})
