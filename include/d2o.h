@@ -217,6 +217,18 @@ d2o_status d2o_decode_step_host(d2o_ctx* ctx, int32_t l0, int32_t l1, const void
                                 const void* k_host, const void* v_host, void* out_host,
                                 void* stream);
 
+/* n_steps consecutive tokens with HOST buffers (pinned memory, or the copies do not overlap
+ * anything): q_host [n_steps, l1-l0, B, Hq, d], k_host and v_host [n_steps, l1-l0, B, Hkv, d],
+ * out_host [n_steps, l1-l0, B, Hq, d].  Per step the same work as d2o_decode_step_host, but
+ * pipelined over three streams (the caller's for the kernels, two of the library's own for the
+ * copies, created with the first call; no device memory): while step t computes, the inputs of
+ * step t+1 travel to the device and the output of step t-1 travels back, through two staging
+ * sets in `scratch`.  As with d2o_decode_steps a step's inputs cannot depend on an earlier
+ * step's output.  Returns after everything, the last copy back included, has completed. */
+d2o_status d2o_decode_steps_host(d2o_ctx* ctx, int32_t l0, int32_t l1, int32_t n_steps,
+                                 const void* q_host, const void* k_host, const void* v_host,
+                                 void* out_host, void* stream);
+
 /* Uncompressed decode attention (Eq. 2-3), the comparison kernel: appends k, v at row `len`
  * of k_cache/v_cache DEVICE [n_slices, capacity, d] (n_slices = B*Hkv) and attends over
  * len+1 rows.  q, out DEVICE [n_slices, group, d]; k, v DEVICE [n_slices, d].

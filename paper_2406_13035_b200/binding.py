@@ -24,7 +24,7 @@ TORCH_DTYPE = {D2O_F32: torch.float32, D2O_F16: torch.float16, D2O_BF16: torch.b
 EXPORTS = [
     "d2o_status_string", "d2o_last_cuda_error", "d2o_workspace_size", "d2o_create", "d2o_destroy",
     "d2o_layer_stats", "d2o_layer_budgets", "d2o_budgets_from_density", "d2o_prefill_compress",
-    "d2o_prefill_compress_layers", "d2o_decode_step", "d2o_decode_steps", "d2o_decode_step_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
+    "d2o_prefill_compress_layers", "d2o_decode_step", "d2o_decode_steps", "d2o_decode_step_host", "d2o_decode_steps_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
     "d2o_set_tuning", "d2o_layer_stats_static", "d2o_set_fault_injection", "d2o_set_prompt_lens",
 ]
 STATIC_LSE_FLOATS = 1 << 20      # D2O_STATIC_LSE_FLOATS of include/d2o.h
@@ -96,6 +96,7 @@ def load_library() -> C.CDLL:
     lib.d2o_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.d2o_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.d2o_decode_steps.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.d2o_decode_steps_host.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.d2o_full_decode_step.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.d2o_get_view.argtypes = [vp, i32, C.POINTER(D2OView)]
     lib.d2o_get_stats.argtypes = [vp, C.POINTER(D2OStats), vp]
@@ -221,6 +222,12 @@ class D2OContext:
             assert t.device.type == "cpu"
         _check(self.lib.d2o_decode_step_host(self.handle, l0, l1, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream()),
                "d2o_decode_step_host")
+
+    def d2o_decode_steps_host(self, l0: int, l1: int, n_steps: int, q, k, v, out):
+        for t in (q, k, v, out):
+            assert t.device.type == "cpu"
+        _check(self.lib.d2o_decode_steps_host(self.handle, l0, l1, n_steps, _ptr(q), _ptr(k), _ptr(v), _ptr(out),
+                                              _stream()), "d2o_decode_steps_host")
 
     def d2o_set_tuning(self, decode_stages: int = 0, decode_l2_hints: int = 1, similarity_path: int = 0,
                        stats_path: int = 0, decode_warps: int = 0, decode_smem_rows: int = 0,

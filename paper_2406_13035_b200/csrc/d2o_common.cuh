@@ -150,6 +150,7 @@ struct Layout {            // byte offsets into `state`
 };
 struct ScratchLayout {     // byte offsets into `scratch`
   size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, seg_tmp, part_key, pl_spill, stage_q, stage_k, stage_v, stage_out, end;
+  size_t stage_stride;     // stage_q .. stage_out exist twice, this far apart (d2o_decode_steps_host alternates)
   size_t lane_stride;      // evict_idx .. part_key are the working set of one layer's compression: kCompressLanes copies, this far apart
 };
 constexpr int kCompressLanes = 4;   // layers that d2o_prefill_compress_layers works on side by side
@@ -198,6 +199,10 @@ struct d2o_ctx {
   cudaEvent_t lane_done[d2o::kCompressLanes];
   cudaEvent_t lane_fork;
   bool lanes_ready;
+  // d2o_decode_steps_host: a stream for the copies to the device, one for the copies back; created with the first call
+  cudaStream_t io_in, io_out;
+  cudaEvent_t io_start, io_in_done[2], io_step_done[2], io_out_done[2];
+  bool io_ready;
 };
 
 namespace d2o {

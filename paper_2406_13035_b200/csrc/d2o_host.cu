@@ -133,6 +133,8 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   s->stage_k = take(L * B * Hkv * d * e);
   s->stage_v = take(L * B * Hkv * d * e);
   s->stage_out = take(L * B * Hq * d * e);
+  s->stage_stride = o - s->stage_q;                        // a second set of the four for the pipelined host path
+  o += s->stage_stride;
   s->end = o;
 }
 
@@ -210,6 +212,12 @@ extern "C" d2o_status d2o_create(const d2o_config* cfg, void* state, size_t stat
 
 extern "C" void d2o_destroy(d2o_ctx* c) {
   if (!c) return;
+  if (c->io_ready) {
+    cudaStreamDestroy(c->io_in); cudaStreamDestroy(c->io_out); cudaEventDestroy(c->io_start);
+    for (int i = 0; i < 2; ++i) {
+      cudaEventDestroy(c->io_in_done[i]); cudaEventDestroy(c->io_step_done[i]); cudaEventDestroy(c->io_out_done[i]);
+    }
+  }
   if (c->lanes_ready) {
     for (int i = 0; i < kCompressLanes; ++i) { cudaStreamDestroy(c->lane_stream[i]); cudaEventDestroy(c->lane_done[i]); }
     cudaEventDestroy(c->lane_fork);
@@ -434,6 +442,65 @@ extern "C" d2o_status d2o_decode_step_host(d2o_ctx* c, int32_t l0, int32_t l1, c
   CUDA_TRY(cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, s));
   CUDA_TRY(cudaStreamSynchronize(s));
   for (int l = l0; l < l1; ++l) c->layer_steps[l] += 1;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_decode_steps_host(d2o_ctx* c, int32_t l0, int32_t l1, int32_t n_steps, const void* q_host,
+                                            const void* k_host, const void* v_host, void* out_host, void* stream) {
+  d2o_status st = check_decode_range(c, l0, l1);
+  if (st != D2O_OK) return st;
+  if (n_steps < 1 || !q_host || !k_host || !v_host || !out_host) return D2O_ERR_INVALID_ARG;
+  if (c->layer_steps[l0] + n_steps > c->cfg.max_new_tokens) return D2O_ERR_STATE;
+  const d2o_config& g = c->cfg;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (!c->io_ready) {
+    // streams and events only: no device memory
+    CUDA_TRY(cudaStreamCreateWithFlags(&c->io_in, cudaStreamNonBlocking));
+    CUDA_TRY(cudaStreamCreateWithFlags(&c->io_out, cudaStreamNonBlocking));
+    CUDA_TRY(cudaEventCreateWithFlags(&c->io_start, cudaEventDisableTiming));
+    for (int i = 0; i < 2; ++i) {
+      CUDA_TRY(cudaEventCreateWithFlags(&c->io_in_done[i], cudaEventDisableTiming));
+      CUDA_TRY(cudaEventCreateWithFlags(&c->io_step_done[i], cudaEventDisableTiming));
+      CUDA_TRY(cudaEventCreateWithFlags(&c->io_out_done[i], cudaEventDisableTiming));
+    }
+    c->io_ready = true;
+  }
+  const size_t nl = (size_t)(l1 - l0);
+  const size_t qb = nl * g.batch * g.n_q_heads * g.d_head * c->elem_size;
+  const size_t kb = nl * g.batch * g.n_kv_heads * g.d_head * c->elem_size;
+  // Step t uses staging set t % 2.  Three streams: the copies of step t + 1 to the device and of step t - 1 back run
+  // beside the kernels of step t.  A set is refilled once the step that read it is done (io_step_done), and its
+  // output is overwritten once the copy back of the step before last is done (io_out_done).
+  CUDA_TRY(cudaEventRecord(c->io_start, s));
+  CUDA_TRY(cudaStreamWaitEvent(c->io_in, c->io_start, 0));
+  CUDA_TRY(cudaStreamWaitEvent(c->io_out, c->io_start, 0));
+  for (int t = 0; t < n_steps; ++t) {
+    const int set = t & 1;
+    char* base = c->scratch + (size_t)set * c->slay.stage_stride;
+    char* dq = base + c->slay.stage_q; char* dk = base + c->slay.stage_k;
+    char* dv = base + c->slay.stage_v; char* dout = base + c->slay.stage_out;
+    if (t >= 2) CUDA_TRY(cudaStreamWaitEvent(c->io_in, c->io_step_done[set], 0));
+    CUDA_TRY(cudaMemcpyAsync(dq, (const char*)q_host + t * qb, qb, cudaMemcpyHostToDevice, c->io_in));
+    CUDA_TRY(cudaMemcpyAsync(dk, (const char*)k_host + t * kb, kb, cudaMemcpyHostToDevice, c->io_in));
+    CUDA_TRY(cudaMemcpyAsync(dv, (const char*)v_host + t * kb, kb, cudaMemcpyHostToDevice, c->io_in));
+    CUDA_TRY(cudaEventRecord(c->io_in_done[set], c->io_in));
+    CUDA_TRY(cudaStreamWaitEvent(s, c->io_in_done[set], 0));
+    if (t >= 2) CUDA_TRY(cudaStreamWaitEvent(s, c->io_out_done[set], 0));
+    d2o_status why = D2O_OK;
+    cudaError_t e = launch_decode(c, l0, l1, dq, dk, dv, dout, s, &why);
+    if (why != D2O_OK || e != cudaSuccess) {
+      (void)cudaStreamSynchronize(c->io_in); (void)cudaStreamSynchronize(c->io_out); (void)cudaStreamSynchronize(s);
+      return why != D2O_OK ? why : cuda_fail(e, "launch_decode");
+    }
+    for (int l = l0; l < l1; ++l) c->layer_steps[l] += 1;
+    CUDA_TRY(cudaEventRecord(c->io_step_done[set], s));
+    CUDA_TRY(cudaStreamWaitEvent(c->io_out, c->io_step_done[set], 0));
+    CUDA_TRY(cudaMemcpyAsync((char*)out_host + t * qb, dout, qb, cudaMemcpyDeviceToHost, c->io_out));
+    CUDA_TRY(cudaEventRecord(c->io_out_done[set], c->io_out));
+  }
+  // the caller's stream ends behind the last copies back; then wait for all of it
+  for (int i = 0; i < (n_steps > 1 ? 2 : 1); ++i) CUDA_TRY(cudaStreamWaitEvent(s, c->io_out_done[(n_steps - 1 - i) & 1], 0));
+  CUDA_TRY(cudaStreamSynchronize(s));
   return D2O_OK;
 }
 

@@ -144,6 +144,27 @@ def test_chained_steps_full_size_config_1():
     _run_pair(wl, [48], slices=picks)
 
 
+@pytest.mark.parametrize("name,steps", [("cfg0", 16), ("cfg2", 9), ("cfg1", 1)])
+def test_pipelined_host_steps_equal_device_steps(name, steps):
+    """d2o_decode_steps_host (copies of neighbouring steps beside the kernels, two staging sets): same outputs and
+    state as stepping with device tensors."""
+    wl = W.CONFIGS["cfg0"] if name == "cfg0" else dataclasses.replace(W.twin(name), decode_steps=steps)
+    wl = dataclasses.replace(wl, decode_steps=steps)
+    (a, b), _, dq, dk, dv = _prepare(wl, 2)
+    L = wl.n_layers
+    out_a = torch.empty_like(dq)
+    for s in range(steps):
+        a.d2o_decode_step(0, L, dq[s], dk[s], dv[s], out_a[s])
+    hq, hk, hv = dq.cpu().pin_memory(), dk.cpu().pin_memory(), dv.cpu().pin_memory()
+    ho = torch.full_like(hq, float("nan")).pin_memory()
+    b.d2o_decode_steps_host(0, L, steps, hq, hk, hv, ho)       # returns when the last copy back has completed
+    assert torch.equal(out_a.cpu().view(torch.uint8), ho.view(torch.uint8))
+    for c in (a, b):
+        assert c.d2o_get_stats().error_word == 0
+    _same_state(a, b, _all_slices(wl))
+    a.close(); b.close()
+
+
 def test_chained_outputs_against_the_oracle():
     """Config 0, every slice: the oracle steps beside the outputs of one multi-step call."""
     wl = W.CONFIGS["cfg0"]
