@@ -50,6 +50,12 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// maximum of three; a NaN operand is ignored
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 }  // namespace tc
 
 template <int D, int FMT, int SWEEP>
@@ -189,7 +195,8 @@ attn_tc_kernel(ColsumTcArgs a, const __grid_constant__ CUtensorMap map_q, const 
       if (SWEEP == kSweepRows) {
         // B rows are keys: valid iff key <= query (keys >= P are > every stored query)
         const bool need_mask = brow0 + 63 > a0 + at * kCsTile + quarter * 32;     // warp-uniform
-        float bm = -INFINITY;
+        // four independent chains of three-input maxima: the block maximum is on every thread's critical path
+        float bmx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           float x = __uint_as_float(ra[i]), y = __uint_as_float(rb[i]);
@@ -198,8 +205,9 @@ attn_tc_kernel(ColsumTcArgs a, const __grid_constant__ CUtensorMap map_q, const 
             if (brow0 + 32 + i > arow) y = -INFINITY;
             ra[i] = __float_as_uint(x); rb[i] = __float_as_uint(y);
           }
-          bm = fmaxf(bm, fmaxf(x, y));
+          bmx[i & 3] = tc::max3(bmx[i & 3], x, y);
         }
+        const float bm = fmaxf(fmaxf(bmx[0], bmx[1]), fmaxf(bmx[2], bmx[3]));
         if (bm > m_run) { l_run *= exp2f((m_run - bm) * c); m_run = bm; }      // exp2f(-inf) = 0 on the first block
         if (m_run > -INFINITY) {
           const float mc = m_run * c;
