@@ -473,6 +473,8 @@ struct MergeArgs {
   int value_feature;       // 1: the cached inverse norms belong to the value rows
 };
 
+constexpr int kMergeFlight = 4;     // merged tokens whose rows a row group has in flight
+
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
 merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* __restrict__ kpool,
@@ -507,8 +509,9 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
   for (int i = 0; i < EPV; ++i) va[i] = own * f[i];
   float den = own;
   // The lanes of the row first fetch the list entries of up to LPR merged tokens side by side (entry -> similarity and
-  // prompt position), then the rows are added in list order, two tokens' key and value rows in flight at a time: the
-  // chain entry -> position -> row is three dependent loads per token otherwise.
+  // prompt position), then the rows are added in list order, four tokens' key and value rows in flight at a time: the
+  // chain entry -> position -> row is three dependent loads per token otherwise, and a retained token that is the
+  // neighbour of hundreds of evicted ones is the launch's critical path.
   const unsigned gm = group_mask<LPR>();
   for (int s = s0; s < s1; s += LPR) {
     const int cnt = min(LPR, s1 - s);
@@ -520,26 +523,27 @@ merge_kernel(MergeArgs a, const T* __restrict__ K, const T* __restrict__ V, T* _
         if (D2O_GUARD(pj >= 0 && pj < a.plen[b], a.status, 0xC4EC0006u)) { my_pj = pj; my_w = a.average ? 1.0f : expf(mx[i]); }
       }
     }
-    for (int t = 0; t < cnt; t += 2) {
-      const float w0 = __shfl_sync(gm, my_w, t, LPR), w1 = t + 1 < cnt ? __shfl_sync(gm, my_w, t + 1, LPR) : 0.f;
-      const int p0 = __shfl_sync(gm, my_pj, t, LPR), p1 = t + 1 < cnt ? __shfl_sync(gm, my_pj, t + 1, LPR) : p0;
-      const uint4 k0 = ld_global_v4(Ks + (size_t)p0 * D + lig * EPV), v0 = ld_global_v4(Vs + (size_t)p0 * D + lig * EPV);
-      const uint4 k1 = ld_global_v4(Ks + (size_t)p1 * D + lig * EPV), v1 = ld_global_v4(Vs + (size_t)p1 * D + lig * EPV);
-      den += w0;
-      Elem<T>::unpack(k0, f);
+    for (int t = 0; t < cnt; t += kMergeFlight) {
+      float w[kMergeFlight]; uint4 kr[kMergeFlight], vr[kMergeFlight];
 #pragma unroll
-      for (int e = 0; e < EPV; ++e) ka[e] = fmaf(w0, f[e], ka[e]);
-      Elem<T>::unpack(v0, f);
+      for (int u = 0; u < kMergeFlight; ++u) {
+        const int tu = t + u < cnt ? t + u : t;              // past the list: the first row once more, never added
+        w[u] = __shfl_sync(gm, my_w, tu, LPR);
+        const int pu = __shfl_sync(gm, my_pj, tu, LPR);
+        kr[u] = ld_global_v4(Ks + (size_t)pu * D + lig * EPV);
+        vr[u] = ld_global_v4(Vs + (size_t)pu * D + lig * EPV);
+      }
 #pragma unroll
-      for (int e = 0; e < EPV; ++e) va[e] = fmaf(w0, f[e], va[e]);
-      if (t + 1 < cnt) {                                   // a token whose check failed has weight 0: its terms are +0
-        den += w1;
-        Elem<T>::unpack(k1, f);
+      for (int u = 0; u < kMergeFlight; ++u) {
+        if (t + u < cnt) {                                   // list order; a token whose check failed has weight 0: its terms are +0
+          den += w[u];
+          Elem<T>::unpack(kr[u], f);
 #pragma unroll
-        for (int e = 0; e < EPV; ++e) ka[e] = fmaf(w1, f[e], ka[e]);
-        Elem<T>::unpack(v1, f);
+          for (int e = 0; e < EPV; ++e) ka[e] = fmaf(w[u], f[e], ka[e]);
+          Elem<T>::unpack(vr[u], f);
 #pragma unroll
-        for (int e = 0; e < EPV; ++e) va[e] = fmaf(w1, f[e], va[e]);
+          for (int e = 0; e < EPV; ++e) va[e] = fmaf(w[u], f[e], va[e]);
+        }
       }
     }
   }

@@ -320,58 +320,89 @@ struct NnReduceArgs {
   int L, layer, Hkv, P, n_chunks_max;
 };
 
+constexpr int kNnRows = 4;                  // evicted rows per row group and pass: their loads are issued together
+
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
 neighbour_reduce_kernel(NnReduceArgs a, const T* __restrict__ K, const T* __restrict__ kpool) {
   constexpr int EPV = Elem<T>::kPerVec;
   constexpr int LPR = D / EPV;
+  constexpr int NGRP = 256 / LPR;
   const int slice = blockIdx.y;
   const int b = slice / a.Hkv, h = slice % a.Hkv;
   const int S = a.budgets[slice_entry(b, a.layer, h, a.L, a.Hkv)];
-  const int Le = a.plen[b] - S;
+  const int Pb = a.plen[b];
+  const int Le = Pb - S;
   const int grp = threadIdx.x / LPR, lig = threadIdx.x % LPR;
-  const int i = blockIdx.x * (blockDim.x / LPR) + grp;
-  if (i >= Le) return;
+  const int i0 = blockIdx.x * (NGRP * kNnRows) + grp;       // this group's rows: i0 + r * NGRP
+  if (i0 >= Le) return;
   const unsigned gmask = group_mask<LPR>();
-  const int pos = a.evict_idx[(size_t)slice * a.P + i];
-  if (!D2O_GUARD(pos >= 0 && pos < a.plen[b], a.status, 0xC4EC0008u)) return;      // uniform for the row's lanes
-  float f[EPV];
-  Elem<T>::unpack(ld_global_v4(K + ((size_t)slice * a.P + pos) * D + lig * EPV), f);
-  float ss = 0.f;
-#pragma unroll
-  for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
-  ss = group_sum<LPR>(ss, gmask);
-  const float rn = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
   const int n_chunks = (S + kChunkN - 1) / kChunkN;
-  unsigned long long key = 0ull;
-  for (int c = 0; c < n_chunks; ++c) {
-    const unsigned long long k2 = a.part_key[((size_t)slice * a.n_chunks_max + c) * a.P + pos];
-    key = k2 > key ? k2 : key;
-  }
-  int slot = 0x7fffffff - (int)(uint32_t)(key & 0xffffffffu);
-  float mx = ord_float((uint32_t)(key >> 32)) * rn;
-  bool found = key != 0ull && (unsigned)slot < (unsigned)S;
-  if (!found) {
-    // No chunk reported a maximum (no finite similarity in the row: non-finite keys).  The row is redone here in
-    // fp32, all retained rows in slot order (the first maximum stays); without any finite similarity it gets maximum
-    // -inf and neighbour 0 and is never merged.
-    const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
-    float best = -INFINITY; int bj = 0;
-    for (int j = 0; j < S; ++j) {
-      float g[EPV];
-      Elem<T>::unpack(ld_global_v4(kpool + (row0 + j) * D + lig * EPV), g);
-      float dot = 0.f;
+  // The three dependent loads of a row (its position, its key, its partial maxima) are issued for four rows at a
+  // time; the partial maxima of a row are spread over the lanes of its group (chunk c is lane c mod LPR's).
+  int pos[kNnRows];
 #pragma unroll
-      for (int e = 0; e < EPV; ++e) dot = fmaf(f[e], g[e], dot);
-      dot = group_sum<LPR>(dot, gmask);
-      const float u = __fadd_rn(dot * rn * a.rnorm[row0 + j], 0.f);
-      if (u > best) { best = u; bj = j; }
-    }
-    mx = best; slot = bj;
+  for (int r = 0; r < kNnRows; ++r) {
+    const int i = i0 + r * NGRP;
+    pos[r] = i < Le ? a.evict_idx[(size_t)slice * a.P + i] : -1;
+    if (pos[r] >= 0 && !D2O_GUARD(pos[r] < Pb, a.status, 0xC4EC0008u)) pos[r] = -1;    // uniform for the row's lanes
   }
-  if (lig == 0) {
-    a.evict_mx[(size_t)slice * a.P + i] = mx;
-    a.evict_nn[(size_t)slice * a.P + i] = slot;
+  uint4 raw[kNnRows];
+  unsigned long long key[kNnRows];
+#pragma unroll
+  for (int r = 0; r < kNnRows; ++r) {
+    raw[r] = make_uint4(0, 0, 0, 0);
+    key[r] = 0ull;
+    if (pos[r] >= 0) {
+      raw[r] = ld_global_v4(K + ((size_t)slice * a.P + pos[r]) * D + lig * EPV);
+      for (int c = lig; c < n_chunks; c += LPR) {
+        const unsigned long long k2 = a.part_key[((size_t)slice * a.n_chunks_max + c) * a.P + pos[r]];
+        key[r] = k2 > key[r] ? k2 : key[r];
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kNnRows; ++r) {
+    if (pos[r] < 0) continue;                                // uniform for the row's lanes
+    float f[EPV];
+    Elem<T>::unpack(raw[r], f);
+    float ss = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) ss = fmaf(f[e], f[e], ss);
+    ss = group_sum<LPR>(ss, gmask);
+    const float rn = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+    unsigned long long kk = key[r];
+#pragma unroll
+    for (int o = LPR / 2; o >= 1; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(gmask, kk, o);
+      kk = other > kk ? other : kk;
+    }
+    int slot = 0x7fffffff - (int)(uint32_t)(kk & 0xffffffffu);
+    float mx = ord_float((uint32_t)(kk >> 32)) * rn;
+    const bool found = kk != 0ull && (unsigned)slot < (unsigned)S;
+    if (!found) {
+      // No chunk reported a maximum (no finite similarity in the row: non-finite keys).  The row is redone here in
+      // fp32, all retained rows in slot order (the first maximum stays); without any finite similarity it gets maximum
+      // -inf and neighbour 0 and is never merged.
+      const int64_t row0 = a.row_off[slice_entry(b, a.layer, h, a.L, a.Hkv)];
+      float best = -INFINITY; int bj = 0;
+      for (int j = 0; j < S; ++j) {
+        float g[EPV];
+        Elem<T>::unpack(ld_global_v4(kpool + (row0 + j) * D + lig * EPV), g);
+        float dot = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) dot = fmaf(f[e], g[e], dot);
+        dot = group_sum<LPR>(dot, gmask);
+        const float u = __fadd_rn(dot * rn * a.rnorm[row0 + j], 0.f);
+        if (u > best) { best = u; bj = j; }
+      }
+      mx = best; slot = bj;
+    }
+    if (lig == 0) {
+      const int i = i0 + r * NGRP;
+      a.evict_mx[(size_t)slice * a.P + i] = mx;
+      a.evict_nn[(size_t)slice * a.P + i] = slot;
+    }
   }
 }
 
@@ -522,7 +553,8 @@ cudaError_t launch_similarity_tc(const d2o_ctx* c, int layer, const void* K, int
     for (int hh = 0; hh < Hkv; ++hh) maxLe = max(maxLe, c->h_plen[bb] - c->h_budgets[(bb * g.n_layers + layer) * Hkv + hh]);
   if (maxLe <= 0) return cudaSuccess;
   const int lpr = D * 2 / 16;
-  dim3 rgrid((maxLe + 256 / lpr - 1) / (256 / lpr), n_slices);
+  const int rows_per_cta = (256 / lpr) * kNnRows;
+  dim3 rgrid((maxLe + rows_per_cta - 1) / rows_per_cta, n_slices);
   if (g.dtype == D2O_F16) {
     if (D == 128) neighbour_reduce_kernel<__half, 128><<<rgrid, 256, 0, st>>>(r, (const __half*)K, (const __half*)pool);
     else neighbour_reduce_kernel<__half, 64><<<rgrid, 256, 0, st>>>(r, (const __half*)K, (const __half*)pool);
