@@ -3,12 +3,15 @@
 
 One bench *step* is one pass of the whole path over one synthetic batch:
   per layer: column sums + density (d2o_layer_stats) -> budgets (d2o_layer_budgets)
-  -> per layer: eviction + similarity + merge (d2o_prefill_compress)
-  -> the decode loop (d2o_decode_step, all layers per call, `decode_steps` tokens).
+  -> all layers: eviction + similarity + merge (d2o_prefill_compress_layers)
+  -> the decode loop (`decode_steps` tokens, all layers per step, through d2o_decode_steps: the inputs
+     of every step are resident, which is what that entry point asks for).
 The headline value is compressed decode steps/s (tokens/s = steps/s x sequences); the
-prompt-stage times are reported beside it.  Inputs are generated once, seeded, and are
-resident in HBM before the timed region; the `e2e` leg repeats the decode loop through the
-host-buffer entry point with pinned host q/k/v/out every step.
+prompt-stage times are reported beside it, and so is the decode loop with one d2o_decode_step call
+per token.  Inputs are generated once, seeded, and are resident in HBM before the timed region; the
+`e2e` leg repeats the decode loop through the host-buffer entry points with pinned host q/k/v/out,
+every step's bytes crossing inside the timed region.  `--single-step-calls` runs every leg through the
+one-call-per-layer / one-call-per-token entry points instead.
 
 The default workload is the Llama-3-8B-shaped config (16 sequences, prompt 8192, 1.7 GB of cache
 streamed per decode step).  `per_config` holds a shorter measurement of the other configs (fewer

@@ -120,6 +120,26 @@ def test_chained_steps_with_two_launch_classes():
     _run_pair(wl, [12], long_pairs=2)
 
 
+def test_chained_steps_on_layer_ranges():
+    """Layer ranges are stepped independently of one another: every range in one multi-step call of its own."""
+    wl = dataclasses.replace(W.twin("cfg1"), decode_steps=10)
+    (a, b), _, dq, dk, dv = _prepare(wl, 2)
+    n = wl.decode_steps
+    out_a, out_b = torch.empty_like(dq), torch.full_like(dq, float("nan"))
+    for s in range(n):
+        a.d2o_decode_step(0, wl.n_layers, dq[s], dk[s], dv[s], out_a[s])
+    for l0, l1 in ((0, 1), (1, 4)):
+        q, k, v = (t[:, l0:l1].contiguous() for t in (dq, dk, dv))
+        o = torch.empty_like(q)
+        b.d2o_decode_steps(l0, l1, n, q, k, v, o)
+        out_b[:, l0:l1] = o
+    torch.cuda.synchronize()
+    assert b.d2o_get_stats().error_word == 0
+    assert torch.equal(out_a.view(torch.uint8), out_b.view(torch.uint8))
+    _same_state(a, b, _all_slices(wl))
+    a.close(); b.close()
+
+
 def test_chained_steps_argument_checks():
     wl = dataclasses.replace(W.CONFIGS["cfg0"], decode_steps=4)
     (c,), _, dq, dk, dv = _prepare(wl, 1)
