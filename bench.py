@@ -514,33 +514,49 @@ def run_ours(args, wl, rank, world, device):
         hk = [hall[s, nq:nq + nk].view(dk[0].shape) for s in range(n_e2e)]
         hv = [hall[s, nq + nk:].view(dv[0].shape) for s in range(n_e2e)]
         ho = torch.empty(dq[0].shape, dtype=dq.dtype).pin_memory()
-        sync_all()
-        e0, e1 = ev(), ev()
-        e0.record()
-        for s in range(n_e2e):
+        n_warm = min(3, n_e2e)
+
+        def recompress():
+            ctx.d2o_prefill_compress_layers(0, L, [p[1] for p in prompts], [p[2] for p in prompts])
+
+        for s in range(n_warm):                           # untimed: the entry point's first calls
             ctx.d2o_decode_step_host(0, L, hq[s], hk[s], hv[s], ho)
-        e1.record()
-        sync_all()
-        ms_single = max_over_ranks([e0.elapsed_time(e1)], world, device)[0]
-        ms = ms_single
+        n_rep = 3                                         # timed runs of n_e2e steps each; the median is reported
+
+        def timed(run):
+            times = []
+            for _ in range(n_rep):
+                recompress()
+                sync_all()
+                e0, e1 = ev(), ev()
+                e0.record()
+                run()
+                e1.record()
+                sync_all()
+                times.append(max_over_ranks([e0.elapsed_time(e1)], world, device)[0])
+            return statistics.median(times), times
+
+        def run_single():
+            for s in range(n_e2e):
+                ctx.d2o_decode_step_host(0, L, hq[s], hk[s], hv[s], ho)
+
+        ms_single, all_single = timed(run_single)
+        ms, all_ms = ms_single, all_single
         if not NO_CHAIN:
             # the same steps through the multi-step host entry point: every step's inputs still cross from pinned
             # host memory and its output crosses back inside the timed region, but beside the neighbouring steps' kernels
-            for l in range(L):
-                ctx.d2o_prefill_compress(l, prompts[l][1], prompts[l][2])
+            recompress()
             hq2 = dq[:n_e2e].cpu().pin_memory(); hk2 = dk[:n_e2e].cpu().pin_memory(); hv2 = dv[:n_e2e].cpu().pin_memory()
             ho2 = torch.empty_like(hq2).pin_memory()
-            sync_all()
-            e0, e1 = ev(), ev()
-            e0.record()
-            ctx.d2o_decode_steps_host(0, L, n_e2e, hq2, hk2, hv2, ho2)
-            e1.record()
-            sync_all()
-            ms = max_over_ranks([e0.elapsed_time(e1)], world, device)[0]
+            # untimed: the first call creates the library's two copy streams
+            ctx.d2o_decode_steps_host(0, L, n_warm, hq2[:n_warm], hk2[:n_warm], hv2[:n_warm], ho2[:n_warm])
+            ms, all_ms = timed(lambda: ctx.d2o_decode_steps_host(0, L, n_e2e, hq2, hk2, hv2, ho2))
             del hq2, hk2, hv2, ho2
         e2e = {"value": round(whole_job_rate(wl.batch * n_e2e, world, ms), 2), "unit": "token-steps/s",
                "h2d_bytes_per_step": int((nq + 2 * nk) * hall.element_size()),
                "d2h_bytes_per_step": int(ho.numel() * ho.element_size()), "steps": n_e2e,
+               "runs": f"median of {n_rep} timed runs of {n_e2e} steps after {n_warm} untimed steps",
+               "us_per_step_runs": [round(x * 1e3 / n_e2e, 2) for x in all_ms],
                "us_per_step": round(ms * 1e3 / n_e2e, 2),
                "entry_point": "d2o_decode_step_host" if NO_CHAIN else "d2o_decode_steps_host",
                "us_per_step_single_calls": round(ms_single * 1e3 / n_e2e, 2)}

@@ -1455,18 +1455,20 @@ cudaError_t launch_decode(const d2o_ctx* c, int l0, int l1, const void* q, const
     const int rest = (n_pairs - n_long) * Hkv;
     int rest_max = rows_of_pair(n_long);
     const int cw = (c->decode_warps == 4 || c->decode_warps == 8) ? c->decode_warps
-                   : ((G <= 2 && rest >= 8 * c->n_sms * 4 && rest_max <= 1536) ? 4 : 8);
+                   : ((G <= 2 && rest >= 8 * c->n_sms * 4 && rest_max <= 2304) ? 4 : 8);
     return launch_class(n_long, n_pairs, cw, true);
   }
   // Consumer warps per CTA.  One head per KV head and enough small slices for seven and more CTAs on every SM:
-  // four warps (measured on the serving-shaped config, 8192 slices of ~410 rows: 350 vs 370 us per step).
+  // four warps (measured on the serving-shaped config, 8192 slices of ~410 rows: 350 vs 370 us per step; with the
+  // upper clamp of the budgets removed, slices up to 2048 rows: 306 vs 348 us chained, 354 vs 350 in single calls,
+  // and at 32 sequences 1299 vs 1453 us).
   // Grouped queries with slices several times the mean and few of them: sixteen warps, one CTA per SM, so that the
   // longest slice streams twice as fast.  Otherwise eight.
   const int n_slices = n_pairs * Hkv;
   int cw = c->decode_warps;
   if (cw == 0) {
     cw = 8;
-    if (G <= 2 && n_slices >= 8 * c->n_sms * 4 && max_rows <= 1536) cw = 4;
+    if (G <= 2 && n_slices >= 8 * c->n_sms * 4 && max_rows <= 2304) cw = 4;
     if (G >= 4 && n_slices <= c->n_sms * 8 && max_rows > 2.0 * mean_rows) cw = 16;
   }
   return launch_class(0, n_pairs, cw, chained);
