@@ -217,8 +217,11 @@ def measure_resident(ctx, wl, prompts, dq, dk, dv, nd, lpc, warmup, steps, world
     def one_pass(timed: bool, step_events=None):
         e = [ev() for _ in range(5)]
         e[0].record()
-        for l in range(L):
-            ctx.d2o_layer_stats(l, prompts[l][0], prompts[l][1])
+        if NO_CHAIN:
+            for l in range(L):
+                ctx.d2o_layer_stats(l, prompts[l][0], prompts[l][1])
+        else:
+            ctx.d2o_layer_stats_layers(0, L, [p[0] for p in prompts], [p[1] for p in prompts])
         e[1].record()
         budgets = ctx.d2o_layer_budgets()
         e[2].record()
@@ -296,12 +299,22 @@ def measure_streamed(B, wl, nd, warmup, steps, device, args, with_lse=False):
     for it in range(warmup + steps):
         t_stats = t_comp = 0.0
         pend = []
-        for l in range(L):
-            Q, K, _ = W.LayerStream(wl, l, device).prompt()
+        sgroup = 1 if NO_CHAIN else 2                     # layers whose Q and K are on the device together
+        for l0 in range(0, L, sgroup):
+            l1 = min(L, l0 + sgroup)
+            Qs, Ks = [], []
+            for l in range(l0, l1):
+                Q, K, _ = W.LayerStream(wl, l, device).prompt()
+                Qs.append(Q); Ks.append(K)
             a, b = ev(), ev()
-            a.record(); ctx.d2o_layer_stats(l, Q, K); b.record()
+            a.record()
+            if sgroup == 1:
+                ctx.d2o_layer_stats(l0, Qs[0], Ks[0])
+            else:
+                ctx.d2o_layer_stats_layers(l0, l1, Qs, Ks)
+            b.record()
             pend.append((0, a, b))
-            del Q, K
+            del Qs, Ks, Q, K
         a, b = ev(), ev()
         a.record(); budgets = ctx.d2o_layer_budgets(); b.record()
         pend.append((1, a, b))

@@ -151,6 +151,16 @@ d2o_status d2o_set_prompt_lens(d2o_ctx* ctx, const int32_t* lens, void* stream);
 d2o_status d2o_layer_stats(d2o_ctx* ctx, int32_t layer, const void* Q, const void* K,
                            const float* lse, void* stream);
 
+/* The same for layers [l0, l1) in one call (Eq. 4 acts per layer; a caller that holds several
+ * layers' Q and K can hand them over together).  Q, K: HOST arrays of l1-l0 DEVICE pointers;
+ * lse: NULL, or a HOST array of l1-l0 DEVICE pointers (entries may be NULL).  Two layers are
+ * worked on side by side on streams of the library's own (as d2o_prefill_compress_layers does,
+ * same fork / join on `stream`, same first-call creation of streams and events), each with its
+ * own row-normaliser scratch, so that one layer's last CTAs share the GPU with the next layer's
+ * first.  Results are those of l1-l0 calls of d2o_layer_stats, bit for bit. */
+d2o_status d2o_layer_stats_layers(d2o_ctx* ctx, int32_t l0, int32_t l1, const void* const* Q,
+                                  const void* const* K, const float* const* lse, void* stream);
+
 /* (1') Eq. 5 / Appendix A.2 once every layer has been fed: the cache size of every slice.
  * Writes budgets_host (HOST int32 [B, L, Hkv], may be NULL).  Synchronises `stream`: the host
  * needs the sizes to lay out the cache and to plan the decode launches.  */

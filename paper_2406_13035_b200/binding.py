@@ -23,7 +23,7 @@ TORCH_DTYPE = {D2O_F32: torch.float32, D2O_F16: torch.float16, D2O_BF16: torch.b
 
 EXPORTS = [
     "d2o_status_string", "d2o_last_cuda_error", "d2o_workspace_size", "d2o_create", "d2o_destroy",
-    "d2o_layer_stats", "d2o_layer_budgets", "d2o_budgets_from_density", "d2o_prefill_compress",
+    "d2o_layer_stats", "d2o_layer_stats_layers", "d2o_layer_budgets", "d2o_budgets_from_density", "d2o_prefill_compress",
     "d2o_prefill_compress_layers", "d2o_decode_step", "d2o_decode_steps", "d2o_decode_step_host", "d2o_decode_steps_host", "d2o_full_decode_step", "d2o_get_view", "d2o_get_stats",
     "d2o_set_tuning", "d2o_layer_stats_static", "d2o_set_fault_injection", "d2o_set_prompt_lens",
 ]
@@ -88,6 +88,7 @@ def load_library() -> C.CDLL:
     lib.d2o_destroy.argtypes = [vp]
     lib.d2o_destroy.restype = None
     lib.d2o_layer_stats.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.d2o_layer_stats_layers.argtypes = [vp, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp]
     lib.d2o_layer_budgets.argtypes = [vp, vp, vp]
     lib.d2o_budgets_from_density.argtypes = [vp, i32, i32, i32, i32, i32, f32, i32, i32, f32, i32, i32, i32, i32, f32,
                                              vp, vp, vp, vp, vp]
@@ -190,6 +191,15 @@ class D2OContext:
 
     def d2o_layer_stats(self, layer: int, Q: torch.Tensor, K: torch.Tensor, lse: Optional[torch.Tensor] = None):
         _check(self.lib.d2o_layer_stats(self.handle, layer, _ptr(Q), _ptr(K), _ptr(lse), _stream()), "d2o_layer_stats")
+
+    def d2o_layer_stats_layers(self, l0: int, l1: int, Qs, Ks, lses=None):
+        """`Qs`, `Ks` (and `lses`, entries may be None): one device tensor per layer of [l0, l1)."""
+        n = l1 - l0
+        assert len(Qs) == n and len(Ks) == n and (lses is None or len(lses) == n)
+        qa = (C.c_void_p * n)(*[_ptr(t) for t in Qs])
+        ka = (C.c_void_p * n)(*[_ptr(t) for t in Ks])
+        la = None if lses is None else (C.c_void_p * n)(*[_ptr(t) for t in lses])
+        _check(self.lib.d2o_layer_stats_layers(self.handle, l0, l1, qa, ka, la, _stream()), "d2o_layer_stats_layers")
 
     def d2o_layer_budgets(self) -> torch.Tensor:
         out = torch.empty(self.cfg.batch, self.cfg.n_layers, self.cfg.n_kv_heads, dtype=torch.int32)

@@ -291,14 +291,14 @@ bool colsum_tc_supported(const d2o_config* cfg) {
 
 // Column sums of one layer on the tensor cores.  `lse_in` (natural log, may be NULL) replaces sweep 1.
 cudaError_t launch_colsum_tc(const d2o_ctx* c, const void* Q, const void* K, const float* lse_in, float* colsum,
-                             cudaStream_t st) {
+                             cudaStream_t st, int lane) {
   const d2o_config& g = c->cfg;
   const int B = g.batch, Hq = g.n_q_heads, Hkv = g.n_kv_heads, P = g.prompt_len, D = g.d_head;
   CUtensorMap map_q, map_k;
   if (!encode_rows_2d(&map_q, g.dtype, Q, (uint64_t)B * Hq * P, D, kCsTile)) return cudaErrorNotSupported;
   if (!encode_rows_2d(&map_k, g.dtype, K, (uint64_t)B * Hkv * P, D, kCsTile)) return cudaErrorNotSupported;
   ColsumTcArgs a;
-  a.lse2 = (float*)(c->scratch + c->slay.lse);
+  a.lse2 = (float*)(c->scratch + c->slay.lse + (size_t)lane * c->slay.lse_stride);
   a.colsum = colsum;
   a.status = (uint32_t*)(c->state + c->lay.status);
   a.P = P; a.Hq = Hq; a.group = c->group;

@@ -150,9 +150,11 @@ struct Layout {            // byte offsets into `state`
 };
 struct ScratchLayout {     // byte offsets into `scratch`
   size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, seg_tmp, part_key, pl_spill, stage_q, stage_k, stage_v, stage_out, end;
+  size_t lse_stride;       // `lse` exists kStatsLanes times, this far apart (d2o_layer_stats_layers)
   size_t stage_stride;     // stage_q .. stage_out exist twice, this far apart (d2o_decode_steps_host alternates)
   size_t lane_stride;      // evict_idx .. part_key are the working set of one layer's compression: kCompressLanes copies, this far apart
 };
+constexpr int kStatsLanes = 2;      // layers whose column sums d2o_layer_stats_layers computes side by side
 constexpr int kCompressLanes = 4;   // layers that d2o_prefill_compress_layers works on side by side
 
 }  // namespace d2o
@@ -209,7 +211,7 @@ namespace d2o {
 
 // launchers (one per .cu file); all return cudaError_t of the launch
 cudaError_t launch_layer_stats(const d2o_ctx* c, int layer, const void* Q, const void* K, const float* lse,
-                               cudaStream_t st);
+                               cudaStream_t st, int lane = 0);
 cudaError_t launch_budgets(const double* density, int B, int L, int H, int Hkv, int P, float rho, int min_budget,
                            int max_budget, float gamma, int head_reduce, int budget_rule, int n_sink, int window,
                            float nm_ratio, int32_t* budgets, int32_t* windows, int64_t* row_off, uint32_t* status_word,
@@ -229,7 +231,7 @@ void sim_tc_build_items(const d2o_ctx* c, int n_sms, int4* items, int32_t* count
 // tensor-core column sums of the prompt attention for 16-bit Q/K (d2o_colsum_tc.cu)
 bool colsum_tc_supported(const d2o_config* cfg);
 cudaError_t launch_colsum_tc(const d2o_ctx* c, const void* Q, const void* K, const float* lse_in, float* colsum,
-                             cudaStream_t st);
+                             cudaStream_t st, int lane = 0);
 
 // remembers the text of a failed CUDA runtime call for d2o_last_cuda_error(); returns D2O_ERR_CUDA
 d2o_status record_cuda_error(cudaError_t e, const char* where);

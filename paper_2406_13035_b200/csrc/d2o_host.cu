@@ -119,6 +119,8 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   l->end = o;
   o = 0;
   s->lse = take(B * Hq * P * 4);
+  s->lse_stride = o - s->lse;
+  o += (size_t)(kStatsLanes - 1) * s->lse_stride;
   s->evict_idx = take(B * Hkv * P * 4);
   s->evict_mx = take(B * Hkv * P * 4);
   s->evict_nn = take(B * Hkv * P * 4);
@@ -238,6 +240,46 @@ extern "C" d2o_status d2o_layer_stats(d2o_ctx* c, int32_t layer, const void* Q, 
   return D2O_OK;
 }
 
+// the library's own streams for the multi-layer calls: streams and events only, no device memory
+static d2o_status ensure_lanes(d2o_ctx* c) {
+  if (c->lanes_ready) return D2O_OK;
+  for (int i = 0; i < kCompressLanes; ++i) {
+    CUDA_TRY(cudaStreamCreateWithFlags(&c->lane_stream[i], cudaStreamNonBlocking));
+    CUDA_TRY(cudaEventCreateWithFlags(&c->lane_done[i], cudaEventDisableTiming));
+  }
+  CUDA_TRY(cudaEventCreateWithFlags(&c->lane_fork, cudaEventDisableTiming));
+  c->lanes_ready = true;
+  return D2O_OK;
+}
+
+extern "C" d2o_status d2o_layer_stats_layers(d2o_ctx* c, int32_t l0, int32_t l1, const void* const* Q,
+                                             const void* const* K, const float* const* lse, void* stream) {
+  if (!c || !Q || !K || l0 < 0 || l1 > c->cfg.n_layers || l0 >= l1) return D2O_ERR_INVALID_ARG;
+  for (int l = l0; l < l1; ++l)
+    if (!aligned16(Q[l - l0]) || !aligned16(K[l - l0]) || (lse && lse[l - l0] && !aligned16(lse[l - l0])))
+      return D2O_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (l1 - l0 == 1) {
+    CUDA_TRY(launch_layer_stats(c, l0, Q[0], K[0], lse ? lse[0] : nullptr, st));
+  } else {
+    const d2o_status ls = ensure_lanes(c);
+    if (ls != D2O_OK) return ls;
+    const int lanes = min(kStatsLanes, l1 - l0);
+    CUDA_TRY(cudaEventRecord(c->lane_fork, st));
+    for (int i = 0; i < lanes; ++i) CUDA_TRY(cudaStreamWaitEvent(c->lane_stream[i], c->lane_fork, 0));
+    for (int l = l0; l < l1; ++l) {
+      const int lane = (l - l0) % lanes;                     // a lane's layers follow one another on its stream
+      CUDA_TRY(launch_layer_stats(c, l, Q[l - l0], K[l - l0], lse ? lse[l - l0] : nullptr, c->lane_stream[lane], lane));
+    }
+    for (int i = 0; i < lanes; ++i) {
+      CUDA_TRY(cudaEventRecord(c->lane_done[i], c->lane_stream[i]));
+      CUDA_TRY(cudaStreamWaitEvent(st, c->lane_done[i], 0));
+    }
+  }
+  for (int l = l0; l < l1; ++l) c->layer_fed[l] = 1;
+  return D2O_OK;
+}
+
 extern "C" d2o_status d2o_budgets_from_density(const double* density, int32_t batch, int32_t n_layers,
                                                int32_t n_heads, int32_t n_kv_heads, int32_t prompt_len, float rho,
                                                int32_t min_budget, int32_t max_budget, float density_temp,
@@ -335,15 +377,8 @@ extern "C" d2o_status d2o_prefill_compress_layers(d2o_ctx* c, int32_t l0, int32_
   if (l1 - l0 == 1) {
     CUDA_TRY(launch_prefill_compress(c, l0, K[0], V[0], st));
   } else {
-    if (!c->lanes_ready) {
-      // streams and events only: no device memory
-      for (int i = 0; i < kCompressLanes; ++i) {
-        CUDA_TRY(cudaStreamCreateWithFlags(&c->lane_stream[i], cudaStreamNonBlocking));
-        CUDA_TRY(cudaEventCreateWithFlags(&c->lane_done[i], cudaEventDisableTiming));
-      }
-      CUDA_TRY(cudaEventCreateWithFlags(&c->lane_fork, cudaEventDisableTiming));
-      c->lanes_ready = true;
-    }
+    const d2o_status ls = ensure_lanes(c);
+    if (ls != D2O_OK) return ls;
     // the lanes start behind everything the caller's stream holds, the caller's stream goes on behind every lane
     const int lanes = min(kCompressLanes, l1 - l0);
     CUDA_TRY(cudaEventRecord(c->lane_fork, st));

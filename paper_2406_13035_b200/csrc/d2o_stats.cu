@@ -383,7 +383,7 @@ __global__ void budget_kernel(const double* __restrict__ density, int B, int L, 
 
 template <typename T, int D>
 static cudaError_t run_stats(const d2o_ctx* c, int layer, const void* Q, const void* K, const float* lse_in,
-                             cudaStream_t st) {
+                             cudaStream_t st, int lane) {
   const d2o_config& g = c->cfg;
   const int P = g.prompt_len, Hq = g.n_q_heads, B = g.batch;
   const int nT = (P + kTile - 1) / kTile;
@@ -391,7 +391,7 @@ static cudaError_t run_stats(const d2o_ctx* c, int layer, const void* Q, const v
   double* density = (double*)(c->state + c->lay.density);
   const int32_t* plen = (const int32_t*)(c->state + c->lay.plen);
   if (c->stats_path == 0 && colsum_tc_supported(&g)) {
-    cudaError_t e = launch_colsum_tc(c, Q, K, lse_in, colsum, st);
+    cudaError_t e = launch_colsum_tc(c, Q, K, lse_in, colsum, st, lane);
     if (e != cudaSuccess) return e;
     density_kernel<<<B * Hq, 256, 0, st>>>(colsum, density, P, Hq, g.n_layers, layer, plen);
     return cudaGetLastError();
@@ -399,7 +399,7 @@ static cudaError_t run_stats(const d2o_ctx* c, int layer, const void* Q, const v
   const float* lse = lse_in;
   dim3 grid(nT, B * Hq);
   if (!lse) {
-    float* lse_buf = (float*)(c->scratch + c->slay.lse);
+    float* lse_buf = (float*)(c->scratch + c->slay.lse + (size_t)lane * c->slay.lse_stride);
     const size_t sm = (size_t)2 * D * kTile * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(lse_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
@@ -415,13 +415,13 @@ static cudaError_t run_stats(const d2o_ctx* c, int layer, const void* Q, const v
 }
 
 cudaError_t launch_layer_stats(const d2o_ctx* c, int layer, const void* Q, const void* K, const float* lse,
-                               cudaStream_t st) {
+                               cudaStream_t st, int lane) {
   const int d = c->cfg.d_head;
   switch (c->cfg.dtype) {
-    case D2O_F32: return d == 64 ? run_stats<float, 64>(c, layer, Q, K, lse, st) : run_stats<float, 128>(c, layer, Q, K, lse, st);
-    case D2O_F16: return d == 64 ? run_stats<__half, 64>(c, layer, Q, K, lse, st) : run_stats<__half, 128>(c, layer, Q, K, lse, st);
-    default: return d == 64 ? run_stats<__nv_bfloat16, 64>(c, layer, Q, K, lse, st)
-                            : run_stats<__nv_bfloat16, 128>(c, layer, Q, K, lse, st);
+    case D2O_F32: return d == 64 ? run_stats<float, 64>(c, layer, Q, K, lse, st, lane) : run_stats<float, 128>(c, layer, Q, K, lse, st, lane);
+    case D2O_F16: return d == 64 ? run_stats<__half, 64>(c, layer, Q, K, lse, st, lane) : run_stats<__half, 128>(c, layer, Q, K, lse, st, lane);
+    default: return d == 64 ? run_stats<__nv_bfloat16, 64>(c, layer, Q, K, lse, st, lane)
+                            : run_stats<__nv_bfloat16, 128>(c, layer, Q, K, lse, st, lane);
   }
 }
 

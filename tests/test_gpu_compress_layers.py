@@ -86,6 +86,28 @@ def test_fp32_config_0_shape():
     _run(wl, [(0, 6)])
 
 
+@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfg2"])
+def test_layer_stats_of_several_layers_in_one_call(name):
+    """d2o_layer_stats_layers against layer-by-layer calls: column sums, densities and budgets bit for bit."""
+    wl = (dataclasses.replace(W.CONFIGS["cfg0"], n_layers=5, density_temp=50.0, min_budget=64) if name == "cfg0"
+          else W.twin(name).scaled(n_layers=5, prompt_div=1, batch=2, steps=2))
+    a, b = make_ctx(wl), make_ctx(wl)
+    streams = [W.LayerStream(wl, l, "cuda:0") for l in range(wl.n_layers)]
+    QK = [s.prompt()[:2] for s in streams]
+    for l, (Q, K) in enumerate(QK):
+        a.d2o_layer_stats(l, Q, K)
+    b.d2o_layer_stats_layers(0, 3, [q for q, _ in QK[:3]], [k for _, k in QK[:3]])
+    b.d2o_layer_stats_layers(3, 4, [QK[3][0]], [QK[3][1]])
+    b.d2o_layer_stats_layers(4, 5, [QK[4][0]], [QK[4][1]], [None])
+    for l in range(wl.n_layers):
+        assert torch.equal(a.colsum(l).view(torch.uint8), b.colsum(l).view(torch.uint8)), l
+    assert torch.equal(a.density().view(torch.uint8), b.density().view(torch.uint8))
+    assert torch.equal(a.d2o_layer_budgets(), b.d2o_layer_budgets())
+    for c in (a, b):
+        assert c.d2o_get_stats().error_word == 0
+    a.close(); b.close()
+
+
 def test_argument_checks():
     wl = dataclasses.replace(W.twin("cfg1"), decode_steps=2)
     c = make_ctx(wl)
