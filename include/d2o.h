@@ -231,9 +231,10 @@ d2o_status d2o_decode_step_host(d2o_ctx* ctx, int32_t l0, int32_t l1, const void
  * anything): q_host [n_steps, l1-l0, B, Hq, d], k_host and v_host [n_steps, l1-l0, B, Hkv, d],
  * out_host [n_steps, l1-l0, B, Hq, d].  Per step the same work as d2o_decode_step_host, but
  * pipelined over three streams (the caller's for the kernels, two of the library's own for the
- * copies, created with the first call; no device memory): while step t computes, the inputs of
- * step t+1 travel to the device and the output of step t-1 travels back, through two staging
- * sets in `scratch`.  As with d2o_decode_steps a step's inputs cannot depend on an earlier
+ * copies, created with the first call; no device memory), in blocks of four steps: while a
+ * block computes, the inputs of the next block travel to the device and the outputs of the
+ * previous one travel back, through two blocks of staging sets in `scratch`; the steps of a
+ * block are chained as in d2o_decode_steps.  As with d2o_decode_steps a step's inputs cannot depend on an earlier
  * step's output.  Returns after everything, the last copy back included, has completed. */
 d2o_status d2o_decode_steps_host(d2o_ctx* ctx, int32_t l0, int32_t l1, int32_t n_steps,
                                  const void* q_host, const void* k_host, const void* v_host,

@@ -151,9 +151,10 @@ struct Layout {            // byte offsets into `state`
 struct ScratchLayout {     // byte offsets into `scratch`
   size_t lse, evict_idx, evict_mx, evict_nn, seg_start, seg_items, seg_tmp, part_key, pl_spill, stage_q, stage_k, stage_v, stage_out, end;
   size_t lse_stride;       // `lse` exists kStatsLanes times, this far apart (d2o_layer_stats_layers)
-  size_t stage_stride;     // stage_q .. stage_out exist twice, this far apart (d2o_decode_steps_host alternates)
+  size_t stage_stride;     // stage_q .. stage_out exist 2 * kHostBlock times, this far apart (d2o_decode_steps_host)
   size_t lane_stride;      // evict_idx .. part_key are the working set of one layer's compression: kCompressLanes copies, this far apart
 };
+constexpr int kHostBlock = 4;       // steps per block of d2o_decode_steps_host (two blocks of staging sets)
 constexpr int kStatsLanes = 2;      // layers whose column sums d2o_layer_stats_layers computes side by side
 constexpr int kCompressLanes = 4;   // layers that d2o_prefill_compress_layers works on side by side
 

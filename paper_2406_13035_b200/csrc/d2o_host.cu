@@ -135,8 +135,8 @@ static void layouts(const d2o_config* c, int64_t total_budget, int max_budget, L
   s->stage_k = take(L * B * Hkv * d * e);
   s->stage_v = take(L * B * Hkv * d * e);
   s->stage_out = take(L * B * Hq * d * e);
-  s->stage_stride = o - s->stage_q;                        // a second set of the four for the pipelined host path
-  o += s->stage_stride;
+  s->stage_stride = o - s->stage_q;                        // further sets of the four for the pipelined host path
+  o += (size_t)(2 * kHostBlock - 1) * s->stage_stride;
   s->end = o;
 }
 
@@ -503,38 +503,49 @@ extern "C" d2o_status d2o_decode_steps_host(d2o_ctx* c, int32_t l0, int32_t l1, 
   const size_t nl = (size_t)(l1 - l0);
   const size_t qb = nl * g.batch * g.n_q_heads * g.d_head * c->elem_size;
   const size_t kb = nl * g.batch * g.n_kv_heads * g.d_head * c->elem_size;
-  // Step t uses staging set t % 2.  Three streams: the copies of step t + 1 to the device and of step t - 1 back run
-  // beside the kernels of step t.  A set is refilled once the step that read it is done (io_step_done), and its
-  // output is overwritten once the copy back of the step before last is done (io_out_done).
+  // Steps go in blocks of kHostBlock; block b uses the staging sets of parity b % 2.  Three streams: the copies of
+  // block b + 1 to the device and of block b - 1 back run beside the kernels of block b.  Inside a block the inputs of
+  // every step are on the device before its first step is launched, so its steps are chained like those of
+  // d2o_decode_steps.  A parity's sets are refilled once the block that read them is done (io_step_done), and their
+  // outputs are overwritten once the copies back of the block before last are done (io_out_done).
   CUDA_TRY(cudaEventRecord(c->io_start, s));
   CUDA_TRY(cudaStreamWaitEvent(c->io_in, c->io_start, 0));
   CUDA_TRY(cudaStreamWaitEvent(c->io_out, c->io_start, 0));
-  for (int t = 0; t < n_steps; ++t) {
-    const int set = t & 1;
-    char* base = c->scratch + (size_t)set * c->slay.stage_stride;
-    char* dq = base + c->slay.stage_q; char* dk = base + c->slay.stage_k;
-    char* dv = base + c->slay.stage_v; char* dout = base + c->slay.stage_out;
-    if (t >= 2) CUDA_TRY(cudaStreamWaitEvent(c->io_in, c->io_step_done[set], 0));
-    CUDA_TRY(cudaMemcpyAsync(dq, (const char*)q_host + t * qb, qb, cudaMemcpyHostToDevice, c->io_in));
-    CUDA_TRY(cudaMemcpyAsync(dk, (const char*)k_host + t * kb, kb, cudaMemcpyHostToDevice, c->io_in));
-    CUDA_TRY(cudaMemcpyAsync(dv, (const char*)v_host + t * kb, kb, cudaMemcpyHostToDevice, c->io_in));
-    CUDA_TRY(cudaEventRecord(c->io_in_done[set], c->io_in));
-    CUDA_TRY(cudaStreamWaitEvent(s, c->io_in_done[set], 0));
-    if (t >= 2) CUDA_TRY(cudaStreamWaitEvent(s, c->io_out_done[set], 0));
-    d2o_status why = D2O_OK;
-    cudaError_t e = launch_decode(c, l0, l1, dq, dk, dv, dout, s, &why);
-    if (why != D2O_OK || e != cudaSuccess) {
-      (void)cudaStreamSynchronize(c->io_in); (void)cudaStreamSynchronize(c->io_out); (void)cudaStreamSynchronize(s);
-      return why != D2O_OK ? why : cuda_fail(e, "launch_decode");
+  const int n_blocks = (n_steps + kHostBlock - 1) / kHostBlock;
+  for (int b = 0; b < n_blocks; ++b) {
+    const int par = b & 1, t0 = b * kHostBlock, cnt = min(kHostBlock, n_steps - t0);
+    auto set_base = [&](int i) { return c->scratch + (size_t)(par * kHostBlock + i) * c->slay.stage_stride; };
+    if (b >= 2) CUDA_TRY(cudaStreamWaitEvent(c->io_in, c->io_step_done[par], 0));
+    for (int i = 0; i < cnt; ++i) {
+      char* base = set_base(i);
+      const size_t t = (size_t)(t0 + i);
+      CUDA_TRY(cudaMemcpyAsync(base + c->slay.stage_q, (const char*)q_host + t * qb, qb, cudaMemcpyHostToDevice, c->io_in));
+      CUDA_TRY(cudaMemcpyAsync(base + c->slay.stage_k, (const char*)k_host + t * kb, kb, cudaMemcpyHostToDevice, c->io_in));
+      CUDA_TRY(cudaMemcpyAsync(base + c->slay.stage_v, (const char*)v_host + t * kb, kb, cudaMemcpyHostToDevice, c->io_in));
     }
-    for (int l = l0; l < l1; ++l) c->layer_steps[l] += 1;
-    CUDA_TRY(cudaEventRecord(c->io_step_done[set], s));
-    CUDA_TRY(cudaStreamWaitEvent(c->io_out, c->io_step_done[set], 0));
-    CUDA_TRY(cudaMemcpyAsync((char*)out_host + t * qb, dout, qb, cudaMemcpyDeviceToHost, c->io_out));
-    CUDA_TRY(cudaEventRecord(c->io_out_done[set], c->io_out));
+    CUDA_TRY(cudaEventRecord(c->io_in_done[par], c->io_in));
+    CUDA_TRY(cudaStreamWaitEvent(s, c->io_in_done[par], 0));
+    if (b >= 2) CUDA_TRY(cudaStreamWaitEvent(s, c->io_out_done[par], 0));
+    for (int i = 0; i < cnt; ++i) {
+      char* base = set_base(i);
+      d2o_status why = D2O_OK;
+      cudaError_t e = launch_decode(c, l0, l1, base + c->slay.stage_q, base + c->slay.stage_k, base + c->slay.stage_v,
+                                    base + c->slay.stage_out, s, &why, i > 0, i + 1 < cnt);
+      if (why != D2O_OK || e != cudaSuccess) {
+        (void)cudaStreamSynchronize(c->io_in); (void)cudaStreamSynchronize(c->io_out); (void)cudaStreamSynchronize(s);
+        return why != D2O_OK ? why : cuda_fail(e, "launch_decode");
+      }
+      for (int l = l0; l < l1; ++l) c->layer_steps[l] += 1;
+    }
+    CUDA_TRY(cudaEventRecord(c->io_step_done[par], s));
+    CUDA_TRY(cudaStreamWaitEvent(c->io_out, c->io_step_done[par], 0));
+    for (int i = 0; i < cnt; ++i)
+      CUDA_TRY(cudaMemcpyAsync((char*)out_host + (size_t)(t0 + i) * qb, set_base(i) + c->slay.stage_out, qb,
+                               cudaMemcpyDeviceToHost, c->io_out));
+    CUDA_TRY(cudaEventRecord(c->io_out_done[par], c->io_out));
   }
   // the caller's stream ends behind the last copies back; then wait for all of it
-  for (int i = 0; i < (n_steps > 1 ? 2 : 1); ++i) CUDA_TRY(cudaStreamWaitEvent(s, c->io_out_done[(n_steps - 1 - i) & 1], 0));
+  for (int i = 0; i < (n_blocks > 1 ? 2 : 1); ++i) CUDA_TRY(cudaStreamWaitEvent(s, c->io_out_done[(n_blocks - 1 - i) & 1], 0));
   CUDA_TRY(cudaStreamSynchronize(s));
   return D2O_OK;
 }
