@@ -57,7 +57,7 @@ struct DecodeArgs {
   int row_cap;                      // rows of a slice whose logits / probabilities live in shared memory (multiple of 8)
   float* spill;                     // the same for rows >= row_cap: [(row0 + 8 slice) G + g (stride(S) + 8) + row], stays in L2
   int stages;                       // stages of the ring
-  int l2_hints;                     // 1: pass K asks L2 to keep its lines, later passes to drop theirs
+  int l2_hints;                     // 1: the streamed rows are marked evict-first in L2 (each is read once per step)
   const int32_t* order;             // NULL: CTAs take (layer, b, h) in index order; else (layer * B + b) per group of Hkv CTAs
   int pair_base;                    // first entry of `order` this launch works on
   int average;                      // 1: average merge (both rows weigh 1/2) instead of the weights of Eq. 12
@@ -418,11 +418,8 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
     if (lane == 0) {
       // rows that the previous step's CTA wrote with ordinary stores are read here by bulk copies
       if (a.chained) asm volatile("fence.proxy.async.global;" ::: "memory");
-      unsigned long long keep = 0, drop = 0;
-      if (a.l2_hints) {
-        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
-        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
-      }
+      unsigned long long drop = 0;
+      if (a.l2_hints) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
       int slot = 0, q = 0;
       uint32_t ph = 1;                                               // parity of the previous use of a slot
       bool stopped = false;
@@ -431,8 +428,10 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
         const T* pool = is_v ? vpool : kpool;
         const T* fresh = is_v ? v_new : k_new;
         const bool hint = a.l2_hints != 0;
-        // keys may be read once more (a victim that was not guessed): they leave L2 after the values
-        const unsigned long long pol = (p == 0 && evict) ? keep : drop;
+        // Keys and values cross once per step, so their lines are the first to leave L2; what stays is the per-row
+        // state, which is read twice and written.  (Keeping the keys for the rare second look after a wrong guess
+        // cost 3 - 8 % of the step; that look now goes to DRAM.)
+        const unsigned long long pol = drop;
         for (int s = 0; s < n_st; ++s, ++q, ring_next(slot, ph, NS)) {
           if (q >= NS) stage_wait(&s_empty[slot], ph, &s_timeout, a.wait_ns);
           // a wait ran out somewhere in this CTA, or the failure-detection tests asked for a stage that never
@@ -935,7 +934,7 @@ decode_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap map_k, const __g
       for (int c = 0; c < NC; ++c) if (hit == c) { best = cbest[c]; best_li = cbest_li[c]; }
     } else {
       // The victim was not among the guessed rows (or is the new token itself): the keys once more, straight from
-      // global memory, where L2 still holds most of them.  One row per group of LPR lanes.
+      // global memory.  One row per group of LPR lanes.
       if (tid == 0) atomicAdd(&a.counters[kCntGuessMisses], 1ull);
       for (int li = grp; li < n_old; li += NGRP) {
         float f[EPV];
