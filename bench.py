@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS = 8000.0          # the figure the metric quotes; the measured c
 # dram__bytes_read.sum + dram__bytes_write.sum of the decode_kernel launches of one step under ncu (the full-size
 # workload, counters that take one pass), divided by the algorithmic bytes of that step, per workload the counters were
 # taken on (None: not captured for this kernel build)
-DECODE_TRAFFIC_RATIO = {"cfg1": 1.022, "cfg2": 1.056}
+DECODE_TRAFFIC_RATIO = {"cfg1": 1.005, "cfg2": 1.040}
 NO_CHAIN = False                  # --single-step-calls: one d2o_decode_step call per token in the timed passes too
 
 
